@@ -1,0 +1,305 @@
+"""Pins for the oracle's verify / propose / commit chain (CPU only).
+
+Every expectation here comes from the paper's statements or from mathematics,
+never from the oracle itself: the p/q rule's closed forms, the laws the rule is
+proved to preserve, brute-force products on tiny vocabularies, the TPF closed
+form (Eq. 3) and the worked example of the step-by-step figure.
+"""
+import os
+
+import numpy as np
+import pytest
+import scipy.stats
+
+import oracle
+from helpers import oracle_step, tiny_state
+from paper_2604_11035_b200.workloads import Workload
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def wl_tiny(B, N, V, seed, propose_mode=0, q_mode=0):
+    return Workload("t", batch=B, stride=N, vocab=V, logits_dtype="f32", propose_mode=propose_mode,
+                    q_mode=q_mode, seed=seed)
+
+
+def rows_from_probs(B, N, probs_by_row):
+    """[B, Q, V] fp32 logits whose row r is log(probs_by_row[r]) for every slot."""
+    Q = 2 * N - 1
+    lg = np.log(np.asarray(probs_by_row, dtype=np.float64))
+    assert lg.shape[0] == Q
+    return np.ascontiguousarray(np.broadcast_to(lg[None], (B,) + lg.shape)).astype(np.float32)
+
+
+def softmax32(row):
+    """Law actually encoded by fp32 logits."""
+    r = np.asarray(row, np.float32).astype(np.float64)
+    e = np.exp(r - r.max())
+    return e / e.sum()
+
+
+def chi2_p(counts, probs):
+    counts, probs = np.asarray(counts, float), np.asarray(probs, float)
+    keep = probs > 0
+    assert counts[~keep].sum() == 0
+    return scipy.stats.chisquare(counts[keep], probs[keep] / probs[keep].sum() * counts[keep].sum()).pvalue
+
+
+def two_step(B, N, V, q_rows, p_rows, seed, propose_mode=0, tau=0.0, q_mode=0):
+    """Step 0 = NP step proposing from q_rows (rows 1..N-1), step 1 = P step judging with p_rows."""
+    Q = 2 * N - 1
+    w = wl_tiny(B, N, V, seed, propose_mode, q_mode)
+    s = tiny_state(B, N, V)
+    pad = [np.full(V, 1.0 / V)] * Q
+    l0 = rows_from_probs(B, N, ([pad[0]] + list(q_rows) + pad)[:Q])
+    _, _, v0, _ = oracle_step(w, s, None, None, None, l0, None, 0, do_attn=False)
+    assert np.all(s["n_ver"] == N - 1) and np.all(s["q_row0"] == 1)
+    l1 = rows_from_probs(B, N, (list(p_rows) + pad)[:Q])
+    s_before = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in s.items()}
+    _, _, v1, _ = oracle_step(w, s, None, None, None, l1, l0, 1, do_attn=False, tau=tau)
+    return w, s_before, s, v0, v1, l0, l1
+
+
+# --------------------------------------------------------------------------- accept rule
+def test_identical_laws_always_accept():
+    # "For AR models p = q by construction, yielding alpha = 1" (Sec. 2): ratio 1 accepts for every u.
+    B, N, V = 4000, 4, 8
+    rng = np.random.default_rng(1)
+    laws = rng.dirichlet(np.ones(V), size=N - 1)
+    _, _, s, v0, v1, _, _ = two_step(B, N, V, laws, list(laws) + [np.full(V, 1 / V)], seed=5)
+    assert np.all(v1.accept == 1) and np.all(v1.accept_len == N - 1) and np.all(v1.n_emit == N)
+    assert np.allclose(v1.alpha, 1.0)
+    assert np.all(s["n_ver"] == N - 1)
+    assert np.array_equal(v1.out_tok[:, :N - 1], v0.new_prop_tok)
+
+
+def test_zero_anchor_probability_never_accepts():
+    B, N, V = 3000, 2, 4
+    q = np.array([0.7, 0.1, 0.1, 0.1])
+    w = wl_tiny(B, N, V, 9, propose_mode=1)     # argmax proposals: always token 0
+    s = tiny_state(B, N, V)
+    l0 = rows_from_probs(B, N, [np.full(V, .25), q, np.full(V, .25)])
+    oracle_step(w, s, None, None, None, l0, None, 0, do_attn=False)
+    assert np.all(s["block_tok"][:, 1] == 0)
+    l1 = rows_from_probs(B, N, [np.full(V, .25)] * 3)
+    l1[:, 0, 0] = -np.inf                        # p(x^) = 0
+    _, _, v1, _ = oracle_step(w, s, None, None, None, l1, l0, 1, do_attn=False)
+    assert np.all(v1.accept[:, 0] == 0) and np.all(v1.accept_len == 0) and np.all(v1.n_emit == 1)
+    assert np.all(v1.alpha[:, 0] == 0.0)
+    assert np.all(v1.repl_tok != 0)              # residual excludes the rejected token
+    assert np.all(s["n_ver"] == 0)               # next step is a pure stride
+
+
+def test_accept_decision_is_u_below_ratio_and_counts_match():
+    # accept iff u < min(1, p(x)/q(x)), u on the 2^-24 lattice (Algorithm 1, strict <)
+    B, N, V = 20000, 2, 4
+    q = np.array([0.4, 0.3, 0.2, 0.1])
+    p = np.array([0.1, 0.2, 0.3, 0.4])
+    w, sb, s, v0, v1, l0, l1 = two_step(B, N, V, [q], [p, np.full(V, .25)], seed=21)
+    p32, q32 = softmax32(l1[0, 0]), softmax32(l0[0, 1])
+    x = v0.new_prop_tok[:, 0]
+    ratio = np.minimum(1.0, p32[x] / q32[x])
+    assert np.allclose(v1.alpha[:, 0], ratio, rtol=1e-12)
+    u = np.array([oracle.uniform(w.seed, 1, b, 1) for b in range(B)])
+    assert np.array_equal(v1.u[:, 0], u)
+    assert np.array_equal(v1.accept[:, 0] == 1, u < ratio)
+    # closed form: for fixed alpha exactly ceil(alpha * 2^24) lattice points accept
+    for tok in range(V):
+        a = ratio[x == tok][0]
+        thresh = int(np.ceil(a * 2 ** 24))
+        k = (u[x == tok] * 2 ** 24).astype(np.int64)
+        assert np.array_equal(v1.accept[x == tok, 0] == 1, k < thresh)
+    # mean acceptance over x^ ~ q equals sum_i min(p_i, q_i)
+    want = np.minimum(p32, q32).sum()
+    got = (v1.accept[:, 0] == 1).mean()
+    assert abs(got - want) < 4 * np.sqrt(want * (1 - want) / B)
+
+
+def test_relaxed_acceptance_is_monotone_in_tau():
+    B, N, V = 5000, 3, 8
+    rng = np.random.default_rng(3)
+    q = rng.dirichlet(np.ones(V), size=N - 1)
+    p = rng.dirichlet(np.ones(V), size=N)
+    lens = []
+    for tau in (0.0, 0.5, 1.0):
+        _, _, _, v0, v1, l0, l1 = two_step(B, N, V, q, p, seed=33, tau=tau)
+        lens.append(v1.accept_len.copy())
+        x = v0.new_prop_tok[:, 0]
+        ratio = np.minimum(1.0, (1 + tau) * softmax32(l1[0, 0])[x] / softmax32(l0[0, 1])[x])
+        assert np.allclose(v1.alpha[:, 0], ratio, rtol=1e-6)
+    assert np.all(lens[0] <= lens[1]) and np.all(lens[1] <= lens[2])
+    assert lens[2].sum() > lens[0].sum()
+
+
+# --------------------------------------------------------------------------- laws
+def test_proposal_residual_final_and_bonus_laws():
+    B, N, V = 120000, 2, 4
+    q = np.array([0.50, 0.25, 0.15, 0.10])
+    p = np.array([0.20, 0.20, 0.35, 0.25])
+    bonus = np.array([0.1, 0.6, 0.1, 0.2])
+    free = np.array([0.3, 0.3, 0.2, 0.2])
+    Q = 3
+    w = wl_tiny(B, N, V, 77)
+    s = tiny_state(B, N, V)
+    l0 = rows_from_probs(B, N, [free, q, np.full(V, .25)])
+    _, _, v0, _ = oracle_step(w, s, None, None, None, l0, None, 0, do_attn=False)
+    l1 = rows_from_probs(B, N, [p, bonus, np.full(V, .25)])
+    _, _, v1, _ = oracle_step(w, s, None, None, None, l1, l0, 1, do_attn=False)
+    p32, q32 = softmax32(l1[0, 0]), softmax32(l0[0, 1])
+    cnt = lambda t: np.bincount(t, minlength=V)
+    # NP step: the free token is an exact AR sample of row 0 (Algorithm 1, "quality-guaranteed")
+    assert chi2_p(cnt(v0.repl_tok), softmax32(l0[0, 0])) > 1e-3
+    assert np.all(v0.n_emit == 1) and np.all(v0.accept_len == 0)
+    # proposals follow q
+    assert chi2_p(cnt(v0.new_prop_tok[:, 0]), q32) > 1e-3
+    rej = v1.accept[:, 0] == 0
+    acc = ~rej
+    # on rejection the replacement follows normalize(max(0, p - q)) and avoids tokens with p <= q
+    resid = np.maximum(0.0, p32 - q32)
+    assert chi2_p(cnt(v1.repl_tok[rej]), resid) > 1e-3
+    # the finalised token at the judged position follows p exactly (losslessness)
+    assert chi2_p(cnt(v1.out_tok[:, 0]), p32) > 1e-3
+    # all accepted -> bonus token from the final anchor row
+    assert chi2_p(cnt(v1.repl_tok[acc]), softmax32(l1[0, 1])) > 1e-3
+    assert np.all(v1.n_emit[acc] == 2) and np.all(v1.n_emit[rej] == 1)
+    assert np.all(v1.out_tok[acc, 0] == v0.new_prop_tok[acc, 0])
+    assert np.all(v1.out_tok[rej, 1] == -1)
+
+
+def test_two_token_vocab_residual_is_a_point_mass():
+    B, N, V = 4000, 2, 2
+    _, _, _, v0, v1, _, _ = two_step(B, N, V, [np.array([0.8, 0.2])], [np.array([0.3, 0.7]), np.array([.5, .5])], seed=4)
+    rej = v1.accept[:, 0] == 0
+    assert rej.sum() > 100
+    assert np.all(v0.new_prop_tok[rej, 0] == 0)   # only the over-proposed token can be rejected
+    assert np.all(v1.repl_tok[rej] == 1)
+
+
+def test_one_hot_q_mode():
+    # argmax proposals judged against a point mass: accept w.p. p(x^); residual = p without x^
+    B, N, V = 60000, 2, 4
+    p = np.array([0.55, 0.25, 0.15, 0.05])
+    w = wl_tiny(B, N, V, 13, propose_mode=1, q_mode=1)
+    s = tiny_state(B, N, V)
+    l0 = rows_from_probs(B, N, [np.full(V, .25), np.array([0.4, 0.3, 0.2, 0.1]), np.full(V, .25)])
+    oracle_step(w, s, None, None, None, l0, None, 0, do_attn=False)
+    l1 = rows_from_probs(B, N, [p, np.full(V, .25), np.full(V, .25)])
+    _, _, v1, _ = oracle_step(w, s, None, None, None, l1, None, 1, do_attn=False)
+    p32 = softmax32(l1[0, 0])
+    acc = v1.accept[:, 0] == 1
+    assert abs(acc.mean() - p32[0]) < 4 * np.sqrt(p32[0] * (1 - p32[0]) / B)
+    resid = p32.copy(); resid[0] = 0
+    assert chi2_p(np.bincount(v1.repl_tok[~acc], minlength=V), resid) > 1e-3
+    assert chi2_p(np.bincount(v1.out_tok[:, 0], minlength=V), p32) > 1e-3
+
+
+# --------------------------------------------------------------------------- prefix structure / brute force
+def test_prefix_structure_bounds_and_brute_force_products():
+    B, N, V = 100000, 3, 3
+    rng = np.random.default_rng(8)
+    q = rng.dirichlet(np.ones(V) * 2, size=N - 1)
+    p = rng.dirichlet(np.ones(V) * 2, size=N)
+    _, sb, s, v0, v1, l0, l1 = two_step(B, N, V, q, p, seed=99)
+    acc = v1.accept
+    for b in range(0, B, 997):
+        row = list(acc[b])
+        k = v1.accept_len[b]
+        assert row[:k] == [1] * k
+        if k < N - 1:
+            assert row[k] == 0 and row[k + 1:] == [-1] * (N - 2 - k)
+    assert v1.accept_len.min() >= 0 and v1.accept_len.max() <= N - 1
+    assert np.array_equal(v1.n_emit, v1.accept_len + 1)
+    assert v1.n_emit.min() >= 1 and v1.n_emit.max() <= N
+    # brute force: P(a >= j) = prod_{k <= j} sum_i min(p_k,i , q_k,i)
+    prod = 1.0
+    for j in range(1, N):
+        prod *= np.minimum(softmax32(l1[0, j - 1]), softmax32(l0[0, j])).sum()
+        got = (v1.accept_len >= j).mean()
+        assert abs(got - prod) < 4.5 * np.sqrt(prod * (1 - prod) / B), (j, got, prod)
+    # joint law of (a, y) by enumeration for a = 0: P(a=0, y) = residual_1(y) * (1 - sum min)
+    p1, q1 = softmax32(l1[0, 0]), softmax32(l0[0, 1])
+    joint = np.maximum(0, p1 - q1)
+    sel = v1.accept_len == 0
+    emp = np.bincount(v1.repl_tok[sel], minlength=V) / B
+    assert np.all(np.abs(emp - joint) < 4.5 * np.sqrt(np.maximum(joint, 1e-4) / B))
+    # state machine after the step
+    allacc = v1.accept_len == sb["n_ver"]
+    assert np.array_equal(s["n_ver"], np.where(allacc, N - 1, 0))
+    assert np.array_equal(s["ctx_len"], sb["ctx_len"] + v1.n_emit)
+    assert np.array_equal(s["block_tok"][:, 0], v1.repl_tok)
+
+
+# --------------------------------------------------------------------------- worked example + TPF
+def _golden_rows():
+    rows = []
+    for line in open(os.path.join(GOLDEN, "isd_steps_figure.txt")):
+        if line.strip() and not line.startswith("#"):
+            f = line.split()
+            rows.append((f[0],) + tuple(int(x) for x in f[1:]))
+    return rows
+
+
+@pytest.mark.parametrize("case", _golden_rows(), ids=lambda c: c[0])
+def test_step_by_step_figure(case):
+    name, N, n_ver, rejected, want_a, want_emit, want_next, want_growth = case
+    B, V, Q = 3, 8, 2 * N - 1
+    w = wl_tiny(B, N, V, 1, propose_mode=1)
+    s = tiny_state(B, N, V)
+    law = np.array([0.3, 0.2, 0.1, 0.1, 0.1, 0.1, 0.05, 0.05])
+    l0 = rows_from_probs(B, N, [law] * Q)
+    oracle_step(w, s, None, None, None, l0, None, 0, do_attn=False)
+    if n_ver == 0:
+        s = tiny_state(B, N, V)      # judge the bootstrap step itself
+        ctx0 = s["ctx_len"].copy()
+        _, _, v, _ = oracle_step(w, s, None, None, None, l0, None, 0, do_attn=False)
+    else:
+        ctx0 = s["ctx_len"].copy()
+        l1 = rows_from_probs(B, N, [law] * Q)     # identical laws: accepted ...
+        if rejected:
+            l1[:, rejected - 1, 0] = -np.inf       # ... except one proposal with p(x^) = 0
+        _, _, v, _ = oracle_step(w, s, None, None, None, l1, l0, 1, do_attn=False)
+    assert np.all(v.accept_len == want_a) and np.all(v.n_emit == want_emit)
+    assert np.all(s["n_ver"] == want_next)
+    assert np.all(s["ctx_len"] - ctx0 == want_growth)
+    mask = V - 1
+    if want_next == 0:   # "propose only": anchor followed by MASK rows
+        assert np.all(s["block_tok"][:, 1:] == mask)
+    else:                # next block = [bonus, fresh proposals, MASK...]
+        assert np.array_equal(s["block_tok"][:, 1:N], v.new_prop_tok)
+        assert np.all(s["block_tok"][:, N:] == mask)
+
+
+def tpf_closed_form(N, c):
+    # Eq. 3 with uniform per-position acceptance c
+    return sum([2.0] + [c ** k for k in range(1, N - 1)]) / (2.0 - c ** (N - 1))
+
+
+@pytest.mark.parametrize("N,c", [(2, 0.9), (4, 0.9), (8, 0.9), (4, 1.0), (4, 0.0), (3, 0.5)])
+def test_free_running_chain_matches_tpf_closed_form(N, c):
+    B, V, steps, Q = 300, 2, 240, 2 * N - 1
+    if c == 0.0:
+        p_law, q_law = np.array([1.0, 1e-30]), np.array([1e-30, 1.0])
+    else:
+        d = (1.0 - c) / 2
+        p_law, q_law = np.array([0.5 + d, 0.5 - d]), np.array([0.5 - d, 0.5 + d])
+    w = wl_tiny(B, N, V, 1234 + N)
+    s = tiny_state(B, N, V, ctx=16, pages_per_slot=(16 + steps * N + Q) // 16 + 3)
+    lp, lq = np.log(p_law).astype(np.float32), np.log(q_law).astype(np.float32)
+    prev = None
+    emitted = 0
+    for t in range(steps):
+        rows = np.arange(Q)[None, :]
+        clean = rows <= s["n_ver"][:, None]            # anchor + proposals give p, MASK rows give q
+        cur = np.where(clean[:, :, None], lp[None, None, :], lq[None, None, :]).astype(np.float32)
+        cur = np.ascontiguousarray(cur)
+        _, _, v, _ = oracle_step(w, s, None, None, None, cur, prev, t, do_attn=False)
+        assert np.all(s["slot_status"] == 0)
+        emitted += int(v.n_emit.sum())
+        prev = cur
+    tpf = emitted / (B * steps)
+    want = tpf_closed_form(N, c)
+    if c in (0.0, 1.0):
+        # limits stated with Eq. 3: TPF = N at p = 1 and 1 at p = 0 (first NP step costs a little)
+        assert abs(tpf - want) < N / steps + 1e-9
+    else:
+        assert abs(tpf - want) < 0.035, (tpf, want)
