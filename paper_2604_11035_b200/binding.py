@@ -1,0 +1,181 @@
+"""Thin ctypes binding of libisd.so: argument marshalling only.
+
+Every step of the ISD path runs inside the CUDA library; this module turns torch
+tensors into device pointers and forwards them.  There is no CPU fallback: if the
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libisd.so")
+
+ST_POOL_EXHAUSTED, ST_SLOT_CAPACITY, ST_BAD_TOKEN_ID = 1, 2, 4
+ST_BAD_PAGE_ID, ST_NONFINITE_LOGIT, ST_EMPTY_RESIDUAL = 8, 16, 32
+
+EXPORTS = ["isd_create", "isd_destroy", "isd_attn", "isd_verify", "isd_commit", "isd_step",
+           "isd_release", "isd_read_status", "isd_launch_count", "isd_strerror"]
+
+
+class IsdConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "batch", "stride", "n_q_heads", "n_kv_heads", "head_dim", "page_size", "vocab",
+        "max_pages_per_slot", "num_pages", "logits_dtype", "q_mode", "propose_mode", "mask_token_id",
+        "attn_impl")] + [("sm_scale", C.c_float), ("inv_temperature", C.c_float), ("tau", C.c_float),
+                         ("seed", C.c_uint64)]
+
+
+class IsdBatchState(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "ctx_len", "n_ver", "block_tok", "q_row0", "q_stats", "page_table", "free_stack", "free_top",
+        "active", "slot_status")]
+
+
+class IsdVerifyOut(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "accept", "alpha", "accept_len", "n_emit", "repl_tok", "out_tok", "new_prop_tok", "new_q_stats")]
+
+
+class IsdStepArgs(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "q", "k_new", "v_new", "k_pool", "v_pool", "attn_out", "attn_lse", "logits_cur", "q_prev_logits")] + \
+        [("out", IsdVerifyOut)]
+
+
+_lib = None
+
+
+def load():
+    """Load libisd.so (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2604_11035_b200.build` "
+                               "(there is no fallback path)")
+        lib = C.CDLL(LIB_PATH)
+        vp = C.c_void_p
+        lib.isd_create.argtypes = [C.POINTER(IsdConfig), C.POINTER(vp)]
+        lib.isd_destroy.argtypes = [vp]
+        lib.isd_attn.argtypes = [vp, C.POINTER(IsdBatchState)] + [vp] * 8
+        lib.isd_verify.argtypes = [vp, C.POINTER(IsdBatchState), vp, vp, C.c_uint64, C.POINTER(IsdVerifyOut), vp]
+        lib.isd_commit.argtypes = [vp, C.POINTER(IsdBatchState), C.POINTER(IsdVerifyOut), vp]
+        lib.isd_step.argtypes = [vp, C.POINTER(IsdBatchState), C.POINTER(IsdStepArgs), C.c_uint64, vp]
+        lib.isd_release.argtypes = [vp, C.POINTER(IsdBatchState), vp, C.c_int32, vp]
+        lib.isd_read_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        lib.isd_launch_count.argtypes = [vp]
+        lib.isd_launch_count.restype = C.c_int64
+        lib.isd_strerror.argtypes = [C.c_int]
+        lib.isd_strerror.restype = C.c_char_p
+        for n in EXPORTS[:8]:
+            getattr(lib, n).restype = C.c_int
+        _lib = lib
+    return _lib
+
+
+class IsdError(RuntimeError):
+    pass
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise IsdError(f"{what} failed: {load().isd_strerror(rc).decode()} ({rc})")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device, contiguous tensors only"
+    return t.data_ptr() if t.numel() > 0 else None
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def alloc_verify_out(B: int, N: int, device) -> dict:
+    NP = N - 1
+    i32 = dict(dtype=torch.int32, device=device)
+    return dict(
+        accept=torch.zeros(B, NP, dtype=torch.int8, device=device),
+        alpha=torch.zeros(B, NP, dtype=torch.float32, device=device),
+        accept_len=torch.zeros(B, **i32), n_emit=torch.zeros(B, **i32), repl_tok=torch.zeros(B, **i32),
+        out_tok=torch.zeros(B, N, **i32), new_prop_tok=torch.zeros(B, NP, **i32),
+        new_q_stats=torch.zeros(B, NP, 2, dtype=torch.float32, device=device))
+
+
+class Isd:
+    """One ISD context (scratch owner).  Methods mirror the C entry points by name."""
+
+    def __init__(self, *, batch, stride, n_q_heads, n_kv_heads, vocab, max_pages_per_slot, num_pages,
+                 logits_dtype, head_dim=128, page_size=16, q_mode=0, propose_mode=1, mask_token_id=None,
+                 attn_impl=0, sm_scale=0.0, inv_temperature=1.0, tau=0.0, seed=0):
+        if not torch.cuda.is_available():
+            raise IsdError("a CUDA device is required (there is no CPU path)")
+        self.lib = load()
+        ld = {"f32": 0, "bf16": 1, torch.float32: 0, torch.bfloat16: 1, 0: 0, 1: 1}[logits_dtype]
+        self.cfg = IsdConfig(batch, stride, n_q_heads, n_kv_heads, head_dim, page_size, vocab,
+                             max_pages_per_slot, num_pages, ld, q_mode, propose_mode,
+                             vocab - 1 if mask_token_id is None else mask_token_id, attn_impl,
+                             sm_scale, inv_temperature, tau, seed)
+        self.ctx = C.c_void_p()
+        _check(self.lib.isd_create(C.byref(self.cfg), C.byref(self.ctx)), "isd_create")
+        self.N, self.B = stride, batch
+
+    def close(self):
+        if getattr(self, "ctx", None) and self.ctx.value:
+            self.lib.isd_destroy(self.ctx)
+            self.ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- struct marshalling
+    @staticmethod
+    def state_struct(st: dict) -> IsdBatchState:
+        return IsdBatchState(*[_ptr(st[n]) for n, _ in IsdBatchState._fields_])
+
+    @staticmethod
+    def out_struct(out: dict) -> IsdVerifyOut:
+        return IsdVerifyOut(*[_ptr(out[n]) for n, _ in IsdVerifyOut._fields_])
+
+    # -- entry points
+    def isd_attn(self, st, q, k_new, v_new, k_pool, v_pool, attn_out, attn_lse=None):
+        s = self.state_struct(st)
+        _check(self.lib.isd_attn(self.ctx, C.byref(s), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool),
+                                 _ptr(v_pool), _ptr(attn_out), _ptr(attn_lse), _stream()), "isd_attn")
+
+    def isd_verify(self, st, logits_cur, q_prev_logits, step, out):
+        s, o = self.state_struct(st), self.out_struct(out)
+        _check(self.lib.isd_verify(self.ctx, C.byref(s), _ptr(logits_cur), _ptr(q_prev_logits), step,
+                                   C.byref(o), _stream()), "isd_verify")
+
+    def isd_commit(self, st, out):
+        s, o = self.state_struct(st), self.out_struct(out)
+        _check(self.lib.isd_commit(self.ctx, C.byref(s), C.byref(o), _stream()), "isd_commit")
+
+    def step_args(self, *, q, k_new, v_new, k_pool, v_pool, attn_out, attn_lse, logits_cur, q_prev_logits, out):
+        return IsdStepArgs(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(attn_out),
+                           _ptr(attn_lse), _ptr(logits_cur), _ptr(q_prev_logits), self.out_struct(out))
+
+    def isd_step(self, st, args: IsdStepArgs, step: int, st_struct: IsdBatchState | None = None):
+        s = st_struct if st_struct is not None else self.state_struct(st)
+        _check(self.lib.isd_step(self.ctx, C.byref(s), C.byref(args), step, _stream()), "isd_step")
+
+    def isd_release(self, st, slots):
+        s = self.state_struct(st)
+        _check(self.lib.isd_release(self.ctx, C.byref(s), _ptr(slots), slots.numel(), _stream()), "isd_release")
+
+    def isd_read_status(self) -> int:
+        v = C.c_uint32(0)
+        _check(self.lib.isd_read_status(self.ctx, C.byref(v), _stream()), "isd_read_status")
+        return int(v.value)
+
+    def isd_launch_count(self) -> int:
+        return int(self.lib.isd_launch_count(self.ctx))

@@ -1,0 +1,206 @@
+// Host side of the C ABI: configuration checks, scratch ownership, launch sequencing.
+#include <math.h>
+#include <new>
+#include <stdio.h>
+
+#include "isd_internal.cuh"
+
+int isd_launch_kv_append(isd_ctx* ctx, const isd_batch_state* st, const void* k_new, const void* v_new,
+                         void* k_pool, void* v_pool, cudaStream_t stream);
+int isd_attn_tc_create(isd_ctx* ctx);
+void isd_attn_tc_destroy(isd_ctx* ctx);
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+int dev_alloc(T** p, size_t n) {
+  *p = nullptr;
+  if (n == 0) n = 1;
+  return cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T)) == cudaSuccess ? ISD_OK : ISD_ERR_NO_MEMORY;
+}
+
+int check_state(const isd_batch_state* st) {
+  if (!st) return ISD_ERR_INVALID_ARG;
+  if (!st->ctx_len || !st->n_ver || !st->block_tok || !st->q_row0 || !st->page_table || !st->free_stack ||
+      !st->free_top || !st->active || !st->slot_status)
+    return ISD_ERR_INVALID_ARG;
+  return ISD_OK;
+}
+
+int check_out(const isd_ctx* ctx, const isd_verify_out* o) {
+  if (!o) return ISD_ERR_INVALID_ARG;
+  if (!o->accept_len || !o->n_emit || !o->repl_tok || !o->out_tok) return ISD_ERR_INVALID_ARG;
+  if (ctx->cfg.stride > 1 && (!o->accept || !o->alpha || !o->new_prop_tok || !o->new_q_stats))
+    return ISD_ERR_INVALID_ARG;
+  return ISD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int isd_create(const isd_config* cfg, isd_ctx** out) {
+  if (!cfg || !out) return ISD_ERR_INVALID_ARG;
+  *out = nullptr;
+  const isd_config& c = *cfg;
+  if (c.batch < 1 || c.batch > 65535 || c.stride < 1 || c.n_q_heads < 1 || c.n_kv_heads < 1 || c.vocab < 8 ||
+      c.max_pages_per_slot < 1 || c.num_pages < 1 || c.n_q_heads % c.n_kv_heads != 0)
+    return ISD_ERR_INVALID_ARG;
+  if (c.logits_dtype != ISD_LOGITS_F32 && c.logits_dtype != ISD_LOGITS_BF16) return ISD_ERR_INVALID_ARG;
+  if (c.q_mode < 0 || c.q_mode > 1 || c.propose_mode < 0 || c.propose_mode > 1) return ISD_ERR_INVALID_ARG;
+  if (c.attn_impl < 0 || c.attn_impl > 1) return ISD_ERR_INVALID_ARG;
+  if (!(c.inv_temperature > 0.f) || !(c.tau >= 0.f)) return ISD_ERR_INVALID_ARG;
+  const int Q = 2 * c.stride - 1;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  if (c.head_dim != ISD_HEAD_DIM || c.page_size != ISD_PAGE || Q > ISD_MAX_Q || G * Q > 128 || c.vocab % 8 != 0)
+    return ISD_ERR_UNSUPPORTED;
+
+  isd_ctx* ctx = new (std::nothrow) isd_ctx();
+  if (!ctx) return ISD_ERR_NO_MEMORY;
+  ctx->cfg = c;
+  ctx->Q = Q;
+  ctx->G = G;
+  ctx->sm_scale = c.sm_scale > 0.f ? c.sm_scale : 1.0f / sqrtf((float)c.head_dim);
+  ctx->launches = 0;
+  if (cudaGetDevice(&ctx->device) != cudaSuccess) { delete ctx; return ISD_ERR_CUDA; }
+  int sms = 0;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
+  ctx->num_sms = sms > 0 ? sms : ISD_NUM_SMS_DEFAULT;
+
+  // Enough CTAs to fill the machine at small batch; one CTA per row once rows are plentiful.
+  const int rows = c.batch * Q;
+  const int target = ctx->num_sms * 4;
+  int rs = (target + rows - 1) / rows;
+  const int max_by_len = (c.vocab + 8191) / 8192;  // keep at least 8k elements per CTA
+  rs = rs < 1 ? 1 : rs;
+  rs = rs > 16 ? 16 : rs;
+  rs = rs > max_by_len ? max_by_len : rs;
+  ctx->row_splits = rs;
+  int ps = (target + c.batch - 1) / c.batch;
+  ps = ps < 1 ? 1 : ps;
+  ps = ps > 16 ? 16 : ps;
+  ps = ps > max_by_len ? max_by_len : ps;
+  ctx->resid_splits = ps;
+
+  int rc = ISD_OK;
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->row_part, (size_t)rows * rs);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->resid_part, (size_t)c.batch * ps);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->row_ticket, c.batch);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->resid_ticket, c.batch);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->reject_pos, c.batch);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->lse_p_rej, c.batch);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->global_status, 1);
+  if (rc == ISD_OK) {
+    cudaMemset(ctx->row_ticket, 0, sizeof(int) * c.batch);
+    cudaMemset(ctx->resid_ticket, 0, sizeof(int) * c.batch);
+    cudaMemset(ctx->reject_pos, 0, sizeof(int) * c.batch);
+    cudaMemset(ctx->global_status, 0, sizeof(uint32_t));
+  }
+  if (rc == ISD_OK && c.attn_impl == 0) rc = isd_attn_tc_create(ctx);
+  if (rc == ISD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ISD_ERR_CUDA;
+  if (rc != ISD_OK) {
+    isd_destroy(ctx);
+    return rc;
+  }
+  *out = ctx;
+  return ISD_OK;
+}
+
+int isd_destroy(isd_ctx* ctx) {
+  if (!ctx) return ISD_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  isd_attn_tc_destroy(ctx);
+  cudaFree(ctx->row_part);
+  cudaFree(ctx->resid_part);
+  cudaFree(ctx->row_ticket);
+  cudaFree(ctx->resid_ticket);
+  cudaFree(ctx->reject_pos);
+  cudaFree(ctx->lse_p_rej);
+  cudaFree(ctx->global_status);
+  delete ctx;
+  return ISD_OK;
+}
+
+int isd_attn(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void* k_new, const void* v_new,
+             void* k_pool, void* v_pool, void* attn_out, float* attn_lse, void* cuda_stream) {
+  if (!ctx) return ISD_ERR_INVALID_ARG;
+  int rc = check_state(st);
+  if (rc != ISD_OK) return rc;
+  if (!q || !k_new || !v_new || !k_pool || !v_pool || !attn_out) return ISD_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(k_pool) || !aligned16(v_pool) ||
+      !aligned16(attn_out))
+    return ISD_ERR_ALIGNMENT;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (ctx->cfg.attn_impl == 1)
+    return isd_launch_attn_plain(ctx, st, q, k_new, v_new, k_pool, v_pool, attn_out, attn_lse, s);
+  rc = isd_launch_kv_append(ctx, st, k_new, v_new, k_pool, v_pool, s);
+  if (rc != ISD_OK) return rc;
+  return isd_launch_attn_tc(ctx, st, q, k_new, v_new, k_pool, v_pool, attn_out, attn_lse, s);
+}
+
+int isd_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur, const void* q_prev_logits,
+               uint64_t step, const isd_verify_out* out, void* cuda_stream) {
+  if (!ctx) return ISD_ERR_INVALID_ARG;
+  int rc = check_state(st);
+  if (rc != ISD_OK) return rc;
+  rc = check_out(ctx, out);
+  if (rc != ISD_OK) return rc;
+  if (!logits_cur || step > 0xFFFFFFFFull) return ISD_ERR_INVALID_ARG;
+  if (ctx->cfg.stride > 1 && !st->q_stats) return ISD_ERR_INVALID_ARG;
+  if (!aligned16(logits_cur) || (q_prev_logits && !aligned16(q_prev_logits))) return ISD_ERR_ALIGNMENT;
+  return isd_launch_verify(ctx, st, logits_cur, q_prev_logits, (uint32_t)step, out,
+                           reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int isd_commit(isd_ctx* ctx, isd_batch_state* st, const isd_verify_out* out, void* cuda_stream) {
+  if (!ctx) return ISD_ERR_INVALID_ARG;
+  int rc = check_state(st);
+  if (rc != ISD_OK) return rc;
+  rc = check_out(ctx, out);
+  if (rc != ISD_OK) return rc;
+  return isd_launch_commit(ctx, st, out, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int isd_step(isd_ctx* ctx, isd_batch_state* st, const isd_step_args* a, uint64_t step, void* cuda_stream) {
+  if (!ctx || !a) return ISD_ERR_INVALID_ARG;
+  int rc = isd_attn(ctx, st, a->q, a->k_new, a->v_new, a->k_pool, a->v_pool, a->attn_out, a->attn_lse, cuda_stream);
+  if (rc != ISD_OK) return rc;
+  rc = isd_verify(ctx, st, a->logits_cur, a->q_prev_logits, step, &a->out, cuda_stream);
+  if (rc != ISD_OK) return rc;
+  return isd_commit(ctx, st, &a->out, cuda_stream);
+}
+
+int isd_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t n, void* cuda_stream) {
+  if (!ctx || !slots || n < 0) return ISD_ERR_INVALID_ARG;
+  int rc = check_state(st);
+  if (rc != ISD_OK) return rc;
+  return isd_launch_release(ctx, st, slots, n, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int isd_read_status(isd_ctx* ctx, uint32_t* host_status, void* cuda_stream) {
+  if (!ctx || !host_status) return ISD_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(host_status, ctx->global_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return ISD_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->global_status, 0, sizeof(uint32_t), s) != cudaSuccess) return ISD_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return ISD_ERR_CUDA;
+  return ISD_OK;
+}
+
+int64_t isd_launch_count(const isd_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* isd_strerror(int code) {
+  switch (code) {
+    case ISD_OK: return "ok";
+    case ISD_ERR_INVALID_ARG: return "invalid argument";
+    case ISD_ERR_UNSUPPORTED: return "unsupported configuration (head_dim must be 128, page_size 16, (Hq/Hkv)*(2N-1) <= 128, vocab % 8 == 0)";
+    case ISD_ERR_CUDA: return "CUDA runtime error";
+    case ISD_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case ISD_ERR_NO_MEMORY: return "out of memory";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

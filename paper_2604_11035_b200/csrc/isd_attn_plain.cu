@@ -1,0 +1,171 @@
+// K/V append (batched scatter of the block rows into the slot's pages, Sec. 3.3 (2)) and a plain
+// CUDA-core attention kernel.  The plain kernel is the slow, obviously-correct device path
+// (attn_impl = 1): one CTA per (slot, block row, query head), fp32 FMA, online softmax per warp.
+// The tensor-core kernel in isd_attn_tc.cu is the product path.
+#include "isd_internal.cuh"
+
+namespace {
+
+struct AttnParams {
+  int B, Q, N, Hq, Hkv, G, max_pages, num_pages;
+  float sm_scale;
+  const int32_t* ctx_len;
+  const int32_t* n_ver;
+  const uint8_t* active;
+  const int32_t* page_table;
+  uint32_t* slot_status;
+  uint32_t* global_status;
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k_new;
+  const __nv_bfloat16* v_new;
+  __nv_bfloat16* k_pool;
+  __nv_bfloat16* v_pool;
+  __nv_bfloat16* out;
+  float* lse;
+};
+
+__device__ __forceinline__ int slot_q_len(const AttnParams& P, int b) {
+  if (!P.active[b]) return 0;
+  const int nv = P.n_ver[b];
+  if (nv < 0 || nv > P.N - 1) return 0;
+  return nv + P.N;
+}
+
+// one CTA per slot: validate the slot's page-table prefix, then scatter the block rows
+__global__ void __launch_bounds__(128) kv_append_kernel(const AttnParams P) {
+  const int b = blockIdx.x;
+  const int ql = slot_q_len(P, b);
+  if (ql == 0) return;
+  const int ctx = P.ctx_len[b];
+  const int pages = (ctx + ql + ISD_PAGE - 1) / ISD_PAGE;
+  __shared__ int sm_bad;
+  if (threadIdx.x == 0) sm_bad = 0;
+  __syncthreads();
+  if (ctx < 0 || pages > P.max_pages) {
+    if (threadIdx.x == 0) {
+      atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
+      atomicOr(P.global_status, ISD_ST_SLOT_CAPACITY);
+    }
+    return;
+  }
+  for (int pg = threadIdx.x; pg < pages; pg += blockDim.x) {
+    const int id = P.page_table[(size_t)b * P.max_pages + pg];
+    if (id < 0 || id >= P.num_pages) sm_bad = 1;
+  }
+  __syncthreads();
+  if (sm_bad) {
+    if (threadIdx.x == 0) {
+      atomicOr(&P.slot_status[b], ISD_ST_BAD_PAGE_ID);
+      atomicOr(P.global_status, ISD_ST_BAD_PAGE_ID);
+    }
+    return;
+  }
+  // each (row, kv head, K|V) is 256 bytes = 16 x 16-byte vectors
+  const int vecs = ql * P.Hkv * 2 * 16;
+  for (int i = threadIdx.x; i < vecs; i += blockDim.x) {
+    const int v16 = i & 15;
+    const int kv = (i >> 4) & 1;
+    const int g = (i >> 5) % P.Hkv;
+    const int r = (i >> 5) / P.Hkv;
+    const int pos = ctx + r;
+    const int page = P.page_table[(size_t)b * P.max_pages + pos / ISD_PAGE];
+    const size_t src = (((size_t)b * P.Q + r) * P.Hkv + g) * ISD_HEAD_DIM;
+    const size_t dst = (((size_t)page * P.Hkv + g) * ISD_PAGE + (pos % ISD_PAGE)) * ISD_HEAD_DIM;
+    const uint4* s = reinterpret_cast<const uint4*>((kv ? P.v_new : P.k_new) + src) + v16;
+    uint4* d = reinterpret_cast<uint4*>((kv ? P.v_pool : P.k_pool) + dst) + v16;
+    *d = *s;
+  }
+}
+
+__global__ void __launch_bounds__(128) attn_plain_kernel(const AttnParams P) {
+  const int h = blockIdx.x, r = blockIdx.y, b = blockIdx.z;
+  const int ql = slot_q_len(P, b);
+  if (r >= ql) return;
+  if (P.slot_status[b] & (ISD_ST_BAD_PAGE_ID | ISD_ST_SLOT_CAPACITY)) return;
+  const int ctx = P.ctx_len[b];
+  const int g = h / P.G;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nkeys = ctx + r + 1;
+
+  const __nv_bfloat16* qp = P.q + (((size_t)b * P.Q + r) * P.Hq + h) * ISD_HEAD_DIM + lane * 4;
+  float qv[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) qv[i] = __bfloat162float(qp[i]) * P.sm_scale;
+
+  float m = -INFINITY, l = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int j = warp; j < nkeys; j += 4) {
+    int page = P.page_table[(size_t)b * P.max_pages + j / ISD_PAGE];
+    page = min(max(page, 0), P.num_pages - 1);
+    const size_t off = (((size_t)page * P.Hkv + g) * ISD_PAGE + (j % ISD_PAGE)) * ISD_HEAD_DIM + lane * 4;
+    const uint2 kb = *reinterpret_cast<const uint2*>(P.k_pool + off);
+    float s = qv[0] * __uint_as_float(kb.x << 16) + qv[1] * __uint_as_float(kb.x & 0xFFFF0000u) +
+              qv[2] * __uint_as_float(kb.y << 16) + qv[3] * __uint_as_float(kb.y & 0xFFFF0000u);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const float mn = fmaxf(m, s);
+    const float corr = __expf(m - mn);
+    const float p = __expf(s - mn);
+    const uint2 vb = *reinterpret_cast<const uint2*>(P.v_pool + off);
+    l = l * corr + p;
+    acc[0] = acc[0] * corr + p * __uint_as_float(vb.x << 16);
+    acc[1] = acc[1] * corr + p * __uint_as_float(vb.x & 0xFFFF0000u);
+    acc[2] = acc[2] * corr + p * __uint_as_float(vb.y << 16);
+    acc[3] = acc[3] * corr + p * __uint_as_float(vb.y & 0xFFFF0000u);
+    m = mn;
+  }
+  __shared__ float sm_m[4], sm_l[4], sm_acc[4][ISD_HEAD_DIM];
+  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) sm_acc[warp][lane * 4 + i] = acc[i];
+  __syncthreads();
+  if (warp == 0) {
+    float M = fmaxf(fmaxf(sm_m[0], sm_m[1]), fmaxf(sm_m[2], sm_m[3]));
+    float L = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float c = (sm_m[w] == -INFINITY) ? 0.f : __expf(sm_m[w] - M);
+      L += sm_l[w] * c;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) o[i] += sm_acc[w][lane * 4 + i] * c;
+    }
+    __nv_bfloat16* op = P.out + (((size_t)b * P.Q + r) * P.Hq + h) * ISD_HEAD_DIM + lane * 4;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) op[i] = __float2bfloat16_rn(o[i] / L);
+    if (P.lse && lane == 0) P.lse[((size_t)b * P.Q + r) * P.Hq + h] = M + logf(L);
+  }
+}
+
+AttnParams make_params(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void* k_new,
+                       const void* v_new, void* k_pool, void* v_pool, void* out, float* lse) {
+  const isd_config& c = ctx->cfg;
+  AttnParams P;
+  P.B = c.batch; P.Q = ctx->Q; P.N = c.stride; P.Hq = c.n_q_heads; P.Hkv = c.n_kv_heads; P.G = ctx->G;
+  P.max_pages = c.max_pages_per_slot; P.num_pages = c.num_pages; P.sm_scale = ctx->sm_scale;
+  P.ctx_len = st->ctx_len; P.n_ver = st->n_ver; P.active = st->active; P.page_table = st->page_table;
+  P.slot_status = st->slot_status; P.global_status = ctx->global_status;
+  P.q = (const __nv_bfloat16*)q; P.k_new = (const __nv_bfloat16*)k_new; P.v_new = (const __nv_bfloat16*)v_new;
+  P.k_pool = (__nv_bfloat16*)k_pool; P.v_pool = (__nv_bfloat16*)v_pool; P.out = (__nv_bfloat16*)out; P.lse = lse;
+  return P;
+}
+
+}  // namespace
+
+int isd_launch_kv_append(isd_ctx* ctx, const isd_batch_state* st, const void* k_new, const void* v_new,
+                         void* k_pool, void* v_pool, cudaStream_t stream) {
+  AttnParams P = make_params(ctx, st, nullptr, k_new, v_new, k_pool, v_pool, nullptr, nullptr);
+  kv_append_kernel<<<ctx->cfg.batch, 128, 0, stream>>>(P);
+  ctx->launches++;
+  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}
+
+int isd_launch_attn_plain(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void* k_new,
+                          const void* v_new, void* k_pool, void* v_pool, void* out, float* lse,
+                          cudaStream_t stream) {
+  int rc = isd_launch_kv_append(ctx, st, k_new, v_new, k_pool, v_pool, stream);
+  if (rc != ISD_OK) return rc;
+  AttnParams P = make_params(ctx, st, q, k_new, v_new, k_pool, v_pool, out, lse);
+  const dim3 grid(ctx->cfg.n_q_heads, ctx->Q, ctx->cfg.batch);
+  attn_plain_kernel<<<grid, 128, 0, stream>>>(P);
+  ctx->launches++;
+  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}

@@ -1,0 +1,557 @@
+// isd_verify: vocab-wide softmax statistics, p/q introspective acceptance, residual resample /
+// bonus token and next proposals (Algorithm 1; Sec. 3.2; Sec. 3.3 (3) fused verification with
+// online softmax and Gumbel-max correction).
+//
+// Two launches, neither of which waits on anything:
+//   1. verify_rows_kernel  one CTA per (slot, block row, split): a single streaming pass over the
+//      logits row (16-byte loads) that yields, per role of the row,
+//        anchor rows (r < n_ver)        online-softmax (max, sum)            -> LSE_p
+//        final row   (r = n_ver)        Gumbel-max top-2                      -> bonus / free token
+//        MASK rows   (r > n_ver)        (max, sum) + argmax or Gumbel top-2   -> proposals, q_stats
+//      The last CTA of a slot to finish (atomic ticket, nobody waits) merges the partials, runs the
+//      sequential accept test and writes every output except a residual replacement.
+//   2. verify_resid_kernel  only for slots whose first rejection needs a replacement drawn from
+//      normalize(max(0, p - q)): a second pass over the rejecting anchor row and the proposal-law
+//      row; CTAs of slots without a rejection exit at once (the common accept path costs one pass).
+//
+// Gumbel noise is a pure function of (seed, step, slot, tag, position, vocab index), so any
+// reduction order gives the same sample.  Noise is evaluated exactly only for elements that can
+// still win: with E = -ln u' >= 1 - u', an element whose cheap bound cannot reach the running best
+// score is skipped.  The two best candidates of a row are re-judged in fp64 when their fp32 scores
+// are closer than ISD_TIE_EPS.
+#include "isd_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct VerifyParams {
+  int B, N, Q, V;
+  int logits_dtype, q_mode, propose_mode;
+  float inv_t, tau;
+  uint32_t seed_lo, seed_hi, step;
+  int row_splits, resid_splits;
+  const int32_t* n_ver;
+  const uint8_t* active;
+  const int32_t* block_tok;
+  const int32_t* q_row0;
+  const float* q_stats;
+  uint32_t* slot_status;
+  uint32_t* global_status;
+  const void* logits_cur;
+  const void* q_prev;
+  isd_verify_out out;
+  RowPartial* row_part;
+  ResidPartial* resid_part;
+  int* row_ticket;
+  int* resid_ticket;
+  int* reject_pos;
+  float* lse_p_rej;
+};
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Eight consecutive logits starting at element e (e % 8 == 0) as fp32.
+template <int DT>
+__device__ __forceinline__ void load8(const void* row, int e, float (&l)[8]) {
+  if (DT == ISD_LOGITS_BF16) {
+    const uint4 v = ld_stream_16B(reinterpret_cast<const uint16_t*>(row) + e);
+    l[0] = __uint_as_float(v.x << 16); l[1] = __uint_as_float(v.x & 0xFFFF0000u);
+    l[2] = __uint_as_float(v.y << 16); l[3] = __uint_as_float(v.y & 0xFFFF0000u);
+    l[4] = __uint_as_float(v.z << 16); l[5] = __uint_as_float(v.z & 0xFFFF0000u);
+    l[6] = __uint_as_float(v.w << 16); l[7] = __uint_as_float(v.w & 0xFFFF0000u);
+  } else {
+    const uint4 a = ld_stream_16B(reinterpret_cast<const float*>(row) + e);
+    const uint4 b = ld_stream_16B(reinterpret_cast<const float*>(row) + e + 4);
+    l[0] = __uint_as_float(a.x); l[1] = __uint_as_float(a.y); l[2] = __uint_as_float(a.z); l[3] = __uint_as_float(a.w);
+    l[4] = __uint_as_float(b.x); l[5] = __uint_as_float(b.y); l[6] = __uint_as_float(b.z); l[7] = __uint_as_float(b.w);
+  }
+}
+
+__device__ __forceinline__ void chunk_range(int V, int splits, int split, int& lo, int& hi) {
+  // chunks are multiples of 8 * kThreads elements so that every thread's vector stays aligned
+  const int per = ((V + splits - 1) / splits + 8 * kThreads - 1) / (8 * kThreads) * (8 * kThreads);
+  lo = split * per;
+  hi = min(V, lo + per);
+}
+
+// Block-wide merge helpers (8 warps) ------------------------------------------------------------
+__device__ __forceinline__ void block_merge_lse(float& m, float& s, float* sm_m, float* sm_s) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, off);
+    const float os = __shfl_xor_sync(0xffffffffu, s, off);
+    lse_merge(m, s, om, os);
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { sm_m[warp] = m; sm_s[warp] = s; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kThreads / 32; ++w) lse_merge(m, s, sm_m[w], sm_s[w]);
+  }
+  __syncthreads();
+}
+
+__device__ __forceinline__ void block_merge_top2(Top2& t, float* sm_s1, int* sm_i1, float* sm_s2, int* sm_i2) {
+  warp_merge_top2(t);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { sm_s1[warp] = t.s1; sm_i1[warp] = t.i1; sm_s2[warp] = t.s2; sm_i2[warp] = t.i2; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kThreads / 32; ++w) t.merge(sm_s1[w], sm_i1[w], sm_s2[w], sm_i2[w]);
+  }
+  __syncthreads();
+}
+
+// fp64 score of vocabulary index i of a Gumbel row: logit * invT + g
+__device__ double noisy_score_f64(const VerifyParams& P, const void* row, int i, uint32_t slot, uint32_t tagpos) {
+  const uint4 r = philox4x32_10((uint32_t)i >> 2, P.step, slot, tagpos, P.seed_lo, P.seed_hi);
+  const double l = (double)load_logit(row, P.logits_dtype, (size_t)i) * (double)P.inv_t;
+  return l + gumbel_f64(philox_word(r, i & 3));
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pass 1: row statistics + decision
+// ------------------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParams P) {
+  const int split = blockIdx.x, r = blockIdx.y, b = blockIdx.z;
+  if (!P.active[b]) return;
+  const int nv = P.n_ver[b];
+  if (nv < 0 || nv > P.N - 1) {
+    if (split == 0 && r == 0 && threadIdx.x == 0) {
+      atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
+      atomicOr(P.global_status, ISD_ST_SLOT_CAPACITY);
+    }
+    return;
+  }
+  const int q_len = nv + P.N;
+  if (r >= q_len) return;
+
+  __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
+  __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
+  __shared__ int sm_last;
+
+  const bool is_final = (r == nv);
+  const bool is_prop = (r > nv);
+  const bool noise = is_final || (is_prop && P.propose_mode == 0);
+  const bool raw_argmax = is_prop && P.propose_mode == 1;
+  const uint32_t tagpos = is_final ? ((ISD_TAG_FINAL << 16) | (uint32_t)(nv + 1))
+                                   : ((ISD_TAG_PROPOSE << 16) | (uint32_t)(r - nv));
+  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
+
+  int lo, hi;
+  chunk_range(P.V, P.row_splits, split, lo, hi);
+
+  const float scale2 = P.inv_t * kLog2e;  // logits -> log2 domain
+  float M2 = -INFINITY, S = 0.f;          // online softmax in the log2 domain
+  float raw_best = -INFINITY;
+  int raw_idx = -1;
+  Top2 top;
+  top.init();
+  float best_nat = -INFINITY;  // lower bound of the best noisy score seen by this warp
+  float K = INFINITY;          // skip an element iff (2^24 (1-u') floor) >= e_i * K
+  int iter = 0;
+
+  // uniform trip count per block (the warp shares its bound with shuffles inside the loop)
+  for (int base = lo; base < hi; base += kThreads * 8, ++iter) {
+    const int e = base + threadIdx.x * 8;
+    const bool valid = e < hi;
+    float l[8];
+    if (valid) {
+      load8<DT>(row, e, l);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) l[i] = -INFINITY;
+    }
+    float x2[8];
+    float vmax = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      x2[i] = l[i] * scale2;
+      vmax = fmaxf(vmax, x2[i]);
+    }
+    if (vmax > M2) {
+      S *= ex2f(M2 - vmax);  // M2 = -inf gives 0 * S(=0)
+      if (noise) K = 1.002f * 0x1p24f * ex2f(vmax - best_nat * kLog2e);
+      M2 = vmax;
+    }
+    float ex[8];
+    if (M2 > -INFINITY) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        ex[i] = ex2f(x2[i] - M2);
+        S += ex[i];
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ex[i] = 0.f;
+    }
+    if (raw_argmax) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (l[i] > raw_best) { raw_best = l[i]; raw_idx = e + i; }
+      }
+    }
+    if (noise) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (!valid) break;
+        const uint4 rnd = philox4x32_10((uint32_t)(e + 4 * h) >> 2, P.step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
+        const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float nf = (float)((~w[i]) >> 8);  // floor(2^24 (1 - u'))
+          // -ln u' >= 1 - u' >= nf 2^-24, so g_i <= -ln(nf 2^-24); the element cannot come within
+          // 2e-3 of the running best when nf >= ex[i] * K
+          if (!(nf >= ex[4 * h + i] * K) && l[4 * h + i] > -INFINITY) {
+            const float s = l[4 * h + i] * P.inv_t + gumbel_f32(w[i]);
+            top.push(s, e + 4 * h + i);
+            if (top.s1 > best_nat) {
+              best_nat = top.s1;
+              K = 1.002f * 0x1p24f * ex2f(M2 - best_nat * kLog2e);
+            }
+          }
+        }
+      }
+      if ((iter & 3) == 3) {  // share the bound inside the warp
+        float bn = best_nat;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) bn = fmaxf(bn, __shfl_xor_sync(0xffffffffu, bn, off));
+        if (bn > best_nat) {
+          best_nat = bn;
+          K = 1.002f * 0x1p24f * ex2f(M2 - best_nat * kLog2e);
+        }
+      }
+    }
+  }
+
+  // ---- block reduction -> partial
+  float m_nat = M2 * kLn2;  // back to natural-log units of the scaled logits
+  block_merge_lse(m_nat, S, sm_f0, sm_f1);
+  if (raw_argmax) {
+    top.init();
+    top.push(raw_best, raw_idx);
+  }
+  block_merge_top2(top, sm_f0, sm_i0, sm_f1, sm_i1);
+  if (threadIdx.x == 0) {
+    RowPartial rp;
+    rp.m = m_nat; rp.s = S; rp.best1 = top.s1; rp.idx1 = top.i1; rp.best2 = top.s2; rp.idx2 = top.i2;
+    P.row_part[((size_t)b * P.Q + r) * P.row_splits + split] = rp;
+    __threadfence();
+    const int arrived = atomicAdd(&P.row_ticket[b], 1);
+    sm_last = (arrived == q_len * P.row_splits - 1);
+  }
+  __syncthreads();
+  if (!sm_last) return;
+
+  // ---- decision phase: last CTA of the slot, warp 0 -------------------------------------------
+  if (threadIdx.x >= 32) return;
+  __threadfence();
+  const int lane = threadIdx.x;
+  __shared__ float d_lse[32];
+  __shared__ int d_tok[32];
+  __shared__ int d_bad[32];
+  if (lane == 0) P.row_ticket[b] = 0;  // ready for the next call
+  {
+    // lane = block row: merge its splits
+    float m = -INFINITY, s = 0.f;
+    Top2 t;
+    t.init();
+    int bad = 0;
+    int tok = -1;
+    if (lane < q_len) {
+      const volatile RowPartial* rp = P.row_part + ((size_t)b * P.Q + lane) * P.row_splits;
+      for (int k = 0; k < P.row_splits; ++k) {  // empty splits wrote neutral values
+        lse_merge(m, s, rp[k].m, rp[k].s);
+        t.merge(rp[k].best1, rp[k].idx1, rp[k].best2, rp[k].idx2);
+      }
+      // NaN anywhere poisons s; +inf logits give m = +inf
+      bad = (s != s) || (m == INFINITY) || (m != m);
+      const bool row_noise = (lane == nv) || (lane > nv && P.propose_mode == 0);
+      tok = t.i1;
+      if (row_noise && t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
+        const uint32_t tp = (lane == nv) ? ((ISD_TAG_FINAL << 16) | (uint32_t)(nv + 1))
+                                         : ((ISD_TAG_PROPOSE << 16) | (uint32_t)(lane - nv));
+        const char* rw = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + lane) * (size_t)P.V * elt;
+        const double a = noisy_score_f64(P, rw, t.i1, (uint32_t)b, tp);
+        const double c = noisy_score_f64(P, rw, t.i2, (uint32_t)b, tp);
+        if (c > a || (c == a && t.i2 < t.i1)) tok = t.i2;
+      }
+    }
+    d_lse[lane] = m + logf(s);
+    d_tok[lane] = tok;
+    d_bad[lane] = bad;
+  }
+  __syncwarp();
+
+  const int NP = P.N - 1;
+  // proposals + cached proposal-law statistics (lanes 1..N-1 = MASK row m)
+  if (lane >= 1 && lane <= NP) {
+    const int rr = nv + lane;
+    const int xh = d_tok[rr];
+    P.out.new_prop_tok[(size_t)b * NP + lane - 1] = xh;
+    const char* rw = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + rr) * (size_t)P.V * elt;
+    P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 0] = d_lse[rr];
+    P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 1] =
+        xh >= 0 ? load_logit(rw, P.logits_dtype, (size_t)xh) * P.inv_t : NAN;
+  }
+  if (lane != 0) return;
+
+  // sequential accept test (Algorithm 1, introspection loop)
+  uint32_t status = 0;
+  int a = nv, rej = 0;
+  for (int m = 1; m <= NP; ++m) status |= d_bad[nv + m] ? ISD_ST_NONFINITE_LOGIT : 0u;
+  for (int j = 1; j <= NP; ++j) {
+    P.out.accept[(size_t)b * NP + j - 1] = -1;
+    P.out.alpha[(size_t)b * NP + j - 1] = NAN;
+  }
+  for (int j = 1; j <= nv; ++j) {
+    const int x = P.block_tok[(size_t)b * P.Q + j];
+    if (x < 0 || x >= P.V) {
+      status |= ISD_ST_BAD_TOKEN_ID;
+      a = -1;
+      break;
+    }
+    if (d_bad[j - 1]) status |= ISD_ST_NONFINITE_LOGIT;
+    const char* rw = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + (j - 1)) * (size_t)P.V * elt;
+    const float logp = load_logit(rw, P.logits_dtype, (size_t)x) * P.inv_t - d_lse[j - 1];
+    float logq = 0.f;
+    if (P.q_mode == 0) {
+      const float* qs = P.q_stats + ((size_t)b * NP + j - 1) * 2;
+      logq = qs[1] - qs[0];
+    }
+    float al = (1.f + P.tau) * expf(logp - logq);
+    al = fminf(al, 1.f);
+    if (al != al) al = 0.f;
+    const uint4 rnd = philox4x32_10(0u, P.step, (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)j, P.seed_lo, P.seed_hi);
+    const float u = (float)(rnd.x >> 8) * 0x1p-24f;
+    P.out.alpha[(size_t)b * NP + j - 1] = al;
+    if (u < al) {
+      P.out.accept[(size_t)b * NP + j - 1] = 1;
+    } else {
+      P.out.accept[(size_t)b * NP + j - 1] = 0;
+      a = j - 1;
+      rej = j;
+      P.lse_p_rej[b] = d_lse[j - 1];
+      break;
+    }
+  }
+  if (a >= 0 && rej == 0 && d_bad[nv]) status |= ISD_ST_NONFINITE_LOGIT;
+  for (int j = 0; j < P.N; ++j) P.out.out_tok[(size_t)b * P.N + j] = -1;
+  if (a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL)) {
+    P.out.accept_len[b] = 0;
+    P.out.n_emit[b] = 0;
+    P.out.repl_tok[b] = -1;
+    P.reject_pos[b] = 0;
+    atomicOr(&P.slot_status[b], status);
+    atomicOr(P.global_status, status);
+    return;
+  }
+  P.out.accept_len[b] = a;
+  P.out.n_emit[b] = a + 1;
+  for (int j = 1; j <= a; ++j) P.out.out_tok[(size_t)b * P.N + j - 1] = P.block_tok[(size_t)b * P.Q + j];
+  if (rej == 0) {
+    const int y = d_tok[nv];
+    P.out.repl_tok[b] = y;
+    P.out.out_tok[(size_t)b * P.N + a] = y;
+  } else {
+    P.out.repl_tok[b] = -1;  // filled by the residual pass
+  }
+  P.reject_pos[b] = rej;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pass 2: residual resample for slots with a rejection
+// ------------------------------------------------------------------------------------------------
+__device__ double resid_score_f64(const VerifyParams& P, const void* prow, const void* qrow, int i, int x,
+                                  double lse_p, double lse_q, uint32_t slot, uint32_t tagpos) {
+  const double pi = exp((double)load_logit(prow, P.logits_dtype, (size_t)i) * (double)P.inv_t - lse_p);
+  double qi;
+  if (P.q_mode == 0) qi = exp((double)load_logit(qrow, P.logits_dtype, (size_t)i) * (double)P.inv_t - lse_q);
+  else qi = (i == x) ? 1.0 : 0.0;
+  const double rres = pi - qi;
+  if (!(rres > 0.0)) return -INFINITY;
+  const uint4 r = philox4x32_10((uint32_t)i >> 2, P.step, slot, tagpos, P.seed_lo, P.seed_hi);
+  return log(rres) + gumbel_f64(philox_word(r, i & 3));
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) verify_resid_kernel(const VerifyParams P) {
+  const int split = blockIdx.x, b = blockIdx.y;
+  if (!P.active[b]) return;
+  const int j = P.reject_pos[b];
+  if (j <= 0) return;
+
+  __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
+  __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
+  __shared__ int sm_last;
+
+  const int NP = P.N - 1;
+  const int x = P.block_tok[(size_t)b * P.Q + j];
+  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  const char* prow = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + (j - 1)) * (size_t)P.V * elt;
+  const char* qrow = P.q_mode == 0
+      ? reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + (P.q_row0[b] + j - 1)) * (size_t)P.V * elt
+      : prow;
+  const float lse_p = P.lse_p_rej[b];
+  const float lse_q = P.q_mode == 0 ? P.q_stats[((size_t)b * NP + j - 1) * 2 + 0] : 0.f;
+  const uint32_t tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)j;
+
+  int lo, hi;
+  chunk_range(P.V, P.resid_splits, split, lo, hi);
+  Top2 top;
+  top.init();
+  float best_nat = -INFINITY;
+  // bound: ln r_i <= ln p_i = lp_i - lse_p; skip iff nf >= 1.002 2^24 exp(lp_i - lse_p - best)
+  const float scale2 = P.inv_t * kLog2e;
+  float K2 = INFINITY;  // log2 offset: skip iff nf >= ex2(x2 + K2)
+  int iter = 0;
+  for (int base = lo; base < hi; base += kThreads * 8, ++iter) {
+    const int e = base + threadIdx.x * 8;
+    const bool valid = e < hi;
+    float lp[8], lq[8];
+    if (valid) {
+      load8<DT>(prow, e, lp);
+      if (P.q_mode == 0) load8<DT>(qrow, e, lq);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (!valid) break;
+      const uint4 rnd = philox4x32_10((uint32_t)(e + 4 * h) >> 2, P.step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
+      const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int idx = e + 4 * h + i;
+        const float nf = (float)((~w[i]) >> 8);
+        const float bound = ex2f(lp[4 * h + i] * scale2 + K2);  // K2 = +inf -> inf (never skip)
+        if (!(nf >= bound)) {
+          const float pi = expf(lp[4 * h + i] * P.inv_t - lse_p);
+          const float qi = P.q_mode == 0 ? expf(lq[4 * h + i] * P.inv_t - lse_q) : (idx == x ? 1.f : 0.f);
+          const float rr = pi - qi;
+          if (rr > 0.f) {
+            const float s = logf(rr) + gumbel_f32(w[i]);
+            top.push(s, idx);
+            if (top.s1 > best_nat) {
+              best_nat = top.s1;
+              K2 = 24.f + 0.0028853901f - (lse_p + best_nat) * kLog2e;  // log2(1.002) = 0.00288539
+            }
+          }
+        }
+      }
+    }
+    if ((iter & 3) == 3) {
+      float bn = best_nat;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) bn = fmaxf(bn, __shfl_xor_sync(0xffffffffu, bn, off));
+      if (bn > best_nat) {
+        best_nat = bn;
+        K2 = 24.f + 0.0028853901f - (lse_p + best_nat) * kLog2e;
+      }
+    }
+  }
+  block_merge_top2(top, sm_f0, sm_i0, sm_f1, sm_i1);
+  if (threadIdx.x == 0) {
+    ResidPartial rp;
+    rp.best1 = top.s1; rp.idx1 = top.i1; rp.best2 = top.s2; rp.idx2 = top.i2;
+    P.resid_part[(size_t)b * P.resid_splits + split] = rp;
+    __threadfence();
+    const int arrived = atomicAdd(&P.resid_ticket[b], 1);
+    sm_last = (arrived == P.resid_splits - 1);
+  }
+  __syncthreads();
+  if (!sm_last) return;
+  __threadfence();
+
+  // last CTA of the slot: merge, fp64 tie-break, write the replacement
+  __shared__ int sm_tok;
+  if (threadIdx.x == 0) {
+    P.resid_ticket[b] = 0;
+    Top2 t;
+    t.init();
+    for (int k = 0; k < P.resid_splits; ++k) {
+      const volatile ResidPartial* rp = P.resid_part + (size_t)b * P.resid_splits + k;
+      t.merge(rp->best1, rp->idx1, rp->best2, rp->idx2);
+    }
+    int y = t.i1;
+    if (t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
+      const double a = resid_score_f64(P, prow, qrow, t.i1, x, lse_p, lse_q, (uint32_t)b, tagpos);
+      const double c = resid_score_f64(P, prow, qrow, t.i2, x, lse_p, lse_q, (uint32_t)b, tagpos);
+      if (c > a || (c == a && t.i2 < t.i1)) y = t.i2;
+    }
+    sm_tok = y;
+  }
+  __syncthreads();
+  int y = sm_tok;
+  if (y < 0) {
+    // Residual empty in fp32 (p and q numerically equal): fall back to a sample of p with the same
+    // noise.  Rare; done by this one CTA over the whole row.
+    Top2 t;
+    t.init();
+    for (int e = threadIdx.x * 8; e < P.V; e += kThreads * 8) {
+      float lp[8];
+      load8<DT>(prow, e, lp);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint4 rnd = philox4x32_10((uint32_t)(e + 4 * h) >> 2, P.step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
+        const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (lp[4 * h + i] > -INFINITY) t.push(lp[4 * h + i] * P.inv_t + gumbel_f32(w[i]), e + 4 * h + i);
+      }
+    }
+    block_merge_top2(t, sm_f0, sm_i0, sm_f1, sm_i1);
+    if (threadIdx.x == 0) {
+      y = t.i1;
+      if (t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
+        const double a = noisy_score_f64(P, prow, t.i1, (uint32_t)b, tagpos);
+        const double c = noisy_score_f64(P, prow, t.i2, (uint32_t)b, tagpos);
+        if (c > a || (c == a && t.i2 < t.i1)) y = t.i2;
+      }
+      atomicOr(&P.slot_status[b], ISD_ST_EMPTY_RESIDUAL);
+      atomicOr(P.global_status, ISD_ST_EMPTY_RESIDUAL);
+    }
+  }
+  if (threadIdx.x == 0) {
+    P.out.repl_tok[b] = y;
+    P.out.out_tok[(size_t)b * P.N + (j - 1)] = y;
+  }
+}
+
+}  // namespace
+
+int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
+                      const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
+                      cudaStream_t stream) {
+  const isd_config& c = ctx->cfg;
+  VerifyParams P;
+  P.B = c.batch; P.N = c.stride; P.Q = ctx->Q; P.V = c.vocab;
+  P.logits_dtype = c.logits_dtype; P.q_mode = c.q_mode; P.propose_mode = c.propose_mode;
+  P.inv_t = c.inv_temperature; P.tau = c.tau;
+  P.seed_lo = (uint32_t)c.seed; P.seed_hi = (uint32_t)(c.seed >> 32); P.step = step;
+  P.row_splits = ctx->row_splits; P.resid_splits = ctx->resid_splits;
+  P.n_ver = st->n_ver; P.active = st->active; P.block_tok = st->block_tok; P.q_row0 = st->q_row0;
+  P.q_stats = st->q_stats; P.slot_status = st->slot_status; P.global_status = ctx->global_status;
+  P.logits_cur = logits_cur; P.q_prev = q_prev_logits; P.out = *out;
+  P.row_part = ctx->row_part; P.resid_part = ctx->resid_part; P.row_ticket = ctx->row_ticket;
+  P.resid_ticket = ctx->resid_ticket; P.reject_pos = ctx->reject_pos; P.lse_p_rej = ctx->lse_p_rej;
+
+  const dim3 grid1(ctx->row_splits, ctx->Q, c.batch);
+  if (c.logits_dtype == ISD_LOGITS_BF16) verify_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads, 0, stream>>>(P);
+  else verify_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads, 0, stream>>>(P);
+  ctx->launches++;
+  if (c.stride > 1 && (c.q_mode == 1 || q_prev_logits != nullptr)) {
+    const dim3 grid2(ctx->resid_splits, c.batch);
+    if (c.logits_dtype == ISD_LOGITS_BF16) verify_resid_kernel<ISD_LOGITS_BF16><<<grid2, kThreads, 0, stream>>>(P);
+    else verify_resid_kernel<ISD_LOGITS_F32><<<grid2, kThreads, 0, stream>>>(P);
+    ctx->launches++;
+  }
+  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}

@@ -1,0 +1,194 @@
+"""GPU-vs-oracle parity harness for chained ISD steps (used by the GPU tests and the smoke check).
+
+Both sides run free from the same seeded inputs.  Every input the oracle sees comes from the
+seeded generators or from the oracle's own state; nothing computed by the CUDA path is ever fed to
+the oracle.  After each step the GPU's outputs and state are compared with the oracle's:
+
+  bit-exact   accept flags, accept_len, n_emit, repl_tok, out_tok, new_prop_tok, ctx_len, n_ver,
+              block_tok, q_row0, page-table prefix, free_top, free stack, slot_status, KV pool rows
+  <= 2e-2     attention output / LSE (max-abs), alpha, cached proposal-law statistics
+
+The one exemption: a position whose acceptance probability lies within 1e-4 of its uniform draw may
+flip; such slot-steps are counted, their downstream fields skipped, and the GPU state is then
+overwritten with the oracle's so that the chain stays comparable.
+"""
+from __future__ import annotations
+
+import os
+import time
+
+import numpy as np
+import torch
+
+import oracle
+import paper_2604_11035_b200 as isd_pkg
+from paper_2604_11035_b200 import workloads as wl
+from helpers import STATE_KEYS, bits16, logits_np, oracle_step, state_to_np
+
+TOL = 2e-2
+EXEMPT = 1e-4
+
+
+def _bf16_to_f64(bits):
+    return torch.from_numpy(bits.astype(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+
+
+def run_chain_parity(w: wl.Workload, steps: int, device="cuda:0", attn_slots=None, attn_impl=None,
+                     oracle_threads=None, check_pools=True, verbose=False, **isd_kw):
+    dev = torch.device(device)
+    N, B, Q, NP = w.stride, w.batch, w.Q, w.stride - 1
+    if attn_impl is None:
+        attn_impl = int(os.environ.get("ISD_TEST_ATTN_IMPL", "0"))
+    oracle.set_threads(oracle_threads or oracle.max_threads())
+    st = wl.make_state(w, dev)
+    s = state_to_np(st)                      # oracle state (inputs come from the generator)
+    eng = isd_pkg.isd_for_workload(w, st, attn_impl=attn_impl, **isd_kw)
+    out = isd_pkg.alloc_verify_out(B, N, dev)
+    attn_out = torch.zeros(B, Q, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
+    attn_lse = torch.zeros(B, Q, w.n_q_heads, dtype=torch.float32, device=dev)
+    attn_sel = np.arange(B) if attn_slots is None else np.asarray(attn_slots)
+    attn_active = np.zeros(B, np.uint8)
+    attn_active[attn_sel] = 1
+
+    rep = dict(workload=w.name, steps=steps, mismatches=0, exempt_flips=0, near_threshold=0,
+               fragile_samples=0, attn_max_abs_err=0.0, lse_max_abs_err=0.0, alpha_max_abs_err=0.0,
+               qstats_max_abs_err=0.0, positions=0, emitted=0, rejections=0, details=[],
+               oracle_seconds=0.0)
+
+    def bad(msg):
+        rep["mismatches"] += 1
+        if len(rep["details"]) < 20:
+            rep["details"].append(msg)
+
+    prev_dev = prev_np = None
+    for t in range(steps):
+        q, k, v = wl.make_qkv(w, t, dev)
+        ctx_dev = torch.from_numpy(s["ctx_len"]).to(dev)          # oracle's lengths drive the generator
+        lg = wl.make_logits(w, t, ctx_dev)
+        lg_np = logits_np(lg)
+        q_np, k_np, v_np = bits16(q), bits16(k), bits16(v)
+        n_ver_before = s["n_ver"].copy()
+        ctx_before = s["ctx_len"].copy()
+
+        # ---- CUDA path: one isd_step through the C ABI
+        args = eng.step_args(q=q, k_new=k, v_new=v, k_pool=st["k_pool"], v_pool=st["v_pool"],
+                             attn_out=attn_out, attn_lse=attn_lse, logits_cur=lg, q_prev_logits=prev_dev, out=out)
+        eng.isd_step(st, args, t)
+        torch.cuda.synchronize()
+
+        # ---- oracle: attention on the selected slots, verify + commit on all slots
+        t0 = time.time()
+        save_active = s["active"]
+        s["active"] = (save_active & attn_active).astype(np.uint8)
+        q_len = np.where(s["active"] != 0, s["n_ver"] + N, 0).astype(np.int32)
+        o_attn, o_lse = oracle.attn(
+            Hq=w.n_q_heads, Hkv=w.n_kv_heads, D=w.head_dim, page_size=wl.PAGE, num_pages=s["num_pages"],
+            sm_scale=1.0 / np.sqrt(w.head_dim), ctx_len=s["ctx_len"], q_len=q_len, active=s["active"],
+            page_table=s["page_table"], q=q_np, k_new=k_np, v_new=v_np, k_pool=s["k_pool"], v_pool=s["v_pool"],
+            slot_status=s["slot_status"])
+        s["active"] = save_active
+        _, _, vr, q_len_all = oracle_step(w, s, None, None, None, lg_np, prev_np, t, do_attn=False)
+        rep["oracle_seconds"] += time.time() - t0
+
+        # ---- compare attention
+        g_out = attn_out.to(torch.float64).cpu().numpy()
+        g_lse = attn_lse.to(torch.float64).cpu().numpy()
+        for b in attn_sel:
+            ql = int(q_len[b])
+            if ql == 0:
+                continue
+            e = np.abs(g_out[b, :ql] - o_attn[b, :ql]).max()
+            rep["attn_max_abs_err"] = max(rep["attn_max_abs_err"], float(e))
+            rep["lse_max_abs_err"] = max(rep["lse_max_abs_err"], float(np.abs(g_lse[b, :ql] - o_lse[b, :ql]).max()))
+            if not (e < TOL):
+                bad(f"step {t} slot {b}: attention max-abs err {e:.3e}")
+        # ---- compare KV rows: every logical position below the new committed length
+        if check_pools:
+            gk, gv = bits16(st["k_pool"]), bits16(st["v_pool"])
+            for b in attn_sel:
+                n = int(ctx_before[b] + q_len[b])
+                pages = s["page_table"][b, :(n + 15) // 16]
+                if not (np.array_equal(gk[pages], s["k_pool"][pages]) and np.array_equal(gv[pages], s["v_pool"][pages])):
+                    bad(f"step {t} slot {b}: KV pages differ after append")
+
+        # ---- compare verify outputs
+        g = {kk: vv.cpu().numpy() for kk, vv in out.items()}
+        gst = {kk: st[kk].cpu().numpy() for kk in STATE_KEYS}
+        gst["slot_status"] = gst["slot_status"].view(np.uint32)
+        resync = False
+        for b in range(B):
+            if not s["active"][b]:
+                continue
+            if (s["slot_status"][b] & ~oracle.ST_EMPTY_RESIDUAL) or (gst["slot_status"][b] & ~oracle.ST_EMPTY_RESIDUAL):
+                if s["slot_status"][b] != gst["slot_status"][b]:
+                    bad(f"step {t} slot {b}: status {gst['slot_status'][b]} vs oracle {s['slot_status'][b]}")
+                continue
+            nv = int(n_ver_before[b])
+            rep["positions"] += nv + N
+            evaluated = vr.accept[b] >= 0
+            near = evaluated & (np.abs(vr.alpha[b] - vr.u[b]) < EXEMPT)
+            rep["near_threshold"] += int(near.sum())
+            acc_equal = np.array_equal(g["accept"][b], vr.accept[b])
+            if not acc_equal:
+                first = int(np.argmax(g["accept"][b] != vr.accept[b]))
+                if near[first]:
+                    rep["exempt_flips"] += 1
+                    resync = True
+                    continue                     # downstream fields of this slot-step are skipped
+                bad(f"step {t} slot {b}: accept {g['accept'][b]} vs oracle {vr.accept[b]} "
+                    f"(alpha {vr.alpha[b]}, u {vr.u[b]})")
+                resync = True
+                continue
+            ev = np.where(evaluated)[0]
+            if len(ev):
+                rep["alpha_max_abs_err"] = max(rep["alpha_max_abs_err"],
+                                               float(np.abs(g["alpha"][b][ev] - vr.alpha[b][ev]).max()))
+            rep["emitted"] += int(vr.n_emit[b])
+            rep["rejections"] += int(vr.accept_len[b] < nv)
+            if vr.final_margin[b] < 1e-4:
+                rep["fragile_samples"] += 1
+            if NP:
+                rep["fragile_samples"] += int((vr.prop_margin[b] < 1e-4).sum()) if w.propose_mode == 0 else 0
+            for name in ("accept_len", "n_emit", "repl_tok", "out_tok", "new_prop_tok"):
+                if not np.array_equal(g[name][b], getattr(vr, name)[b]):
+                    bad(f"step {t} slot {b}: {name} {g[name][b]} vs oracle {getattr(vr, name)[b]} "
+                        f"(final margin {vr.final_margin[b]:.3e})")
+                    resync = True
+            if NP:
+                dq = np.abs(g["new_q_stats"][b] - vr.new_q_stats[b]).max()
+                rep["qstats_max_abs_err"] = max(rep["qstats_max_abs_err"], float(dq))
+                if not (dq < TOL):
+                    bad(f"step {t} slot {b}: q_stats err {dq:.3e}")
+            # ---- committed state
+            for name in ("ctx_len", "n_ver", "q_row0"):
+                if gst[name][b] != s[name][b]:
+                    bad(f"step {t} slot {b}: state {name} {gst[name][b]} vs oracle {s[name][b]}")
+                    resync = True
+            if not np.array_equal(gst["block_tok"][b], s["block_tok"][b]):
+                bad(f"step {t} slot {b}: block_tok {gst['block_tok'][b]} vs {s['block_tok'][b]}")
+                resync = True
+            own = (int(s["ctx_len"][b]) + Q + 15) // 16
+            if not np.array_equal(gst["page_table"][b, :own], s["page_table"][b, :own]):
+                bad(f"step {t} slot {b}: page table prefix differs")
+                resync = True
+        if not resync:
+            top = int(s["free_top"][0])
+            if gst["free_top"][0] != top or not np.array_equal(gst["free_stack"][:top], s["free_stack"][:top]):
+                bad(f"step {t}: free stack differs (top {gst['free_top'][0]} vs {top})")
+        if resync:
+            # GPU inputs may come from the oracle (never the reverse): continue from the oracle's state
+            for kk in STATE_KEYS:
+                a = s[kk]
+                if kk == "slot_status":
+                    a = a.view(np.int32)
+                if kk == "q_stats":
+                    a = a.astype(np.float32)
+                st[kk].copy_(torch.from_numpy(np.ascontiguousarray(a)).to(dev))
+        prev_dev, prev_np = lg, lg_np
+        if verbose:
+            print(f"step {t}: mism {rep['mismatches']} exempt {rep['exempt_flips']} attn_err {rep['attn_max_abs_err']:.2e}")
+    rep["global_status"] = eng.isd_read_status()
+    rep["gpu_launches"] = eng.isd_launch_count()
+    rep["tpf"] = rep["emitted"] / max(1, B * steps)
+    eng.close()
+    return rep

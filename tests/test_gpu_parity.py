@@ -1,0 +1,229 @@
+"""CUDA path vs fp64 oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2604_11035_b200 as isd_pkg
+from helpers import STATE_KEYS, bits16, logits_np, oracle_step, state_to_np
+from paper_2604_11035_b200 import workloads as wl
+from paper_2604_11035_b200.workloads import Workload
+from parity import run_chain_parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def assert_clean(rep, allow_exempt=2):
+    assert rep["mismatches"] == 0, rep["details"]
+    assert rep["exempt_flips"] <= allow_exempt, rep
+    assert rep["attn_max_abs_err"] < 2e-2 and rep["lse_max_abs_err"] < 2e-2, rep
+    assert rep["alpha_max_abs_err"] < 2e-2 and rep["qstats_max_abs_err"] < 2e-2, rep
+    assert rep["gpu_launches"] > 0
+
+
+@pytest.mark.parametrize("attn_impl", [0, 1])
+def test_config0_tiny(attn_impl):
+    rep = run_chain_parity(wl.config(0), steps=4, device=DEV, attn_impl=attn_impl)
+    assert_clean(rep)
+    assert rep["positions"] > 0 and rep["emitted"] >= 4
+
+
+@pytest.mark.parametrize("attn_impl", [0, 1])
+@pytest.mark.parametrize("dtype,propose_mode,q_mode,N", [
+    ("f32", 0, 0, 4), ("bf16", 0, 0, 4), ("bf16", 1, 0, 8), ("bf16", 1, 1, 3), ("f32", 0, 0, 2), ("bf16", 0, 0, 16)])
+def test_ragged_multi_tile_chain(attn_impl, dtype, propose_mode, q_mode, N):
+    # several 128-key tiles per slot, ragged tails, mixed P / NP steps, pages shuffled
+    w = Workload("ragged", batch=5, stride=N, n_q_heads=32, n_kv_heads=8, vocab=4096 + 8 * 37, ctx_min=3,
+                 ctx_max=700, logits_dtype=dtype, logit_sigma=2.0, peaked_frac=0.6, steps=8,
+                 propose_mode=propose_mode, q_mode=q_mode, seed=40 + N)
+    rep = run_chain_parity(w, steps=8, device=DEV, attn_impl=attn_impl)
+    assert_clean(rep)
+    assert rep["rejections"] > 0 and rep["tpf"] > 1.0
+
+
+def test_temperature_and_relaxed_acceptance():
+    w = Workload("temp", batch=6, stride=4, n_q_heads=8, n_kv_heads=2, vocab=2048, ctx_min=20, ctx_max=200,
+                 logits_dtype="f32", logit_sigma=2.0, peaked_frac=0.5, steps=6, propose_mode=0, seed=77)
+    st_kw = dict(inv_temperature=0.7, tau=0.5)
+    # the oracle helper takes the same scalars
+    import parity
+    orig = parity.oracle_step
+    parity.oracle_step = lambda *a, **k: orig(*a, inv_temperature=0.7, tau=0.5, **k)
+    try:
+        rep = run_chain_parity(w, steps=6, device=DEV, **st_kw)
+    finally:
+        parity.oracle_step = orig
+    assert_clean(rep)
+
+
+def test_config1_moderate_full():
+    rep = run_chain_parity(wl.config(1), steps=2, device=DEV, attn_slots=[0, 7, 31])
+    assert_clean(rep)
+    assert rep["rejections"] > 0
+
+
+def test_config2_stationary_batch_full_size_sampled_attention():
+    # full launch configuration of the benchmark; verify/commit compared on all 256 slots,
+    # attention on sampled slots (the oracle needs ~1 s per slot)
+    w = wl.config(2, steps=4)
+    rep = run_chain_parity(w, steps=3, device=DEV, attn_slots=[0, 100, 255], check_pools=True)
+    assert_clean(rep)
+    assert rep["positions"] >= 256 * 8
+
+
+def test_config3_long_context_sampled():
+    rep = run_chain_parity(wl.config(3), steps=2, device=DEV, attn_slots=[3])
+    assert_clean(rep)
+
+
+def _fresh(w, **kw):
+    import os
+    kw.setdefault("attn_impl", int(os.environ.get("ISD_TEST_ATTN_IMPL", "0")))
+    st = wl.make_state(w, DEV)
+    eng = isd_pkg.isd_for_workload(w, st, **kw)
+    out = isd_pkg.alloc_verify_out(w.batch, w.stride, DEV)
+    return st, eng, out
+
+
+def _step(w, st, eng, out, t, prev, logits=None):
+    q, k, v = wl.make_qkv(w, t, DEV)
+    lg = wl.make_logits(w, t, st["ctx_len"]) if logits is None else logits
+    ao = torch.zeros(w.batch, w.Q, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=DEV)
+    args = eng.step_args(q=q, k_new=k, v_new=v, k_pool=st["k_pool"], v_pool=st["v_pool"], attn_out=ao,
+                         attn_lse=None, logits_cur=lg, q_prev_logits=prev, out=out)
+    eng.isd_step(st, args, t)
+    torch.cuda.synchronize()
+    return lg, ao
+
+
+def test_run_to_run_determinism():
+    w = Workload("det", batch=7, stride=4, n_q_heads=32, n_kv_heads=8, vocab=8192, ctx_min=50, ctx_max=900,
+                 logits_dtype="bf16", peaked_frac=0.5, steps=4, propose_mode=0, seed=5)
+    snaps = []
+    for _ in range(2):
+        st, eng, out = _fresh(w)
+        prev = None
+        acc = []
+        for t in range(4):
+            prev, ao = _step(w, st, eng, out, t, prev)
+            acc.append([x.clone() for x in out.values()] + [ao.clone()] + [st[k].clone() for k in STATE_KEYS])
+        snaps.append(acc)
+        eng.close()
+    for a, b in zip(snaps[0], snaps[1]):
+        for x, y in zip(a, b):
+            assert torch.equal(x.view(torch.uint8) if x.dtype.is_floating_point else x,
+                               y.view(torch.uint8) if y.dtype.is_floating_point else y)
+
+
+def test_inactive_slots_and_empty_batch():
+    w = Workload("inact", batch=4, stride=3, n_q_heads=8, n_kv_heads=2, vocab=1024, ctx_min=10, ctx_max=90,
+                 logits_dtype="f32", steps=3, propose_mode=0, seed=8)
+    st, eng, out = _fresh(w)
+    st["active"][1] = 0
+    before = {k: st[k].clone() for k in STATE_KEYS}
+    kp = st["k_pool"].clone()
+    _step(w, st, eng, out, 0, None)
+    assert st["ctx_len"][1] == before["ctx_len"][1] and torch.equal(st["block_tok"][1], before["block_tok"][1])
+    assert (st["ctx_len"][[0, 2, 3]] == before["ctx_len"][[0, 2, 3]] + 1).all()
+    st["active"][:] = 0
+    snap = {k: st[k].clone() for k in STATE_KEYS}
+    kp = st["k_pool"].clone()
+    _step(w, st, eng, out, 1, None)
+    for k in STATE_KEYS:
+        assert torch.equal(st[k], snap[k])
+    assert torch.equal(st["k_pool"], kp)
+    assert eng.isd_read_status() == 0
+    eng.close()
+
+
+def test_faults_set_status_bits_and_freeze_the_slot():
+    w = Workload("fault", batch=5, stride=3, n_q_heads=8, n_kv_heads=2, vocab=1024, ctx_min=30, ctx_max=60,
+                 logits_dtype="f32", steps=4, propose_mode=0, seed=9)
+    st, eng, out = _fresh(w)
+    s_np = state_to_np(st)                              # oracle starts from the same generated state
+    lg0 = wl.make_logits(w, 0, torch.from_numpy(s_np["ctx_len"]).to(DEV))
+    prev, _ = _step(w, st, eng, out, 0, None, logits=lg0)   # bootstrap: everyone proposes
+    q0, k0, v0 = wl.make_qkv(w, 0, DEV)
+    oracle_step(w, s_np, bits16(q0), bits16(k0), bits16(v0), logits_np(lg0), None, 0)
+    assert (st["n_ver"] == 2).all() and np.all(s_np["n_ver"] == 2)
+    lg = wl.make_logits(w, 1, torch.from_numpy(s_np["ctx_len"]).to(DEV))
+    lg[1, 0, 5] = float("nan")                          # non-finite anchor row
+    st["block_tok"][2, 1] = w.vocab + 3                 # proposal id out of range
+    st["page_table"][3, 0] = st["num_pages"] + 9        # page id out of range
+    s_np["block_tok"][2, 1] = w.vocab + 3
+    s_np["page_table"][3, 0] = st["num_pages"] + 9
+    before = {k: st[k].clone() for k in STATE_KEYS}
+    q, k, v = wl.make_qkv(w, 1, DEV)
+    _step(w, st, eng, out, 1, prev, logits=lg)
+    oracle_step(w, s_np, bits16(q), bits16(k), bits16(v), logits_np(lg), logits_np(prev), 1)
+    status = st["slot_status"].cpu().numpy().view(np.uint32)
+    assert status[1] & isd_pkg.binding.ST_NONFINITE_LOGIT
+    assert status[2] & isd_pkg.binding.ST_BAD_TOKEN_ID
+    assert status[3] & isd_pkg.binding.ST_BAD_PAGE_ID
+    assert status[0] == 0 and status[4] == 0
+    assert np.array_equal(status != 0, s_np["slot_status"] != 0)
+    for b in (1, 2, 3):                                 # frozen
+        assert st["ctx_len"][b] == before["ctx_len"][b] and st["n_ver"][b] == before["n_ver"][b]
+    for b in (0, 4):                                    # healthy slots advanced exactly like the oracle's
+        assert st["ctx_len"][b].item() == s_np["ctx_len"][b]
+        assert np.array_equal(st["block_tok"][b].cpu().numpy(), s_np["block_tok"][b])
+    g = eng.isd_read_status()
+    assert g & 4 and g & 8 and g & 16
+    assert eng.isd_read_status() == 0                   # cleared by the read
+    eng.close()
+
+
+def test_pool_exhaustion_and_capacity_match_the_oracle():
+    w = Workload("pool", batch=6, stride=4, n_q_heads=8, n_kv_heads=2, vocab=512, ctx_min=40, ctx_max=56,
+                 logits_dtype="f32", peaked_frac=1.0, steps=1, propose_mode=1, seed=10)
+    st, eng, out = _fresh(w)
+    st["free_top"][0] = 3                               # nearly empty pool
+    s_np = state_to_np(st)
+    prev = prev_np = None
+    for t in range(12):
+        q, k, v = wl.make_qkv(w, t, DEV)
+        lg = wl.make_logits(w, t, torch.from_numpy(s_np["ctx_len"]).to(DEV))
+        ao = torch.zeros(w.batch, w.Q, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=DEV)
+        args = eng.step_args(q=q, k_new=k, v_new=v, k_pool=st["k_pool"], v_pool=st["v_pool"], attn_out=ao,
+                             attn_lse=None, logits_cur=lg, q_prev_logits=prev, out=out)
+        eng.isd_step(st, args, t)
+        torch.cuda.synchronize()
+        oracle_step(w, s_np, bits16(q), bits16(k), bits16(v), logits_np(lg), prev_np, t)
+        prev, prev_np = lg, logits_np(lg)
+        for name in ("ctx_len", "n_ver", "free_top"):
+            assert np.array_equal(st[name].cpu().numpy(), s_np[name]), (t, name)
+        assert np.array_equal(st["slot_status"].cpu().numpy().view(np.uint32), s_np["slot_status"]), t
+    status = s_np["slot_status"]
+    assert np.any(status & oracle.ST_POOL_EXHAUSTED) or np.any(status & oracle.ST_SLOT_CAPACITY)
+    eng.close()
+
+
+def test_release_returns_pages():
+    w = Workload("rel", batch=3, stride=2, n_q_heads=8, n_kv_heads=2, vocab=256, ctx_min=20, ctx_max=40,
+                 logits_dtype="f32", steps=2, seed=12)
+    st, eng, out = _fresh(w)
+    s_np = state_to_np(st)
+    slots = torch.tensor([2, 0], dtype=torch.int32, device=DEV)
+    eng.isd_release(st, slots)
+    torch.cuda.synchronize()
+    oracle.release(N=w.stride, page_size=16, ctx_len=s_np["ctx_len"], n_ver=s_np["n_ver"],
+                   page_table=s_np["page_table"], free_stack=s_np["free_stack"], free_top=s_np["free_top"],
+                   active=s_np["active"], slots=[2, 0])
+    top = int(s_np["free_top"][0])
+    assert st["free_top"].item() == top
+    assert np.array_equal(st["free_stack"].cpu().numpy()[:top], s_np["free_stack"][:top])
+    assert np.array_equal(st["active"].cpu().numpy(), s_np["active"])
+    eng.close()
+
+
+def test_invalid_arguments_return_error_codes():
+    with pytest.raises(isd_pkg.IsdError, match="unsupported"):
+        isd_pkg.Isd(batch=1, stride=2, n_q_heads=8, n_kv_heads=2, vocab=64, max_pages_per_slot=4, num_pages=8,
+                    logits_dtype="f32", head_dim=64)
+    with pytest.raises(isd_pkg.IsdError, match="unsupported"):
+        isd_pkg.Isd(batch=1, stride=16, n_q_heads=64, n_kv_heads=8, vocab=64, max_pages_per_slot=4, num_pages=8,
+                    logits_dtype="f32")
+    with pytest.raises(isd_pkg.IsdError, match="invalid"):
+        isd_pkg.Isd(batch=0, stride=2, n_q_heads=8, n_kv_heads=2, vocab=64, max_pages_per_slot=4, num_pages=8,
+                    logits_dtype="f32")
