@@ -211,6 +211,13 @@ int isd_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t
  * last call into *host_status (host pointer), then clears the global word. */
 int isd_read_status(isd_ctx* ctx, uint32_t* host_status, void* cuda_stream);
 
+/* Optional instrumentation (the paper has no counterpart): cudaEvent_t handles, passed as void*,
+ * that later calls record on their stream immediately before / after the attention main kernel
+ * (attn_*) and the row-statistics kernel of isd_verify (verify_*).  NULL switches a pair off.
+ * The events stay owned by the caller. */
+int isd_set_profile_events(isd_ctx* ctx, void* attn_start, void* attn_stop, void* verify_start,
+                           void* verify_stop);
+
 /* Number of kernel launches the library has issued through this context. */
 int64_t isd_launch_count(const isd_ctx* ctx);
 

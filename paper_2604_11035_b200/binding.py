@@ -18,7 +18,7 @@ ST_POOL_EXHAUSTED, ST_SLOT_CAPACITY, ST_BAD_TOKEN_ID = 1, 2, 4
 ST_BAD_PAGE_ID, ST_NONFINITE_LOGIT, ST_EMPTY_RESIDUAL = 8, 16, 32
 
 EXPORTS = ["isd_create", "isd_destroy", "isd_attn", "isd_verify", "isd_commit", "isd_step",
-           "isd_release", "isd_read_status", "isd_launch_count", "isd_strerror"]
+           "isd_release", "isd_read_status", "isd_set_profile_events", "isd_launch_count", "isd_strerror"]
 
 
 class IsdConfig(C.Structure):
@@ -66,6 +66,8 @@ def load():
         lib.isd_step.argtypes = [vp, C.POINTER(IsdBatchState), C.POINTER(IsdStepArgs), C.c_uint64, vp]
         lib.isd_release.argtypes = [vp, C.POINTER(IsdBatchState), vp, C.c_int32, vp]
         lib.isd_read_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        lib.isd_set_profile_events.argtypes = [vp] * 5
+        lib.isd_set_profile_events.restype = C.c_int
         lib.isd_launch_count.argtypes = [vp]
         lib.isd_launch_count.restype = C.c_int64
         lib.isd_strerror.argtypes = [C.c_int]
@@ -176,6 +178,11 @@ class Isd:
         v = C.c_uint32(0)
         _check(self.lib.isd_read_status(self.ctx, C.byref(v), _stream()), "isd_read_status")
         return int(v.value)
+
+    def isd_set_profile_events(self, attn_start=None, attn_stop=None, verify_start=None, verify_stop=None):
+        """Events are torch.cuda.Event objects (created with enable_timing=True and already recorded once)."""
+        h = [None if e is None else e.cuda_event for e in (attn_start, attn_stop, verify_start, verify_stop)]
+        _check(self.lib.isd_set_profile_events(self.ctx, *h), "isd_set_profile_events")
 
     def isd_launch_count(self) -> int:
         return int(self.lib.isd_launch_count(self.ctx))

@@ -189,6 +189,15 @@ int isd_read_status(isd_ctx* ctx, uint32_t* host_status, void* cuda_stream) {
   return ISD_OK;
 }
 
+int isd_set_profile_events(isd_ctx* ctx, void* attn_start, void* attn_stop, void* verify_start, void* verify_stop) {
+  if (!ctx) return ISD_ERR_INVALID_ARG;
+  ctx->ev_attn0 = reinterpret_cast<cudaEvent_t>(attn_start);
+  ctx->ev_attn1 = reinterpret_cast<cudaEvent_t>(attn_stop);
+  ctx->ev_verify0 = reinterpret_cast<cudaEvent_t>(verify_start);
+  ctx->ev_verify1 = reinterpret_cast<cudaEvent_t>(verify_stop);
+  return ISD_OK;
+}
+
 int64_t isd_launch_count(const isd_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 const char* isd_strerror(int code) {

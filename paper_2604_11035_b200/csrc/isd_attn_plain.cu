@@ -75,6 +75,20 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const AttnParams P) {
     uint4* d = reinterpret_cast<uint4*>((kv ? P.v_pool : P.k_pool) + dst) + v16;
     *d = *s;
   }
+  // Rows of the last page beyond the block are zeroed: they are never attended (masked), but the
+  // tensor-core kernel multiplies them by a zero probability, which needs finite values.
+  const int end = ctx + ql;
+  const int tail = (ISD_PAGE - end % ISD_PAGE) % ISD_PAGE;
+  const int zvecs = tail * P.Hkv * 2 * 16;
+  for (int i = threadIdx.x; i < zvecs; i += blockDim.x) {
+    const int v16 = i & 15;
+    const int kv = (i >> 4) & 1;
+    const int g = (i >> 5) % P.Hkv;
+    const int pos = end + (i >> 5) / P.Hkv;
+    const int page = P.page_table[(size_t)b * P.max_pages + pos / ISD_PAGE];
+    const size_t dst = (((size_t)page * P.Hkv + g) * ISD_PAGE + (pos % ISD_PAGE)) * ISD_HEAD_DIM;
+    reinterpret_cast<uint4*>((kv ? P.v_pool : P.k_pool) + dst)[v16] = make_uint4(0, 0, 0, 0);
+  }
 }
 
 __global__ void __launch_bounds__(128) attn_plain_kernel(const AttnParams P) {

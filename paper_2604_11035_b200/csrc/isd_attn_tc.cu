@@ -1,6 +1,728 @@
-// placeholder until the tensor-core kernel lands
+// isd_attn tensor-core path (sm_100a): strict-causal attention of every slot's ISD query block
+// against its paged bf16 KV cache (Sec. 3.1 mask; Sec. 3.3 (1) "single paged-only kernel" for the
+// 2N-1 row extend), re-designed for B200:
+//
+//   * GQA packing: the G = Hq/Hkv query heads that share a KV head and the q_len block rows form one
+//     M = 128 row tile (row m = r * G + head-in-group), so each KV byte is read once per step.
+//   * KV pages (16 tokens x 128 dims, 4 KiB per head) are staged by TMA (cp.async.bulk.tensor, no
+//     multicast) into a 4-deep shared-memory ring in the 128-byte-swizzled layout tcgen05 consumes;
+//     one 128-key tile = 8 pages.
+//   * S = Q K^T and O += P V run on the 5th-gen tensor cores (tcgen05.mma, cta_group::1, M=128,
+//     N=128, K=16, bf16 -> fp32) with accumulators in TMEM; S is double-buffered so that the
+//     softmax of tile j overlaps the QK^T of tile j+1.
+//   * Softmax: 128 threads, one TMEM lane (= row) each, so row max / sum need no shuffles; the
+//     running maximum is only raised when it grows by more than 2^8 (lazy rescale of O in TMEM).
+//   * Persistent CTAs, one per SM.  All (slot, kv-head) KV ranges are laid end to end in units of
+//     128-key tiles and cut into equal contiguous shares, so every CTA streams the same number of
+//     bytes; a share's ragged first/last pieces go to a small fp32 scratch and are merged by a
+//     second kernel (log-sum-exp combine).  Nothing waits on another CTA.
+//   * Warp roles: warps 0-3 softmax/epilogue, warp 4 TMA producer, warp 5 MMA issuer.
+//
+// Every mbarrier wait is bounded; on expiry the CTA raises ISD_ST_KERNEL_TIMEOUT in the global status
+// word, stops issuing work, drains, frees its TMEM and returns.
+#include <cuda.h>
+#include <new>
+
 #include "isd_internal.cuh"
-int isd_attn_tc_create(isd_ctx*) { return ISD_OK; }
-void isd_attn_tc_destroy(isd_ctx*) {}
-int isd_launch_attn_tc(isd_ctx*, const isd_batch_state*, const void*, const void*, const void*, void*, void*,
-                       void*, float*, cudaStream_t) { return ISD_ERR_UNSUPPORTED; }
+
+#define ISD_ST_KERNEL_TIMEOUT 0x80000000u
+
+namespace {
+
+constexpr int kTile = 128;                 // keys per tile
+constexpr int kStageBytes = 32768;         // one K or V tile: [half(2)][page(8)][tok(16)][128 B]
+constexpr int kStages = 4;
+constexpr int kThreads = 192;
+constexpr int kSmQ = 0;                    // [half(2)][row group(16)][8 rows][128 B]
+constexpr int kSmP = 32768;                // 2 buffers, same layout over keys
+constexpr int kSmRing = 98304;
+constexpr int kSmBar = kSmRing + kStages * kStageBytes;  // 229376
+constexpr int kSmemBytes = kSmBar + 256;
+constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// barrier slots (8 bytes each) inside the barrier block
+enum { BAR_FULL = 0, BAR_EMPTY = kStages, BAR_SFULL = 2 * kStages, BAR_SEMPTY = 2 * kStages + 2,
+       BAR_PFULL = 2 * kStages + 4, BAR_ODONE = 2 * kStages + 6, BAR_OFREE = 2 * kStages + 8,
+       BAR_QFULL = 2 * kStages + 9, BAR_COUNT = 2 * kStages + 10 };
+
+struct TcParams {
+  int B, Q, N, Hq, Hkv, G, max_pages, num_pages;
+  float scale2;  // sm_scale * log2(e)
+  const int32_t* ctx_len;
+  const int32_t* n_ver;
+  const uint8_t* active;
+  const int32_t* page_table;
+  const uint32_t* slot_status;
+  uint32_t* global_status;
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  float* lse;
+  int* tile_prefix;  // [B + 1] tiles per kv head, exclusive prefix over slots
+  float* part_o;     // [ctas * 2][128][128]
+  float* part_ml;    // [ctas * 2][128][2]
+  int num_ctas;
+};
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: returns false (and raises the abort flag) when the limit is reached.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
+}
+
+// K-major / MN-major shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+  const uint32_t hi = (sbo_bytes >> 4) | (1u << 14) | (2u << 29);
+  return ((uint64_t)hi << 32) | lo;
+}
+
+#define TMEM_LD32(taddr, v, o)                                                                          \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                         \
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25," \
+      "%26,%27,%28,%29,%30,%31}, [%32];"                                                                \
+      : "=r"(v[o + 0]), "=r"(v[o + 1]), "=r"(v[o + 2]), "=r"(v[o + 3]), "=r"(v[o + 4]), "=r"(v[o + 5]), \
+        "=r"(v[o + 6]), "=r"(v[o + 7]), "=r"(v[o + 8]), "=r"(v[o + 9]), "=r"(v[o + 10]),                \
+        "=r"(v[o + 11]), "=r"(v[o + 12]), "=r"(v[o + 13]), "=r"(v[o + 14]), "=r"(v[o + 15]),            \
+        "=r"(v[o + 16]), "=r"(v[o + 17]), "=r"(v[o + 18]), "=r"(v[o + 19]), "=r"(v[o + 20]),            \
+        "=r"(v[o + 21]), "=r"(v[o + 22]), "=r"(v[o + 23]), "=r"(v[o + 24]), "=r"(v[o + 25]),            \
+        "=r"(v[o + 26]), "=r"(v[o + 27]), "=r"(v[o + 28]), "=r"(v[o + 29]), "=r"(v[o + 30]),            \
+        "=r"(v[o + 31])                                                                                 \
+      : "r"(taddr))
+
+#define TMEM_ST32(taddr, v, o)                                                                          \
+  asm volatile(                                                                                         \
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "                                                   \
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26," \
+      "%27,%28,%29,%30,%31,%32};"                                                                       \
+      ::"r"(taddr), "r"(v[o + 0]), "r"(v[o + 1]), "r"(v[o + 2]), "r"(v[o + 3]), "r"(v[o + 4]),          \
+        "r"(v[o + 5]), "r"(v[o + 6]), "r"(v[o + 7]), "r"(v[o + 8]), "r"(v[o + 9]), "r"(v[o + 10]),      \
+        "r"(v[o + 11]), "r"(v[o + 12]), "r"(v[o + 13]), "r"(v[o + 14]), "r"(v[o + 15]), "r"(v[o + 16]), \
+        "r"(v[o + 17]), "r"(v[o + 18]), "r"(v[o + 19]), "r"(v[o + 20]), "r"(v[o + 21]), "r"(v[o + 22]), \
+        "r"(v[o + 23]), "r"(v[o + 24]), "r"(v[o + 25]), "r"(v[o + 26]), "r"(v[o + 27]), "r"(v[o + 28]), \
+        "r"(v[o + 29]), "r"(v[o + 30]), "r"(v[o + 31])                                                  \
+      : "memory")
+
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Work split: identical, independent enumeration in every warp role
+// ------------------------------------------------------------------------------------------------
+struct Segment {
+  int b, g;      // slot, kv head
+  int j0, j1;    // tiles [j0, j1) of the pair
+  int T;         // tiles of the whole pair
+  int kv_len;    // ctx_len + q_len
+  int ctx, q_len;
+  int part_slot; // scratch slot when the segment does not cover the whole pair, else -1
+};
+
+struct WorkIter {
+  const int* prefix;
+  int B, Hkv, b;
+  long long t, t_begin, t_end;
+  __device__ void init(const TcParams& P, int cta) {
+    prefix = P.tile_prefix;
+    B = P.B; Hkv = P.Hkv;
+    const long long total = (long long)prefix[B] * Hkv;
+    const long long per = (total + P.num_ctas - 1) / P.num_ctas;
+    t_begin = t = (long long)cta * per;
+    t_end = t + per < total ? t + per : total;
+    // first slot whose range ends after t
+    int lo = 0, hi = B;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if ((long long)prefix[mid + 1] * Hkv > t) hi = mid; else lo = mid + 1;
+    }
+    b = lo;
+  }
+  __device__ bool next(const TcParams& P, int cta, Segment& s) {
+    if (t >= t_end) return false;
+    while (b < B && (long long)prefix[b + 1] * Hkv <= t) ++b;
+    if (b >= B) return false;
+    const int T = prefix[b + 1] - prefix[b];
+    const long long off = t - (long long)prefix[b] * Hkv;
+    s.b = b; s.T = T;
+    s.g = (int)(off / T);
+    s.j0 = (int)(off % T);
+    const long long room = t_end - t;
+    s.j1 = (long long)(T - s.j0) <= room ? T : s.j0 + (int)room;
+    s.ctx = P.ctx_len[b];
+    s.q_len = P.n_ver[b] + P.N;
+    s.kv_len = s.ctx + s.q_len;
+    const bool whole = (s.j0 == 0 && s.j1 == T);
+    s.part_slot = whole ? -1 : cta * 2 + (t == t_begin ? 0 : 1);
+    t += s.j1 - s.j0;
+    return true;
+  }
+};
+
+// ------------------------------------------------------------------------------------------------
+// Plan: tiles per slot (per kv head) and their exclusive prefix, one CTA
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) attn_plan_kernel(const TcParams P) {
+  __shared__ int sm_warp[33];
+  __shared__ int sm_carry;
+  if (threadIdx.x == 0) sm_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < P.B; base += 1024) {
+    const int b = base + threadIdx.x;
+    int tiles = 0;
+    if (b < P.B && P.active[b]) {
+      const int nv = P.n_ver[b];
+      const int ctx = P.ctx_len[b];
+      const bool ok = nv >= 0 && nv <= P.N - 1 && ctx >= 0 &&
+                      (P.slot_status[b] & (ISD_ST_BAD_PAGE_ID | ISD_ST_SLOT_CAPACITY)) == 0;
+      if (ok) tiles = (ctx + nv + P.N + kTile - 1) / kTile;
+    }
+    // inclusive scan
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = tiles;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
+    }
+    if (lane == 31) sm_warp[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      int w = sm_warp[lane], winc = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += v;
+      }
+      sm_warp[lane] = winc - w;
+      if (lane == 31) sm_warp[32] = winc;
+    }
+    __syncthreads();
+    const int excl = sm_carry + sm_warp[warp] + inc - tiles;
+    if (b < P.B) P.tile_prefix[b] = excl;
+    __syncthreads();
+    if (threadIdx.x == 0) sm_carry += sm_warp[32];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) P.tile_prefix[P.B] = sm_carry;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Main kernel
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sm_base = smem_u32(smem);
+  const uint32_t bar_base = sm_base + kSmBar;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kSmBar + BAR_COUNT * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kSmBar + BAR_COUNT * 8 + 8);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x;
+  auto bar = [&](int i) { return bar_base + 8u * (uint32_t)i; };
+
+  if (sm_base & 1023u) {  // the swizzled layouts below assume a 1 KiB aligned window
+    if (threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+    return;
+  }
+  // ---- setup: barriers, TMEM, zero the ring (stale V rows of a ragged tile must be finite)
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kStages; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_SFULL + i), 1); mbar_init(bar(BAR_SEMPTY + i), 4); mbar_init(bar(BAR_PFULL + i), 4); }
+    mbar_init(bar(BAR_ODONE), 1);
+    mbar_init(bar(BAR_ODONE + 1), 1);
+    mbar_init(bar(BAR_OFREE), 4);
+    mbar_init(bar(BAR_QFULL), 4);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  {
+    uint4* z = reinterpret_cast<uint4*>(smem);
+    for (int i = threadIdx.x; i < kSmBar / 16; i += kThreads) z[i] = make_uint4(0, 0, 0, 0);
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem_s0 = tmem, tmem_o = tmem + 256;
+
+  if (warp == 4) {
+    // =========================================================================== TMA producer
+    WorkIter it;
+    it.init(P, cta);
+    Segment sg;
+    uint32_t fill = 0;
+    while (it.next(P, cta, sg) && !*abort_flag) {
+      const int cnt = sg.j1 - sg.j0;
+      const int32_t* pt = P.page_table + (size_t)sg.b * P.max_pages;
+      // fill order = consumption order: K(0), then for each i: K(i+1), V(i)
+      auto issue = [&](int j, bool is_v) -> bool {
+        const int first_page = j * 8;
+        const int valid = min(8, (sg.kv_len - j * kTile + ISD_PAGE - 1) / ISD_PAGE);
+        int id = 0;
+        if (lane < valid) id = pt[first_page + lane];
+        id = min(max(id, 0), P.num_pages - 1);
+        const uint32_t s = fill % kStages, ph = (fill / kStages) & 1u;
+        if (!mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag)) return false;
+        if (lane == 0) mbar_arrive_expect_tx(bar(BAR_FULL + s), (uint32_t)valid * 4096u);
+        __syncwarp();
+        const int pg = lane >> 1, half = lane & 1;
+        const int pid = __shfl_sync(0xffffffffu, id, pg & 7);
+        if (lane < 16 && pg < valid) {
+          const uint32_t dst = sm_base + kSmRing + s * kStageBytes + half * 16384 + pg * 2048;
+          tma_load_3d(dst, is_v ? &tmap_v : &tmap_k, half * 64, 0, pid * P.Hkv + sg.g, bar(BAR_FULL + s));
+        }
+        ++fill;
+        return true;
+      };
+      bool ok = issue(sg.j0, false);
+      for (int i = 0; i < cnt && ok; ++i) {
+        if (i + 1 < cnt) ok = issue(sg.j0 + i + 1, false);
+        if (ok) ok = issue(sg.j0 + i, true);
+      }
+      if (!ok) break;
+    }
+    // drain: every issued copy must have landed before the CTA may exit
+    // (the consumer waits on every FULL barrier it was promised; on abort wait here, bounded)
+    if (*abort_flag) {
+      for (uint32_t f = (fill > kStages ? fill - kStages : 0); f < fill; ++f)
+        mbar_wait(bar(BAR_FULL + f % kStages), (f / kStages) & 1u, abort_flag);
+    }
+  } else if (warp == 5) {
+    // =========================================================================== MMA issuer
+    WorkIter it;
+    it.init(P, cta);
+    Segment sg;
+    uint32_t cons = 0, n = 0, seg = 0;
+    const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+    const uint32_t idesc_pv = idesc_qk | (1u << 16);  // B (= V) is MN-major
+    bool ok = true;
+    while (ok && it.next(P, cta, sg) && !*abort_flag) {
+      const int cnt = sg.j1 - sg.j0;
+      ok = mbar_wait(bar(BAR_QFULL), seg & 1u, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      auto qk = [&](uint32_t nn) -> bool {
+        const uint32_t s = cons % kStages, ph = (cons / kStages) & 1u;
+        if (!mbar_wait(bar(BAR_FULL + s), ph, abort_flag)) return false;
+        if (nn >= 2 && !mbar_wait(bar(BAR_SEMPTY + (nn & 1u)), ((nn >> 1) - 1u) & 1u, abort_flag)) return false;
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t kb = sm_base + kSmRing + s * kStageBytes;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t off = (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u;
+            tc_mma(tmem_s0 + (nn & 1u) * 128u, smem_desc(sm_base + kSmQ + off, 16, 1024),
+                   smem_desc(kb + off, 16, 1024), idesc_qk, k > 0);
+          }
+          tc_commit(bar(BAR_EMPTY + s));
+          tc_commit(bar(BAR_SFULL + (nn & 1u)));
+        }
+        __syncwarp();
+        ++cons;
+        return true;
+      };
+      auto pv = [&](uint32_t nn, bool first) -> bool {
+        const uint32_t s = cons % kStages, ph = (cons / kStages) & 1u;
+        if (!mbar_wait(bar(BAR_FULL + s), ph, abort_flag)) return false;
+        if (!mbar_wait(bar(BAR_PFULL + (nn & 1u)), (nn >> 1) & 1u, abort_flag)) return false;
+        if (first && seg > 0 && !mbar_wait(bar(BAR_OFREE), (seg - 1u) & 1u, abort_flag)) return false;
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t vb = sm_base + kSmRing + s * kStageBytes;
+          const uint32_t pb = sm_base + kSmP + (nn & 1u) * 32768u;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t aoff = (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u;
+            tc_mma(tmem_o, smem_desc(pb + aoff, 16, 1024), smem_desc(vb + (uint32_t)k * 2048u, 16384, 1024),
+                   idesc_pv, !(first && k == 0));
+          }
+          tc_commit(bar(BAR_EMPTY + s));
+          tc_commit(bar(BAR_ODONE + (nn & 1u)));
+        }
+        __syncwarp();
+        ++cons;
+        return true;
+      };
+      ok = qk(n);
+      for (int i = 0; i < cnt && ok; ++i) {
+        if (i + 1 < cnt) ok = qk(n + i + 1);
+        if (ok) ok = pv(n + i, i == 0);
+      }
+      n += cnt;
+      ++seg;
+    }
+  } else {
+    // =========================================================================== softmax / epilogue
+    WorkIter it;
+    it.init(P, cta);
+    Segment sg;
+    uint32_t n = 0, seg = 0;
+    const int row = warp * 32 + lane;          // TMEM lane = row of the M = 128 tile
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    bool ok = true;
+    while (ok && it.next(P, cta, sg) && !*abort_flag) {
+      const int cnt = sg.j1 - sg.j0;
+      const int rows_valid = sg.q_len * P.G;
+      const int r = row / P.G, hg = row % P.G;
+      const bool row_ok = row < rows_valid;
+      // ---- stage Q (rows m = r * G + hg) into the swizzled K-major layout; padding rows stay zero
+      {
+        // previous segment's QK MMAs are complete (its last S tile was consumed), so Q may be overwritten
+        const uint4* src = reinterpret_cast<const uint4*>(
+            P.q + (((size_t)sg.b * P.Q + (row_ok ? r : 0)) * P.Hq + sg.g * P.G + hg) * ISD_HEAD_DIM);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          uint4 v = make_uint4(0, 0, 0, 0);
+          if (row_ok) v = src[c];
+          const int half = c >> 3, cc = c & 7;
+          uint8_t* dst = smem + kSmQ + half * 16384 + (row >> 3) * 1024 + (row & 7) * 128 + ((cc ^ (row & 7)) << 4);
+          *reinterpret_cast<uint4*>(dst) = v;
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_QFULL));
+      }
+      float m2 = -INFINITY, l = 0.f;  // running max (log2 domain) and sum of this row
+      for (int i = 0; i < cnt && ok; ++i) {
+        const uint32_t nn = n + i;
+        const int j = sg.j0 + i;
+        ok = mbar_wait(bar(BAR_SFULL + (nn & 1u)), (nn >> 1) & 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t sv[128];
+        const uint32_t ts = tmem_s0 + (nn & 1u) * 128u + lane_base;
+        TMEM_LD32(ts, sv, 0);
+        TMEM_LD32(ts + 32, sv, 32);
+        TMEM_LD32(ts + 64, sv, 64);
+        TMEM_LD32(ts + 96, sv, 96);
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_SEMPTY + (nn & 1u)));
+        // ---- scale, mask, row max
+        const int kb = j * kTile;
+        const int limit = row_ok ? (sg.ctx + r - kb) : -1;  // columns c <= limit are visible
+        float mx = -INFINITY;
+        if (limit >= kTile - 1) {
+#pragma unroll
+          for (int c = 0; c < 128; ++c) {
+            const float x = __uint_as_float(sv[c]) * P.scale2;
+            sv[c] = __float_as_uint(x);
+            mx = fmaxf(mx, x);
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 128; ++c) {
+            const float x = c <= limit ? __uint_as_float(sv[c]) * P.scale2 : -INFINITY;
+            sv[c] = __float_as_uint(x);
+            mx = fmaxf(mx, x);
+          }
+        }
+        // ---- lazy rescale: raise the reference maximum only when it grows by more than 2^8
+        float m_use = m2;
+        const bool grow = mx > m2 + 8.f || (m2 == -INFINITY && mx > -INFINITY);
+        const bool any_grow = __any_sync(0xffffffffu, grow && i > 0);
+        if (grow) m_use = mx;
+        if (any_grow) {
+          // PV(nn-1) must have finished before O is touched.  PV completions alternate between two
+          // barriers: a waiter may lag one PV behind (PV(x-2) is known complete once S(x) arrived),
+          // which a single barrier's phase parity could not tell apart.
+          ok = mbar_wait(bar(BAR_ODONE + ((nn - 1u) & 1u)), ((nn - 1u) >> 1) & 1u, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const float f = (grow && m2 > -INFINITY) ? ex2f(m2 - m_use) : 1.f;
+          uint32_t ov[32];
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            TMEM_LD32(tmem_o + lane_base + q4 * 32, ov, 0);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * f);
+            TMEM_ST32(tmem_o + lane_base + q4 * 32, ov, 0);
+          }
+          tmem_wait_st();
+          l *= f;
+        } else if (grow) {
+          // first tile of the segment (nothing accumulated yet)
+          l = 0.f;
+        }
+        m2 = m_use;
+        // ---- probabilities, row sum, P tile (bf16, swizzled K-major) for the PV MMA
+        const float mref = (m2 == -INFINITY) ? 0.f : m2;
+        uint8_t* pbase = smem + kSmP + (nn & 1u) * 32768 + (row >> 3) * 1024 + (row & 7) * 128;
+        float lsum = 0.f;
+#pragma unroll
+        for (int c16 = 0; c16 < 16; ++c16) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float p0 = ex2f(__uint_as_float(sv[c16 * 8 + 2 * e]) - mref);
+            const float p1 = ex2f(__uint_as_float(sv[c16 * 8 + 2 * e + 1]) - mref);
+            lsum += p0 + p1;
+            pk[e] = pack_bf16(p0, p1);
+          }
+          const int half = c16 >> 3, cc = c16 & 7;
+          *reinterpret_cast<uint4*>(pbase + half * 16384 + ((cc ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+        l += lsum;
+        fence_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_PFULL + (nn & 1u)));
+      }
+      if (!ok) break;
+      // ---- epilogue: wait for the last PV, read O, write the result or the partial
+      const uint32_t last = n + cnt - 1;
+      ok = mbar_wait(bar(BAR_ODONE + (last & 1u)), (last >> 1) & 1u, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint32_t ov[32];
+        TMEM_LD32(tmem_o + lane_base + q4 * 32, ov, 0);
+        tmem_wait_ld();
+        if (row_ok) {
+          if (sg.part_slot < 0) {
+            uint4* dst = reinterpret_cast<uint4*>(
+                P.out + (((size_t)sg.b * P.Q + r) * P.Hq + sg.g * P.G + hg) * ISD_HEAD_DIM + q4 * 32);
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              dst[c] = make_uint4(pack_bf16(__uint_as_float(ov[c * 8 + 0]) * inv_l, __uint_as_float(ov[c * 8 + 1]) * inv_l),
+                                  pack_bf16(__uint_as_float(ov[c * 8 + 2]) * inv_l, __uint_as_float(ov[c * 8 + 3]) * inv_l),
+                                  pack_bf16(__uint_as_float(ov[c * 8 + 4]) * inv_l, __uint_as_float(ov[c * 8 + 5]) * inv_l),
+                                  pack_bf16(__uint_as_float(ov[c * 8 + 6]) * inv_l, __uint_as_float(ov[c * 8 + 7]) * inv_l));
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(P.part_o + ((size_t)sg.part_slot * 128 + row) * 128 + q4 * 32);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) dst[c] = make_uint4(ov[c * 4], ov[c * 4 + 1], ov[c * 4 + 2], ov[c * 4 + 3]);
+          }
+        }
+      }
+      if (row_ok) {
+        if (sg.part_slot < 0) {
+          if (P.lse) P.lse[((size_t)sg.b * P.Q + r) * P.Hq + sg.g * P.G + hg] = (m2 + log2f(l)) * kLn2;
+        } else {
+          P.part_ml[((size_t)sg.part_slot * 128 + row) * 2 + 0] = m2;
+          P.part_ml[((size_t)sg.part_slot * 128 + row) * 2 + 1] = l;
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_OFREE));
+      n += cnt;
+      ++seg;
+    }
+  }
+
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Combine: pairs whose tiles were split over several CTAs (log-sum-exp merge of the partials)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) attn_combine_kernel(const TcParams P) {
+  const int g = blockIdx.x, b = blockIdx.y;
+  const int T = P.tile_prefix[b + 1] - P.tile_prefix[b];
+  if (T == 0) return;
+  const long long total = (long long)P.tile_prefix[P.B] * P.Hkv;
+  const long long per = (total + P.num_ctas - 1) / P.num_ctas;
+  const long long p0 = (long long)P.tile_prefix[b] * P.Hkv + (long long)g * T, p1 = p0 + T;
+  const int c_first = (int)(p0 / per), c_last = (int)((p1 - 1) / per);
+  if (c_first == c_last) return;  // written directly by one CTA
+  const int q_len = P.n_ver[b] + P.N;
+  const int rows_valid = q_len * P.G;
+  for (int row = threadIdx.x >> 5; row < rows_valid; row += 4) {
+    const int lane = threadIdx.x & 31;
+    float M = -INFINITY;
+    for (int c = c_first; c <= c_last; ++c) {
+      const int slot = c * 2 + (((long long)c * per >= p0) ? 0 : 1);
+      M = fmaxf(M, P.part_ml[((size_t)slot * 128 + row) * 2]);
+    }
+    float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int c = c_first; c <= c_last; ++c) {
+      const int slot = c * 2 + (((long long)c * per >= p0) ? 0 : 1);
+      const float m = P.part_ml[((size_t)slot * 128 + row) * 2], l = P.part_ml[((size_t)slot * 128 + row) * 2 + 1];
+      const float w = (m == -INFINITY) ? 0.f : ex2f(m - M);
+      L += l * w;
+      const float4 o = *reinterpret_cast<const float4*>(P.part_o + ((size_t)slot * 128 + row) * 128 + lane * 4);
+      acc[0] += o.x * w; acc[1] += o.y * w; acc[2] += o.z * w; acc[3] += o.w * w;
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    const int r = row / P.G, hg = row % P.G;
+    const size_t o_off = (((size_t)b * P.Q + r) * P.Hq + g * P.G + hg) * ISD_HEAD_DIM + lane * 4;
+    *reinterpret_cast<uint2*>(P.out + o_off) = make_uint2(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv));
+    if (P.lse && lane == 0) P.lse[((size_t)b * P.Q + r) * P.Hq + g * P.G + hg] = (M + log2f(L)) * kLn2;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// pool viewed as [num_pages * Hkv][16 tokens][128 dims]; box = 64 dims x 16 tokens of one (page, head)
+int encode_pool_map(CUtensorMap* map, const void* pool, int num_pages, int Hkv) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return ISD_ERR_CUDA;
+  const cuuint64_t dims[3] = {ISD_HEAD_DIM, ISD_PAGE, (cuuint64_t)num_pages * (cuuint64_t)Hkv};
+  const cuuint64_t strides[2] = {ISD_HEAD_DIM * 2, ISD_HEAD_DIM * 2 * ISD_PAGE};
+  const cuuint32_t box[3] = {64, ISD_PAGE, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(pool), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ISD_OK : ISD_ERR_CUDA;
+}
+
+struct TcHost {
+  CUtensorMap map_k, map_v;
+  int* tile_prefix;
+};
+
+}  // namespace
+
+int isd_attn_tc_create(isd_ctx* ctx) {
+  TcHost* h = new (std::nothrow) TcHost();
+  if (!h) return ISD_ERR_NO_MEMORY;
+  h->tile_prefix = nullptr;
+  ctx->tmap_k = h;
+  ctx->tmap_k_base = ctx->tmap_v_base = nullptr;
+  ctx->attn_ctas = ctx->num_sms;
+  if (cudaMalloc(&h->tile_prefix, sizeof(int) * (ctx->cfg.batch + 1)) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  if (cudaMalloc(&ctx->attn_part_o, sizeof(float) * (size_t)ctx->attn_ctas * 2 * 128 * 128) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  if (cudaMalloc(&ctx->attn_part_ml, sizeof(float) * (size_t)ctx->attn_ctas * 2 * 128 * 2) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+    return ISD_ERR_CUDA;
+  if (!get_encode()) return ISD_ERR_CUDA;
+  return ISD_OK;
+}
+
+void isd_attn_tc_destroy(isd_ctx* ctx) {
+  TcHost* h = reinterpret_cast<TcHost*>(ctx->tmap_k);
+  if (h) {
+    cudaFree(h->tile_prefix);
+    delete h;
+  }
+  cudaFree(ctx->attn_part_o);
+  cudaFree(ctx->attn_part_ml);
+  ctx->tmap_k = nullptr;
+}
+
+int isd_launch_attn_tc(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void* k_new, const void* v_new,
+                       void* k_pool, void* v_pool, void* out, float* lse, cudaStream_t stream) {
+  (void)k_new; (void)v_new;  // already appended to the pages by the scatter kernel
+  TcHost* h = reinterpret_cast<TcHost*>(ctx->tmap_k);
+  if (!h) return ISD_ERR_INVALID_ARG;
+  const isd_config& c = ctx->cfg;
+  if (ctx->tmap_k_base != k_pool || ctx->tmap_v_base != v_pool) {
+    int rc = encode_pool_map(&h->map_k, k_pool, c.num_pages, c.n_kv_heads);
+    if (rc == ISD_OK) rc = encode_pool_map(&h->map_v, v_pool, c.num_pages, c.n_kv_heads);
+    if (rc != ISD_OK) return rc;
+    ctx->tmap_k_base = k_pool;
+    ctx->tmap_v_base = v_pool;
+  }
+  TcParams P;
+  P.B = c.batch; P.Q = ctx->Q; P.N = c.stride; P.Hq = c.n_q_heads; P.Hkv = c.n_kv_heads; P.G = ctx->G;
+  P.max_pages = c.max_pages_per_slot; P.num_pages = c.num_pages;
+  P.scale2 = ctx->sm_scale * kLog2e;
+  P.ctx_len = st->ctx_len; P.n_ver = st->n_ver; P.active = st->active; P.page_table = st->page_table;
+  P.slot_status = st->slot_status; P.global_status = ctx->global_status;
+  P.q = (const __nv_bfloat16*)q; P.out = (__nv_bfloat16*)out; P.lse = lse;
+  P.tile_prefix = h->tile_prefix; P.part_o = ctx->attn_part_o; P.part_ml = ctx->attn_part_ml;
+  P.num_ctas = ctx->attn_ctas;
+  attn_plan_kernel<<<1, 1024, 0, stream>>>(P);
+  if (ctx->ev_attn0) cudaEventRecord(ctx->ev_attn0, stream);
+  attn_tc_kernel<<<ctx->attn_ctas, kThreads, kSmemBytes, stream>>>(P, h->map_k, h->map_v);
+  if (ctx->ev_attn1) cudaEventRecord(ctx->ev_attn1, stream);
+  attn_combine_kernel<<<dim3(c.n_kv_heads, c.batch), 128, 0, stream>>>(P);
+  ctx->launches += 3;
+  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}

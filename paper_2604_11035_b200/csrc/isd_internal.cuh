@@ -62,6 +62,8 @@ struct isd_ctx {
   void* tmap_v;
   const void* tmap_k_base;  // pool pointers the tensor maps were encoded for
   const void* tmap_v_base;
+  // ---- optional instrumentation events (owned by the caller)
+  cudaEvent_t ev_attn0, ev_attn1, ev_verify0, ev_verify1;
   // ---- status
   uint32_t* global_status;  // [1]
   int64_t launches;

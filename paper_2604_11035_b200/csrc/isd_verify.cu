@@ -544,8 +544,10 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   P.resid_ticket = ctx->resid_ticket; P.reject_pos = ctx->reject_pos; P.lse_p_rej = ctx->lse_p_rej;
 
   const dim3 grid1(ctx->row_splits, ctx->Q, c.batch);
+  if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
   if (c.logits_dtype == ISD_LOGITS_BF16) verify_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads, 0, stream>>>(P);
   else verify_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads, 0, stream>>>(P);
+  if (ctx->ev_verify1) cudaEventRecord(ctx->ev_verify1, stream);
   ctx->launches++;
   if (c.stride > 1 && (c.q_mode == 1 || q_prev_logits != nullptr)) {
     const dim3 grid2(ctx->resid_splits, c.batch);

@@ -22,14 +22,14 @@ def assert_clean(rep, allow_exempt=2):
     assert rep["gpu_launches"] > 0
 
 
-@pytest.mark.parametrize("attn_impl", [0, 1])
+@pytest.mark.parametrize("attn_impl", [0, 1], ids=["tcgen05", "plain"])
 def test_config0_tiny(attn_impl):
     rep = run_chain_parity(wl.config(0), steps=4, device=DEV, attn_impl=attn_impl)
     assert_clean(rep)
     assert rep["positions"] > 0 and rep["emitted"] >= 4
 
 
-@pytest.mark.parametrize("attn_impl", [0, 1])
+@pytest.mark.parametrize("attn_impl", [0, 1], ids=["tcgen05", "plain"])
 @pytest.mark.parametrize("dtype,propose_mode,q_mode,N", [
     ("f32", 0, 0, 4), ("bf16", 0, 0, 4), ("bf16", 1, 0, 8), ("bf16", 1, 1, 3), ("f32", 0, 0, 2), ("bf16", 0, 0, 16)])
 def test_ragged_multi_tile_chain(attn_impl, dtype, propose_mode, q_mode, N):
