@@ -319,30 +319,45 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
     while (it.next(P, cta, sg) && !*abort_flag) {
       const int cnt = sg.j1 - sg.j0;
       const int32_t* pt = P.page_table + (size_t)sg.b * P.max_pages;
-      // fill order = consumption order: K(0), then for each i: K(i+1), V(i)
-      auto issue = [&](int j, bool is_v) -> bool {
-        const int first_page = j * 8;
-        const int valid = min(8, (sg.kv_len - j * kTile + ISD_PAGE - 1) / ISD_PAGE);
+      // Page ids are fetched 32 at a time (4 tiles) and one chunk ahead, so that the table lookup is
+      // off the critical path of the copies; lane l of a chunk register holds the id of page 32c + l.
+      const int total_pages = (sg.kv_len + ISD_PAGE - 1) / ISD_PAGE;
+      const int base_page = sg.j0 * 8;
+      auto load_chunk = [&](int c) -> int {
+        const int pg = base_page + c * 32 + lane;
         int id = 0;
-        if (lane < valid) id = pt[first_page + lane];
-        id = min(max(id, 0), P.num_pages - 1);
+        if (pg < total_pages) id = pt[pg];
+        return min(max(id, 0), P.num_pages - 1);
+      };
+      int cur_c = 0;
+      int ids_cur = load_chunk(0), ids_nxt = load_chunk(1);
+      // fill order = consumption order: K(0), then for each i: K(i+1), V(i)
+      auto issue = [&](int i, bool is_v) -> bool {
+        const int j = sg.j0 + i;
+        const int valid = min(8, (sg.kv_len - j * kTile + ISD_PAGE - 1) / ISD_PAGE);
+        const int src = ((i >> 2) == cur_c) ? ids_cur : ids_nxt;
         const uint32_t s = fill % kStages, ph = (fill / kStages) & 1u;
         if (!mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag)) return false;
         if (lane == 0) mbar_arrive_expect_tx(bar(BAR_FULL + s), (uint32_t)valid * 4096u);
         __syncwarp();
         const int pg = lane >> 1, half = lane & 1;
-        const int pid = __shfl_sync(0xffffffffu, id, pg & 7);
+        const int pid = __shfl_sync(0xffffffffu, src, ((i & 3) << 3) + (pg & 7));
         if (lane < 16 && pg < valid) {
           const uint32_t dst = sm_base + kSmRing + s * kStageBytes + half * 16384 + pg * 2048;
           tma_load_3d(dst, is_v ? &tmap_v : &tmap_k, half * 64, 0, pid * P.Hkv + sg.g, bar(BAR_FULL + s));
         }
         ++fill;
+        if (is_v && (i & 3) == 3) {  // V(i) is the last user of chunk i / 4
+          ++cur_c;
+          ids_cur = ids_nxt;
+          ids_nxt = load_chunk(cur_c + 1);
+        }
         return true;
       };
-      bool ok = issue(sg.j0, false);
+      bool ok = issue(0, false);
       for (int i = 0; i < cnt && ok; ++i) {
-        if (i + 1 < cnt) ok = issue(sg.j0 + i + 1, false);
-        if (ok) ok = issue(sg.j0 + i, true);
+        if (i + 1 < cnt) ok = issue(i + 1, false);
+        if (ok) ok = issue(i, true);
       }
       if (!ok) break;
     }

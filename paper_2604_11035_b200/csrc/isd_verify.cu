@@ -116,6 +116,162 @@ __device__ double noisy_score_f64(const VerifyParams& P, const void* row, int i,
   return l + gumbel_f64(philox_word(r, i & 3));
 }
 
+// Packed fp32x2 arithmetic (two lanes per instruction on sm_100) and 3-input max
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// Philox4x32-10 with the ten round keys precomputed (they depend on the seed only)
+struct PhiloxKeys {
+  uint32_t k0[10], k1[10];
+  __device__ __forceinline__ void init(uint32_t lo, uint32_t hi) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+      k0[r] = lo + (uint32_t)r * 0x9E3779B9u;
+      k1[r] = hi + (uint32_t)r * 0xBB67AE85u;
+    }
+  }
+  __device__ __forceinline__ uint4 draw(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3) const {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+      const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+      const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+      const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0[r];
+      const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1[r];
+      c1 = (uint32_t)p1; c3 = (uint32_t)p0; c0 = n0; c2 = n2;
+    }
+    return make_uint4(c0, c1, c2, c3);
+  }
+};
+
+// One streaming pass over elements [lo, hi) of a logits row.
+//   always   online softmax: running max M of the raw logits and S = sum exp((l - M) * invT)
+//   RAW      argmax of the raw logits (lowest index on ties): the running max itself
+//   NOISE    Gumbel-max top-2 of l * invT + g with the bound-based skip
+// Returns m_nat = M * invT (natural-log units of the scaled logits), S and the candidates.
+template <int DT, bool NOISE, bool RAW>
+__device__ __forceinline__ void row_pass(const VerifyParams& P, const char* row, int lo, int hi, int b,
+                                         uint32_t tagpos, float& m_nat, float& S_out, Top2& top) {
+  const float scale2 = P.inv_t * kLog2e;  // raw logit -> log2 domain
+  const uint64_t scale22 = pack2(scale2, scale2);
+  float M = -INFINITY;                    // running max of the raw logits
+  float neg_ms = 0.f;                     // -M * scale2 (0 while M = -inf, so that -inf logits give e = 0)
+  uint64_t Sa = pack2(0.f, 0.f), Sb = Sa; // two packed partial sums
+  int raw_idx = -1;
+  top.init();
+  float best_nat = -INFINITY;             // lower bound of the best noisy score seen by this warp
+  float K = INFINITY;                     // skip an element iff floor(2^24 (1 - u')) >= e_i * K
+  PhiloxKeys keys;
+  if (NOISE) keys.init(P.seed_lo, P.seed_hi);
+  int iter = 0;
+  // uniform trip count per block (the warp shares its bound with shuffles inside the loop)
+  for (int base = lo; base < hi; base += kThreads * 8, ++iter) {
+    const int e = base + threadIdx.x * 8;
+    const bool valid = e < hi;
+    float l[8];
+    if (valid) {
+      load8<DT>(row, e, l);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) l[i] = -INFINITY;
+    }
+    const float vmax = fmaxf(max3(l[0], l[1], l[2]), max3(max3(l[3], l[4], l[5]), l[6], l[7]));
+    if (vmax > M) {  // rare after the first iterations
+      const float f = (M == -INFINITY) ? 0.f : ex2f((M - vmax) * scale2);
+      const uint64_t f2 = pack2(f, f);
+      Sa = mul2(Sa, f2);
+      Sb = mul2(Sb, f2);
+      M = vmax;
+      neg_ms = -M * scale2;
+      if (NOISE) K = 1.002f * 0x1p24f * ex2f(M * scale2 - best_nat * kLog2e);
+      if (RAW) {
+#pragma unroll
+        for (int i = 7; i >= 0; --i)
+          if (l[i] == vmax) raw_idx = e + i;
+      }
+    }
+    const uint64_t nm2 = pack2(neg_ms, neg_ms);
+    float ex[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float x0, x1;
+      unpack2(fma2(pack2(l[2 * i], l[2 * i + 1]), scale22, nm2), x0, x1);
+      ex[2 * i] = ex2f(x0);
+      ex[2 * i + 1] = ex2f(x1);
+    }
+    Sa = add2(Sa, pack2(ex[0], ex[1]));
+    Sb = add2(Sb, pack2(ex[2], ex[3]));
+    Sa = add2(Sa, pack2(ex[4], ex[5]));
+    Sb = add2(Sb, pack2(ex[6], ex[7]));
+    if (NOISE) {
+      if (valid) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint4 rnd = keys.draw((uint32_t)(e + 4 * h) >> 2, P.step, (uint32_t)b, tagpos);
+          const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float nf = (float)((~w[i]) >> 8);  // floor(2^24 (1 - u'))
+            // -ln u' >= 1 - u' >= nf 2^-24, so g_i <= -ln(nf 2^-24): the element cannot come within
+            // 2e-3 of the running best when nf >= e_i * K
+            if (!(nf >= ex[4 * h + i] * K) && l[4 * h + i] > -INFINITY) {
+              const float sc = l[4 * h + i] * P.inv_t + gumbel_f32(w[i]);
+              top.push(sc, e + 4 * h + i);
+              if (top.s1 > best_nat) {
+                best_nat = top.s1;
+                K = 1.002f * 0x1p24f * ex2f(M * scale2 - best_nat * kLog2e);
+              }
+            }
+          }
+        }
+      }
+      if ((iter & 3) == 3) {  // share the bound inside the warp
+        float bn = best_nat;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) bn = fmaxf(bn, __shfl_xor_sync(0xffffffffu, bn, off));
+        if (bn > best_nat) {
+          best_nat = bn;
+          K = 1.002f * 0x1p24f * ex2f(M * scale2 - best_nat * kLog2e);
+        }
+      }
+    }
+  }
+  float s0, s1, s2, s3;
+  unpack2(Sa, s0, s1);
+  unpack2(Sb, s2, s3);
+  S_out = (s0 + s1) + (s2 + s3);
+  m_nat = M * P.inv_t;
+  if (RAW) {
+    top.init();
+    top.push(M, raw_idx);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Pass 1: row statistics + decision
 // ------------------------------------------------------------------------------------------------
@@ -150,96 +306,14 @@ __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParam
   int lo, hi;
   chunk_range(P.V, P.row_splits, split, lo, hi);
 
-  const float scale2 = P.inv_t * kLog2e;  // logits -> log2 domain
-  float M2 = -INFINITY, S = 0.f;          // online softmax in the log2 domain
-  float raw_best = -INFINITY;
-  int raw_idx = -1;
+  float m_nat, S;
   Top2 top;
-  top.init();
-  float best_nat = -INFINITY;  // lower bound of the best noisy score seen by this warp
-  float K = INFINITY;          // skip an element iff (2^24 (1-u') floor) >= e_i * K
-  int iter = 0;
-
-  // uniform trip count per block (the warp shares its bound with shuffles inside the loop)
-  for (int base = lo; base < hi; base += kThreads * 8, ++iter) {
-    const int e = base + threadIdx.x * 8;
-    const bool valid = e < hi;
-    float l[8];
-    if (valid) {
-      load8<DT>(row, e, l);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) l[i] = -INFINITY;
-    }
-    float x2[8];
-    float vmax = -INFINITY;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      x2[i] = l[i] * scale2;
-      vmax = fmaxf(vmax, x2[i]);
-    }
-    if (vmax > M2) {
-      S *= ex2f(M2 - vmax);  // M2 = -inf gives 0 * S(=0)
-      if (noise) K = 1.002f * 0x1p24f * ex2f(vmax - best_nat * kLog2e);
-      M2 = vmax;
-    }
-    float ex[8];
-    if (M2 > -INFINITY) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        ex[i] = ex2f(x2[i] - M2);
-        S += ex[i];
-      }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) ex[i] = 0.f;
-    }
-    if (raw_argmax) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (l[i] > raw_best) { raw_best = l[i]; raw_idx = e + i; }
-      }
-    }
-    if (noise) {
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        if (!valid) break;
-        const uint4 rnd = philox4x32_10((uint32_t)(e + 4 * h) >> 2, P.step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
-        const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float nf = (float)((~w[i]) >> 8);  // floor(2^24 (1 - u'))
-          // -ln u' >= 1 - u' >= nf 2^-24, so g_i <= -ln(nf 2^-24); the element cannot come within
-          // 2e-3 of the running best when nf >= ex[i] * K
-          if (!(nf >= ex[4 * h + i] * K) && l[4 * h + i] > -INFINITY) {
-            const float s = l[4 * h + i] * P.inv_t + gumbel_f32(w[i]);
-            top.push(s, e + 4 * h + i);
-            if (top.s1 > best_nat) {
-              best_nat = top.s1;
-              K = 1.002f * 0x1p24f * ex2f(M2 - best_nat * kLog2e);
-            }
-          }
-        }
-      }
-      if ((iter & 3) == 3) {  // share the bound inside the warp
-        float bn = best_nat;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) bn = fmaxf(bn, __shfl_xor_sync(0xffffffffu, bn, off));
-        if (bn > best_nat) {
-          best_nat = bn;
-          K = 1.002f * 0x1p24f * ex2f(M2 - best_nat * kLog2e);
-        }
-      }
-    }
-  }
+  if (noise) row_pass<DT, true, false>(P, row, lo, hi, b, tagpos, m_nat, S, top);
+  else if (raw_argmax) row_pass<DT, false, true>(P, row, lo, hi, b, tagpos, m_nat, S, top);
+  else row_pass<DT, false, false>(P, row, lo, hi, b, tagpos, m_nat, S, top);
 
   // ---- block reduction -> partial
-  float m_nat = M2 * kLn2;  // back to natural-log units of the scaled logits
   block_merge_lse(m_nat, S, sm_f0, sm_f1);
-  if (raw_argmax) {
-    top.init();
-    top.push(raw_best, raw_idx);
-  }
   block_merge_top2(top, sm_f0, sm_i0, sm_f1, sm_i1);
   if (threadIdx.x == 0) {
     RowPartial rp;
@@ -557,3 +631,4 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   }
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }
+
