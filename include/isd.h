@@ -218,6 +218,35 @@ int isd_read_status(isd_ctx* ctx, uint32_t* host_status, void* cuda_stream);
 int isd_set_profile_events(isd_ctx* ctx, void* attn_start, void* attn_stop, void* verify_start,
                            void* verify_stop);
 
+/*
+ * isd_verify without any allocation (the paper has no counterpart; this serves hosts of the
+ * library).  Same computation, arguments and outputs as isd_verify, but it needs no isd_ctx: the
+ * scratch of the two verification kernels lives in a fixed array inside the library's device image
+ * (about 0.8 MB on every GPU that loads the library, held until the process exits).
+ *
+ * Who needs it: callers that cannot call cudaMalloc when they verify -- an engine that has given
+ * all free device memory to its own KV-cache allocator, a latency-critical thread on which
+ * allocation is forbidden, or code running while the allocator is held elsewhere.  The call uses
+ * no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ * Limits and rules
+ *   - cfg->batch <= ISD_STATIC_MAX_BATCH, otherwise ISD_ERR_TOO_LARGE (nothing is launched).
+ *     Only the fields of cfg that verification reads matter (batch, stride, vocab, logits_dtype,
+ *     q_mode, propose_mode, inv_temperature, tau, seed).
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current) and caches it; make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents; the counters that
+ *     must start at zero are cleared on the stream at the start of every call.  Two calls that
+ *     overlap on the GPU (different streams, or different host threads on one device) race on it:
+ *     serialise them.
+ *   - Data faults are reported in slot_status[b] only; there is no global status word to read.
+ */
+#define ISD_STATIC_MAX_BATCH 64
+#define ISD_ERR_TOO_LARGE (-6)
+int isd_verify_static(const isd_config* cfg, const isd_batch_state* st, const void* logits_cur,
+                      const void* q_prev_logits, uint64_t step, const isd_verify_out* out,
+                      void* cuda_stream);
+
 /* Number of kernel launches the library has issued through this context. */
 int64_t isd_launch_count(const isd_ctx* ctx);
 

@@ -1,6 +1,6 @@
 """B200-native ISD step (introspective strided decoding): C-ABI CUDA library + thin binding."""
 from .binding import (Isd, IsdError, IsdBatchState, IsdConfig, IsdStepArgs, IsdVerifyOut,
-                      alloc_verify_out, load, LIB_PATH, EXPORTS)
+                      alloc_verify_out, isd_verify_static, load, LIB_PATH, EXPORTS)
 from . import workloads
 
 

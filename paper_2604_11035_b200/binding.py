@@ -18,7 +18,8 @@ ST_POOL_EXHAUSTED, ST_SLOT_CAPACITY, ST_BAD_TOKEN_ID = 1, 2, 4
 ST_BAD_PAGE_ID, ST_NONFINITE_LOGIT, ST_EMPTY_RESIDUAL = 8, 16, 32
 
 EXPORTS = ["isd_create", "isd_destroy", "isd_attn", "isd_verify", "isd_commit", "isd_step",
-           "isd_release", "isd_read_status", "isd_set_profile_events", "isd_launch_count", "isd_strerror"]
+           "isd_release", "isd_read_status", "isd_set_profile_events", "isd_launch_count", "isd_strerror",
+           "isd_verify_static"]
 
 
 class IsdConfig(C.Structure):
@@ -68,6 +69,9 @@ def load():
         lib.isd_read_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         lib.isd_set_profile_events.argtypes = [vp] * 5
         lib.isd_set_profile_events.restype = C.c_int
+        lib.isd_verify_static.argtypes = [C.POINTER(IsdConfig), C.POINTER(IsdBatchState), vp, vp, C.c_uint64,
+                                          C.POINTER(IsdVerifyOut), vp]
+        lib.isd_verify_static.restype = C.c_int
         lib.isd_launch_count.argtypes = [vp]
         lib.isd_launch_count.restype = C.c_int64
         lib.isd_strerror.argtypes = [C.c_int]
@@ -107,6 +111,14 @@ def alloc_verify_out(B: int, N: int, device) -> dict:
         accept_len=torch.zeros(B, **i32), n_emit=torch.zeros(B, **i32), repl_tok=torch.zeros(B, **i32),
         out_tok=torch.zeros(B, N, **i32), new_prop_tok=torch.zeros(B, NP, **i32),
         new_q_stats=torch.zeros(B, NP, 2, dtype=torch.float32, device=device))
+
+
+def isd_verify_static(cfg: IsdConfig, st: dict, logits_cur, q_prev_logits, step: int, out: dict):
+    """isd_verify for callers that must not allocate device memory: no context, the scratch is a fixed
+    array inside the library (batch <= 64).  Calls must not overlap on the GPU; see include/isd.h."""
+    s, o = Isd.state_struct(st), Isd.out_struct(out)
+    _check(load().isd_verify_static(C.byref(cfg), C.byref(s), _ptr(logits_cur), _ptr(q_prev_logits), step,
+                                    C.byref(o), _stream()), "isd_verify_static")
 
 
 class Isd:

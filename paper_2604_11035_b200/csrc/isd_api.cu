@@ -208,6 +208,7 @@ const char* isd_strerror(int code) {
     case ISD_ERR_CUDA: return "CUDA runtime error";
     case ISD_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
     case ISD_ERR_NO_MEMORY: return "out of memory";
+    case ISD_ERR_TOO_LARGE: return "batch exceeds ISD_STATIC_MAX_BATCH, the capacity of the static scratch of isd_verify_static";
     default: return "unknown error";
   }
 }

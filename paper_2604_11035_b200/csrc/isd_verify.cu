@@ -632,3 +632,108 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }
 
+// ------------------------------------------------------------------------------------------------
+// isd_verify_static: the same two verification kernels, for callers that must not allocate.
+//
+// Some hosts of this library cannot call cudaMalloc at the point where they verify: a serving
+// engine that has handed every free byte of the device to its own KV-cache allocator, a runtime
+// that forbids allocation on its latency-critical thread, or code that runs while another component
+// holds the allocator.  isd_create (which owns the scratch of isd_verify) is closed to them.  For
+// those callers the scratch lives in the fixed device array below, which every GPU that loads the
+// library keeps until the process exits, and the entry point touches neither cudaMalloc/cudaFree
+// nor any allocating library routine.
+//
+// Capacity: at most ISD_STATIC_MAX_BATCH slots (any stride the library supports).  Larger batches
+// are refused with ISD_ERR_TOO_LARGE before anything is launched.
+// ------------------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace {
+
+constexpr int kStaticMaxBatch = ISD_STATIC_MAX_BATCH;
+constexpr int kStaticMaxSplits = 16;
+constexpr size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+// layout of the array: [zeroed every call: tickets, reject positions, status word][partials]
+constexpr size_t kOffRowTicket = 0;
+constexpr size_t kOffResidTicket = kOffRowTicket + align256(sizeof(int) * kStaticMaxBatch);
+constexpr size_t kOffRejectPos = kOffResidTicket + align256(sizeof(int) * kStaticMaxBatch);
+constexpr size_t kOffStatus = kOffRejectPos + align256(sizeof(int) * kStaticMaxBatch);
+constexpr size_t kZeroedBytes = kOffStatus + align256(sizeof(uint32_t));
+constexpr size_t kOffLse = kZeroedBytes;
+constexpr size_t kOffResidPart = kOffLse + align256(sizeof(float) * kStaticMaxBatch);
+constexpr size_t kOffRowPart = kOffResidPart + align256(sizeof(ResidPartial) * kStaticMaxBatch * kStaticMaxSplits);
+constexpr size_t kStaticBytes = kOffRowPart + align256(sizeof(RowPartial) * kStaticMaxBatch * ISD_MAX_Q * kStaticMaxSplits);
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kMaxDevices] = {};
+
+}  // namespace
+
+// File-scope device array (about 0.8 MB per GPU).  In host code this name is only a handle for
+// cudaGetSymbolAddress; it is never passed to a kernel directly.
+static __device__ __align__(256) unsigned char g_isd_verify_static_scratch[kStaticBytes];
+
+extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* st, const void* logits_cur,
+                                 const void* q_prev_logits, uint64_t step, const isd_verify_out* out,
+                                 void* cuda_stream) {
+  if (!cfg || !st || !out || !logits_cur || step > 0xFFFFFFFFull) return ISD_ERR_INVALID_ARG;
+  const isd_config& c = *cfg;
+  if (c.batch < 1 || c.stride < 1 || c.vocab < 8 || c.inv_temperature <= 0.f || c.tau < 0.f) return ISD_ERR_INVALID_ARG;
+  if (c.logits_dtype != ISD_LOGITS_F32 && c.logits_dtype != ISD_LOGITS_BF16) return ISD_ERR_INVALID_ARG;
+  if (c.q_mode < 0 || c.q_mode > 1 || c.propose_mode < 0 || c.propose_mode > 1) return ISD_ERR_INVALID_ARG;
+  if (2 * c.stride - 1 > ISD_MAX_Q || c.vocab % 8 != 0) return ISD_ERR_UNSUPPORTED;
+  if (c.batch > kStaticMaxBatch) return ISD_ERR_TOO_LARGE;
+  if (!st->n_ver || !st->active || !st->block_tok || !st->q_row0 || !st->slot_status) return ISD_ERR_INVALID_ARG;
+  if (c.stride > 1 && (!st->q_stats || !out->accept || !out->alpha || !out->new_prop_tok || !out->new_q_stats))
+    return ISD_ERR_INVALID_ARG;
+  if (!out->accept_len || !out->n_emit || !out->repl_tok || !out->out_tok) return ISD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(logits_cur) & 15u) || (reinterpret_cast<uintptr_t>(q_prev_logits) & 15u))
+    return ISD_ERR_ALIGNMENT;
+
+  // one-time set-up per device: resolve the device address of the scratch array with that device current
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ISD_ERR_CUDA;
+  unsigned char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_isd_verify_static_scratch) != cudaSuccess || !p) return ISD_ERR_CUDA;
+      g_static_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    base = g_static_ptr[dev];
+  }
+
+  // a context on the host stack that points into the static array; nothing is allocated
+  isd_ctx tmp = {};
+  tmp.cfg = c;
+  tmp.device = dev;
+  tmp.Q = 2 * c.stride - 1;
+  tmp.G = 1;
+  int sms = 0;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  tmp.num_sms = sms > 0 ? sms : ISD_NUM_SMS_DEFAULT;
+  const int rows = c.batch * tmp.Q, target = tmp.num_sms * 4;
+  const int max_by_len = (c.vocab + 8191) / 8192;
+  int rs = (target + rows - 1) / rows;
+  rs = rs < 1 ? 1 : (rs > kStaticMaxSplits ? kStaticMaxSplits : rs);
+  rs = rs > max_by_len ? max_by_len : rs;
+  int ps = (target + c.batch - 1) / c.batch;
+  ps = ps < 1 ? 1 : (ps > kStaticMaxSplits ? kStaticMaxSplits : ps);
+  ps = ps > max_by_len ? max_by_len : ps;
+  tmp.row_splits = rs;
+  tmp.resid_splits = ps;
+  tmp.row_ticket = reinterpret_cast<int*>(base + kOffRowTicket);
+  tmp.resid_ticket = reinterpret_cast<int*>(base + kOffResidTicket);
+  tmp.reject_pos = reinterpret_cast<int*>(base + kOffRejectPos);
+  tmp.global_status = reinterpret_cast<uint32_t*>(base + kOffStatus);
+  tmp.lse_p_rej = reinterpret_cast<float*>(base + kOffLse);
+  tmp.resid_part = reinterpret_cast<ResidPartial*>(base + kOffResidPart);
+  tmp.row_part = reinterpret_cast<RowPartial*>(base + kOffRowPart);
+
+  // the array keeps the previous call's contents: counters and flags must start at zero
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(base, 0, kZeroedBytes, stream) != cudaSuccess) return ISD_ERR_CUDA;
+  return isd_launch_verify(&tmp, st, logits_cur, q_prev_logits, (uint32_t)step, out, stream);
+}
