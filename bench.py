@@ -120,6 +120,10 @@ def run_ours(args):
     K, W = args.steps, args.warmup
     from dataclasses import replace
     w = replace(w, steps=max(w.steps, K + W + args.e2e_steps + 2))
+    if args.sequential_pages:
+        w = replace(w, shuffle_pages=False, name=w.name + "[sequential pages]")
+    if args.batch:
+        w = replace(w, batch=args.batch, name=w.name + f"[batch {args.batch}]")
     st = wl.make_state(w, dev)
     eng = pkg.isd_for_workload(w, st)
     out = pkg.alloc_verify_out(w.batch, w.stride, dev)
@@ -375,6 +379,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-slots", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (smaller captures under ncu)")
+    ap.add_argument("--sequential-pages", action="store_true", help="identity page order instead of a shuffled pool")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

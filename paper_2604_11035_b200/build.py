@@ -28,6 +28,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
     if verbose:
         flags += ["-Xptxas", "-v"]
+    if os.environ.get("ISD_DEBUG_TIMING"):
+        flags += ["-DISD_DEBUG_TIMING"]
     objs = []
     procs = []
     for src in SOURCES:

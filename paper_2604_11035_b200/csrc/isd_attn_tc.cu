@@ -5,18 +5,21 @@
 //   * GQA packing: the G = Hq/Hkv query heads that share a KV head and the q_len block rows form one
 //     M = 128 row tile (row m = r * G + head-in-group), so each KV byte is read once per step.
 //   * KV pages (16 tokens x 128 dims, 4 KiB per head) are staged by TMA (cp.async.bulk.tensor, no
-//     multicast) into a 4-deep shared-memory ring in the 128-byte-swizzled layout tcgen05 consumes;
+//     multicast) into a 6-deep shared-memory ring in the 128-byte-swizzled layout tcgen05 consumes;
 //     one 128-key tile = 8 pages.
 //   * S = Q K^T and O += P V run on the 5th-gen tensor cores (tcgen05.mma, cta_group::1, M=128,
 //     N=128, K=16, bf16 -> fp32) with accumulators in TMEM; S is double-buffered so that the
-//     softmax of tile j overlaps the QK^T of tile j+1.
+//     softmax of tile j overlaps the QK^T of tile j+1.  Both A operands live in TMEM (Q for QK^T,
+//     P -- written over its own S tile -- for PV), so shared memory holds nothing but the KV ring and
+//     each MMA fetches only its 4 KiB B operand from it.
 //   * Softmax: 128 threads, one TMEM lane (= row) each, so row max / sum need no shuffles; the
 //     running maximum is only raised when it grows by more than 2^8 (lazy rescale of O in TMEM).
 //   * Persistent CTAs, one per SM.  All (slot, kv-head) KV ranges are laid end to end in units of
 //     128-key tiles and cut into equal contiguous shares, so every CTA streams the same number of
 //     bytes; a share's ragged first/last pieces go to a small fp32 scratch and are merged by a
 //     second kernel (log-sum-exp combine).  Nothing waits on another CTA.
-//   * Warp roles: warps 0-3 softmax/epilogue, warp 4 TMA producer, warp 5 MMA issuer.
+//   * Warp roles: warps 0-3 softmax/epilogue, warps 4-6 TMA producers (round-robin over the ring
+//     stages: issuing the 16 copies of a stage costs one warp about a microsecond), warp 7 MMA issuer.
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises ISD_ST_KERNEL_TIMEOUT in the global status
 // word, stops issuing work, drains, frees its TMEM and returns.
@@ -31,21 +34,25 @@ namespace {
 
 constexpr int kTile = 128;                 // keys per tile
 constexpr int kStageBytes = 32768;         // one K or V tile: [half(2)][page(8)][tok(16)][128 B]
-constexpr int kStages = 4;
-constexpr int kThreads = 192;
-constexpr int kSmQ = 0;                    // [half(2)][row group(16)][8 rows][128 B]
-constexpr int kSmP = 32768;                // 2 buffers, same layout over keys
-constexpr int kSmRing = 98304;
-constexpr int kSmBar = kSmRing + kStages * kStageBytes;  // 229376
-constexpr int kSmemBytes = kSmBar + 256;
+constexpr int kStages = 6;
+constexpr int kThreads = 256;
+constexpr int kProducerWarps = 3;        // warps 4..6 issue the TMA copies round-robin, warp 7 issues the MMAs
+constexpr int kSmRing = 0;
+constexpr int kSmBar = kSmRing + kStages * kStageBytes;  // 196608
+constexpr int kSmMl = kSmBar + 256;     // [128][2] floats: (max, sum) of every replica row at segment end
+constexpr int kSmXchg = kSmMl + 1024;   // [3][32 rows] or [1][64 rows] x 32 floats: rows handed to replica 0
+// TMEM columns (512 allocated): S double buffer (P, as bf16 pairs, overwrites the first 64 columns of
+// its S buffer once the scores are in registers), O, and the query block Q (bf16 pairs, 64 columns)
+constexpr uint32_t kTmS = 0, kTmO = 256, kTmQ = 384;
+constexpr int kSmemBytes = kSmXchg + 12288;
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
 // barrier slots (8 bytes each) inside the barrier block
-enum { BAR_FULL = 0, BAR_EMPTY = kStages, BAR_SFULL = 2 * kStages, BAR_SEMPTY = 2 * kStages + 2,
-       BAR_PFULL = 2 * kStages + 4, BAR_ODONE = 2 * kStages + 6, BAR_OFREE = 2 * kStages + 8,
-       BAR_QFULL = 2 * kStages + 9, BAR_COUNT = 2 * kStages + 10 };
+enum { BAR_FULL = 0, BAR_EMPTY = kStages, BAR_SFULL = 2 * kStages,
+       BAR_PFULL = 2 * kStages + 2, BAR_ODONE = 2 * kStages + 4, BAR_OFREE = 2 * kStages + 6,
+       BAR_QFULL = 2 * kStages + 7, BAR_COUNT = 2 * kStages + 8 };
 
 struct TcParams {
   int B, Q, N, Hq, Hkv, G, max_pages, num_pages;
@@ -88,6 +95,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+#ifdef ISD_DEBUG_TIMING
+// cycles spent waiting, per CTA: [0] producer on EMPTY, [1] MMA on K FULL, [2] MMA on V FULL, [3] MMA on
+// S buffer free, [4] MMA on P ready, [5] softmax on S ready, [6] softmax busy, [7] total
+__device__ unsigned long long g_isd_dbg[160 * 12];
+#define DBG_T0() const long long _t0 = clock64()
+#define DBG_ADD(slot) dbg_acc[slot] += clock64() - _t0
+#else
+#define DBG_T0()
+#define DBG_ADD(slot)
+#endif
+
 // Bounded wait: returns false (and raises the abort flag) when the limit is reached.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
@@ -104,12 +122,32 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
 
+// One lane of a converged warp; unlike `lane == 0` the compiler keeps the surrounding code uniform, so
+// that MMA descriptors stay in uniform registers instead of being moved there one by one.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile(
+      "{\n.reg .b32 rx;\n.reg .pred px;\n"
+      "elect.sync rx|px, 0xffffffff;\n"
+      "selp.u32 %0, 1, 0, px;\n}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// A operand read from tensor memory (row = lane, 2 bf16 per 32-bit column), B from shared memory
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
 }
 
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
@@ -164,6 +202,15 @@ __device__ __forceinline__ float ex2f(float x) {
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
+}
+// bf16 pair of two non-negative finite floats, rounded half up, with integer ALU operations only: the
+// conversion instruction shares the transcendental unit with ex2, which is the busiest pipe of the
+// softmax warps.
+__device__ __forceinline__ uint32_t pack_bf16_alu(float a, float b) {
+  const uint32_t ra = __float_as_uint(a) + 0x8000u, rb = __float_as_uint(b) + 0x8000u;
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, 0x7632;" : "=r"(d) : "r"(ra), "r"(rb));
+  return d;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -267,6 +314,262 @@ __global__ void __launch_bounds__(1024) attn_plan_kernel(const TcParams P) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// Softmax / epilogue of one segment, executed by the 128 threads of warps 0-3 (thread = TMEM lane).
+//
+// Key split across lane groups: when a block has at most 128 / F valid rows (F = 2 or 4) the query
+// rows are replicated F times along M, and replica `part` only keeps the keys
+// [part * 128 / F, (part + 1) * 128 / F) of every tile (the others get probability 0).  Each thread then
+// evaluates 128 / F exponentials per tile instead of 128 -- the transcendental unit is the busiest pipe
+// of this kernel -- and all four schedulers share the valid rows.  The replicas are independent
+// online-softmax streams with their own running maximum; they are merged (log-sum-exp) once per
+// segment through a small shared-memory buffer, or by the combine kernel for split segments.
+// ------------------------------------------------------------------------------------------------
+struct SoftmaxCtx {
+  uint8_t* smem;
+  uint32_t bar_base;
+  volatile int* abort_flag;
+  uint32_t tmem_s0, tmem_o, tmem_q;
+  uint32_t n, seg;
+#ifdef ISD_DEBUG_TIMING
+  long long* dbg;
+#endif
+};
+
+__device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+template <int F>
+__device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment& sg, SoftmaxCtx& sc) {
+  constexpr int RG = 128 / F;  // rows per replica group
+  constexpr int C = 128 / F;   // key columns per thread and tile
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m = warp * 32 + lane;  // TMEM lane
+  const int v = m % RG, part = m / RG;
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+  volatile int* abort_flag = sc.abort_flag;
+  auto bar = [&](int i) { return sc.bar_base + 8u * (uint32_t)i; };
+#ifdef ISD_DEBUG_TIMING
+  long long* dbg_acc = sc.dbg;
+#endif
+  const int cnt = sg.j1 - sg.j0;
+  const int rows_valid = sg.q_len * P.G;
+  const int r = v / P.G, hg = v % P.G;
+  const bool row_ok = v < rows_valid;
+  // ---- stage Q (logical row v = r * G + hg, 128 bf16 = 64 packed columns) into tensor memory; padding
+  // rows are zero.  The previous segment's QK MMAs are complete (its last S tile was consumed).
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(
+        P.q + (((size_t)sg.b * P.Q + (row_ok ? r : 0)) * P.Hq + sg.g * P.G + hg) * ISD_HEAD_DIM);
+    uint32_t qv[64];
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      uint4 x = make_uint4(0, 0, 0, 0);
+      if (row_ok) x = src[c];
+      qv[4 * c] = x.x; qv[4 * c + 1] = x.y; qv[4 * c + 2] = x.z; qv[4 * c + 3] = x.w;
+    }
+    TMEM_ST32(sc.tmem_q + lane_base, qv, 0);
+    TMEM_ST32(sc.tmem_q + lane_base + 32, qv, 32);
+    tmem_wait_st();
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(BAR_QFULL));
+  }
+  float m2 = -INFINITY, l = 0.f;  // running max (log2 domain) and sum of this (row, replica)
+  bool ok = true;
+  for (int i = 0; i < cnt && ok; ++i) {
+    const uint32_t nn = sc.n + i;
+    const int j = sg.j0 + i;
+    {
+      DBG_T0();
+      ok = mbar_wait(bar(BAR_SFULL + (nn & 1u)), (nn >> 1) & 1u, abort_flag);
+      DBG_ADD(5);
+    }
+    if (!ok) break;
+    tc_fence_after();
+    DBG_T0();
+    uint32_t sv[C];
+    const uint32_t ts = sc.tmem_s0 + (nn & 1u) * 128u + lane_base;
+#pragma unroll
+    for (int q4 = 0; q4 < C / 32; ++q4) TMEM_LD32(ts + part * C + q4 * 32, sv, q4 * 32);
+    tmem_wait_ld();
+    // ---- mask (last tiles only) and row max; independent chains of 3-input max keep the single
+    // softmax warp of each scheduler busy (no other warp hides the latency)
+    const int kb = j * kTile + part * C;
+    const int limit = row_ok ? (sg.ctx + r - kb) : -1;  // own columns c <= limit are visible
+    if (limit < C - 1) {
+#pragma unroll
+      for (int c = 0; c < C; ++c)
+        if (c > limit) sv[c] = 0xFF800000u;  // -inf
+    }
+    float mxa = -INFINITY, mxb = -INFINITY, mxc = -INFINITY, mxd = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < C; c += 8) {
+      mxa = max3(mxa, __uint_as_float(sv[c]), __uint_as_float(sv[c + 1]));
+      mxb = max3(mxb, __uint_as_float(sv[c + 2]), __uint_as_float(sv[c + 3]));
+      mxc = max3(mxc, __uint_as_float(sv[c + 4]), __uint_as_float(sv[c + 5]));
+      mxd = max3(mxd, __uint_as_float(sv[c + 6]), __uint_as_float(sv[c + 7]));
+    }
+    const float mx = fmaxf(fmaxf(mxa, mxb), fmaxf(mxc, mxd)) * P.scale2;  // log2 domain (scale2 > 0)
+    // ---- lazy rescale: raise the reference maximum only when it grows by more than 2^8
+    float m_use = m2;
+    const bool grow = mx > m2 + 8.f || (m2 == -INFINITY && mx > -INFINITY);
+    const bool any_grow = __any_sync(0xffffffffu, grow && i > 0);
+    if (grow) m_use = mx;
+    if (any_grow) {
+      // PV(nn-1) must have finished before O is touched.  PV completions alternate between two
+      // barriers: a waiter may lag one PV behind (PV(x-2) is known complete once S(x) arrived),
+      // which a single barrier's phase parity could not tell apart.
+      ok = mbar_wait(bar(BAR_ODONE + ((nn - 1u) & 1u)), ((nn - 1u) >> 1) & 1u, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      const float f = (grow && m2 > -INFINITY) ? ex2f(m2 - m_use) : 1.f;
+      uint32_t ov[32];
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        TMEM_LD32(sc.tmem_o + lane_base + q4 * 32, ov, 0);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * f);
+        TMEM_ST32(sc.tmem_o + lane_base + q4 * 32, ov, 0);
+      }
+      tmem_wait_st();
+      l *= f;
+    }
+    m2 = m_use;
+    // ---- probabilities and row sum; P (bf16 pairs) overwrites the first 64 columns of S(nn): own
+    // keys carry the probabilities, the other replicas' keys are zero
+    const float mref = (m2 == -INFINITY) ? 0.f : m2;
+    const uint64_t sc2 = pack2(P.scale2, P.scale2), nm2 = pack2(-mref, -mref);
+    uint64_t acc[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
+    uint32_t pk[64];
+#pragma unroll
+    for (int c = 0; c < 64; ++c) pk[c] = 0u;
+#pragma unroll
+    for (int c = 0; c < C / 2; ++c) {
+      float x0, x1;
+      unpack2(fma2(pack2(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1])), sc2, nm2), x0, x1);
+      const float p0 = ex2f(x0), p1 = ex2f(x1);
+      acc[c & 3] = add2(acc[c & 3], pack2(p0, p1));
+      const uint32_t w = pack_bf16_alu(p0, p1);
+      // static placement: replica `part` owns packed columns [part * C / 2, (part + 1) * C / 2)
+#pragma unroll
+      for (int pp = 0; pp < F; ++pp)
+        if (pp == part) pk[pp * (C / 2) + c] = w;
+    }
+    float lsum;
+    {
+      float a0, a1, b0, b1;
+      unpack2(add2(acc[0], acc[1]), a0, a1);
+      unpack2(add2(acc[2], acc[3]), b0, b1);
+      lsum = (a0 + a1) + (b0 + b1);
+    }
+#ifdef ISD_DEBUG_TIMING
+    const long long _t1 = clock64();
+#endif
+    TMEM_ST32(ts, pk, 0);
+    TMEM_ST32(ts + 32, pk, 32);
+    tmem_wait_st();
+#ifdef ISD_DEBUG_TIMING
+    dbg_acc[11] += clock64() - _t1;
+#endif
+    l += lsum;
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(BAR_PFULL + (nn & 1u)));
+    DBG_ADD(6);
+  }
+  if (!ok) return false;
+  // ---- epilogue: wait for the last PV, read O, write the result or the partial
+  const uint32_t last = sc.n + cnt - 1;
+  ok = mbar_wait(bar(BAR_ODONE + (last & 1u)), (last >> 1) & 1u, abort_flag);
+  if (!ok) return false;
+  tc_fence_after();
+  if (sg.part_slot >= 0) {
+    // split segment: every replica's un-normalised row goes to the scratch, the combine kernel merges
+#pragma unroll
+    for (int q4 = 0; q4 < 4; ++q4) {
+      uint32_t ov[32];
+      TMEM_LD32(sc.tmem_o + lane_base + q4 * 32, ov, 0);
+      tmem_wait_ld();
+      if (row_ok) {
+        uint4* dst = reinterpret_cast<uint4*>(P.part_o + ((size_t)sg.part_slot * 128 + m) * 128 + q4 * 32);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) dst[c] = make_uint4(ov[c * 4], ov[c * 4 + 1], ov[c * 4 + 2], ov[c * 4 + 3]);
+      }
+    }
+    if (row_ok) {
+      P.part_ml[((size_t)sg.part_slot * 128 + m) * 2 + 0] = m2;
+      P.part_ml[((size_t)sg.part_slot * 128 + m) * 2 + 1] = l;
+    }
+  } else {
+    // whole segment: merge the F replicas of a row (log-sum-exp), normalise, write bf16
+    float* sm_ml = reinterpret_cast<float*>(sc.smem + kSmMl);
+    float* sm_x = reinterpret_cast<float*>(sc.smem + kSmXchg);
+    float w = (l > 0.f) ? 1.f / l : 0.f, Mrow = m2, Lrow = l;
+    if (F > 1) {
+      sm_ml[2 * m] = m2;
+      sm_ml[2 * m + 1] = l;
+      softmax_group_sync();
+      Mrow = -INFINITY;
+#pragma unroll
+      for (int pp = 0; pp < F; ++pp) Mrow = fmaxf(Mrow, sm_ml[2 * (pp * RG + v)]);
+      Lrow = 0.f;
+#pragma unroll
+      for (int pp = 0; pp < F; ++pp) {
+        const float mp = sm_ml[2 * (pp * RG + v)], lp = sm_ml[2 * (pp * RG + v) + 1];
+        Lrow += (mp == -INFINITY) ? 0.f : lp * ex2f(mp - Mrow);
+      }
+      w = (m2 == -INFINITY || !(Lrow > 0.f)) ? 0.f : ex2f(m2 - Mrow) / Lrow;
+    }
+#pragma unroll
+    for (int q4 = 0; q4 < 4; ++q4) {
+      uint32_t ov[32];
+      TMEM_LD32(sc.tmem_o + lane_base + q4 * 32, ov, 0);
+      tmem_wait_ld();
+      float o[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) o[c] = __uint_as_float(ov[c]) * w;
+      if (F > 1) {
+        // replicas 1..F-1 hand their scaled rows to replica 0 through shared memory (32 columns a round)
+        if (part > 0) {
+          float4* dst = reinterpret_cast<float4*>(sm_x + ((size_t)(part - 1) * RG + v) * 32);
+#pragma unroll
+          for (int c = 0; c < 8; ++c) dst[c] = make_float4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+        }
+        softmax_group_sync();
+        if (part == 0) {
+#pragma unroll
+          for (int pp = 1; pp < F; ++pp) {
+            const float4* src = reinterpret_cast<const float4*>(sm_x + ((size_t)(pp - 1) * RG + v) * 32);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              const float4 t = src[c];
+              o[4 * c] += t.x; o[4 * c + 1] += t.y; o[4 * c + 2] += t.z; o[4 * c + 3] += t.w;
+            }
+          }
+        }
+        softmax_group_sync();
+      }
+      if (row_ok && part == 0) {
+        uint4* dst = reinterpret_cast<uint4*>(
+            P.out + (((size_t)sg.b * P.Q + r) * P.Hq + sg.g * P.G + hg) * ISD_HEAD_DIM + q4 * 32);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          dst[c] = make_uint4(pack_bf16(o[c * 8 + 0], o[c * 8 + 1]), pack_bf16(o[c * 8 + 2], o[c * 8 + 3]),
+                              pack_bf16(o[c * 8 + 4], o[c * 8 + 5]), pack_bf16(o[c * 8 + 6], o[c * 8 + 7]));
+      }
+    }
+    if (row_ok && part == 0 && P.lse)
+      P.lse[((size_t)sg.b * P.Q + r) * P.Hq + sg.g * P.G + hg] = (Mrow + log2f(Lrow)) * kLn2;
+  }
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar(BAR_OFREE));
+  sc.n += cnt;
+  ++sc.seg;
+  return true;
+}
+
+// ------------------------------------------------------------------------------------------------
 // Main kernel
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads, 1)
@@ -287,7 +590,7 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   // ---- setup: barriers, TMEM, zero the ring (stale V rows of a ragged tile must be finite)
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_SFULL + i), 1); mbar_init(bar(BAR_SEMPTY + i), 4); mbar_init(bar(BAR_PFULL + i), 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_SFULL + i), 1); mbar_init(bar(BAR_PFULL + i), 4); }
     mbar_init(bar(BAR_ODONE), 1);
     mbar_init(bar(BAR_ODONE + 1), 1);
     mbar_init(bar(BAR_OFREE), 4);
@@ -308,10 +611,17 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_s0 = tmem, tmem_o = tmem + 256;
+#ifdef ISD_DEBUG_TIMING
+  long long dbg_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  const long long dbg_start = clock64();
+  unsigned long long dbg_gt0;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(dbg_gt0));
+#endif
+  const uint32_t tmem_s0 = tmem + kTmS, tmem_o = tmem + kTmO, tmem_q = tmem + kTmQ;
 
-  if (warp == 4) {
-    // =========================================================================== TMA producer
+  if (warp >= 4 && warp < 4 + kProducerWarps) {
+    // =========================================================================== TMA producers
+    const uint32_t pw = (uint32_t)(warp - 4);  // this warp serves the fills f with f % kProducerWarps == pw
     WorkIter it;
     it.init(P, cta);
     Segment sg;
@@ -337,14 +647,23 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
         const int valid = min(8, (sg.kv_len - j * kTile + ISD_PAGE - 1) / ISD_PAGE);
         const int src = ((i >> 2) == cur_c) ? ids_cur : ids_nxt;
         const uint32_t s = fill % kStages, ph = (fill / kStages) & 1u;
-        if (!mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag)) return false;
-        if (lane == 0) mbar_arrive_expect_tx(bar(BAR_FULL + s), (uint32_t)valid * 4096u);
-        __syncwarp();
-        const int pg = lane >> 1, half = lane & 1;
-        const int pid = __shfl_sync(0xffffffffu, src, ((i & 3) << 3) + (pg & 7));
-        if (lane < 16 && pg < valid) {
-          const uint32_t dst = sm_base + kSmRing + s * kStageBytes + half * 16384 + pg * 2048;
-          tma_load_3d(dst, is_v ? &tmap_v : &tmap_k, half * 64, 0, pid * P.Hkv + sg.g, bar(BAR_FULL + s));
+        if (fill % kProducerWarps == pw) {
+          {
+            DBG_T0();
+            if (!mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag)) return false;
+            DBG_ADD(0);
+          }
+          DBG_T0();
+          if (lane == 0) mbar_arrive_expect_tx(bar(BAR_FULL + s), (uint32_t)valid * 4096u);
+          __syncwarp();
+          const int pg = lane >> 1, half = lane & 1;
+          const int pid = __shfl_sync(0xffffffffu, src, ((i & 3) << 3) + (pg & 7));
+          if (lane < 16 && pg < valid) {
+            const uint32_t dst = sm_base + kSmRing + s * kStageBytes + half * 16384 + pg * 2048;
+            tma_load_3d(dst, is_v ? &tmap_v : &tmap_k, half * 64, 0, pid * P.Hkv + sg.g, bar(BAR_FULL + s));
+          }
+          __syncwarp();
+          DBG_ADD(3);
         }
         ++fill;
         if (is_v && (i & 3) == 3) {  // V(i) is the last user of chunk i / 4
@@ -367,7 +686,7 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
       for (uint32_t f = (fill > kStages ? fill - kStages : 0); f < fill; ++f)
         mbar_wait(bar(BAR_FULL + f % kStages), (f / kStages) & 1u, abort_flag);
     }
-  } else if (warp == 5) {
+  } else if (warp == 7) {
     // =========================================================================== MMA issuer
     WorkIter it;
     it.init(P, cta);
@@ -383,42 +702,56 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
       tc_fence_after();
       auto qk = [&](uint32_t nn) -> bool {
         const uint32_t s = cons % kStages, ph = (cons / kStages) & 1u;
-        if (!mbar_wait(bar(BAR_FULL + s), ph, abort_flag)) return false;
-        if (nn >= 2 && !mbar_wait(bar(BAR_SEMPTY + (nn & 1u)), ((nn >> 1) - 1u) & 1u, abort_flag)) return false;
+        {
+          DBG_T0();
+          if (!mbar_wait(bar(BAR_FULL + s), ph, abort_flag)) return false;
+          DBG_ADD(1);
+        }
+        // S[nn & 1] is free: QK(nn) follows PV(nn-2) in issue order, and PV(nn-2) was issued only after
+        // the softmax warps had read S(nn-2) and stored P(nn-2) over it
         tc_fence_after();
-        if (lane == 0) {
+        DBG_T0();
+        if (elect_one()) {
           const uint32_t kb = sm_base + kSmRing + s * kStageBytes;
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
+          for (int k = 0; k < 8; ++k) {  // 16 dims = 8 packed columns of Q per step
             const uint32_t off = (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u;
-            tc_mma(tmem_s0 + (nn & 1u) * 128u, smem_desc(sm_base + kSmQ + off, 16, 1024),
-                   smem_desc(kb + off, 16, 1024), idesc_qk, k > 0);
+            tc_mma_ts(tmem_s0 + (nn & 1u) * 128u, tmem_q + (uint32_t)k * 8u, smem_desc(kb + off, 16, 1024), idesc_qk, k > 0);
           }
           tc_commit(bar(BAR_EMPTY + s));
           tc_commit(bar(BAR_SFULL + (nn & 1u)));
         }
+        DBG_ADD(8);
         __syncwarp();
         ++cons;
         return true;
       };
       auto pv = [&](uint32_t nn, bool first) -> bool {
         const uint32_t s = cons % kStages, ph = (cons / kStages) & 1u;
-        if (!mbar_wait(bar(BAR_FULL + s), ph, abort_flag)) return false;
-        if (!mbar_wait(bar(BAR_PFULL + (nn & 1u)), (nn >> 1) & 1u, abort_flag)) return false;
+        {
+          DBG_T0();
+          if (!mbar_wait(bar(BAR_FULL + s), ph, abort_flag)) return false;
+          DBG_ADD(2);
+        }
+        {
+          DBG_T0();
+          if (!mbar_wait(bar(BAR_PFULL + (nn & 1u)), (nn >> 1) & 1u, abort_flag)) return false;
+          DBG_ADD(4);
+        }
         if (first && seg > 0 && !mbar_wait(bar(BAR_OFREE), (seg - 1u) & 1u, abort_flag)) return false;
         tc_fence_after();
-        if (lane == 0) {
+        DBG_T0();
+        if (elect_one()) {
           const uint32_t vb = sm_base + kSmRing + s * kStageBytes;
-          const uint32_t pb = sm_base + kSmP + (nn & 1u) * 32768u;
+          const uint32_t pt_ = tmem_s0 + (nn & 1u) * 128u;
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint32_t aoff = (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u;
-            tc_mma(tmem_o, smem_desc(pb + aoff, 16, 1024), smem_desc(vb + (uint32_t)k * 2048u, 16384, 1024),
-                   idesc_pv, !(first && k == 0));
-          }
+          for (int k = 0; k < 8; ++k)  // 16 keys = 8 packed columns of P per step
+            tc_mma_ts(tmem_o, pt_ + (uint32_t)k * 8u, smem_desc(vb + (uint32_t)k * 2048u, 16384, 1024),
+                      idesc_pv, !(first && k == 0));
           tc_commit(bar(BAR_EMPTY + s));
           tc_commit(bar(BAR_ODONE + (nn & 1u)));
         }
+        DBG_ADD(9);
         __syncwarp();
         ++cons;
         return true;
@@ -431,172 +764,40 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
       n += cnt;
       ++seg;
     }
-  } else {
+  } else if (warp < 4) {
     // =========================================================================== softmax / epilogue
     WorkIter it;
     it.init(P, cta);
     Segment sg;
-    uint32_t n = 0, seg = 0;
-    const int row = warp * 32 + lane;          // TMEM lane = row of the M = 128 tile
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    SoftmaxCtx sc;
+    sc.smem = smem; sc.bar_base = bar_base; sc.abort_flag = abort_flag;
+    sc.tmem_s0 = tmem_s0; sc.tmem_o = tmem_o; sc.tmem_q = tmem_q;
+    sc.n = 0; sc.seg = 0;
+#ifdef ISD_DEBUG_TIMING
+    sc.dbg = dbg_acc;
+#endif
     bool ok = true;
     while (ok && it.next(P, cta, sg) && !*abort_flag) {
-      const int cnt = sg.j1 - sg.j0;
       const int rows_valid = sg.q_len * P.G;
-      const int r = row / P.G, hg = row % P.G;
-      const bool row_ok = row < rows_valid;
-      // ---- stage Q (rows m = r * G + hg) into the swizzled K-major layout; padding rows stay zero
-      {
-        // previous segment's QK MMAs are complete (its last S tile was consumed), so Q may be overwritten
-        const uint4* src = reinterpret_cast<const uint4*>(
-            P.q + (((size_t)sg.b * P.Q + (row_ok ? r : 0)) * P.Hq + sg.g * P.G + hg) * ISD_HEAD_DIM);
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          uint4 v = make_uint4(0, 0, 0, 0);
-          if (row_ok) v = src[c];
-          const int half = c >> 3, cc = c & 7;
-          uint8_t* dst = smem + kSmQ + half * 16384 + (row >> 3) * 1024 + (row & 7) * 128 + ((cc ^ (row & 7)) << 4);
-          *reinterpret_cast<uint4*>(dst) = v;
-        }
-        fence_async_smem();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_QFULL));
-      }
-      float m2 = -INFINITY, l = 0.f;  // running max (log2 domain) and sum of this row
-      for (int i = 0; i < cnt && ok; ++i) {
-        const uint32_t nn = n + i;
-        const int j = sg.j0 + i;
-        ok = mbar_wait(bar(BAR_SFULL + (nn & 1u)), (nn >> 1) & 1u, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t sv[128];
-        const uint32_t ts = tmem_s0 + (nn & 1u) * 128u + lane_base;
-        TMEM_LD32(ts, sv, 0);
-        TMEM_LD32(ts + 32, sv, 32);
-        TMEM_LD32(ts + 64, sv, 64);
-        TMEM_LD32(ts + 96, sv, 96);
-        tmem_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_SEMPTY + (nn & 1u)));
-        // ---- scale, mask, row max
-        const int kb = j * kTile;
-        const int limit = row_ok ? (sg.ctx + r - kb) : -1;  // columns c <= limit are visible
-        float mx = -INFINITY;
-        if (limit >= kTile - 1) {
-#pragma unroll
-          for (int c = 0; c < 128; ++c) {
-            const float x = __uint_as_float(sv[c]) * P.scale2;
-            sv[c] = __float_as_uint(x);
-            mx = fmaxf(mx, x);
-          }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 128; ++c) {
-            const float x = c <= limit ? __uint_as_float(sv[c]) * P.scale2 : -INFINITY;
-            sv[c] = __float_as_uint(x);
-            mx = fmaxf(mx, x);
-          }
-        }
-        // ---- lazy rescale: raise the reference maximum only when it grows by more than 2^8
-        float m_use = m2;
-        const bool grow = mx > m2 + 8.f || (m2 == -INFINITY && mx > -INFINITY);
-        const bool any_grow = __any_sync(0xffffffffu, grow && i > 0);
-        if (grow) m_use = mx;
-        if (any_grow) {
-          // PV(nn-1) must have finished before O is touched.  PV completions alternate between two
-          // barriers: a waiter may lag one PV behind (PV(x-2) is known complete once S(x) arrived),
-          // which a single barrier's phase parity could not tell apart.
-          ok = mbar_wait(bar(BAR_ODONE + ((nn - 1u) & 1u)), ((nn - 1u) >> 1) & 1u, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const float f = (grow && m2 > -INFINITY) ? ex2f(m2 - m_use) : 1.f;
-          uint32_t ov[32];
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            TMEM_LD32(tmem_o + lane_base + q4 * 32, ov, 0);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * f);
-            TMEM_ST32(tmem_o + lane_base + q4 * 32, ov, 0);
-          }
-          tmem_wait_st();
-          l *= f;
-        } else if (grow) {
-          // first tile of the segment (nothing accumulated yet)
-          l = 0.f;
-        }
-        m2 = m_use;
-        // ---- probabilities, row sum, P tile (bf16, swizzled K-major) for the PV MMA
-        const float mref = (m2 == -INFINITY) ? 0.f : m2;
-        uint8_t* pbase = smem + kSmP + (nn & 1u) * 32768 + (row >> 3) * 1024 + (row & 7) * 128;
-        float lsum = 0.f;
-#pragma unroll
-        for (int c16 = 0; c16 < 16; ++c16) {
-          uint32_t pk[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float p0 = ex2f(__uint_as_float(sv[c16 * 8 + 2 * e]) - mref);
-            const float p1 = ex2f(__uint_as_float(sv[c16 * 8 + 2 * e + 1]) - mref);
-            lsum += p0 + p1;
-            pk[e] = pack_bf16(p0, p1);
-          }
-          const int half = c16 >> 3, cc = c16 & 7;
-          *reinterpret_cast<uint4*>(pbase + half * 16384 + ((cc ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-        }
-        l += lsum;
-        fence_async_smem();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_PFULL + (nn & 1u)));
-      }
-      if (!ok) break;
-      // ---- epilogue: wait for the last PV, read O, write the result or the partial
-      const uint32_t last = n + cnt - 1;
-      ok = mbar_wait(bar(BAR_ODONE + (last & 1u)), (last >> 1) & 1u, abort_flag);
-      if (!ok) break;
-      tc_fence_after();
-      const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
-#pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        uint32_t ov[32];
-        TMEM_LD32(tmem_o + lane_base + q4 * 32, ov, 0);
-        tmem_wait_ld();
-        if (row_ok) {
-          if (sg.part_slot < 0) {
-            uint4* dst = reinterpret_cast<uint4*>(
-                P.out + (((size_t)sg.b * P.Q + r) * P.Hq + sg.g * P.G + hg) * ISD_HEAD_DIM + q4 * 32);
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-              dst[c] = make_uint4(pack_bf16(__uint_as_float(ov[c * 8 + 0]) * inv_l, __uint_as_float(ov[c * 8 + 1]) * inv_l),
-                                  pack_bf16(__uint_as_float(ov[c * 8 + 2]) * inv_l, __uint_as_float(ov[c * 8 + 3]) * inv_l),
-                                  pack_bf16(__uint_as_float(ov[c * 8 + 4]) * inv_l, __uint_as_float(ov[c * 8 + 5]) * inv_l),
-                                  pack_bf16(__uint_as_float(ov[c * 8 + 6]) * inv_l, __uint_as_float(ov[c * 8 + 7]) * inv_l));
-          } else {
-            uint4* dst = reinterpret_cast<uint4*>(P.part_o + ((size_t)sg.part_slot * 128 + row) * 128 + q4 * 32);
-#pragma unroll
-            for (int c = 0; c < 8; ++c) dst[c] = make_uint4(ov[c * 4], ov[c * 4 + 1], ov[c * 4 + 2], ov[c * 4 + 3]);
-          }
-        }
-      }
-      if (row_ok) {
-        if (sg.part_slot < 0) {
-          if (P.lse) P.lse[((size_t)sg.b * P.Q + r) * P.Hq + sg.g * P.G + hg] = (m2 + log2f(l)) * kLn2;
-        } else {
-          P.part_ml[((size_t)sg.part_slot * 128 + row) * 2 + 0] = m2;
-          P.part_ml[((size_t)sg.part_slot * 128 + row) * 2 + 1] = l;
-        }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_OFREE));
-      n += cnt;
-      ++seg;
+      if (rows_valid > 64) ok = softmax_segment<1>(P, sg, sc);
+      else if (rows_valid > 32) ok = softmax_segment<2>(P, sg, sc);
+      else ok = softmax_segment<4>(P, sg, sc);
     }
   }
 
   // ---- teardown
+#ifdef ISD_DEBUG_TIMING
+  if (lane == 0 && (warp == 0 || warp >= 4)) {
+    dbg_acc[7] = clock64() - dbg_start;
+    if (warp == 0) {
+      unsigned long long gt1;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1));
+      dbg_acc[2] = (long long)(gt1 - dbg_gt0);  // nanoseconds (slot 2 of warp 0 is otherwise unused)
+    }
+    for (int i = 0; i < 12; ++i)
+      if (dbg_acc[i]) g_isd_dbg[cta * 12 + i] = dbg_acc[i];
+  }
+#endif
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
@@ -620,21 +821,27 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const TcParams P) {
   if (c_first == c_last) return;  // written directly by one CTA
   const int q_len = P.n_ver[b] + P.N;
   const int rows_valid = q_len * P.G;
+  // replicas of a row (key split across lane groups, see softmax_segment) are further partials
+  const int F = rows_valid > 64 ? 1 : (rows_valid > 32 ? 2 : 4);
+  const int RG = 128 / F;
   for (int row = threadIdx.x >> 5; row < rows_valid; row += 4) {
     const int lane = threadIdx.x & 31;
     float M = -INFINITY;
     for (int c = c_first; c <= c_last; ++c) {
       const int slot = c * 2 + (((long long)c * per >= p0) ? 0 : 1);
-      M = fmaxf(M, P.part_ml[((size_t)slot * 128 + row) * 2]);
+      for (int pp = 0; pp < F; ++pp) M = fmaxf(M, P.part_ml[((size_t)slot * 128 + pp * RG + row) * 2]);
     }
     float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
     for (int c = c_first; c <= c_last; ++c) {
       const int slot = c * 2 + (((long long)c * per >= p0) ? 0 : 1);
-      const float m = P.part_ml[((size_t)slot * 128 + row) * 2], l = P.part_ml[((size_t)slot * 128 + row) * 2 + 1];
-      const float w = (m == -INFINITY) ? 0.f : ex2f(m - M);
-      L += l * w;
-      const float4 o = *reinterpret_cast<const float4*>(P.part_o + ((size_t)slot * 128 + row) * 128 + lane * 4);
-      acc[0] += o.x * w; acc[1] += o.y * w; acc[2] += o.z * w; acc[3] += o.w * w;
+      for (int pp = 0; pp < F; ++pp) {
+        const size_t rr = (size_t)slot * 128 + pp * RG + row;
+        const float m = P.part_ml[rr * 2], l = P.part_ml[rr * 2 + 1];
+        const float w = (m == -INFINITY) ? 0.f : ex2f(m - M);
+        L += l * w;
+        const float4 o = *reinterpret_cast<const float4*>(P.part_o + rr * 128 + lane * 4);
+        acc[0] += o.x * w; acc[1] += o.y * w; acc[2] += o.z * w; acc[3] += o.w * w;
+      }
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
     const int r = row / P.G, hg = row % P.G;
@@ -683,6 +890,12 @@ struct TcHost {
 };
 
 }  // namespace
+
+#ifdef ISD_DEBUG_TIMING
+extern "C" int isd_debug_timing(unsigned long long* host_out, int n) {
+  return cudaMemcpyFromSymbol(host_out, g_isd_dbg, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 int isd_attn_tc_create(isd_ctx* ctx) {
   TcHost* h = new (std::nothrow) TcHost();
