@@ -30,6 +30,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         flags += ["-Xptxas", "-v"]
     if os.environ.get("ISD_DEBUG_TIMING"):
         flags += ["-DISD_DEBUG_TIMING"]
+    if os.environ.get("ISD_EXTRA_DEFS"):
+        flags += os.environ["ISD_EXTRA_DEFS"].split()
     objs = []
     procs = []
     for src in SOURCES:

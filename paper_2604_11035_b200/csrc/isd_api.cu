@@ -78,9 +78,9 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   rs = rs > 16 ? 16 : rs;
   rs = rs > max_by_len ? max_by_len : rs;
   ctx->row_splits = rs;
-  int ps = (target + c.batch - 1) / c.batch;
-  ps = ps < 1 ? 1 : ps;
-  ps = ps > 16 ? 16 : ps;
+  // rejections are sparse at realistic accept rates and the CTAs of slots without one exit at once,
+  // so the residual pass is always cut as finely as the row length allows
+  int ps = 16;
   ps = ps > max_by_len ? max_by_len : ps;
   ctx->resid_splits = ps;
 

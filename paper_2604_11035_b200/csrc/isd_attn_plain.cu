@@ -31,9 +31,9 @@ __device__ __forceinline__ int slot_q_len(const AttnParams& P, int b) {
   return nv + P.N;
 }
 
-// one CTA per slot: validate the slot's page-table prefix, then scatter the block rows
+// one CTA per (slot, kv head): validate the slot's page-table prefix, then scatter the block rows
 __global__ void __launch_bounds__(128) kv_append_kernel(const AttnParams P) {
-  const int b = blockIdx.x;
+  const int b = blockIdx.x, g = blockIdx.y;
   const int ql = slot_q_len(P, b);
   if (ql == 0) return;
   const int ctx = P.ctx_len[b];
@@ -42,7 +42,7 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const AttnParams P) {
   if (threadIdx.x == 0) sm_bad = 0;
   __syncthreads();
   if (ctx < 0 || pages > P.max_pages) {
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0 && g == 0) {
       atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
       atomicOr(P.global_status, ISD_ST_SLOT_CAPACITY);
     }
@@ -54,19 +54,18 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const AttnParams P) {
   }
   __syncthreads();
   if (sm_bad) {
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0 && g == 0) {
       atomicOr(&P.slot_status[b], ISD_ST_BAD_PAGE_ID);
       atomicOr(P.global_status, ISD_ST_BAD_PAGE_ID);
     }
     return;
   }
-  // each (row, kv head, K|V) is 256 bytes = 16 x 16-byte vectors
-  const int vecs = ql * P.Hkv * 2 * 16;
+  // each (row, K|V) of this head is 256 bytes = 16 x 16-byte vectors
+  const int vecs = ql * 2 * 16;
   for (int i = threadIdx.x; i < vecs; i += blockDim.x) {
     const int v16 = i & 15;
     const int kv = (i >> 4) & 1;
-    const int g = (i >> 5) % P.Hkv;
-    const int r = (i >> 5) / P.Hkv;
+    const int r = i >> 5;
     const int pos = ctx + r;
     const int page = P.page_table[(size_t)b * P.max_pages + pos / ISD_PAGE];
     const size_t src = (((size_t)b * P.Q + r) * P.Hkv + g) * ISD_HEAD_DIM;
@@ -79,12 +78,11 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const AttnParams P) {
   // tensor-core kernel multiplies them by a zero probability, which needs finite values.
   const int end = ctx + ql;
   const int tail = (ISD_PAGE - end % ISD_PAGE) % ISD_PAGE;
-  const int zvecs = tail * P.Hkv * 2 * 16;
+  const int zvecs = tail * 2 * 16;
   for (int i = threadIdx.x; i < zvecs; i += blockDim.x) {
     const int v16 = i & 15;
     const int kv = (i >> 4) & 1;
-    const int g = (i >> 5) % P.Hkv;
-    const int pos = end + (i >> 5) / P.Hkv;
+    const int pos = end + (i >> 5);
     const int page = P.page_table[(size_t)b * P.max_pages + pos / ISD_PAGE];
     const size_t dst = (((size_t)page * P.Hkv + g) * ISD_PAGE + (pos % ISD_PAGE)) * ISD_HEAD_DIM;
     reinterpret_cast<uint4*>((kv ? P.v_pool : P.k_pool) + dst)[v16] = make_uint4(0, 0, 0, 0);
@@ -167,7 +165,7 @@ AttnParams make_params(isd_ctx* ctx, const isd_batch_state* st, const void* q, c
 int isd_launch_kv_append(isd_ctx* ctx, const isd_batch_state* st, const void* k_new, const void* v_new,
                          void* k_pool, void* v_pool, cudaStream_t stream) {
   AttnParams P = make_params(ctx, st, nullptr, k_new, v_new, k_pool, v_pool, nullptr, nullptr);
-  kv_append_kernel<<<ctx->cfg.batch, 128, 0, stream>>>(P);
+  kv_append_kernel<<<dim3(ctx->cfg.batch, ctx->cfg.n_kv_heads), 128, 0, stream>>>(P);
   ctx->launches++;
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }

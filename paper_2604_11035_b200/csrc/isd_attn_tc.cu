@@ -44,7 +44,9 @@ constexpr int kSmXchg = kSmMl + 1024;   // [3][32 rows] or [1][64 rows] x 32 flo
 // TMEM columns (512 allocated): S double buffer (P, as bf16 pairs, overwrites the first 64 columns of
 // its S buffer once the scores are in registers), O, and the query block Q (bf16 pairs, 64 columns)
 constexpr uint32_t kTmS = 0, kTmO = 256, kTmQ = 384;
-constexpr int kSmemBytes = kSmXchg + 12288;
+constexpr int kSmPrefix = kSmXchg + 12288;  // tile prefix over slots when the batch fits (else it stays in global memory)
+constexpr int kMaxSmemPrefixSlots = 1024;
+constexpr int kSmemBytes = kSmPrefix + (kMaxSmemPrefixSlots + 1) * 4 + 12;
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -229,8 +231,8 @@ struct WorkIter {
   const int* prefix;
   int B, Hkv, b;
   long long t, t_begin, t_end;
-  __device__ void init(const TcParams& P, int cta) {
-    prefix = P.tile_prefix;
+  __device__ void init(const TcParams& P, int cta, const int* prefix_) {
+    prefix = prefix_;
     B = P.B; Hkv = P.Hkv;
     const long long total = (long long)prefix[B] * Hkv;
     const long long per = (total + P.num_ctas - 1) / P.num_ctas;
@@ -265,8 +267,55 @@ struct WorkIter {
   }
 };
 
+__device__ __forceinline__ int slot_tiles(const TcParams& P, int b) {
+  if (b >= P.B || !P.active[b]) return 0;
+  const int nv = P.n_ver[b];
+  const int ctx = P.ctx_len[b];
+  const bool ok = nv >= 0 && nv <= P.N - 1 && ctx >= 0 &&
+                  (P.slot_status[b] & (ISD_ST_BAD_PAGE_ID | ISD_ST_SLOT_CAPACITY)) == 0;
+  return ok ? (ctx + nv + P.N + kTile - 1) / kTile : 0;
+}
+
+// Exclusive prefix of tiles per slot, computed by the 256 threads of a main-kernel CTA into shared
+// memory (batches up to kMaxSmemPrefixSlots); CTA 0 also publishes it for the combine kernel.
+__device__ void block_tile_prefix(const TcParams& P, int* sm_prefix, int* sm_warp, bool publish) {
+  int carry = 0;
+  for (int base = 0; base < P.B; base += kThreads) {
+    const int b = base + threadIdx.x;
+    const int tiles = slot_tiles(P, b);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = tiles;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
+    }
+    if (lane == 31) sm_warp[warp] = inc;
+    __syncthreads();
+    int woff = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) {
+      const int x = sm_warp[w];
+      if (w < warp) woff += x;
+      tot += x;
+    }
+    if (b < P.B) {
+      const int excl = carry + woff + inc - tiles;
+      sm_prefix[b] = excl;
+      if (publish) P.tile_prefix[b] = excl;
+    }
+    carry += tot;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    sm_prefix[P.B] = carry;
+    if (publish) P.tile_prefix[P.B] = carry;
+  }
+  __syncthreads();
+}
+
 // ------------------------------------------------------------------------------------------------
-// Plan: tiles per slot (per kv head) and their exclusive prefix, one CTA
+// Plan for batches too large for the in-kernel prefix: tiles per slot and their exclusive prefix
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) attn_plan_kernel(const TcParams P) {
   __shared__ int sm_warp[33];
@@ -275,14 +324,7 @@ __global__ void __launch_bounds__(1024) attn_plan_kernel(const TcParams P) {
   __syncthreads();
   for (int base = 0; base < P.B; base += 1024) {
     const int b = base + threadIdx.x;
-    int tiles = 0;
-    if (b < P.B && P.active[b]) {
-      const int nv = P.n_ver[b];
-      const int ctx = P.ctx_len[b];
-      const bool ok = nv >= 0 && nv <= P.N - 1 && ctx >= 0 &&
-                      (P.slot_status[b] & (ISD_ST_BAD_PAGE_ID | ISD_ST_SLOT_CAPACITY)) == 0;
-      if (ok) tiles = (ctx + nv + P.N + kTile - 1) / kTile;
-    }
+    const int tiles = slot_tiles(P, b);
     // inclusive scan
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int inc = tiles;
@@ -611,6 +653,12 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  const int* prefix = P.tile_prefix;
+  if (P.B <= kMaxSmemPrefixSlots) {
+    int* sm_prefix = reinterpret_cast<int*>(smem + kSmPrefix);
+    block_tile_prefix(P, sm_prefix, reinterpret_cast<int*>(smem + kSmMl), cta == 0);
+    prefix = sm_prefix;
+  }
 #ifdef ISD_DEBUG_TIMING
   long long dbg_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
   const long long dbg_start = clock64();
@@ -623,7 +671,7 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
     // =========================================================================== TMA producers
     const uint32_t pw = (uint32_t)(warp - 4);  // this warp serves the fills f with f % kProducerWarps == pw
     WorkIter it;
-    it.init(P, cta);
+    it.init(P, cta, prefix);
     Segment sg;
     uint32_t fill = 0;
     while (it.next(P, cta, sg) && !*abort_flag) {
@@ -689,7 +737,7 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   } else if (warp == 7) {
     // =========================================================================== MMA issuer
     WorkIter it;
-    it.init(P, cta);
+    it.init(P, cta, prefix);
     Segment sg;
     uint32_t cons = 0, n = 0, seg = 0;
     const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
@@ -767,7 +815,7 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   } else if (warp < 4) {
     // =========================================================================== softmax / epilogue
     WorkIter it;
-    it.init(P, cta);
+    it.init(P, cta, prefix);
     Segment sg;
     SoftmaxCtx sc;
     sc.smem = smem; sc.bar_base = bar_base; sc.abort_flag = abort_flag;
@@ -810,21 +858,33 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
 // ------------------------------------------------------------------------------------------------
 // Combine: pairs whose tiles were split over several CTAs (log-sum-exp merge of the partials)
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) attn_combine_kernel(const TcParams P) {
-  const int g = blockIdx.x, b = blockIdx.y;
-  const int T = P.tile_prefix[b + 1] - P.tile_prefix[b];
-  if (T == 0) return;
+// One CTA per share of the main kernel: CTA c merges the pair that starts inside share c and runs on
+// into later shares (every split pair has exactly one such share).
+__global__ void __launch_bounds__(256) attn_combine_kernel(const TcParams P) {
+  const int c0 = blockIdx.x;
   const long long total = (long long)P.tile_prefix[P.B] * P.Hkv;
+  if (total == 0) return;
   const long long per = (total + P.num_ctas - 1) / P.num_ctas;
+  const long long t_last = ((long long)(c0 + 1) * per < total ? (long long)(c0 + 1) * per : total) - 1;
+  if (t_last < (long long)c0 * per) return;  // empty share
+  // slot and kv head of the share's last tile
+  int lo = 0, hi = P.B;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if ((long long)P.tile_prefix[mid + 1] * P.Hkv > t_last) hi = mid; else lo = mid + 1;
+  }
+  const int b = lo;
+  const int T = P.tile_prefix[b + 1] - P.tile_prefix[b];
+  const int g = (int)((t_last - (long long)P.tile_prefix[b] * P.Hkv) / T);
   const long long p0 = (long long)P.tile_prefix[b] * P.Hkv + (long long)g * T, p1 = p0 + T;
   const int c_first = (int)(p0 / per), c_last = (int)((p1 - 1) / per);
-  if (c_first == c_last) return;  // written directly by one CTA
+  if (c_first != c0 || c_last == c0) return;  // merged by an earlier share, or written directly
   const int q_len = P.n_ver[b] + P.N;
   const int rows_valid = q_len * P.G;
   // replicas of a row (key split across lane groups, see softmax_segment) are further partials
   const int F = rows_valid > 64 ? 1 : (rows_valid > 32 ? 2 : 4);
   const int RG = 128 / F;
-  for (int row = threadIdx.x >> 5; row < rows_valid; row += 4) {
+  for (int row = threadIdx.x >> 5; row < rows_valid; row += 8) {
     const int lane = threadIdx.x & 31;
     float M = -INFINITY;
     for (int c = c_first; c <= c_last; ++c) {
@@ -946,11 +1006,11 @@ int isd_launch_attn_tc(isd_ctx* ctx, const isd_batch_state* st, const void* q, c
   P.q = (const __nv_bfloat16*)q; P.out = (__nv_bfloat16*)out; P.lse = lse;
   P.tile_prefix = h->tile_prefix; P.part_o = ctx->attn_part_o; P.part_ml = ctx->attn_part_ml;
   P.num_ctas = ctx->attn_ctas;
-  attn_plan_kernel<<<1, 1024, 0, stream>>>(P);
+  if (c.batch > kMaxSmemPrefixSlots) attn_plan_kernel<<<1, 1024, 0, stream>>>(P);
   if (ctx->ev_attn0) cudaEventRecord(ctx->ev_attn0, stream);
   attn_tc_kernel<<<ctx->attn_ctas, kThreads, kSmemBytes, stream>>>(P, h->map_k, h->map_v);
   if (ctx->ev_attn1) cudaEventRecord(ctx->ev_attn1, stream);
-  attn_combine_kernel<<<dim3(c.n_kv_heads, c.batch), 128, 0, stream>>>(P);
-  ctx->launches += 3;
+  attn_combine_kernel<<<ctx->attn_ctas, 256, 0, stream>>>(P);
+  ctx->launches += 2 + (c.batch > kMaxSmemPrefixSlots ? 1 : 0);
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }

@@ -158,6 +158,71 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
+// 2^x for a pair of non-positive arguments without the transcendental unit, which both streaming kernels
+// saturate: round to the nearest integer with the 1.5 * 2^23 trick, evaluate a polynomial of the
+// remainder f in [-0.5, 0.5] with packed FMAs, and add the integer to the exponent field.
+// DEG = 5: relative error < 3e-7 (as good as ex2.approx); DEG = 3: < 1.1e-4 (enough for bf16 results).
+// Arguments below -125 (including -inf) give a value below 2^-124, i.e. zero for every use here.
+template <int DEG>
+__device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& r0, float& r1) {
+  const float c0 = fmaxf(x0, -125.f), c1 = fmaxf(x1, -125.f);
+  const uint64_t xc = pack2(c0, c1);
+  const uint64_t magic = pack2(12582912.f, 12582912.f), nmagic = pack2(-12582912.f, -12582912.f);
+  const uint64_t t = add2(xc, magic);                       // magic + round(x)
+  const uint64_t f = fma2(add2(t, nmagic), pack2(-1.f, -1.f), xc);  // x - round(x)
+  uint64_t p;
+  if (DEG == 5) {
+    p = pack2(0.0013400432653725147f, 0.0013400432653725147f);
+    p = fma2(p, f, pack2(0.009676037356257439f, 0.009676037356257439f));
+    p = fma2(p, f, pack2(0.05550327152013779f, 0.05550327152013779f));
+    p = fma2(p, f, pack2(0.2402210682630539f, 0.2402210682630539f));
+    p = fma2(p, f, pack2(0.6931471824645996f, 0.6931471824645996f));
+    p = fma2(p, f, pack2(1.0000001192092896f, 1.0000001192092896f));
+  } else {
+    p = pack2(0.05592203512787819f, 0.05592203512787819f);
+    p = fma2(p, f, pack2(0.24264007806777954f, 0.24264007806777954f));
+    p = fma2(p, f, pack2(0.6931210160255432f, 0.6931210160255432f));
+    p = fma2(p, f, pack2(0.9999244809150696f, 0.9999244809150696f));
+  }
+  float t0, t1, p0, p1;
+  unpack2(t, t0, t1);
+  unpack2(p, p0, p1);
+  r0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+  r1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
+
+// -------------------------------------------------------------------------------------------------
+// mbarrier / bulk-copy helpers for shared-memory rings (one producer thread, many consumers)
+// -------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t ring_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void ring_mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void ring_mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void ring_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait on a phase parity; false when the limit expires (the caller raises a status bit and leaves).
+__device__ __forceinline__ bool ring_mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < (1u << 24); ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+// Contiguous global -> shared copy (16-byte aligned addresses, size a multiple of 16) that signals `bar`.
+__device__ __forceinline__ void ring_bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
 // Ordering of (score, index) candidates: higher score wins, ties go to the lower index.
 __device__ __forceinline__ bool cand_better(float sa, int ia, float sb, int ib) {
   if (ib < 0) return ia >= 0;

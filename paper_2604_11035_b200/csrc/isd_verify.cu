@@ -689,8 +689,7 @@ extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* s
   int rs = (target + rows - 1) / rows;
   rs = rs < 1 ? 1 : (rs > kStaticMaxSplits ? kStaticMaxSplits : rs);
   rs = rs > max_by_len ? max_by_len : rs;
-  int ps = (target + c.batch - 1) / c.batch;
-  ps = ps < 1 ? 1 : (ps > kStaticMaxSplits ? kStaticMaxSplits : ps);
+  int ps = kStaticMaxSplits;
   ps = ps > max_by_len ? max_by_len : ps;
   tmp.row_splits = rs;
   tmp.resid_splits = ps;
