@@ -80,7 +80,10 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   ctx->row_splits = rs;
   // rejections are sparse at realistic accept rates and the CTAs of slots without one exit at once,
   // so the residual pass is always cut as finely as the row length allows
-  int ps = 16;
+#ifndef ISD_RESID_SPLITS
+#define ISD_RESID_SPLITS 4
+#endif
+  int ps = ISD_RESID_SPLITS;
   ps = ps > max_by_len ? max_by_len : ps;
   ctx->resid_splits = ps;
 

@@ -469,6 +469,13 @@ __global__ void __launch_bounds__(kThreads) verify_resid_kernel(const VerifyPara
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       if (!valid) break;
+      // Cheap pre-filter before any random number is drawn: ln r_i <= ln p_i and no Gumbel variate on the
+      // 24-bit lattice exceeds 17.33, so a group whose four elements all have ln p_i + 17.34 below the
+      // running best cannot produce a candidate.  At realistic vocabulary sizes this skips almost all
+      // of the Philox work (only logits a few sigma above the mean survive).
+      const float cut = best_nat - 17.34f + lse_p;
+      const float gmax = fmaxf(fmaxf(lp[4 * h], lp[4 * h + 1]), fmaxf(lp[4 * h + 2], lp[4 * h + 3])) * P.inv_t;
+      if (!(gmax > cut)) continue;
       const uint4 rnd = philox4x32_10((uint32_t)(e + 4 * h) >> 2, P.step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
       const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
 #pragma unroll
@@ -491,7 +498,7 @@ __global__ void __launch_bounds__(kThreads) verify_resid_kernel(const VerifyPara
         }
       }
     }
-    if ((iter & 3) == 3) {
+    if (iter == 0 || (iter & 3) == 3) {
       float bn = best_nat;
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) bn = fmaxf(bn, __shfl_xor_sync(0xffffffffu, bn, off));
@@ -689,7 +696,7 @@ extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* s
   int rs = (target + rows - 1) / rows;
   rs = rs < 1 ? 1 : (rs > kStaticMaxSplits ? kStaticMaxSplits : rs);
   rs = rs > max_by_len ? max_by_len : rs;
-  int ps = kStaticMaxSplits;
+  int ps = 4;  // same cut as isd_create uses
   ps = ps > max_by_len ? max_by_len : ps;
   tmp.row_splits = rs;
   tmp.resid_splits = ps;
