@@ -46,7 +46,8 @@ constexpr int kSmXchg = kSmMl + 1024;   // [3][32 rows] or [1][64 rows] x 32 flo
 constexpr uint32_t kTmS = 0, kTmO = 256, kTmQ = 384;
 constexpr int kSmPrefix = kSmXchg + 12288;  // tile prefix over slots when the batch fits (else it stays in global memory)
 constexpr int kMaxSmemPrefixSlots = 1024;
-constexpr int kSmemBytes = kSmPrefix + (kMaxSmemPrefixSlots + 1) * 4 + 12;
+constexpr int kSmSlot = kSmPrefix + (kMaxSmemPrefixSlots + 1) * 4 + 12;  // per slot: ctx_len | q_len << 24 (with the prefix)
+constexpr int kSmemBytes = kSmSlot + kMaxSmemPrefixSlots * 4;
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -229,10 +230,12 @@ struct Segment {
 
 struct WorkIter {
   const int* prefix;
+  const int* slot_info;  // ctx_len | q_len << 24 per slot in shared memory, or nullptr (read the state arrays)
   int B, Hkv, b;
   long long t, t_begin, t_end;
-  __device__ void init(const TcParams& P, int cta, const int* prefix_) {
+  __device__ void init(const TcParams& P, int cta, const int* prefix_, const int* slot_info_) {
     prefix = prefix_;
+    slot_info = slot_info_;
     B = P.B; Hkv = P.Hkv;
     const long long total = (long long)prefix[B] * Hkv;
     const long long per = (total + P.num_ctas - 1) / P.num_ctas;
@@ -257,8 +260,14 @@ struct WorkIter {
     s.j0 = (int)(off % T);
     const long long room = t_end - t;
     s.j1 = (long long)(T - s.j0) <= room ? T : s.j0 + (int)room;
-    s.ctx = P.ctx_len[b];
-    s.q_len = P.n_ver[b] + P.N;
+    if (slot_info) {
+      const int w = slot_info[b];
+      s.ctx = w & 0xFFFFFF;
+      s.q_len = (int)((unsigned)w >> 24);
+    } else {
+      s.ctx = P.ctx_len[b];
+      s.q_len = P.n_ver[b] + P.N;
+    }
     s.kv_len = s.ctx + s.q_len;
     const bool whole = (s.j0 == 0 && s.j1 == T);
     s.part_slot = whole ? -1 : cta * 2 + (t == t_begin ? 0 : 1);
@@ -278,11 +287,12 @@ __device__ __forceinline__ int slot_tiles(const TcParams& P, int b) {
 
 // Exclusive prefix of tiles per slot, computed by the 256 threads of a main-kernel CTA into shared
 // memory (batches up to kMaxSmemPrefixSlots); CTA 0 also publishes it for the combine kernel.
-__device__ void block_tile_prefix(const TcParams& P, int* sm_prefix, int* sm_warp, bool publish) {
+__device__ void block_tile_prefix(const TcParams& P, int* sm_prefix, int* sm_slot, int* sm_warp, bool publish) {
   int carry = 0;
   for (int base = 0; base < P.B; base += kThreads) {
     const int b = base + threadIdx.x;
     const int tiles = slot_tiles(P, b);
+    if (b < P.B && tiles > 0) sm_slot[b] = (P.ctx_len[b] & 0xFFFFFF) | ((P.n_ver[b] + P.N) << 24);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int inc = tiles;
 #pragma unroll
@@ -572,19 +582,21 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
       for (int c = 0; c < 32; ++c) o[c] = __uint_as_float(ov[c]) * w;
       if (F > 1) {
         // replicas 1..F-1 hand their scaled rows to replica 0 through shared memory (32 columns a round)
+        // layout [replica - 1][float4 column c][row v]: consecutive threads touch consecutive 16-byte
+        // words, so neither the writes nor the reads below conflict on shared-memory banks
         if (part > 0) {
-          float4* dst = reinterpret_cast<float4*>(sm_x + ((size_t)(part - 1) * RG + v) * 32);
+          float4* dst = reinterpret_cast<float4*>(sm_x) + (size_t)(part - 1) * 8 * RG + v;
 #pragma unroll
-          for (int c = 0; c < 8; ++c) dst[c] = make_float4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+          for (int c = 0; c < 8; ++c) dst[c * RG] = make_float4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
         }
         softmax_group_sync();
         if (part == 0) {
 #pragma unroll
           for (int pp = 1; pp < F; ++pp) {
-            const float4* src = reinterpret_cast<const float4*>(sm_x + ((size_t)(pp - 1) * RG + v) * 32);
+            const float4* src = reinterpret_cast<const float4*>(sm_x) + (size_t)(pp - 1) * 8 * RG + v;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
-              const float4 t = src[c];
+              const float4 t = src[c * RG];
               o[4 * c] += t.x; o[4 * c + 1] += t.y; o[4 * c + 2] += t.z; o[4 * c + 3] += t.w;
             }
           }
@@ -654,10 +666,13 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const int* prefix = P.tile_prefix;
+  const int* slot_info = nullptr;
   if (P.B <= kMaxSmemPrefixSlots) {
     int* sm_prefix = reinterpret_cast<int*>(smem + kSmPrefix);
-    block_tile_prefix(P, sm_prefix, reinterpret_cast<int*>(smem + kSmMl), cta == 0);
+    int* sm_slot = reinterpret_cast<int*>(smem + kSmSlot);
+    block_tile_prefix(P, sm_prefix, sm_slot, reinterpret_cast<int*>(smem + kSmMl), cta == 0);
     prefix = sm_prefix;
+    slot_info = sm_slot;
   }
 #ifdef ISD_DEBUG_TIMING
   long long dbg_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
@@ -671,7 +686,7 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
     // =========================================================================== TMA producers
     const uint32_t pw = (uint32_t)(warp - 4);  // this warp serves the fills f with f % kProducerWarps == pw
     WorkIter it;
-    it.init(P, cta, prefix);
+    it.init(P, cta, prefix, slot_info);
     Segment sg;
     uint32_t fill = 0;
     while (it.next(P, cta, sg) && !*abort_flag) {
@@ -737,7 +752,7 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   } else if (warp == 7) {
     // =========================================================================== MMA issuer
     WorkIter it;
-    it.init(P, cta, prefix);
+    it.init(P, cta, prefix, slot_info);
     Segment sg;
     uint32_t cons = 0, n = 0, seg = 0;
     const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
@@ -815,7 +830,7 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   } else if (warp < 4) {
     // =========================================================================== softmax / epilogue
     WorkIter it;
-    it.init(P, cta, prefix);
+    it.init(P, cta, prefix, slot_info);
     Segment sg;
     SoftmaxCtx sc;
     sc.smem = smem; sc.bar_base = bar_base; sc.abort_flag = abort_flag;
