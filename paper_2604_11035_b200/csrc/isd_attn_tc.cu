@@ -43,7 +43,7 @@ constexpr int kSmMl = kSmBar + 256;     // [128][2] floats: (max, sum) of every 
 constexpr int kSmXchg = kSmMl + 1024;   // [3][32 rows] or [1][64 rows] x 32 floats: rows handed to replica 0
 // TMEM columns (512 allocated): S double buffer (P, as bf16 pairs, overwrites the first 64 columns of
 // its S buffer once the scores are in registers), O, and the query block Q (bf16 pairs, 64 columns)
-constexpr uint32_t kTmS = 0, kTmO = 256, kTmQ = 384;
+constexpr uint32_t kTmS = 0, kTmO = 256, kTmQ = 384;  // Q: two buffers of 64 columns (segment parity)
 constexpr int kSmPrefix = kSmXchg + 12288;  // tile prefix over slots when the batch fits (else it stays in global memory)
 constexpr int kMaxSmemPrefixSlots = 1024;
 constexpr int kSmSlot = kSmPrefix + (kMaxSmemPrefixSlots + 1) * 4 + 12;  // per slot: ctx_len | q_len << 24 (with the prefix)
@@ -389,8 +389,49 @@ struct SoftmaxCtx {
 
 __device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// Replication factor of a segment's rows along M (see softmax_segment)
+__device__ __forceinline__ int seg_replicas(const TcParams& P, const Segment& sg) {
+  const int rows_valid = sg.q_len * P.G;
+  return rows_valid > 64 ? 1 : (rows_valid > 32 ? 2 : 4);
+}
+
+__device__ __forceinline__ const __nv_bfloat16* q_row_ptr(const TcParams& P, const Segment& sg, int m, bool& row_ok) {
+  const int RG = 128 / seg_replicas(P, sg);
+  const int v = m % RG;
+  const int r = v / P.G, hg = v % P.G;
+  row_ok = v < sg.q_len * P.G;
+  return P.q + (((size_t)sg.b * P.Q + (row_ok ? r : 0)) * P.Hq + sg.g * P.G + hg) * ISD_HEAD_DIM;
+}
+
+// Stage the query block of a segment (logical row v = r * G + head-in-group, 128 bf16 = 64 packed
+// columns, replicated along M, padding rows zero) into Q buffer `seg & 1` of tensor memory and announce
+// it.  The buffer's previous user (segment seg - 2) finished its QK MMAs long ago.  Staging the next
+// segment's block right after the current segment's last P tile lets the MMA warp issue the next QK^T
+// while this segment's last PV and epilogue are still running.
+__device__ __forceinline__ void stage_q(const TcParams& P, const Segment& sg, SoftmaxCtx& sc, uint32_t seg) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+  bool row_ok;
+  const uint4* src = reinterpret_cast<const uint4*>(q_row_ptr(P, sg, warp * 32 + lane, row_ok));
+  uint32_t qv[64];
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    uint4 x = make_uint4(0, 0, 0, 0);
+    if (row_ok) x = src[c];
+    qv[4 * c] = x.x; qv[4 * c + 1] = x.y; qv[4 * c + 2] = x.z; qv[4 * c + 3] = x.w;
+  }
+  const uint32_t tq = sc.tmem_q + (seg & 1u) * 64u + lane_base;
+  TMEM_ST32(tq, qv, 0);
+  TMEM_ST32(tq + 32, qv, 32);
+  tmem_wait_st();
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(sc.bar_base + 8u * (uint32_t)BAR_QFULL);
+}
+
 template <int F>
-__device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment& sg, SoftmaxCtx& sc) {
+__device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment& sg, SoftmaxCtx& sc,
+                                                const Segment* sg_next) {
   constexpr int RG = 128 / F;  // rows per replica group
   constexpr int C = 128 / F;   // key columns per thread and tile
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -406,24 +447,13 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
   const int rows_valid = sg.q_len * P.G;
   const int r = v / P.G, hg = v % P.G;
   const bool row_ok = v < rows_valid;
-  // ---- stage Q (logical row v = r * G + hg, 128 bf16 = 64 packed columns) into tensor memory; padding
-  // rows are zero.  The previous segment's QK MMAs are complete (its last S tile was consumed).
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(
-        P.q + (((size_t)sg.b * P.Q + (row_ok ? r : 0)) * P.Hq + sg.g * P.G + hg) * ISD_HEAD_DIM);
-    uint32_t qv[64];
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-      uint4 x = make_uint4(0, 0, 0, 0);
-      if (row_ok) x = src[c];
-      qv[4 * c] = x.x; qv[4 * c + 1] = x.y; qv[4 * c + 2] = x.z; qv[4 * c + 3] = x.w;
+  if (sg_next != nullptr) {  // pull the next segment's query rows towards L2 well before they are staged
+    bool nok;
+    const __nv_bfloat16* nq = q_row_ptr(P, *sg_next, m, nok);
+    if (nok) {
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(nq));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(nq + 64));
     }
-    TMEM_ST32(sc.tmem_q + lane_base, qv, 0);
-    TMEM_ST32(sc.tmem_q + lane_base + 32, qv, 32);
-    tmem_wait_st();
-    tc_fence_before();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar(BAR_QFULL));
   }
   float m2 = -INFINITY, l = 0.f;  // running max (log2 domain) and sum of this (row, replica)
   bool ok = true;
@@ -530,6 +560,7 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
     DBG_ADD(6);
   }
   if (!ok) return false;
+  if (sg_next != nullptr) stage_q(P, *sg_next, sc, sc.seg + 1);
   // ---- epilogue: wait for the last PV, read O, write the result or the partial
   const uint32_t last = sc.n + cnt - 1;
   ok = mbar_wait(bar(BAR_ODONE + (last & 1u)), (last >> 1) & 1u, abort_flag);
@@ -779,7 +810,7 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
 #pragma unroll
           for (int k = 0; k < 8; ++k) {  // 16 dims = 8 packed columns of Q per step
             const uint32_t off = (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u;
-            tc_mma_ts(tmem_s0 + (nn & 1u) * 128u, tmem_q + (uint32_t)k * 8u, smem_desc(kb + off, 16, 1024), idesc_qk, k > 0);
+            tc_mma_ts(tmem_s0 + (nn & 1u) * 128u, tmem_q + (seg & 1u) * 64u + (uint32_t)k * 8u, smem_desc(kb + off, 16, 1024), idesc_qk, k > 0);
           }
           tc_commit(bar(BAR_EMPTY + s));
           tc_commit(bar(BAR_SFULL + (nn & 1u)));
@@ -840,11 +871,18 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
     sc.dbg = dbg_acc;
 #endif
     bool ok = true;
-    while (ok && it.next(P, cta, sg) && !*abort_flag) {
+    Segment sg_next;
+    bool have = it.next(P, cta, sg);
+    if (have) stage_q(P, sg, sc, 0);
+    while (ok && have && !*abort_flag) {
+      const bool have_next = it.next(P, cta, sg_next);
+      const Segment* nx = have_next ? &sg_next : nullptr;
       const int rows_valid = sg.q_len * P.G;
-      if (rows_valid > 64) ok = softmax_segment<1>(P, sg, sc);
-      else if (rows_valid > 32) ok = softmax_segment<2>(P, sg, sc);
-      else ok = softmax_segment<4>(P, sg, sc);
+      if (rows_valid > 64) ok = softmax_segment<1>(P, sg, sc, nx);
+      else if (rows_valid > 32) ok = softmax_segment<2>(P, sg, sc, nx);
+      else ok = softmax_segment<4>(P, sg, sc, nx);
+      sg = sg_next;
+      have = have_next;
     }
   }
 
