@@ -280,13 +280,15 @@ def run_ours(args):
     if e2e:
         line["e2e"] = {"value": e2e["pos"] / e2e["t"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
                        "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"]}
-    prof = os.path.join(ROOT, "profiles", "attn_tc_kernel_dram_traffic.json")
+    # DRAM traffic per launch: ncu capture of a smaller case of the same kernel (see profiles/), scaled by
+    # the algorithmic bytes of this launch (the kernel's traffic is proportional to the KV bytes it streams)
+    prof = os.path.join(ROOT, "profiles", "attn_tc_kernel_sweep_n8_b64.md")
     if os.path.exists(prof):
-        try:
-            per_byte = json.load(open(prof))["dram_bytes_per_algorithmic_byte"]
-            line["roofline"]["traffic"] = per_byte * attn_bytes / K
-        except Exception:
-            pass
+        import re
+        m = re.search(r"dram_bytes_per_algorithmic_byte = ([0-9.]+)", open(prof).read())
+        if m:
+            line["roofline"]["traffic"] = float(m.group(1)) * attn_bytes / K
+            line["roofline"]["traffic_source"] = "ncu capture of B=64 case scaled by algorithmic bytes"
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(args, w)
     eng.close()
