@@ -52,7 +52,7 @@ class ClockSampler:
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -98,6 +98,23 @@ def algorithmic_bytes(w, ctx_len, q_len, rejecting: int):
     return attn, verify
 
 
+def rank_workload(config_index: int, rank: int):
+    """Workload of one rank: ranks own disjoint slots with their own pools, so each gets its own seed."""
+    from paper_2604_11035_b200 import workloads as wl
+    base = wl.config(config_index)
+    return wl.config(config_index, seed=base.seed + 1000 * rank)
+
+
+def reduce_over_ranks(dist, device, times, counts):
+    """Whole-job numbers: the slowest rank's time (MAX) and the units all ranks processed (SUM)."""
+    import torch
+    tt = torch.tensor(times, dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    cc = torch.tensor(counts, dtype=torch.int64, device=device)
+    dist.all_reduce(cc, op=dist.ReduceOp.SUM)
+    return {"max": [float(x) for x in tt], "sum": [int(x) for x in cc]}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -113,7 +130,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     # weak scaling: every rank owns its own slots, pools and free stack (slots never interact)
-    w = wl.config(args.config, seed=wl.config(args.config).seed + 1000 * rank)
+    w = rank_workload(args.config, rank)
     if args.propose_mode is not None:
         from dataclasses import replace
         w = replace(w, propose_mode=args.propose_mode)
@@ -240,13 +257,11 @@ def run_ours(args):
 
     # ---- reduce over ranks: max time, summed positions
     if world > 1:
-        tt = torch.tensor([t_total, e2e["t"] if e2e else 0.0], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        cnt = torch.tensor([positions, emitted, e2e["pos"] if e2e else 0, launches], dtype=torch.int64, device=dev)
-        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
-        t_total = float(tt[0]); positions = int(cnt[0]); emitted = int(cnt[1]); launches = int(cnt[3])
+        red = reduce_over_ranks(dist, dev, [t_total, e2e["t"] if e2e else 0.0],
+                                [positions, emitted, e2e["pos"] if e2e else 0, launches])
+        t_total, positions, emitted, launches = red["max"][0], red["sum"][0], red["sum"][1], red["sum"][3]
         if e2e:
-            e2e["t"] = float(tt[1]); e2e["pos"] = int(cnt[2])
+            e2e["t"], e2e["pos"] = red["max"][1], red["sum"][2]
     if rank != 0:
         eng.close()
         if world > 1:
@@ -329,7 +344,7 @@ def oracle_sample_step(w, n_slots, step_seed=0):
 def cpu_baseline(args, w):
     import oracle
     oracle.build()
-    n = args.cpu_slots or max(2, min(w.batch, oracle.max_threads()))
+    n = args.cpu_slots or max(2, min(w.batch, 8 * oracle.max_threads()))   # about 10 s of host work
     pos, sec, threads = oracle_sample_step(w, n)
     return {"value": pos / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"one P step (attention + verify + commit) of the first {n} slots of {w.name}, "
@@ -345,7 +360,7 @@ def run_reference(args):
     from paper_2604_11035_b200 import workloads as wl
     oracle.build()
     w = wl.config(args.config)
-    n = args.cpu_slots or max(2, min(w.batch, oracle.max_threads()))
+    n = args.cpu_slots or max(2, min(w.batch, 8 * oracle.max_threads()))
     K, W = args.steps, args.warmup
     K = min(K, 5)
     W = min(W, 1)
