@@ -15,17 +15,19 @@
 //      row; CTAs of slots without a rejection exit at once (the common accept path costs one pass).
 //
 // Gumbel noise is a pure function of (seed, step, slot, tag, position, vocab index), so any
-// reduction order gives the same sample.  Noise is evaluated exactly only for elements that can
-// still win: with E = -ln u' >= 1 - u', an element whose cheap bound cannot reach the running best
-// score is skipped.  The two best candidates of a row are re-judged in fp64 when their fp32 scores
-// are closer than ISD_TIE_EPS.
+// reduction order gives the same sample.  Noise is evaluated only for elements that can still win,
+// in two stages.  (1) No variate on the 24-bit lattice exceeds 25 ln 2 = 17.33, so a group of four
+// logits whose maximum is more than 17.34 below the running best score needs no random numbers at
+// all; the groups that survive are compacted into a per-warp queue so that the Philox work runs on
+// full warps.  (2) With E = -ln u' >= 1 - u', a queued element whose cheap bound cannot reach the
+// running best is skipped before any logarithm.  The two best candidates of a row are re-judged in
+// fp64 when their fp32 scores are closer than ISD_TIE_EPS.
 #include "isd_internal.cuh"
 
 namespace {
 
 constexpr int kThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 
 struct VerifyParams {
   int B, N, Q, V;
@@ -57,22 +59,92 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
-// Eight consecutive logits starting at element e (e % 8 == 0) as fp32.
+// Order-preserving map float -> unsigned (larger float = larger code; code 0 is below every float and
+// decodes to a NaN, which fmaxf ignores): lets the running best score live behind atomicMax.
+__device__ __forceinline__ unsigned enc_ordered(float f) {
+  const unsigned b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float dec_ordered(unsigned u) {
+  return __uint_as_float((u & 0x80000000u) ? (u ^ 0x80000000u) : ~u);
+}
+
+// Eight consecutive logits as fp32 from their raw 16-byte vectors.
 template <int DT>
-__device__ __forceinline__ void load8(const void* row, int e, float (&l)[8]) {
+__device__ __forceinline__ void unpack8(const uint4* v, float (&l)[8]) {
   if (DT == ISD_LOGITS_BF16) {
-    const uint4 v = ld_stream_16B(reinterpret_cast<const uint16_t*>(row) + e);
-    l[0] = __uint_as_float(v.x << 16); l[1] = __uint_as_float(v.x & 0xFFFF0000u);
-    l[2] = __uint_as_float(v.y << 16); l[3] = __uint_as_float(v.y & 0xFFFF0000u);
-    l[4] = __uint_as_float(v.z << 16); l[5] = __uint_as_float(v.z & 0xFFFF0000u);
-    l[6] = __uint_as_float(v.w << 16); l[7] = __uint_as_float(v.w & 0xFFFF0000u);
+    const uint4 a = v[0];
+    l[0] = __uint_as_float(a.x << 16); l[1] = __uint_as_float(a.x & 0xFFFF0000u);
+    l[2] = __uint_as_float(a.y << 16); l[3] = __uint_as_float(a.y & 0xFFFF0000u);
+    l[4] = __uint_as_float(a.z << 16); l[5] = __uint_as_float(a.z & 0xFFFF0000u);
+    l[6] = __uint_as_float(a.w << 16); l[7] = __uint_as_float(a.w & 0xFFFF0000u);
   } else {
-    const uint4 a = ld_stream_16B(reinterpret_cast<const float*>(row) + e);
-    const uint4 b = ld_stream_16B(reinterpret_cast<const float*>(row) + e + 4);
+    const uint4 a = v[0], b = v[1];
     l[0] = __uint_as_float(a.x); l[1] = __uint_as_float(a.y); l[2] = __uint_as_float(a.z); l[3] = __uint_as_float(a.w);
     l[4] = __uint_as_float(b.x); l[5] = __uint_as_float(b.y); l[6] = __uint_as_float(b.z); l[7] = __uint_as_float(b.w);
   }
 }
+
+// Eight consecutive logits starting at element e (e % 8 == 0), straight from global memory.
+template <int DT>
+__device__ __forceinline__ void load8(const void* row, int e, float (&l)[8]) {
+  uint4 v[2];
+  if (DT == ISD_LOGITS_BF16) {
+    v[0] = ld_stream_16B(reinterpret_cast<const uint16_t*>(row) + e);
+  } else {
+    v[0] = ld_stream_16B(reinterpret_cast<const float*>(row) + e);
+    v[1] = ld_stream_16B(reinterpret_cast<const float*>(row) + e + 4);
+  }
+  unpack8<DT>(v, l);
+}
+
+// A row piece streamed through shared memory with per-thread asynchronous copies.  Every thread
+// fetches its own eight logits of the next kDepth iterations ahead of time (64 bytes in flight per
+// thread without holding registers) and later reads back exactly what it fetched itself, so no
+// barrier is needed.  The load latency, which bounds a pass that issues one load per iteration and
+// then computes on it, disappears behind the iterations in between.
+constexpr int kRingBytes = 16384;  // per CTA
+template <int DT>
+struct RowStream {
+  static constexpr int kVec = DT == ISD_LOGITS_BF16 ? 1 : 2;  // 16-byte vectors per thread and iteration
+  static constexpr int kDepth = kRingBytes / (kThreads * 16 * kVec);
+  static constexpr int kStep = kThreads * 8;                  // elements per iteration of the CTA
+  uint4* mine;      // this thread's vectors of stage 0; stage s is kThreads * kVec vectors further
+  const char* row;
+  int hi, stage;
+
+  __device__ __forceinline__ void fetch(int s, int e) const {
+    if (e < hi) {
+      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(mine + s * kThreads * kVec);
+      const char* src = row + (size_t)e * (DT == ISD_LOGITS_BF16 ? 2 : 4);
+#pragma unroll
+      for (int v = 0; v < kVec; ++v)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16 * v), "l"(src + 16 * v) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");  // one group per iteration, empty or not
+  }
+  __device__ __forceinline__ void start(uint4* ring, const char* row_, int lo, int hi_) {
+    mine = ring + threadIdx.x * kVec;
+    row = row_;
+    hi = hi_;
+    stage = 0;
+#pragma unroll
+    for (int s = 0; s < kDepth; ++s) fetch(s, lo + s * kStep + threadIdx.x * 8);
+  }
+  // logits of this thread at element e (the iteration that started kDepth fetches ago); refills the stage
+  __device__ __forceinline__ void next(int e, float (&l)[8]) {
+    asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
+    if (e < hi) {
+      unpack8<DT>(mine + stage * kThreads * kVec, l);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) l[i] = -INFINITY;
+    }
+    fetch(stage, e + kDepth * kStep);
+    stage = (stage + 1) & (kDepth - 1);
+  }
+  __device__ __forceinline__ void finish() const { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+};
 
 __device__ __forceinline__ void chunk_range(int V, int splits, int split, int& lo, int& hi) {
   // chunks are multiples of 8 * kThreads elements so that every thread's vector stays aligned
@@ -116,75 +188,33 @@ __device__ double noisy_score_f64(const VerifyParams& P, const void* row, int i,
   return l + gumbel_f64(philox_word(r, i & 3));
 }
 
-// Philox4x32-10 with the ten round keys precomputed (they depend on the seed only)
-struct PhiloxKeys {
-  uint32_t k0[10], k1[10];
-  __device__ __forceinline__ void init(uint32_t lo, uint32_t hi) {
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-      k0[r] = lo + (uint32_t)r * 0x9E3779B9u;
-      k1[r] = hi + (uint32_t)r * 0xBB67AE85u;
-    }
+// One streaming pass over elements [lo, hi) of a logits row: online softmax, i.e. the running max M
+// of the raw logits and S = sum exp((l - M) * invT); with RAW also the argmax of the raw logits
+// (lowest index on ties), which is the running max itself.
+// Returns m_nat = M * invT (natural-log units of the scaled logits), S and the candidate.
+struct OnlineSoftmax {
+  float M, neg_ms, scale2;
+  uint64_t Sa, Sb, scale22;
+  __device__ __forceinline__ void init(float inv_t) {
+    scale2 = inv_t * kLog2e;  // raw logit -> log2 domain
+    scale22 = pack2(scale2, scale2);
+    M = -INFINITY;            // running max of the raw logits
+    neg_ms = 0.f;             // -M * scale2 (0 while M = -inf, so that -inf logits give e = 0)
+    Sa = pack2(0.f, 0.f);     // two packed partial sums
+    Sb = Sa;
   }
-  __device__ __forceinline__ uint4 draw(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3) const {
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-      const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
-      const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
-      const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0[r];
-      const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1[r];
-      c1 = (uint32_t)p1; c3 = (uint32_t)p0; c0 = n0; c2 = n2;
-    }
-    return make_uint4(c0, c1, c2, c3);
+  // true when the maximum grew (rare after the first iterations)
+  __device__ __forceinline__ bool raise(float vmax) {
+    if (!(vmax > M)) return false;
+    const float f = (M == -INFINITY) ? 0.f : ex2f((M - vmax) * scale2);
+    const uint64_t f2 = pack2(f, f);
+    Sa = mul2(Sa, f2);
+    Sb = mul2(Sb, f2);
+    M = vmax;
+    neg_ms = -M * scale2;
+    return true;
   }
-};
-
-// One streaming pass over elements [lo, hi) of a logits row.
-//   always   online softmax: running max M of the raw logits and S = sum exp((l - M) * invT)
-//   RAW      argmax of the raw logits (lowest index on ties): the running max itself
-//   NOISE    Gumbel-max top-2 of l * invT + g with the bound-based skip
-// Returns m_nat = M * invT (natural-log units of the scaled logits), S and the candidates.
-template <int DT, bool NOISE, bool RAW>
-__device__ __forceinline__ void row_pass(const VerifyParams& P, const char* row, int lo, int hi, int b,
-                                         uint32_t tagpos, float& m_nat, float& S_out, Top2& top) {
-  const float scale2 = P.inv_t * kLog2e;  // raw logit -> log2 domain
-  const uint64_t scale22 = pack2(scale2, scale2);
-  float M = -INFINITY;                    // running max of the raw logits
-  float neg_ms = 0.f;                     // -M * scale2 (0 while M = -inf, so that -inf logits give e = 0)
-  uint64_t Sa = pack2(0.f, 0.f), Sb = Sa; // two packed partial sums
-  int raw_idx = -1;
-  top.init();
-  float best_nat = -INFINITY;             // lower bound of the best noisy score seen by this warp
-  float K = INFINITY;                     // skip an element iff floor(2^24 (1 - u')) >= e_i * K
-  PhiloxKeys keys;
-  if (NOISE) keys.init(P.seed_lo, P.seed_hi);
-  int iter = 0;
-  // uniform trip count per block (the warp shares its bound with shuffles inside the loop)
-  for (int base = lo; base < hi; base += kThreads * 8, ++iter) {
-    const int e = base + threadIdx.x * 8;
-    const bool valid = e < hi;
-    float l[8];
-    if (valid) {
-      load8<DT>(row, e, l);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) l[i] = -INFINITY;
-    }
-    const float vmax = fmaxf(max3(l[0], l[1], l[2]), max3(max3(l[3], l[4], l[5]), l[6], l[7]));
-    if (vmax > M) {  // rare after the first iterations
-      const float f = (M == -INFINITY) ? 0.f : ex2f((M - vmax) * scale2);
-      const uint64_t f2 = pack2(f, f);
-      Sa = mul2(Sa, f2);
-      Sb = mul2(Sb, f2);
-      M = vmax;
-      neg_ms = -M * scale2;
-      if (NOISE) K = 1.002f * 0x1p24f * ex2f(M * scale2 - best_nat * kLog2e);
-      if (RAW) {
-#pragma unroll
-        for (int i = 7; i >= 0; --i)
-          if (l[i] == vmax) raw_idx = e + i;
-      }
-    }
+  __device__ __forceinline__ void add8(const float (&l)[8]) {
     const uint64_t nm2 = pack2(neg_ms, neg_ms);
     float ex[8];
 #pragma unroll
@@ -198,48 +228,137 @@ __device__ __forceinline__ void row_pass(const VerifyParams& P, const char* row,
     Sb = add2(Sb, pack2(ex[2], ex[3]));
     Sa = add2(Sa, pack2(ex[4], ex[5]));
     Sb = add2(Sb, pack2(ex[6], ex[7]));
-    if (NOISE) {
-      if (valid) {
+  }
+  __device__ __forceinline__ float sum() const {
+    float s0, s1, s2, s3;
+    unpack2(Sa, s0, s1);
+    unpack2(Sb, s2, s3);
+    return (s0 + s1) + (s2 + s3);
+  }
+};
+
+template <int DT, bool RAW>
+__device__ __forceinline__ void row_pass(const VerifyParams& P, const char* row, int lo, int hi,
+                                         float& m_nat, float& S_out, Top2& top, uint4* ring) {
+  OnlineSoftmax os;
+  os.init(P.inv_t);
+  int raw_idx = -1;
+  RowStream<DT> in;
+  in.start(ring, row, lo, hi);
+  for (int base = lo; base < hi; base += kThreads * 8) {
+    const int e = base + threadIdx.x * 8;
+    float l[8];
+    in.next(e, l);
+    const float vmax = fmaxf(max3(l[0], l[1], l[2]), max3(max3(l[3], l[4], l[5]), l[6], l[7]));
+    if (os.raise(vmax) && RAW) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const uint4 rnd = keys.draw((uint32_t)(e + 4 * h) >> 2, P.step, (uint32_t)b, tagpos);
-          const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+      for (int i = 7; i >= 0; --i)
+        if (l[i] == vmax) raw_idx = e + i;
+    }
+    os.add8(l);
+  }
+  in.finish();
+  S_out = os.sum();
+  m_nat = os.M * P.inv_t;
+  top.init();
+  if (RAW) top.push(os.M, raw_idx);
+}
+
+// Per-warp queue of groups of four logits that survived the first skip test.
+constexpr int kQueueCap = 128;  // < 32 left over + at most 64 new per iteration
+struct SampleQueue {
+  float4 l[kThreads / 32][kQueueCap];
+  int idx[kThreads / 32][kQueueCap];
+};
+
+// The same pass for a Gumbel-sampled row: online softmax plus the top-2 of l * invT + g.
+template <int DT>
+__device__ __forceinline__ void row_pass_sampled(const VerifyParams& P, const char* row, int lo, int hi, int b,
+                                                 uint32_t tagpos, float& m_nat, float& S_out, Top2& top,
+                                                 SampleQueue& Q, unsigned* sm_best, uint4* ring) {
+  OnlineSoftmax os;
+  os.init(P.inv_t);
+  RowStream<DT> in;
+  in.start(ring, row, lo, hi);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned below = (1u << lane) - 1u;
+  float4* ql = Q.l[warp];
+  int* qi = Q.idx[warp];
+  const float rcp_t = 1.f / P.inv_t;
+  const float cut_off = -17.34f * rcp_t;
+  top.init();
+  // A noisy score that some element of the row really has (so a lower bound of the winner's), shared by
+  // the CTA through sm_best; a stale value only makes the skip tests weaker.
+  float best = -INFINITY;
+  int head = 0, tail = 0;  // warp-uniform queue positions
+
+  // Draw the noise of one queued group and keep its candidates.
+  auto drain = [&](int pos) {
+    const int idx = qi[pos & (kQueueCap - 1)];
+    const float4 v = ql[pos & (kQueueCap - 1)];
+    const float l4[4] = {v.x, v.y, v.z, v.w};
+    const uint4 rnd = philox4x32_10((uint32_t)idx >> 2, P.step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
+    const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+    // -ln u' >= 1 - u' >= nf 2^-24 with nf = floor(2^24 (1 - u')), so g_i <= -ln(nf 2^-24): the element
+    // cannot come within 2e-3 of the running best when nf >= 1.002 * 2^24 * exp(l_i invT - best)
+    float K2 = 24.0028853901f - best * kLog2e;  // log2 of the factor; +inf while there is no best
+    bool improved = false;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float nf = (float)((~w[i]) >> 8);  // floor(2^24 (1 - u'))
-            // -ln u' >= 1 - u' >= nf 2^-24, so g_i <= -ln(nf 2^-24): the element cannot come within
-            // 2e-3 of the running best when nf >= e_i * K
-            if (!(nf >= ex[4 * h + i] * K) && l[4 * h + i] > -INFINITY) {
-              const float sc = l[4 * h + i] * P.inv_t + gumbel_f32(w[i]);
-              top.push(sc, e + 4 * h + i);
-              if (top.s1 > best_nat) {
-                best_nat = top.s1;
-                K = 1.002f * 0x1p24f * ex2f(M * scale2 - best_nat * kLog2e);
-              }
-            }
-          }
-        }
-      }
-      if ((iter & 3) == 3) {  // share the bound inside the warp
-        float bn = best_nat;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) bn = fmaxf(bn, __shfl_xor_sync(0xffffffffu, bn, off));
-        if (bn > best_nat) {
-          best_nat = bn;
-          K = 1.002f * 0x1p24f * ex2f(M * scale2 - best_nat * kLog2e);
+    for (int i = 0; i < 4; ++i) {
+      const float nf = (float)((~w[i]) >> 8);
+      const float bound = ex2f(fmaf(l4[i], os.scale2, K2));
+      if (!(nf >= bound) && l4[i] > -INFINITY) {
+        const float sc = l4[i] * P.inv_t + gumbel_f32(w[i]);
+        top.push(sc, idx + i);
+        if (top.s1 > best) {
+          best = top.s1;
+          K2 = 24.0028853901f - best * kLog2e;
+          improved = true;
         }
       }
     }
+    if (improved) atomicMax(sm_best, enc_ordered(best));
+  };
+
+  // uniform trip count per block (the warp votes inside the loop)
+  for (int base = lo; base < hi; base += kThreads * 8) {
+    const int e = base + threadIdx.x * 8;
+    float l[8];
+    in.next(e, l);
+    best = fmaxf(best, dec_ordered(*reinterpret_cast<volatile unsigned*>(sm_best)));
+    const float cut = fmaf(best, rcp_t, cut_off);  // raw-logit units; -inf while there is no best
+    const float g0 = fmaxf(fmaxf(l[0], l[1]), fmaxf(l[2], l[3]));
+    const float g1 = fmaxf(fmaxf(l[4], l[5]), fmaxf(l[6], l[7]));
+    os.raise(fmaxf(g0, g1));
+    os.add8(l);
+    {
+      const bool p0 = g0 > cut, p1 = g1 > cut;  // false for padding and all -inf groups
+      const unsigned m0 = __ballot_sync(0xffffffffu, p0);
+      const unsigned m1 = __ballot_sync(0xffffffffu, p1);
+      if (p0) {
+        const int s = (tail + __popc(m0 & below)) & (kQueueCap - 1);
+        ql[s] = make_float4(l[0], l[1], l[2], l[3]);
+        qi[s] = e;
+      }
+      tail += __popc(m0);
+      if (p1) {
+        const int s = (tail + __popc(m1 & below)) & (kQueueCap - 1);
+        ql[s] = make_float4(l[4], l[5], l[6], l[7]);
+        qi[s] = e + 4;
+      }
+      tail += __popc(m1);
+    }
+    __syncwarp();
+    while (tail - head >= 32) {
+      drain(head + lane);
+      head += 32;
+    }
   }
-  float s0, s1, s2, s3;
-  unpack2(Sa, s0, s1);
-  unpack2(Sb, s2, s3);
-  S_out = (s0 + s1) + (s2 + s3);
-  m_nat = M * P.inv_t;
-  if (RAW) {
-    top.init();
-    top.push(M, raw_idx);
-  }
+  in.finish();
+  __syncwarp();
+  if (lane < tail - head) drain(head + lane);
+  S_out = os.sum();
+  m_nat = os.M * P.inv_t;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -247,11 +366,16 @@ __device__ __forceinline__ void row_pass(const VerifyParams& P, const char* row,
 // ------------------------------------------------------------------------------------------------
 template <int DT>
 __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParams P) {
-  const int split = blockIdx.x, r = blockIdx.y, b = blockIdx.z;
+  // Launch order = (split, slot, row class): the Gumbel-sampled rows of every slot come first.  They run
+  // several times longer than a streamed row, so starting them all at once and letting the streamed rows
+  // fill the remaining CTA slots keeps the ALU-bound and the HBM-bound work overlapped and the tail short.
+  const int split = blockIdx.x, b = blockIdx.y, k = blockIdx.z;
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
+  const int n_sampled = P.propose_mode == 0 ? P.N : 1;  // rows nv .. nv + n_sampled - 1
+  const int r = k < n_sampled ? nv + k : (k - n_sampled < nv ? k - n_sampled : k);
   if (nv < 0 || nv > P.N - 1) {
-    if (split == 0 && r == 0 && threadIdx.x == 0) {
+    if (split == 0 && k == 0 && threadIdx.x == 0) {
       atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
       atomicOr(P.global_status, ISD_ST_SLOT_CAPACITY);
     }
@@ -263,6 +387,9 @@ __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParam
   __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
   __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
   __shared__ int sm_last;
+  __shared__ unsigned sm_best;
+  __shared__ SampleQueue sm_queue;
+  __shared__ __align__(16) uint4 sm_ring[kRingBytes / 16];
 
   const bool is_final = (r == nv);
   const bool is_prop = (r > nv);
@@ -278,9 +405,15 @@ __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParam
 
   float m_nat, S;
   Top2 top;
-  if (noise) row_pass<DT, true, false>(P, row, lo, hi, b, tagpos, m_nat, S, top);
-  else if (raw_argmax) row_pass<DT, false, true>(P, row, lo, hi, b, tagpos, m_nat, S, top);
-  else row_pass<DT, false, false>(P, row, lo, hi, b, tagpos, m_nat, S, top);
+  if (noise) {
+    if (threadIdx.x == 0) sm_best = 0;
+    __syncthreads();
+    row_pass_sampled<DT>(P, row, lo, hi, b, tagpos, m_nat, S, top, sm_queue, &sm_best, sm_ring);
+  } else if (raw_argmax) {
+    row_pass<DT, true>(P, row, lo, hi, m_nat, S, top, sm_ring);
+  } else {
+    row_pass<DT, false>(P, row, lo, hi, m_nat, S, top, sm_ring);
+  }
 
   // ---- block reduction -> partial
   block_merge_lse(m_nat, S, sm_f0, sm_f1);
@@ -594,7 +727,7 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   P.row_part = ctx->row_part; P.resid_part = ctx->resid_part; P.row_ticket = ctx->row_ticket;
   P.resid_ticket = ctx->resid_ticket; P.reject_pos = ctx->reject_pos; P.lse_p_rej = ctx->lse_p_rej;
 
-  const dim3 grid1(ctx->row_splits, ctx->Q, c.batch);
+  const dim3 grid1(ctx->row_splits, c.batch, ctx->Q);
   if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
   if (c.logits_dtype == ISD_LOGITS_BF16) verify_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads, 0, stream>>>(P);
   else verify_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads, 0, stream>>>(P);
