@@ -288,7 +288,7 @@ def run_ours(args):
         "roofline": {"kernel": "attn_tc_kernel", "bound": "hbm", "achieved": attn_gbs, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": attn_gbs / peak, "frac_of_8TBs": attn_gbs / HBM_NOMINAL_GBS,
                      "traffic": None, "ms_per_launch": sum(attn_ms) / K, "bytes_per_launch": attn_bytes / K},
-        "verify_rows_kernel": {"achieved_gbs": ver_gbs, "ms_per_launch": sum(ver_ms) / K,
+        "verify_kernels": {"kernels": "verify_rows_kernel + verify_sample_kernel", "achieved_gbs": ver_gbs, "ms_per_launch": sum(ver_ms) / K,
                                "frac_of_measured_copy": (ver_gbs / peak) if ver_gbs else None},
         "gpu_launches": launches, "status_word": status, "clocks": clocks, "wall_s": wall,
     }

@@ -78,27 +78,29 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   rs = rs > 16 ? 16 : rs;
   rs = rs > max_by_len ? max_by_len : rs;
   ctx->row_splits = rs;
-  // rejections are sparse at realistic accept rates and the CTAs of slots without one exit at once,
-  // so the residual pass is always cut as finely as the row length allows
-#ifndef ISD_RESID_SPLITS
-#define ISD_RESID_SPLITS 4
+  // every slot samples one row (bonus token or residual replacement; N rows with sampled proposals)
+  // in the second pass; those passes are light, so they are cut as finely as the row length allows
+#ifndef ISD_SAMPLE_SPLITS
+#define ISD_SAMPLE_SPLITS 4
 #endif
-  int ps = ISD_RESID_SPLITS;
+  int ps = ISD_SAMPLE_SPLITS;
   ps = ps > max_by_len ? max_by_len : ps;
-  ctx->resid_splits = ps;
+  ctx->sample_splits = ps;
 
   int rc = ISD_OK;
   if (rc == ISD_OK) rc = dev_alloc(&ctx->row_part, (size_t)rows * rs);
-  if (rc == ISD_OK) rc = dev_alloc(&ctx->resid_part, (size_t)c.batch * ps);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->samp_part, (size_t)c.batch * c.stride * ps);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->row_ticket, c.batch);
-  if (rc == ISD_OK) rc = dev_alloc(&ctx->resid_ticket, c.batch);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->samp_ticket, (size_t)c.batch * c.stride);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->reject_pos, c.batch);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->row_arg, (size_t)rows);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->lse_p_rej, c.batch);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->global_status, 1);
   if (rc == ISD_OK) {
     cudaMemset(ctx->row_ticket, 0, sizeof(int) * c.batch);
-    cudaMemset(ctx->resid_ticket, 0, sizeof(int) * c.batch);
-    cudaMemset(ctx->reject_pos, 0, sizeof(int) * c.batch);
+    cudaMemset(ctx->samp_ticket, 0, sizeof(int) * c.batch * c.stride);
+    cudaMemset(ctx->reject_pos, 0xFF, sizeof(int) * c.batch);
+    cudaMemset(ctx->row_arg, 0xFF, sizeof(int) * rows);
     cudaMemset(ctx->global_status, 0, sizeof(uint32_t));
   }
   if (rc == ISD_OK && c.attn_impl == 0) rc = isd_attn_tc_create(ctx);
@@ -116,10 +118,11 @@ int isd_destroy(isd_ctx* ctx) {
   cudaDeviceSynchronize();
   isd_attn_tc_destroy(ctx);
   cudaFree(ctx->row_part);
-  cudaFree(ctx->resid_part);
+  cudaFree(ctx->samp_part);
   cudaFree(ctx->row_ticket);
-  cudaFree(ctx->resid_ticket);
+  cudaFree(ctx->samp_ticket);
   cudaFree(ctx->reject_pos);
+  cudaFree(ctx->row_arg);
   cudaFree(ctx->lse_p_rej);
   cudaFree(ctx->global_status);
   delete ctx;

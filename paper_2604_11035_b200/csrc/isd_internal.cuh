@@ -22,16 +22,14 @@
 
 // Partial result of one (slot, row, split) CTA of the row-statistics pass.
 struct RowPartial {
-  float m;      // max of scaled logits in the chunk
-  float s;      // sum of exp(l - m) over the chunk
-  float best1;  // best score (raw logit for argmax rows, l*invT + gumbel for sampled rows)
-  int idx1;
-  float best2;  // runner-up score
-  int idx2;
+  float m;        // max of the scaled logits in the chunk
+  float s;        // sum of exp(l - m) over the chunk
+  float raw_max;  // max of the raw logits in the chunk ...
+  int idx;        // ... and the lowest index that attains it (-1: none)
 };
 
-// Partial result of one (slot, split) CTA of the residual pass.
-struct ResidPartial {
+// Partial result of one (slot, sampled row, split) CTA of the sampling pass: the two best noisy scores.
+struct SamplePartial {
   float best1;
   int idx1;
   float best2;
@@ -47,12 +45,13 @@ struct isd_ctx {
   float sm_scale;
   // ---- verify scratch
   int row_splits;        // CTAs per logits row in the row pass
-  int resid_splits;      // CTAs per rejecting slot in the residual pass
+  int sample_splits;     // CTAs per sampled row in the sampling pass
   RowPartial* row_part;  // [B, Q, row_splits]
-  ResidPartial* resid_part;  // [B, resid_splits]
+  SamplePartial* samp_part;  // [B, N, sample_splits]
   int* row_ticket;       // [B] arrivals of the row pass
-  int* resid_ticket;     // [B]
-  int* reject_pos;       // [B] 0 = nothing rejected, j = first rejected proposal
+  int* samp_ticket;      // [B, N] arrivals of the sampling pass
+  int* reject_pos;       // [B] -1 = slot frozen (nothing to sample), 0 = nothing rejected, j = first rejected proposal
+  int* row_arg;          // [B, Q] argmax of every valid row (seeds the sampling pass)
   float* lse_p_rej;      // [B] LSE of the anchor row that rejected
   // ---- attention scratch
   int attn_ctas;         // persistent CTAs of the tensor-core kernel

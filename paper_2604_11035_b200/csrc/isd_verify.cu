@@ -3,38 +3,42 @@
 // online softmax and Gumbel-max correction).
 //
 // Two launches, neither of which waits on anything:
-//   1. verify_rows_kernel  one CTA per (slot, block row, split): a single streaming pass over the
-//      logits row (16-byte loads) that yields, per role of the row,
-//        anchor rows (r < n_ver)        online-softmax (max, sum)            -> LSE_p
-//        final row   (r = n_ver)        Gumbel-max top-2                      -> bonus / free token
-//        MASK rows   (r > n_ver)        (max, sum) + argmax or Gumbel top-2   -> proposals, q_stats
-//      The last CTA of a slot to finish (atomic ticket, nobody waits) merges the partials, runs the
-//      sequential accept test and writes every output except a residual replacement.
-//   2. verify_resid_kernel  only for slots whose first rejection needs a replacement drawn from
-//      normalize(max(0, p - q)): a second pass over the rejecting anchor row and the proposal-law
-//      row; CTAs of slots without a rejection exit at once (the common accept path costs one pass).
+//   1. verify_rows_kernel   one CTA per (slot, block row, split): a single streaming pass over the
+//      logits row that yields the online-softmax pair (max, sum) -> LSE and the argmax of the row.
+//      Every row has the same role here, so the kernel is a lean HBM stream.  The last CTA of a slot
+//      to finish (atomic ticket, nobody waits) merges the partials, runs the sequential accept test
+//      and writes every output that needs no random sample: accept flags, alpha, accept length, the
+//      accepted tokens, argmax proposals and the proposal-law statistics.
+//   2. verify_sample_kernel one CTA per (slot, sampled row, split).  Each slot draws exactly one
+//      token for its emission: the replacement from normalize(max(0, p - q)) when a proposal was
+//      rejected, else the bonus / free token from the row of the last clean token; with sampled
+//      proposals the N - 1 MASK rows are drawn here too.  The pass re-reads the row (mostly from L2:
+//      the rows kernel reads the rows that are sampled last).
 //
 // Gumbel noise is a pure function of (seed, step, slot, tag, position, vocab index), so any
-// reduction order gives the same sample.  Noise is evaluated only for elements that can still win,
-// in two stages.  (1) No variate on the 24-bit lattice exceeds 25 ln 2 = 17.33, so a group of four
-// logits whose maximum is more than 17.34 below the running best score needs no random numbers at
-// all; the groups that survive are compacted into a per-warp queue so that the Philox work runs on
-// full warps.  (2) With E = -ln u' >= 1 - u', a queued element whose cheap bound cannot reach the
-// running best is skipped before any logarithm.  The two best candidates of a row are re-judged in
-// fp64 when their fp32 scores are closer than ISD_TIE_EPS.
+// reduction order gives the same sample, and it is evaluated only for elements that can still win.
+// The sampling pass starts from the true noisy score of the row's argmax (known from pass 1), which
+// is a lower bound of the winner's score from the first element on.  (1) No variate on the 24-bit
+// lattice exceeds 25 ln 2 = 17.33, so a group of four logits whose maximum is more than 17.34 below
+// the running best needs no random numbers at all; the groups that survive are compacted into a
+// per-warp queue so that the Philox work runs on full warps.  (2) With E = -ln u' >= 1 - u', a
+// queued element whose cheap bound cannot reach the running best is skipped before any logarithm.
+// The two best candidates of a row are re-judged in fp64 when their fp32 scores are closer than
+// ISD_TIE_EPS.
 #include "isd_internal.cuh"
 
 namespace {
 
 constexpr int kThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kGumbelMax = 17.34f;  // > 25 ln 2, the largest variate of the 24-bit lattice
 
 struct VerifyParams {
   int B, N, Q, V;
   int logits_dtype, q_mode, propose_mode;
   float inv_t, tau;
   uint32_t seed_lo, seed_hi, step;
-  int row_splits, resid_splits;
+  int row_splits, sample_splits;
   const int32_t* n_ver;
   const uint8_t* active;
   const int32_t* block_tok;
@@ -46,12 +50,16 @@ struct VerifyParams {
   const void* q_prev;
   isd_verify_out out;
   RowPartial* row_part;
-  ResidPartial* resid_part;
+  SamplePartial* samp_part;
   int* row_ticket;
-  int* resid_ticket;
+  int* samp_ticket;
   int* reject_pos;
+  int* row_arg;
   float* lse_p_rej;
 };
+
+// rows nv .. nv + rows_sampled - 1 of a slot are drawn by the sampling pass
+__device__ __forceinline__ int rows_sampled(const VerifyParams& P) { return P.propose_mode == 0 ? P.N : 1; }
 
 __device__ __forceinline__ float ex2f(float x) {
   float y;
@@ -188,10 +196,8 @@ __device__ double noisy_score_f64(const VerifyParams& P, const void* row, int i,
   return l + gumbel_f64(philox_word(r, i & 3));
 }
 
-// One streaming pass over elements [lo, hi) of a logits row: online softmax, i.e. the running max M
-// of the raw logits and S = sum exp((l - M) * invT); with RAW also the argmax of the raw logits
-// (lowest index on ties), which is the running max itself.
-// Returns m_nat = M * invT (natural-log units of the scaled logits), S and the candidate.
+// Online softmax of a thread's share of a row: the running max M of the raw logits and
+// S = sum exp((l - M) * invT), in the log2 domain with packed fp32x2 arithmetic.
 struct OnlineSoftmax {
   float M, neg_ms, scale2;
   uint64_t Sa, Sb, scale22;
@@ -237,12 +243,14 @@ struct OnlineSoftmax {
   }
 };
 
-template <int DT, bool RAW>
+// One streaming pass over elements [lo, hi) of a logits row: online softmax and the raw argmax
+// (lowest index on ties), which is the running max itself.
+template <int DT>
 __device__ __forceinline__ void row_pass(const VerifyParams& P, const char* row, int lo, int hi,
-                                         float& m_nat, float& S_out, Top2& top, uint4* ring) {
+                                         float& m_nat, float& S_out, float& raw_max, int& raw_idx, uint4* ring) {
   OnlineSoftmax os;
   os.init(P.inv_t);
-  int raw_idx = -1;
+  raw_idx = -1;
   RowStream<DT> in;
   in.start(ring, row, lo, hi);
   for (int base = lo; base < hi; base += kThreads * 8) {
@@ -250,7 +258,7 @@ __device__ __forceinline__ void row_pass(const VerifyParams& P, const char* row,
     float l[8];
     in.next(e, l);
     const float vmax = fmaxf(max3(l[0], l[1], l[2]), max3(max3(l[3], l[4], l[5]), l[6], l[7]));
-    if (os.raise(vmax) && RAW) {
+    if (os.raise(vmax)) {
 #pragma unroll
       for (int i = 7; i >= 0; --i)
         if (l[i] == vmax) raw_idx = e + i;
@@ -260,105 +268,7 @@ __device__ __forceinline__ void row_pass(const VerifyParams& P, const char* row,
   in.finish();
   S_out = os.sum();
   m_nat = os.M * P.inv_t;
-  top.init();
-  if (RAW) top.push(os.M, raw_idx);
-}
-
-// Per-warp queue of groups of four logits that survived the first skip test.
-constexpr int kQueueCap = 128;  // < 32 left over + at most 64 new per iteration
-struct SampleQueue {
-  float4 l[kThreads / 32][kQueueCap];
-  int idx[kThreads / 32][kQueueCap];
-};
-
-// The same pass for a Gumbel-sampled row: online softmax plus the top-2 of l * invT + g.
-template <int DT>
-__device__ __forceinline__ void row_pass_sampled(const VerifyParams& P, const char* row, int lo, int hi, int b,
-                                                 uint32_t tagpos, float& m_nat, float& S_out, Top2& top,
-                                                 SampleQueue& Q, unsigned* sm_best, uint4* ring) {
-  OnlineSoftmax os;
-  os.init(P.inv_t);
-  RowStream<DT> in;
-  in.start(ring, row, lo, hi);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const unsigned below = (1u << lane) - 1u;
-  float4* ql = Q.l[warp];
-  int* qi = Q.idx[warp];
-  const float rcp_t = 1.f / P.inv_t;
-  const float cut_off = -17.34f * rcp_t;
-  top.init();
-  // A noisy score that some element of the row really has (so a lower bound of the winner's), shared by
-  // the CTA through sm_best; a stale value only makes the skip tests weaker.
-  float best = -INFINITY;
-  int head = 0, tail = 0;  // warp-uniform queue positions
-
-  // Draw the noise of one queued group and keep its candidates.
-  auto drain = [&](int pos) {
-    const int idx = qi[pos & (kQueueCap - 1)];
-    const float4 v = ql[pos & (kQueueCap - 1)];
-    const float l4[4] = {v.x, v.y, v.z, v.w};
-    const uint4 rnd = philox4x32_10((uint32_t)idx >> 2, P.step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
-    const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-    // -ln u' >= 1 - u' >= nf 2^-24 with nf = floor(2^24 (1 - u')), so g_i <= -ln(nf 2^-24): the element
-    // cannot come within 2e-3 of the running best when nf >= 1.002 * 2^24 * exp(l_i invT - best)
-    float K2 = 24.0028853901f - best * kLog2e;  // log2 of the factor; +inf while there is no best
-    bool improved = false;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float nf = (float)((~w[i]) >> 8);
-      const float bound = ex2f(fmaf(l4[i], os.scale2, K2));
-      if (!(nf >= bound) && l4[i] > -INFINITY) {
-        const float sc = l4[i] * P.inv_t + gumbel_f32(w[i]);
-        top.push(sc, idx + i);
-        if (top.s1 > best) {
-          best = top.s1;
-          K2 = 24.0028853901f - best * kLog2e;
-          improved = true;
-        }
-      }
-    }
-    if (improved) atomicMax(sm_best, enc_ordered(best));
-  };
-
-  // uniform trip count per block (the warp votes inside the loop)
-  for (int base = lo; base < hi; base += kThreads * 8) {
-    const int e = base + threadIdx.x * 8;
-    float l[8];
-    in.next(e, l);
-    best = fmaxf(best, dec_ordered(*reinterpret_cast<volatile unsigned*>(sm_best)));
-    const float cut = fmaf(best, rcp_t, cut_off);  // raw-logit units; -inf while there is no best
-    const float g0 = fmaxf(fmaxf(l[0], l[1]), fmaxf(l[2], l[3]));
-    const float g1 = fmaxf(fmaxf(l[4], l[5]), fmaxf(l[6], l[7]));
-    os.raise(fmaxf(g0, g1));
-    os.add8(l);
-    {
-      const bool p0 = g0 > cut, p1 = g1 > cut;  // false for padding and all -inf groups
-      const unsigned m0 = __ballot_sync(0xffffffffu, p0);
-      const unsigned m1 = __ballot_sync(0xffffffffu, p1);
-      if (p0) {
-        const int s = (tail + __popc(m0 & below)) & (kQueueCap - 1);
-        ql[s] = make_float4(l[0], l[1], l[2], l[3]);
-        qi[s] = e;
-      }
-      tail += __popc(m0);
-      if (p1) {
-        const int s = (tail + __popc(m1 & below)) & (kQueueCap - 1);
-        ql[s] = make_float4(l[4], l[5], l[6], l[7]);
-        qi[s] = e + 4;
-      }
-      tail += __popc(m1);
-    }
-    __syncwarp();
-    while (tail - head >= 32) {
-      drain(head + lane);
-      head += 32;
-    }
-  }
-  in.finish();
-  __syncwarp();
-  if (lane < tail - head) drain(head + lane);
-  S_out = os.sum();
-  m_nat = os.M * P.inv_t;
+  raw_max = os.M;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -366,14 +276,11 @@ __device__ __forceinline__ void row_pass_sampled(const VerifyParams& P, const ch
 // ------------------------------------------------------------------------------------------------
 template <int DT>
 __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParams P) {
-  // Launch order = (split, slot, row class): the Gumbel-sampled rows of every slot come first.  They run
-  // several times longer than a streamed row, so starting them all at once and letting the streamed rows
-  // fill the remaining CTA slots keeps the ALU-bound and the HBM-bound work overlapped and the tail short.
+  // Launch order = (split, slot, k): the rows that the sampling pass reads again come last, so that
+  // they are the most recent lines in L2 when it starts.
   const int split = blockIdx.x, b = blockIdx.y, k = blockIdx.z;
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
-  const int n_sampled = P.propose_mode == 0 ? P.N : 1;  // rows nv .. nv + n_sampled - 1
-  const int r = k < n_sampled ? nv + k : (k - n_sampled < nv ? k - n_sampled : k);
   if (nv < 0 || nv > P.N - 1) {
     if (split == 0 && k == 0 && threadIdx.x == 0) {
       atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
@@ -382,45 +289,33 @@ __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParam
     return;
   }
   const int q_len = nv + P.N;
+  int r = k + nv + rows_sampled(P);  // k = Q - rows_sampled .. Q - 1  <->  r = nv .. nv + rows_sampled - 1
+  if (r >= P.Q) r -= P.Q;
   if (r >= q_len) return;
 
   __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
   __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
   __shared__ int sm_last;
-  __shared__ unsigned sm_best;
-  __shared__ SampleQueue sm_queue;
   __shared__ __align__(16) uint4 sm_ring[kRingBytes / 16];
 
-  const bool is_final = (r == nv);
-  const bool is_prop = (r > nv);
-  const bool noise = is_final || (is_prop && P.propose_mode == 0);
-  const bool raw_argmax = is_prop && P.propose_mode == 1;
-  const uint32_t tagpos = is_final ? ((ISD_TAG_FINAL << 16) | (uint32_t)(nv + 1))
-                                   : ((ISD_TAG_PROPOSE << 16) | (uint32_t)(r - nv));
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
-
   int lo, hi;
   chunk_range(P.V, P.row_splits, split, lo, hi);
 
-  float m_nat, S;
-  Top2 top;
-  if (noise) {
-    if (threadIdx.x == 0) sm_best = 0;
-    __syncthreads();
-    row_pass_sampled<DT>(P, row, lo, hi, b, tagpos, m_nat, S, top, sm_queue, &sm_best, sm_ring);
-  } else if (raw_argmax) {
-    row_pass<DT, true>(P, row, lo, hi, m_nat, S, top, sm_ring);
-  } else {
-    row_pass<DT, false>(P, row, lo, hi, m_nat, S, top, sm_ring);
-  }
+  float m_nat, S, raw_max;
+  int raw_idx;
+  row_pass<DT>(P, row, lo, hi, m_nat, S, raw_max, raw_idx, sm_ring);
 
   // ---- block reduction -> partial
   block_merge_lse(m_nat, S, sm_f0, sm_f1);
+  Top2 top;
+  top.init();
+  top.push(raw_max, raw_idx);
   block_merge_top2(top, sm_f0, sm_i0, sm_f1, sm_i1);
   if (threadIdx.x == 0) {
     RowPartial rp;
-    rp.m = m_nat; rp.s = S; rp.best1 = top.s1; rp.idx1 = top.i1; rp.best2 = top.s2; rp.idx2 = top.i2;
+    rp.m = m_nat; rp.s = S; rp.raw_max = top.s1; rp.idx = top.i1;
     P.row_part[((size_t)b * P.Q + r) * P.row_splits + split] = rp;
     __threadfence();
     const int arrived = atomicAdd(&P.row_ticket[b], 1);
@@ -443,42 +338,35 @@ __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParam
     Top2 t;
     t.init();
     int bad = 0;
-    int tok = -1;
     if (lane < q_len) {
       const volatile RowPartial* rp = P.row_part + ((size_t)b * P.Q + lane) * P.row_splits;
-      for (int k = 0; k < P.row_splits; ++k) {  // empty splits wrote neutral values
-        lse_merge(m, s, rp[k].m, rp[k].s);
-        t.merge(rp[k].best1, rp[k].idx1, rp[k].best2, rp[k].idx2);
+      for (int i = 0; i < P.row_splits; ++i) {  // empty splits wrote neutral values
+        lse_merge(m, s, rp[i].m, rp[i].s);
+        t.push(rp[i].raw_max, rp[i].idx);
       }
       // NaN anywhere poisons s; +inf logits give m = +inf
       bad = (s != s) || (m == INFINITY) || (m != m);
-      const bool row_noise = (lane == nv) || (lane > nv && P.propose_mode == 0);
-      tok = t.i1;
-      if (row_noise && t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
-        const uint32_t tp = (lane == nv) ? ((ISD_TAG_FINAL << 16) | (uint32_t)(nv + 1))
-                                         : ((ISD_TAG_PROPOSE << 16) | (uint32_t)(lane - nv));
-        const char* rw = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + lane) * (size_t)P.V * elt;
-        const double a = noisy_score_f64(P, rw, t.i1, (uint32_t)b, tp);
-        const double c = noisy_score_f64(P, rw, t.i2, (uint32_t)b, tp);
-        if (c > a || (c == a && t.i2 < t.i1)) tok = t.i2;
-      }
+      P.row_arg[(size_t)b * P.Q + lane] = t.i1;
     }
     d_lse[lane] = m + logf(s);
-    d_tok[lane] = tok;
+    d_tok[lane] = t.i1;
     d_bad[lane] = bad;
   }
   __syncwarp();
 
   const int NP = P.N - 1;
-  // proposals + cached proposal-law statistics (lanes 1..N-1 = MASK row m)
+  // proposal-law statistics (lanes 1..N-1 = MASK row m); argmax proposals are final here, sampled ones
+  // and their logit are written by the sampling pass
   if (lane >= 1 && lane <= NP) {
     const int rr = nv + lane;
-    const int xh = d_tok[rr];
-    P.out.new_prop_tok[(size_t)b * NP + lane - 1] = xh;
-    const char* rw = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + rr) * (size_t)P.V * elt;
     P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 0] = d_lse[rr];
-    P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 1] =
-        xh >= 0 ? load_logit(rw, P.logits_dtype, (size_t)xh) * P.inv_t : NAN;
+    if (P.propose_mode == 1) {
+      const int xh = d_tok[rr];
+      const char* rw = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + rr) * (size_t)P.V * elt;
+      P.out.new_prop_tok[(size_t)b * NP + lane - 1] = xh;
+      P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 1] =
+          xh >= 0 ? load_logit(rw, P.logits_dtype, (size_t)xh) * P.inv_t : NAN;
+    }
   }
   if (lane != 0) return;
 
@@ -523,11 +411,11 @@ __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParam
   }
   if (a >= 0 && rej == 0 && d_bad[nv]) status |= ISD_ST_NONFINITE_LOGIT;
   for (int j = 0; j < P.N; ++j) P.out.out_tok[(size_t)b * P.N + j] = -1;
+  P.out.repl_tok[b] = -1;  // the sampling pass fills the drawn token
   if (a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL)) {
     P.out.accept_len[b] = 0;
     P.out.n_emit[b] = 0;
-    P.out.repl_tok[b] = -1;
-    P.reject_pos[b] = 0;
+    P.reject_pos[b] = -1;  // frozen: nothing is drawn for the emission
     atomicOr(&P.slot_status[b], status);
     atomicOr(P.global_status, status);
     return;
@@ -535,19 +423,13 @@ __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParam
   P.out.accept_len[b] = a;
   P.out.n_emit[b] = a + 1;
   for (int j = 1; j <= a; ++j) P.out.out_tok[(size_t)b * P.N + j - 1] = P.block_tok[(size_t)b * P.Q + j];
-  if (rej == 0) {
-    const int y = d_tok[nv];
-    P.out.repl_tok[b] = y;
-    P.out.out_tok[(size_t)b * P.N + a] = y;
-  } else {
-    P.out.repl_tok[b] = -1;  // filled by the residual pass
-  }
   P.reject_pos[b] = rej;
 }
 
 // ------------------------------------------------------------------------------------------------
-// Pass 2: residual resample for slots with a rejection
+// Pass 2: the random draws
 // ------------------------------------------------------------------------------------------------
+// fp64 score of vocabulary index i of the residual law: ln max(0, p_i - q_i) + g
 __device__ double resid_score_f64(const VerifyParams& P, const void* prow, const void* qrow, int i, int x,
                                   double lse_p, double lse_q, uint32_t slot, uint32_t tagpos) {
   const double pi = exp((double)load_logit(prow, P.logits_dtype, (size_t)i) * (double)P.inv_t - lse_p);
@@ -560,152 +442,251 @@ __device__ double resid_score_f64(const VerifyParams& P, const void* prow, const
   return log(rres) + gumbel_f64(philox_word(r, i & 3));
 }
 
+// What one CTA of the sampling pass draws from.
+struct SampleJob {
+  const char* prow;  // the row whose law (or whose law minus q) is sampled
+  const char* qrow;  // residual only, softmax q: the proposal-law row of the previous step
+  int x;             // residual only: the rejected token
+  float lse_p, lse_q;
+  uint32_t tagpos;
+  bool resid;
+};
+
+// fp32 noisy score of element i of the job's law; -inf when the element has no mass.  The same
+// arithmetic scores the seed, the queued candidates and the fallback.
+__device__ __forceinline__ float job_score(const VerifyParams& P, const SampleJob& J, float l, int i, uint32_t w) {
+  if (!(l > -INFINITY)) return -INFINITY;
+  if (!J.resid) return l * P.inv_t + gumbel_f32(w);
+  const float pi = expf(l * P.inv_t - J.lse_p);
+  const float qi = P.q_mode == 0 ? expf(load_logit(J.qrow, P.logits_dtype, (size_t)i) * P.inv_t - J.lse_q)
+                                 : (i == J.x ? 1.f : 0.f);
+  const float rr = pi - qi;
+  return rr > 0.f ? logf(rr) + gumbel_f32(w) : -INFINITY;
+}
+
+// Per-warp queue of groups of four logits that survived the first skip test.
+constexpr int kQueueCap = 128;  // < 32 left over + at most 64 new per iteration
+struct SampleQueue {
+  float4 l[kThreads / 32][kQueueCap];
+  int idx[kThreads / 32][kQueueCap];
+};
+
+// Gumbel-max top-2 of elements [lo, hi) of the job's law.  `best` enters as a noisy score that some
+// element of the row really has (the seed, or -inf), so it is a lower bound of the winner's score; it is
+// shared by the CTA through sm_best, and a stale value only makes the skip tests weaker.
 template <int DT>
-__global__ void __launch_bounds__(kThreads) verify_resid_kernel(const VerifyParams P) {
-  const int split = blockIdx.x, b = blockIdx.y;
-  if (!P.active[b]) return;
-  const int j = P.reject_pos[b];
-  if (j <= 0) return;
-
-  __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
-  __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
-  __shared__ int sm_last;
-
-  const int NP = P.N - 1;
-  const int x = P.block_tok[(size_t)b * P.Q + j];
-  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
-  const char* prow = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + (j - 1)) * (size_t)P.V * elt;
-  const char* qrow = P.q_mode == 0
-      ? reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + (P.q_row0[b] + j - 1)) * (size_t)P.V * elt
-      : prow;
-  const float lse_p = P.lse_p_rej[b];
-  const float lse_q = P.q_mode == 0 ? P.q_stats[((size_t)b * NP + j - 1) * 2 + 0] : 0.f;
-  const uint32_t tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)j;
-
-  int lo, hi;
-  chunk_range(P.V, P.resid_splits, split, lo, hi);
-  Top2 top;
-  top.init();
-  float best_nat = -INFINITY;
-  // bound: ln r_i <= ln p_i = lp_i - lse_p; skip iff nf >= 1.002 2^24 exp(lp_i - lse_p - best)
+__device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJob& J, int lo, int hi, int b,
+                                            float best, Top2& top, SampleQueue& Q, unsigned* sm_best, uint4* ring) {
+  RowStream<DT> in;
+  in.start(ring, J.prow, lo, hi);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned below = (1u << lane) - 1u;
+  float4* ql = Q.l[warp];
+  int* qi = Q.idx[warp];
   const float scale2 = P.inv_t * kLog2e;
-  float K2 = INFINITY;  // log2 offset: skip iff nf >= ex2(x2 + K2)
-  int iter = 0;
-  for (int base = lo; base < hi; base += kThreads * 8, ++iter) {
-    const int e = base + threadIdx.x * 8;
-    const bool valid = e < hi;
-    float lp[8], lq[8];
-    if (valid) {
-      load8<DT>(prow, e, lp);
-      if (P.q_mode == 0) load8<DT>(qrow, e, lq);
-    }
+  const float rcp_t = 1.f / P.inv_t;
+  // the law's log-mass of element i is at most l_i invT - shift (residual: ln r_i <= ln p_i)
+  const float shift = J.resid ? J.lse_p : 0.f;
+  const float cut_off = (shift - kGumbelMax) * rcp_t;
+  top.init();
+  int head = 0, tail = 0;  // warp-uniform queue positions
+
+  // Draw the noise of one queued group and keep its candidates.
+  auto drain = [&](int pos) {
+    const int idx = qi[pos & (kQueueCap - 1)];
+    const float4 v = ql[pos & (kQueueCap - 1)];
+    const float l4[4] = {v.x, v.y, v.z, v.w};
+    const uint4 rnd = philox4x32_10((uint32_t)idx >> 2, P.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
+    const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+    // -ln u' >= 1 - u' >= nf 2^-24 with nf = floor(2^24 (1 - u')), so g_i <= -ln(nf 2^-24): the element
+    // cannot come within 2e-3 of the running best when nf >= 1.002 * 2^24 * exp(l_i invT - shift - best)
+    float K2 = 24.0028853901f - (shift + best) * kLog2e;  // log2 of the factor; +inf while there is no best
+    bool improved = false;
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      if (!valid) break;
-      // Cheap pre-filter before any random number is drawn: ln r_i <= ln p_i and no Gumbel variate on the
-      // 24-bit lattice exceeds 17.33, so a group whose four elements all have ln p_i + 17.34 below the
-      // running best cannot produce a candidate.  At realistic vocabulary sizes this skips almost all
-      // of the Philox work (only logits a few sigma above the mean survive).
-      const float cut = best_nat - 17.34f + lse_p;
-      const float gmax = fmaxf(fmaxf(lp[4 * h], lp[4 * h + 1]), fmaxf(lp[4 * h + 2], lp[4 * h + 3])) * P.inv_t;
-      if (!(gmax > cut)) continue;
-      const uint4 rnd = philox4x32_10((uint32_t)(e + 4 * h) >> 2, P.step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
-      const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int idx = e + 4 * h + i;
-        const float nf = (float)((~w[i]) >> 8);
-        const float bound = ex2f(lp[4 * h + i] * scale2 + K2);  // K2 = +inf -> inf (never skip)
-        if (!(nf >= bound)) {
-          const float pi = expf(lp[4 * h + i] * P.inv_t - lse_p);
-          const float qi = P.q_mode == 0 ? expf(lq[4 * h + i] * P.inv_t - lse_q) : (idx == x ? 1.f : 0.f);
-          const float rr = pi - qi;
-          if (rr > 0.f) {
-            const float s = logf(rr) + gumbel_f32(w[i]);
-            top.push(s, idx);
-            if (top.s1 > best_nat) {
-              best_nat = top.s1;
-              K2 = 24.f + 0.0028853901f - (lse_p + best_nat) * kLog2e;  // log2(1.002) = 0.00288539
-            }
+    for (int i = 0; i < 4; ++i) {
+      const float nf = (float)((~w[i]) >> 8);
+      const float bound = ex2f(fmaf(l4[i], scale2, K2));
+      if (!(nf >= bound)) {
+        const float sc = job_score(P, J, l4[i], idx + i, w[i]);
+        if (sc > -INFINITY) {
+          top.push(sc, idx + i);
+          if (top.s1 > best) {
+            best = top.s1;
+            K2 = 24.0028853901f - (shift + best) * kLog2e;
+            improved = true;
           }
         }
       }
     }
-    if (iter == 0 || (iter & 3) == 3) {
-      float bn = best_nat;
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) bn = fmaxf(bn, __shfl_xor_sync(0xffffffffu, bn, off));
-      if (bn > best_nat) {
-        best_nat = bn;
-        K2 = 24.f + 0.0028853901f - (lse_p + best_nat) * kLog2e;
-      }
+    if (improved) atomicMax(sm_best, enc_ordered(best));
+  };
+
+  // uniform trip count per block (the warp votes inside the loop)
+  for (int base = lo; base < hi; base += kThreads * 8) {
+    const int e = base + threadIdx.x * 8;
+    float l[8];
+    in.next(e, l);
+    best = fmaxf(best, dec_ordered(*reinterpret_cast<volatile unsigned*>(sm_best)));
+    const float cut = fmaf(best, rcp_t, cut_off);  // raw-logit units; -inf while there is no best
+    const float g0 = fmaxf(fmaxf(l[0], l[1]), fmaxf(l[2], l[3]));
+    const float g1 = fmaxf(fmaxf(l[4], l[5]), fmaxf(l[6], l[7]));
+    const bool p0 = g0 > cut, p1 = g1 > cut;  // false for padding and all -inf groups
+    const unsigned m0 = __ballot_sync(0xffffffffu, p0);
+    const unsigned m1 = __ballot_sync(0xffffffffu, p1);
+    if (p0) {
+      const int s = (tail + __popc(m0 & below)) & (kQueueCap - 1);
+      ql[s] = make_float4(l[0], l[1], l[2], l[3]);
+      qi[s] = e;
+    }
+    tail += __popc(m0);
+    if (p1) {
+      const int s = (tail + __popc(m1 & below)) & (kQueueCap - 1);
+      ql[s] = make_float4(l[4], l[5], l[6], l[7]);
+      qi[s] = e + 4;
+    }
+    tail += __popc(m1);
+    __syncwarp();
+    while (tail - head >= 32) {
+      drain(head + lane);
+      head += 32;
     }
   }
-  block_merge_top2(top, sm_f0, sm_i0, sm_f1, sm_i1);
+  in.finish();
+  __syncwarp();
+  if (lane < tail - head) drain(head + lane);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) verify_sample_kernel(const VerifyParams P) {
+  const int split = blockIdx.x, k = blockIdx.y, b = blockIdx.z;
+  if (!P.active[b]) return;
+  const int nv = P.n_ver[b];
+  if (nv < 0 || nv > P.N - 1) return;  // flagged by the row pass; its scratch entries are stale
+  const int rej = P.reject_pos[b];
+  if (k == 0 && rej < 0) return;       // frozen slot: no emission
+
+  __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
+  __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
+  __shared__ int sm_last, sm_tok;
+  __shared__ unsigned sm_best;
+  __shared__ SampleQueue sm_queue;
+  __shared__ __align__(16) uint4 sm_ring[kRingBytes / 16];
+
+  const int NP = P.N - 1;
+  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  const size_t row_bytes = (size_t)P.V * elt;
+  const char* cur = reinterpret_cast<const char*>(P.logits_cur) + (size_t)b * P.Q * row_bytes;
+
+  // ---- what this (slot, k) draws
+  SampleJob J;
+  J.qrow = nullptr; J.x = -1; J.lse_p = 0.f; J.lse_q = 0.f;
+  int r;  // row of this step's logits that is sampled
+  if (k == 0 && rej > 0) {
+    // replacement for the first rejected proposal, from normalize(max(0, p - q))
+    if (P.q_mode == 0 && P.q_prev == nullptr) return;  // nothing to subtract: the caller gave no proposal-law rows
+    r = rej - 1;
+    J.resid = true;
+    J.x = P.block_tok[(size_t)b * P.Q + rej];
+    J.lse_p = P.lse_p_rej[b];
+    if (P.q_mode == 0) {
+      J.qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + (P.q_row0[b] + rej - 1)) * row_bytes;
+      J.lse_q = P.q_stats[((size_t)b * NP + rej - 1) * 2 + 0];
+    }
+    J.tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)rej;
+  } else {
+    r = nv + k;  // k = 0: bonus / free token from the row of the last clean token; k >= 1: MASK row k
+    J.resid = false;
+    J.tagpos = k == 0 ? ((ISD_TAG_FINAL << 16) | (uint32_t)(nv + 1)) : ((ISD_TAG_PROPOSE << 16) | (uint32_t)k);
+  }
+  J.prow = cur + (size_t)r * row_bytes;
+
+  // ---- seed: the true noisy score of the row's argmax (for the residual: if it has residual mass)
   if (threadIdx.x == 0) {
-    ResidPartial rp;
-    rp.best1 = top.s1; rp.idx1 = top.i1; rp.best2 = top.s2; rp.idx2 = top.i2;
-    P.resid_part[(size_t)b * P.resid_splits + split] = rp;
+    float seed = -INFINITY;
+    const int i0 = P.row_arg[(size_t)b * P.Q + r];
+    if (i0 >= 0 && i0 < P.V) {
+      const uint4 rnd = philox4x32_10((uint32_t)i0 >> 2, P.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
+      seed = job_score(P, J, load_logit(J.prow, P.logits_dtype, (size_t)i0), i0, philox_word(rnd, i0 & 3));
+    }
+    sm_best = seed > -INFINITY ? enc_ordered(seed) : 0u;
+  }
+  __syncthreads();
+  const float best0 = dec_ordered(sm_best);  // NaN when there is no seed
+
+  int lo, hi;
+  chunk_range(P.V, P.sample_splits, split, lo, hi);
+  Top2 top;
+  sample_pass<DT>(P, J, lo, hi, b, fmaxf(-INFINITY, best0), top, sm_queue, &sm_best, sm_ring);
+
+  block_merge_top2(top, sm_f0, sm_i0, sm_f1, sm_i1);
+  int* ticket = P.samp_ticket + (size_t)b * P.N + k;
+  SamplePartial* parts = P.samp_part + ((size_t)b * P.N + k) * P.sample_splits;
+  if (threadIdx.x == 0) {
+    SamplePartial sp;
+    sp.best1 = top.s1; sp.idx1 = top.i1; sp.best2 = top.s2; sp.idx2 = top.i2;
+    parts[split] = sp;
     __threadfence();
-    const int arrived = atomicAdd(&P.resid_ticket[b], 1);
-    sm_last = (arrived == P.resid_splits - 1);
+    const int arrived = atomicAdd(ticket, 1);
+    sm_last = (arrived == P.sample_splits - 1);
   }
   __syncthreads();
   if (!sm_last) return;
   __threadfence();
 
-  // last CTA of the slot: merge, fp64 tie-break, write the replacement
-  __shared__ int sm_tok;
+  // ---- last CTA of the (slot, k): merge, fp64 tie-break, write the token
   if (threadIdx.x == 0) {
-    P.resid_ticket[b] = 0;
+    *ticket = 0;  // ready for the next call
     Top2 t;
     t.init();
-    for (int k = 0; k < P.resid_splits; ++k) {
-      const volatile ResidPartial* rp = P.resid_part + (size_t)b * P.resid_splits + k;
-      t.merge(rp->best1, rp->idx1, rp->best2, rp->idx2);
+    for (int i = 0; i < P.sample_splits; ++i) {
+      const volatile SamplePartial* sp = parts + i;
+      t.merge(sp->best1, sp->idx1, sp->best2, sp->idx2);
     }
     int y = t.i1;
     if (t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
-      const double a = resid_score_f64(P, prow, qrow, t.i1, x, lse_p, lse_q, (uint32_t)b, tagpos);
-      const double c = resid_score_f64(P, prow, qrow, t.i2, x, lse_p, lse_q, (uint32_t)b, tagpos);
-      if (c > a || (c == a && t.i2 < t.i1)) y = t.i2;
+      double s1, s2;
+      if (J.resid) {
+        s1 = resid_score_f64(P, J.prow, J.qrow, t.i1, J.x, J.lse_p, J.lse_q, (uint32_t)b, J.tagpos);
+        s2 = resid_score_f64(P, J.prow, J.qrow, t.i2, J.x, J.lse_p, J.lse_q, (uint32_t)b, J.tagpos);
+      } else {
+        s1 = noisy_score_f64(P, J.prow, t.i1, (uint32_t)b, J.tagpos);
+        s2 = noisy_score_f64(P, J.prow, t.i2, (uint32_t)b, J.tagpos);
+      }
+      if (s2 > s1 || (s2 == s1 && t.i2 < t.i1)) y = t.i2;
     }
     sm_tok = y;
   }
   __syncthreads();
   int y = sm_tok;
-  if (y < 0) {
+  if (J.resid && y < 0) {
     // Residual empty in fp32 (p and q numerically equal): fall back to a sample of p with the same
     // noise.  Rare; done by this one CTA over the whole row.
+    J.resid = false;
+    if (threadIdx.x == 0) sm_best = 0u;
+    __syncthreads();
     Top2 t;
-    t.init();
-    for (int e = threadIdx.x * 8; e < P.V; e += kThreads * 8) {
-      float lp[8];
-      load8<DT>(prow, e, lp);
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const uint4 rnd = philox4x32_10((uint32_t)(e + 4 * h) >> 2, P.step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
-        const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          if (lp[4 * h + i] > -INFINITY) t.push(lp[4 * h + i] * P.inv_t + gumbel_f32(w[i]), e + 4 * h + i);
-      }
-    }
+    sample_pass<DT>(P, J, 0, P.V, b, -INFINITY, t, sm_queue, &sm_best, sm_ring);
     block_merge_top2(t, sm_f0, sm_i0, sm_f1, sm_i1);
     if (threadIdx.x == 0) {
       y = t.i1;
       if (t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
-        const double a = noisy_score_f64(P, prow, t.i1, (uint32_t)b, tagpos);
-        const double c = noisy_score_f64(P, prow, t.i2, (uint32_t)b, tagpos);
-        if (c > a || (c == a && t.i2 < t.i1)) y = t.i2;
+        const double s1 = noisy_score_f64(P, J.prow, t.i1, (uint32_t)b, J.tagpos);
+        const double s2 = noisy_score_f64(P, J.prow, t.i2, (uint32_t)b, J.tagpos);
+        if (s2 > s1 || (s2 == s1 && t.i2 < t.i1)) y = t.i2;
       }
       atomicOr(&P.slot_status[b], ISD_ST_EMPTY_RESIDUAL);
       atomicOr(P.global_status, ISD_ST_EMPTY_RESIDUAL);
     }
   }
-  if (threadIdx.x == 0) {
+  if (threadIdx.x != 0) return;
+  if (k == 0) {
+    const int a = rej > 0 ? rej - 1 : nv;
     P.out.repl_tok[b] = y;
-    P.out.out_tok[(size_t)b * P.N + (j - 1)] = y;
+    P.out.out_tok[(size_t)b * P.N + a] = y;
+  } else {
+    P.out.new_prop_tok[(size_t)b * NP + k - 1] = y;
+    P.out.new_q_stats[((size_t)b * NP + k - 1) * 2 + 1] =
+        y >= 0 ? load_logit(J.prow, P.logits_dtype, (size_t)y) * P.inv_t : NAN;
   }
 }
 
@@ -720,25 +701,26 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   P.logits_dtype = c.logits_dtype; P.q_mode = c.q_mode; P.propose_mode = c.propose_mode;
   P.inv_t = c.inv_temperature; P.tau = c.tau;
   P.seed_lo = (uint32_t)c.seed; P.seed_hi = (uint32_t)(c.seed >> 32); P.step = step;
-  P.row_splits = ctx->row_splits; P.resid_splits = ctx->resid_splits;
+  P.row_splits = ctx->row_splits; P.sample_splits = ctx->sample_splits;
   P.n_ver = st->n_ver; P.active = st->active; P.block_tok = st->block_tok; P.q_row0 = st->q_row0;
   P.q_stats = st->q_stats; P.slot_status = st->slot_status; P.global_status = ctx->global_status;
   P.logits_cur = logits_cur; P.q_prev = q_prev_logits; P.out = *out;
-  P.row_part = ctx->row_part; P.resid_part = ctx->resid_part; P.row_ticket = ctx->row_ticket;
-  P.resid_ticket = ctx->resid_ticket; P.reject_pos = ctx->reject_pos; P.lse_p_rej = ctx->lse_p_rej;
+  P.row_part = ctx->row_part; P.samp_part = ctx->samp_part; P.row_ticket = ctx->row_ticket;
+  P.samp_ticket = ctx->samp_ticket; P.reject_pos = ctx->reject_pos; P.row_arg = ctx->row_arg;
+  P.lse_p_rej = ctx->lse_p_rej;
 
   const dim3 grid1(ctx->row_splits, c.batch, ctx->Q);
+  const dim3 grid2(ctx->sample_splits, c.propose_mode == 0 ? c.stride : 1, c.batch);
   if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
-  if (c.logits_dtype == ISD_LOGITS_BF16) verify_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads, 0, stream>>>(P);
-  else verify_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads, 0, stream>>>(P);
-  if (ctx->ev_verify1) cudaEventRecord(ctx->ev_verify1, stream);
-  ctx->launches++;
-  if (c.stride > 1 && (c.q_mode == 1 || q_prev_logits != nullptr)) {
-    const dim3 grid2(ctx->resid_splits, c.batch);
-    if (c.logits_dtype == ISD_LOGITS_BF16) verify_resid_kernel<ISD_LOGITS_BF16><<<grid2, kThreads, 0, stream>>>(P);
-    else verify_resid_kernel<ISD_LOGITS_F32><<<grid2, kThreads, 0, stream>>>(P);
-    ctx->launches++;
+  if (c.logits_dtype == ISD_LOGITS_BF16) {
+    verify_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads, 0, stream>>>(P);
+    verify_sample_kernel<ISD_LOGITS_BF16><<<grid2, kThreads, 0, stream>>>(P);
+  } else {
+    verify_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads, 0, stream>>>(P);
+    verify_sample_kernel<ISD_LOGITS_F32><<<grid2, kThreads, 0, stream>>>(P);
   }
+  if (ctx->ev_verify1) cudaEventRecord(ctx->ev_verify1, stream);
+  ctx->launches += 2;
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }
 
@@ -764,14 +746,17 @@ constexpr int kStaticMaxBatch = ISD_STATIC_MAX_BATCH;
 constexpr int kStaticMaxSplits = 16;
 constexpr size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 // layout of the array: [zeroed every call: tickets, reject positions, status word][partials]
+constexpr int kStaticMaxStride = (ISD_MAX_Q + 1) / 2;
 constexpr size_t kOffRowTicket = 0;
-constexpr size_t kOffResidTicket = kOffRowTicket + align256(sizeof(int) * kStaticMaxBatch);
-constexpr size_t kOffRejectPos = kOffResidTicket + align256(sizeof(int) * kStaticMaxBatch);
-constexpr size_t kOffStatus = kOffRejectPos + align256(sizeof(int) * kStaticMaxBatch);
+constexpr size_t kOffSampTicket = kOffRowTicket + align256(sizeof(int) * kStaticMaxBatch);
+constexpr size_t kOffStatus = kOffSampTicket + align256(sizeof(int) * kStaticMaxBatch * kStaticMaxStride);
 constexpr size_t kZeroedBytes = kOffStatus + align256(sizeof(uint32_t));
-constexpr size_t kOffLse = kZeroedBytes;
-constexpr size_t kOffResidPart = kOffLse + align256(sizeof(float) * kStaticMaxBatch);
-constexpr size_t kOffRowPart = kOffResidPart + align256(sizeof(ResidPartial) * kStaticMaxBatch * kStaticMaxSplits);
+constexpr size_t kOffRejectPos = kZeroedBytes;  // written by the row pass for every slot the sampling pass reads
+constexpr size_t kOffRowArg = kOffRejectPos + align256(sizeof(int) * kStaticMaxBatch);
+constexpr size_t kOffLse = kOffRowArg + align256(sizeof(int) * kStaticMaxBatch * ISD_MAX_Q);
+constexpr size_t kOffSampPart = kOffLse + align256(sizeof(float) * kStaticMaxBatch);
+constexpr size_t kOffRowPart =
+    kOffSampPart + align256(sizeof(SamplePartial) * kStaticMaxBatch * kStaticMaxStride * kStaticMaxSplits);
 constexpr size_t kStaticBytes = kOffRowPart + align256(sizeof(RowPartial) * kStaticMaxBatch * ISD_MAX_Q * kStaticMaxSplits);
 
 constexpr int kMaxDevices = 64;
@@ -832,13 +817,14 @@ extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* s
   int ps = 4;  // same cut as isd_create uses
   ps = ps > max_by_len ? max_by_len : ps;
   tmp.row_splits = rs;
-  tmp.resid_splits = ps;
+  tmp.sample_splits = ps;
   tmp.row_ticket = reinterpret_cast<int*>(base + kOffRowTicket);
-  tmp.resid_ticket = reinterpret_cast<int*>(base + kOffResidTicket);
+  tmp.samp_ticket = reinterpret_cast<int*>(base + kOffSampTicket);
+  tmp.row_arg = reinterpret_cast<int*>(base + kOffRowArg);
   tmp.reject_pos = reinterpret_cast<int*>(base + kOffRejectPos);
   tmp.global_status = reinterpret_cast<uint32_t*>(base + kOffStatus);
   tmp.lse_p_rej = reinterpret_cast<float*>(base + kOffLse);
-  tmp.resid_part = reinterpret_cast<ResidPartial*>(base + kOffResidPart);
+  tmp.samp_part = reinterpret_cast<SamplePartial*>(base + kOffSampPart);
   tmp.row_part = reinterpret_cast<RowPartial*>(base + kOffRowPart);
 
   // the array keeps the previous call's contents: counters and flags must start at zero
