@@ -74,6 +74,9 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   const int target = ctx->num_sms * 4;
   int rs = (target + rows - 1) / rows;
   const int max_by_len = (c.vocab + 8191) / 8192;  // keep at least 8k elements per CTA
+#ifdef ISD_ROW_SPLITS_MIN
+  rs = rs < ISD_ROW_SPLITS_MIN ? ISD_ROW_SPLITS_MIN : rs;
+#endif
   rs = rs < 1 ? 1 : rs;
   rs = rs > 16 ? 16 : rs;
   rs = rs > max_by_len ? max_by_len : rs;

@@ -17,6 +17,11 @@
 #define ISD_TAG_FINAL 1u
 #define ISD_TAG_PROPOSE 2u
 
+// internal status bit (not part of the public set): a bounded wait inside a kernel ran out
+#ifndef ISD_ST_KERNEL_TIMEOUT
+#define ISD_ST_KERNEL_TIMEOUT 0x80000000u
+#endif
+
 // score gap below which two Gumbel-max candidates are re-judged in fp64
 #define ISD_TIE_EPS 1e-3f
 
@@ -215,6 +220,17 @@ __device__ __forceinline__ bool ring_mbar_wait(uint32_t bar, uint32_t parity) {
     if (ok) return true;
   }
   return false;
+}
+// The same wait where the phase has normally completed already: one probe, then the bounded loop.
+__device__ __forceinline__ bool mbar_wait_likely(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  if (__builtin_expect(ok != 0, 1)) return true;
+  return ring_mbar_wait(bar, parity);
 }
 // Contiguous global -> shared copy (16-byte aligned addresses, size a multiple of 16) that signals `bar`.
 __device__ __forceinline__ void ring_bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {

@@ -27,6 +27,19 @@
 // ISD_TIE_EPS.
 #include "isd_internal.cuh"
 
+#ifdef EXP_COUNT
+__device__ unsigned long long g_dbg[8];
+extern "C" int isd_debug_counters(unsigned long long* out) {
+  cudaMemcpyFromSymbol(out, g_dbg, sizeof(g_dbg));
+  unsigned long long z[8] = {};
+  cudaMemcpyToSymbol(g_dbg, z, sizeof(z));
+  return 0;
+}
+#define DBG_COUNT(i, v) atomicAdd(&g_dbg[i], (unsigned long long)(v))
+#else
+#define DBG_COUNT(i, v)
+#endif
+
 namespace {
 
 constexpr int kThreads = 256;
@@ -77,17 +90,16 @@ __device__ __forceinline__ float dec_ordered(unsigned u) {
   return __uint_as_float((u & 0x80000000u) ? (u ^ 0x80000000u) : ~u);
 }
 
-// Eight consecutive logits as fp32 from their raw 16-byte vectors.
+// Eight consecutive logits as fp32 from their raw 16-byte vectors (bf16: byte permutes and masks, which
+// run on the ALU pipe; shifts would be issued as integer multiplies on the busier FMA pipe).
 template <int DT>
-__device__ __forceinline__ void unpack8(const uint4* v, float (&l)[8]) {
+__device__ __forceinline__ void unpack8(const uint4& a, const uint4& b, float (&l)[8]) {
   if (DT == ISD_LOGITS_BF16) {
-    const uint4 a = v[0];
-    l[0] = __uint_as_float(a.x << 16); l[1] = __uint_as_float(a.x & 0xFFFF0000u);
-    l[2] = __uint_as_float(a.y << 16); l[3] = __uint_as_float(a.y & 0xFFFF0000u);
-    l[4] = __uint_as_float(a.z << 16); l[5] = __uint_as_float(a.z & 0xFFFF0000u);
-    l[6] = __uint_as_float(a.w << 16); l[7] = __uint_as_float(a.w & 0xFFFF0000u);
+    l[0] = __uint_as_float(__byte_perm(a.x, 0u, 0x1044)); l[1] = __uint_as_float(a.x & 0xFFFF0000u);
+    l[2] = __uint_as_float(__byte_perm(a.y, 0u, 0x1044)); l[3] = __uint_as_float(a.y & 0xFFFF0000u);
+    l[4] = __uint_as_float(__byte_perm(a.z, 0u, 0x1044)); l[5] = __uint_as_float(a.z & 0xFFFF0000u);
+    l[6] = __uint_as_float(__byte_perm(a.w, 0u, 0x1044)); l[7] = __uint_as_float(a.w & 0xFFFF0000u);
   } else {
-    const uint4 a = v[0], b = v[1];
     l[0] = __uint_as_float(a.x); l[1] = __uint_as_float(a.y); l[2] = __uint_as_float(a.z); l[3] = __uint_as_float(a.w);
     l[4] = __uint_as_float(b.x); l[5] = __uint_as_float(b.y); l[6] = __uint_as_float(b.z); l[7] = __uint_as_float(b.w);
   }
@@ -96,63 +108,83 @@ __device__ __forceinline__ void unpack8(const uint4* v, float (&l)[8]) {
 // Eight consecutive logits starting at element e (e % 8 == 0), straight from global memory.
 template <int DT>
 __device__ __forceinline__ void load8(const void* row, int e, float (&l)[8]) {
-  uint4 v[2];
+  uint4 a, b = make_uint4(0u, 0u, 0u, 0u);
   if (DT == ISD_LOGITS_BF16) {
-    v[0] = ld_stream_16B(reinterpret_cast<const uint16_t*>(row) + e);
+    a = ld_stream_16B(reinterpret_cast<const uint16_t*>(row) + e);
   } else {
-    v[0] = ld_stream_16B(reinterpret_cast<const float*>(row) + e);
-    v[1] = ld_stream_16B(reinterpret_cast<const float*>(row) + e + 4);
+    a = ld_stream_16B(reinterpret_cast<const float*>(row) + e);
+    b = ld_stream_16B(reinterpret_cast<const float*>(row) + e + 4);
   }
-  unpack8<DT>(v, l);
+  unpack8<DT>(a, b, l);
 }
 
 // A row piece streamed through shared memory with per-thread asynchronous copies.  Every thread
-// fetches its own eight logits of the next kDepth iterations ahead of time (64 bytes in flight per
-// thread without holding registers) and later reads back exactly what it fetched itself, so no
-// barrier is needed.  The load latency, which bounds a pass that issues one load per iteration and
-// then computes on it, disappears behind the iterations in between.
-constexpr int kRingBytes = 16384;  // per CTA
-template <int DT>
+// fetches its own logits of the next kDepth iterations ahead of time (no registers held) and later
+// reads back exactly what it fetched itself, so no barrier is needed.  The load latency, which bounds
+// a pass that issues one load per iteration and then computes on it, disappears behind the iterations
+// in between.  U = groups of eight logits per thread and iteration (group g of thread t covers elements
+// base + g * kThreads * 8 + t * 8): the bookkeeping of an iteration is paid once for all of them.
+template <int DT, int U, int RING_BYTES>
 struct RowStream {
-  static constexpr int kVec = DT == ISD_LOGITS_BF16 ? 1 : 2;  // 16-byte vectors per thread and iteration
-  static constexpr int kDepth = kRingBytes / (kThreads * 16 * kVec);
-  static constexpr int kStep = kThreads * 8;                  // elements per iteration of the CTA
-  uint4* mine;      // this thread's vectors of stage 0; stage s is kThreads * kVec vectors further
-  const char* row;
-  int hi, stage;
+  static constexpr int kElt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  static constexpr int kVec = kElt / 2;                        // 16-byte vectors per group of eight logits
+  static constexpr int kGroupBytes = kThreads * 8 * kElt;      // one group of every thread
+  static constexpr int kStageBytes = U * kGroupBytes;
+  static constexpr int kDepth = RING_BYTES / kStageBytes;
+  static constexpr int kGroupStep = kThreads * 8;              // elements between a thread's groups
+  static constexpr int kStep = U * kGroupStep;                 // elements per iteration of the CTA
+  static_assert(kDepth >= 2 && (kDepth & (kDepth - 1)) == 0, "ring depth must be a power of two");
+  uint32_t sbase;   // shared-memory address of this thread's first vector in stage 0
+  uint32_t soff;    // byte offset of the stage that is read (and refilled) next
+  const char* src;  // global address of this thread's next fetch ...
+  int e_fetch;      // ... and its element index
+  int hi;
 
-  __device__ __forceinline__ void fetch(int s, int e) const {
-    if (e < hi) {
-      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(mine + s * kThreads * kVec);
-      const char* src = row + (size_t)e * (DT == ISD_LOGITS_BF16 ? 2 : 4);
+  __device__ __forceinline__ void fetch(uint32_t stage_off) {
 #pragma unroll
-      for (int v = 0; v < kVec; ++v)
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16 * v), "l"(src + 16 * v) : "memory");
+    for (int g = 0; g < U; ++g) {
+      if (e_fetch + g * kGroupStep < hi) {
+#pragma unroll
+        for (int v = 0; v < kVec; ++v)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sbase + stage_off + g * kGroupBytes + 16 * v),
+                       "l"(src + g * kGroupBytes + 16 * v)
+                       : "memory");
+      }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");  // one group per iteration, empty or not
+    src += kStageBytes;
+    e_fetch += kStep;
   }
-  __device__ __forceinline__ void start(uint4* ring, const char* row_, int lo, int hi_) {
-    mine = ring + threadIdx.x * kVec;
-    row = row_;
+  __device__ __forceinline__ void start(uint4* ring, const char* row, int lo, int hi_) {
+    sbase = (uint32_t)__cvta_generic_to_shared(ring) + threadIdx.x * 16 * kVec;
+    soff = 0;
+    e_fetch = lo + threadIdx.x * 8;
+    src = row + (size_t)e_fetch * kElt;
     hi = hi_;
-    stage = 0;
 #pragma unroll
-    for (int s = 0; s < kDepth; ++s) fetch(s, lo + s * kStep + threadIdx.x * 8);
+    for (int s = 0; s < kDepth; ++s) fetch(s * kStageBytes);
   }
-  // logits of this thread at element e (the iteration that started kDepth fetches ago); refills the stage
-  __device__ __forceinline__ void next(int e, float (&l)[8]) {
+  // this thread's logits of the iteration that was fetched kDepth fetches ago (the caller knows which of
+  // them exist); refills the stage
+  __device__ __forceinline__ void next(float (&l)[U][8]) {
     asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
-    if (e < hi) {
-      unpack8<DT>(mine + stage * kThreads * kVec, l);
-    } else {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) l[i] = -INFINITY;
+    for (int g = 0; g < U; ++g) {
+      uint4 a, b = make_uint4(0u, 0u, 0u, 0u);
+      const uint32_t addr = sbase + soff + g * kGroupBytes;
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "r"(addr) : "memory");
+      if (kVec == 2)
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "r"(addr + 16) : "memory");
+      unpack8<DT>(a, b, l[g]);
     }
-    fetch(stage, e + kDepth * kStep);
-    stage = (stage + 1) & (kDepth - 1);
+    fetch(soff);
+    soff = (soff + kStageBytes) & (RING_BYTES - 1);
   }
   __device__ __forceinline__ void finish() const { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 };
+constexpr int kRowStages = 4;            // row pass: bulk-copy ring of kRowStages x kRowStageBytes
+constexpr int kRowStageBytes = 8192;
+constexpr int kSampleRingBytes = 16384;  // sampling pass: one group per iteration
 
 __device__ __forceinline__ void chunk_range(int V, int splits, int split, int& lo, int& hi) {
   // chunks are multiples of 8 * kThreads elements so that every thread's vector stays aligned
@@ -161,7 +193,10 @@ __device__ __forceinline__ void chunk_range(int V, int splits, int split, int& l
   hi = min(V, lo + per);
 }
 
-// Block-wide merge helpers (8 warps) ------------------------------------------------------------
+// Barrier of the kThreads worker threads (a producer warp, where a kernel has one, stays out of it).
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+
+// Block-wide merge helpers (8 worker warps) -------------------------------------------------------
 __device__ __forceinline__ void block_merge_lse(float& m, float& s, float* sm_m, float* sm_s) {
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
@@ -171,22 +206,22 @@ __device__ __forceinline__ void block_merge_lse(float& m, float& s, float* sm_m,
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (lane == 0) { sm_m[warp] = m; sm_s[warp] = s; }
-  __syncthreads();
+  worker_sync();
   if (threadIdx.x == 0) {
     for (int w = 1; w < kThreads / 32; ++w) lse_merge(m, s, sm_m[w], sm_s[w]);
   }
-  __syncthreads();
+  worker_sync();
 }
 
 __device__ __forceinline__ void block_merge_top2(Top2& t, float* sm_s1, int* sm_i1, float* sm_s2, int* sm_i2) {
   warp_merge_top2(t);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (lane == 0) { sm_s1[warp] = t.s1; sm_i1[warp] = t.i1; sm_s2[warp] = t.s2; sm_i2[warp] = t.i2; }
-  __syncthreads();
+  worker_sync();
   if (threadIdx.x == 0) {
     for (int w = 1; w < kThreads / 32; ++w) t.merge(sm_s1[w], sm_i1[w], sm_s2[w], sm_i2[w]);
   }
-  __syncthreads();
+  worker_sync();
 }
 
 // fp64 score of vocabulary index i of a Gumbel row: logit * invT + g
@@ -196,86 +231,191 @@ __device__ double noisy_score_f64(const VerifyParams& P, const void* row, int i,
   return l + gumbel_f64(philox_word(r, i & 3));
 }
 
-// Online softmax of a thread's share of a row: the running max M of the raw logits and
-// S = sum exp((l - M) * invT), in the log2 domain with packed fp32x2 arithmetic.
+// Order-preserving map float <-> signed int (an involution), so that a warp can agree on a maximum with
+// one integer reduction.
+__device__ __forceinline__ int ord_key(float f) {
+  const int b = __float_as_int(f);
+  return b ^ ((b >> 31) & 0x7FFFFFFF);
+}
+__device__ __forceinline__ float ord_val(int k) { return __int_as_float(k ^ ((k >> 31) & 0x7FFFFFFF)); }
+
+// Online softmax of a thread's share of a row: S = sum exp((l - M) * invT) in the log2 domain, plain
+// scalar FFMA / ex2 / FADD with four independent partial sums (the packed fp32x2 forms cost more in
+// register-pair moves here than they save).  The reference point M is the running maximum of the WARP,
+// not of the thread: the warp agrees on it with one integer max-reduction per iteration, which makes
+// "the maximum grew" a warp-uniform and genuinely rare branch (about ln(iterations) times per row),
+// where per-thread maxima would send some lane of the warp into it in most iterations.
 struct OnlineSoftmax {
   float M, neg_ms, scale2;
-  uint64_t Sa, Sb, scale22;
+  int Mkey;
+  float S0, S1, S2, S3;
   __device__ __forceinline__ void init(float inv_t) {
     scale2 = inv_t * kLog2e;  // raw logit -> log2 domain
-    scale22 = pack2(scale2, scale2);
-    M = -INFINITY;            // running max of the raw logits
+    M = -INFINITY;            // running max of the raw logits seen by the warp
+    Mkey = ord_key(M);
     neg_ms = 0.f;             // -M * scale2 (0 while M = -inf, so that -inf logits give e = 0)
-    Sa = pack2(0.f, 0.f);     // two packed partial sums
-    Sb = Sa;
+    S0 = S1 = S2 = S3 = 0.f;
   }
-  // true when the maximum grew (rare after the first iterations)
-  __device__ __forceinline__ bool raise(float vmax) {
-    if (!(vmax > M)) return false;
-    const float f = (M == -INFINITY) ? 0.f : ex2f((M - vmax) * scale2);
-    const uint64_t f2 = pack2(f, f);
-    Sa = mul2(Sa, f2);
-    Sb = mul2(Sb, f2);
-    M = vmax;
+  __device__ __forceinline__ void raise_to(float new_m, int new_key) {
+    const float f = (M == -INFINITY) ? 0.f : ex2f((M - new_m) * scale2);
+    S0 *= f; S1 *= f; S2 *= f; S3 *= f;
+    M = new_m;
+    Mkey = new_key;
     neg_ms = -M * scale2;
-    return true;
   }
   __device__ __forceinline__ void add8(const float (&l)[8]) {
-    const uint64_t nm2 = pack2(neg_ms, neg_ms);
-    float ex[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float x0, x1;
-      unpack2(fma2(pack2(l[2 * i], l[2 * i + 1]), scale22, nm2), x0, x1);
-      ex[2 * i] = ex2f(x0);
-      ex[2 * i + 1] = ex2f(x1);
-    }
-    Sa = add2(Sa, pack2(ex[0], ex[1]));
-    Sb = add2(Sb, pack2(ex[2], ex[3]));
-    Sa = add2(Sa, pack2(ex[4], ex[5]));
-    Sb = add2(Sb, pack2(ex[6], ex[7]));
+    S0 += ex2f(fmaf(l[0], scale2, neg_ms));
+    S1 += ex2f(fmaf(l[1], scale2, neg_ms));
+    S2 += ex2f(fmaf(l[2], scale2, neg_ms));
+    S3 += ex2f(fmaf(l[3], scale2, neg_ms));
+    S0 += ex2f(fmaf(l[4], scale2, neg_ms));
+    S1 += ex2f(fmaf(l[5], scale2, neg_ms));
+    S2 += ex2f(fmaf(l[6], scale2, neg_ms));
+    S3 += ex2f(fmaf(l[7], scale2, neg_ms));
   }
-  __device__ __forceinline__ float sum() const {
-    float s0, s1, s2, s3;
-    unpack2(Sa, s0, s1);
-    unpack2(Sb, s2, s3);
-    return (s0 + s1) + (s2 + s3);
-  }
+  __device__ __forceinline__ float sum() const { return (S0 + S1) + (S2 + S3); }
 };
 
-// One streaming pass over elements [lo, hi) of a logits row: online softmax and the raw argmax
-// (lowest index on ties), which is the running max itself.
+__device__ __forceinline__ float max8(const float (&l)[8]) {
+  return fmaxf(max3(l[0], l[1], l[2]), max3(max3(l[3], l[4], l[5]), l[6], l[7]));
+}
+
+// Shared memory of the row pass: the ring and its barriers.
+struct RowRing {
+  __align__(128) unsigned char stage[kRowStages][kRowStageBytes];
+  __align__(8) uint64_t full[kRowStages];   // a stage's bytes have landed (one arrival + transaction bytes)
+  __align__(8) uint64_t empty[kRowStages];  // every worker warp has read the stage (one arrival per warp)
+};
+
+// Producer (one thread): streams bytes [byte_lo, byte_hi) of a row into the ring, one contiguous bulk copy
+// per stage.  Returns false when a wait ran out.
+__device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t byte_lo, size_t byte_hi) {
+  const uint32_t full0 = ring_smem_u32(R.full), empty0 = ring_smem_u32(R.empty), st0 = ring_smem_u32(R.stage);
+  int c = 0;
+  for (size_t off = byte_lo; off < byte_hi; off += kRowStageBytes, ++c) {
+    const int s = c & (kRowStages - 1);
+    const uint32_t ph = (c / kRowStages) & 1;
+    if (!ring_mbar_wait(empty0 + 8 * s, ph ^ 1)) return false;
+    const size_t left = byte_hi - off;
+    const uint32_t bytes = left < (size_t)kRowStageBytes ? (uint32_t)left : (uint32_t)kRowStageBytes;
+    ring_mbar_expect_tx(full0 + 8 * s, bytes);
+    ring_bulk_g2s(st0 + s * kRowStageBytes, row + off, bytes, full0 + 8 * s);
+  }
+  return true;
+}
+
+// Worker side of one streaming pass over elements [lo, hi) of a logits row: online softmax (m_nat, S
+// relative to the warp's maximum) and this thread's argmax candidate of the raw logits.  A thread
+// records (value, position) only when one of its elements sets a new maximum of the warp, strictly
+// above everything the warp saw before; merging the candidates by (value, lowest index) gives the first
+// occurrence of the row maximum.  Thread t reads vectors t, t + kThreads, ... of a stage (bf16: two
+// groups of eight logits per stage; fp32: one group from two adjacent vectors).
 template <int DT>
-__device__ __forceinline__ void row_pass(const VerifyParams& P, const char* row, int lo, int hi,
-                                         float& m_nat, float& S_out, float& raw_max, int& raw_idx, uint4* ring) {
+__device__ __forceinline__ bool row_pass(const VerifyParams& P, RowRing& R, const char* row, int lo, int hi,
+                                         float& m_nat, float& S_out, float& raw_max, int& raw_idx) {
+  constexpr int kElt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  constexpr int U = DT == ISD_LOGITS_BF16 ? 2 : 1;      // groups of eight logits per thread and stage
+  constexpr int kStageElems = kRowStageBytes / kElt;
+  constexpr int kGroupStep = kStageElems / U;           // elements between a thread's groups
+  const uint32_t full0 = ring_smem_u32(R.full), empty0 = ring_smem_u32(R.empty);
+  const uint32_t mine = ring_smem_u32(R.stage) + threadIdx.x * (DT == ISD_LOGITS_BF16 ? 16 : 32);
+  const int lane = threadIdx.x & 31;
   OnlineSoftmax os;
   os.init(P.inv_t);
+  raw_max = -INFINITY;
   raw_idx = -1;
-  RowStream<DT> in;
-  in.start(ring, row, lo, hi);
-  for (int base = lo; base < hi; base += kThreads * 8) {
-    const int e = base + threadIdx.x * 8;
-    float l[8];
-    in.next(e, l);
-    const float vmax = fmaxf(max3(l[0], l[1], l[2]), max3(max3(l[3], l[4], l[5]), l[6], l[7]));
-    if (os.raise(vmax)) {
-#pragma unroll
-      for (int i = 7; i >= 0; --i)
-        if (l[i] == vmax) raw_idx = e + i;
+  int raw_e = -1;  // first element of the stage in which this thread set the warp's maximum
+  bool ok = true;
+
+  // called by all lanes of the warp together
+  auto consume = [&](const float (&l)[U][8], int e) {
+    float vmax = max8(l[0]);
+    if (U == 2) vmax = fmaxf(vmax, max8(l[U - 1]));
+    const int wkey = __reduce_max_sync(0xffffffffu, ord_key(vmax));
+    if (__builtin_expect(wkey > os.Mkey, 0)) {  // warp-uniform, rare
+      const float wmax = ord_val(wkey);
+      os.raise_to(wmax, wkey);
+      if (vmax == wmax) {  // which element it was is looked up once, after the loop
+        raw_max = wmax;
+        raw_e = e;
+      }
     }
-    os.add8(l);
+#pragma unroll
+    for (int g = 0; g < U; ++g) os.add8(l[g]);
+  };
+  // s = stage (a compile-time constant in the unrolled main loop), ph = parity of its current fill
+  auto read_stage = [&](int s, uint32_t ph, float (&l)[U][8]) {
+    ok = ok && mbar_wait_likely(full0 + 8 * s, ph);
+    const uint32_t base = mine + s * kRowStageBytes;
+#pragma unroll
+    for (int g = 0; g < U; ++g) {
+      uint4 a, b = make_uint4(0u, 0u, 0u, 0u);
+      const uint32_t addr = base + g * (kRowStageBytes / U);
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "r"(addr) : "memory");
+      if (DT != ISD_LOGITS_BF16)
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "r"(addr + 16) : "memory");
+      unpack8<DT>(a, b, l[g]);
+    }
+    __syncwarp();
+    if (lane == 0) ring_mbar_arrive(empty0 + 8 * s);  // the values are in registers: the stage may be refilled
+  };
+
+  // Stages in which every thread has all its data need no checks; the ragged last one is peeled.  The main
+  // loop takes one trip round the ring per iteration, so stage numbers are constants and the parity flips
+  // once per iteration.
+  const int n = hi > lo ? hi - lo : 0;
+  const int full = n / kStageElems;
+  int e = lo + threadIdx.x * 8;
+  int c = 0;
+  uint32_t ph = 0;
+  for (; c + kRowStages <= full; c += kRowStages, ph ^= 1) {
+#pragma unroll
+    for (int s = 0; s < kRowStages; ++s, e += kStageElems) {
+      float l[U][8];
+      read_stage(s, ph, l);
+      consume(l, e);
+    }
   }
-  in.finish();
+  for (; c < full; ++c, e += kStageElems) {  // fewer than kRowStages left: stages 0, 1, ... of this round
+    float l[U][8];
+    read_stage(c & (kRowStages - 1), ph, l);
+    consume(l, e);
+  }
+  if (full * kStageElems < n) {  // uniform over the CTA
+    float l[U][8];
+    read_stage(c & (kRowStages - 1), ph, l);
+#pragma unroll
+    for (int g = 0; g < U; ++g)
+      if (!(e + g * kGroupStep < hi)) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) l[g][i] = -INFINITY;
+      }
+    consume(l, e);
+  }
+  if (raw_e >= 0) {
+    // lowest index among this thread's elements of that stage that holds the recorded maximum
+#pragma unroll
+    for (int g = U - 1; g >= 0; --g) {
+      const int eg = raw_e + g * kGroupStep;
+      if (eg < hi) {
+        float l[8];
+        load8<DT>(row, eg, l);
+#pragma unroll
+        for (int i = 7; i >= 0; --i)
+          if (l[i] == raw_max) raw_idx = eg + i;
+      }
+    }
+  }
   S_out = os.sum();
   m_nat = os.M * P.inv_t;
-  raw_max = os.M;
+  return ok;
 }
 
 // ------------------------------------------------------------------------------------------------
 // Pass 1: row statistics + decision
 // ------------------------------------------------------------------------------------------------
 template <int DT>
-__global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParams P) {
+__global__ void __launch_bounds__(kThreads + 32) verify_rows_kernel(const VerifyParams P) {
   // Launch order = (split, slot, k): the rows that the sampling pass reads again come last, so that
   // they are the most recent lines in L2 when it starts.
   const int split = blockIdx.x, b = blockIdx.y, k = blockIdx.z;
@@ -296,16 +436,34 @@ __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParam
   __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
   __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
   __shared__ int sm_last;
-  __shared__ __align__(16) uint4 sm_ring[kRingBytes / 16];
+  __shared__ RowRing sm_ring;
 
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
   int lo, hi;
   chunk_range(P.V, P.row_splits, split, lo, hi);
 
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kRowStages; ++i) {
+      ring_mbar_init(ring_smem_u32(&sm_ring.full[i]), 1);
+      ring_mbar_init(ring_smem_u32(&sm_ring.empty[i]), kThreads / 32);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x >= kThreads) {
+    // producer warp: one thread feeds the ring, then the warp is done (every copy it issued is consumed
+    // by the workers before they leave; a wait that runs out raises the status bit and stops feeding)
+    if (threadIdx.x == kThreads && hi > lo) {
+      if (!row_producer(sm_ring, row, (size_t)lo * elt, (size_t)hi * elt)) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+    }
+    return;
+  }
+
   float m_nat, S, raw_max;
   int raw_idx;
-  row_pass<DT>(P, row, lo, hi, m_nat, S, raw_max, raw_idx, sm_ring);
+  if (!row_pass<DT>(P, sm_ring, row, lo, hi, m_nat, S, raw_max, raw_idx) && threadIdx.x == 0)
+    atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
 
   // ---- block reduction -> partial
   block_merge_lse(m_nat, S, sm_f0, sm_f1);
@@ -321,7 +479,7 @@ __global__ void __launch_bounds__(kThreads) verify_rows_kernel(const VerifyParam
     const int arrived = atomicAdd(&P.row_ticket[b], 1);
     sm_last = (arrived == q_len * P.row_splits - 1);
   }
-  __syncthreads();
+  worker_sync();
   if (!sm_last) return;
 
   // ---- decision phase: last CTA of the slot, warp 0 -------------------------------------------
@@ -477,7 +635,7 @@ struct SampleQueue {
 template <int DT>
 __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJob& J, int lo, int hi, int b,
                                             float best, Top2& top, SampleQueue& Q, unsigned* sm_best, uint4* ring) {
-  RowStream<DT> in;
+  RowStream<DT, 1, kSampleRingBytes> in;
   in.start(ring, J.prow, lo, hi);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const unsigned below = (1u << lane) - 1u;
@@ -498,6 +656,7 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
     const float l4[4] = {v.x, v.y, v.z, v.w};
     const uint4 rnd = philox4x32_10((uint32_t)idx >> 2, P.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
     const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+    DBG_COUNT(J.resid ? 1 : 0, 1);
     // -ln u' >= 1 - u' >= nf 2^-24 with nf = floor(2^24 (1 - u')), so g_i <= -ln(nf 2^-24): the element
     // cannot come within 2e-3 of the running best when nf >= 1.002 * 2^24 * exp(l_i invT - shift - best)
     float K2 = 24.0028853901f - (shift + best) * kLog2e;  // log2 of the factor; +inf while there is no best
@@ -507,6 +666,7 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
       const float nf = (float)((~w[i]) >> 8);
       const float bound = ex2f(fmaf(l4[i], scale2, K2));
       if (!(nf >= bound)) {
+        DBG_COUNT(J.resid ? 3 : 2, 1);
         const float sc = job_score(P, J, l4[i], idx + i, w[i]);
         if (sc > -INFINITY) {
           top.push(sc, idx + i);
@@ -524,8 +684,13 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
   // uniform trip count per block (the warp votes inside the loop)
   for (int base = lo; base < hi; base += kThreads * 8) {
     const int e = base + threadIdx.x * 8;
-    float l[8];
-    in.next(e, l);
+    float lg[1][8];
+    in.next(lg);
+    float (&l)[8] = lg[0];
+    if (!(e < hi)) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) l[i] = -INFINITY;
+    }
     best = fmaxf(best, dec_ordered(*reinterpret_cast<volatile unsigned*>(sm_best)));
     const float cut = fmaf(best, rcp_t, cut_off);  // raw-logit units; -inf while there is no best
     const float g0 = fmaxf(fmaxf(l[0], l[1]), fmaxf(l[2], l[3]));
@@ -570,7 +735,7 @@ __global__ void __launch_bounds__(kThreads) verify_sample_kernel(const VerifyPar
   __shared__ int sm_last, sm_tok;
   __shared__ unsigned sm_best;
   __shared__ SampleQueue sm_queue;
-  __shared__ __align__(16) uint4 sm_ring[kRingBytes / 16];
+  __shared__ __align__(16) uint4 sm_ring[kSampleRingBytes / 16];
 
   const int NP = P.N - 1;
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
@@ -615,6 +780,7 @@ __global__ void __launch_bounds__(kThreads) verify_sample_kernel(const VerifyPar
 
   int lo, hi;
   chunk_range(P.V, P.sample_splits, split, lo, hi);
+  if (threadIdx.x == 0) { DBG_COUNT(J.resid ? 5 : 4, (hi - lo) / 4); if (J.resid && !(best0 > -INFINITY)) DBG_COUNT(6, 1); }
   Top2 top;
   sample_pass<DT>(P, J, lo, hi, b, fmaxf(-INFINITY, best0), top, sm_queue, &sm_best, sm_ring);
 
@@ -713,10 +879,10 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   const dim3 grid2(ctx->sample_splits, c.propose_mode == 0 ? c.stride : 1, c.batch);
   if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
   if (c.logits_dtype == ISD_LOGITS_BF16) {
-    verify_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads, 0, stream>>>(P);
+    verify_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads + 32, 0, stream>>>(P);
     verify_sample_kernel<ISD_LOGITS_BF16><<<grid2, kThreads, 0, stream>>>(P);
   } else {
-    verify_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads, 0, stream>>>(P);
+    verify_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads + 32, 0, stream>>>(P);
     verify_sample_kernel<ISD_LOGITS_F32><<<grid2, kThreads, 0, stream>>>(P);
   }
   if (ctx->ev_verify1) cudaEventRecord(ctx->ev_verify1, stream);
