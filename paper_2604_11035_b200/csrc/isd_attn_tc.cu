@@ -912,21 +912,32 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
 // Combine: pairs whose tiles were split over several CTAs (log-sum-exp merge of the partials)
 // ------------------------------------------------------------------------------------------------
 // One CTA per share of the main kernel: CTA c merges the pair that starts inside share c and runs on
-// into later shares (every split pair has exactly one such share).
-__global__ void __launch_bounds__(256) attn_combine_kernel(const TcParams P) {
+// into later shares (every split pair has exactly one such share).  The kernel is pure latency (a few
+// dependent rounds of small loads), so it is laid out wide: the slot of the share's last tile is found by
+// a counting vote over the tile prefix instead of a binary search of dependent loads, and one warp per
+// block row merges all partials of its row in a single round.
+constexpr int kCombineThreads = 1024;
+__global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const TcParams P) {
   const int c0 = blockIdx.x;
   const long long total = (long long)P.tile_prefix[P.B] * P.Hkv;
   if (total == 0) return;
   const long long per = (total + P.num_ctas - 1) / P.num_ctas;
   const long long t_last = ((long long)(c0 + 1) * per < total ? (long long)(c0 + 1) * per : total) - 1;
   if (t_last < (long long)c0 * per) return;  // empty share
-  // slot and kv head of the share's last tile
-  int lo = 0, hi = P.B;
-  while (lo < hi) {
-    const int mid = (lo + hi) >> 1;
-    if ((long long)P.tile_prefix[mid + 1] * P.Hkv > t_last) hi = mid; else lo = mid + 1;
+  // slot of the share's last tile = number of slots whose tiles all lie at or before t_last
+  __shared__ int sm_cnt;
+  if (threadIdx.x == 0) sm_cnt = 0;
+  __syncthreads();
+  {
+    int cnt = 0;
+    for (int i = threadIdx.x; i < P.B; i += kCombineThreads)
+      cnt += ((long long)P.tile_prefix[i + 1] * P.Hkv <= t_last) ? 1 : 0;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+    if ((threadIdx.x & 31) == 0 && cnt) atomicAdd(&sm_cnt, cnt);
   }
-  const int b = lo;
+  __syncthreads();
+  const int b = sm_cnt;
   const int T = P.tile_prefix[b + 1] - P.tile_prefix[b];
   const int g = (int)((t_last - (long long)P.tile_prefix[b] * P.Hkv) / T);
   const long long p0 = (long long)P.tile_prefix[b] * P.Hkv + (long long)g * T, p1 = p0 + T;
@@ -937,23 +948,50 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const TcParams P) {
   // replicas of a row (key split across lane groups, see softmax_segment) are further partials
   const int F = rows_valid > 64 ? 1 : (rows_valid > 32 ? 2 : 4);
   const int RG = 128 / F;
-  for (int row = threadIdx.x >> 5; row < rows_valid; row += 8) {
-    const int lane = threadIdx.x & 31;
-    float M = -INFINITY;
-    for (int c = c_first; c <= c_last; ++c) {
-      const int slot = c * 2 + (((long long)c * per >= p0) ? 0 : 1);
-      for (int pp = 0; pp < F; ++pp) M = fmaxf(M, P.part_ml[((size_t)slot * 128 + pp * RG + row) * 2]);
-    }
-    float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int c = c_first; c <= c_last; ++c) {
-      const int slot = c * 2 + (((long long)c * per >= p0) ? 0 : 1);
-      for (int pp = 0; pp < F; ++pp) {
-        const size_t rr = (size_t)slot * 128 + pp * RG + row;
-        const float m = P.part_ml[rr * 2], l = P.part_ml[rr * 2 + 1];
-        const float w = (m == -INFINITY) ? 0.f : ex2f(m - M);
-        L += l * w;
-        const float4 o = *reinterpret_cast<const float4*>(P.part_o + rr * 128 + lane * 4);
-        acc[0] += o.x * w; acc[1] += o.y * w; acc[2] += o.z * w; acc[3] += o.w * w;
+  const int lane = threadIdx.x & 31;
+  const int n_part = (c_last - c_first + 1) * F;  // partials of a row: lane i < n_part fetches the i-th (max, sum)
+  for (int row = threadIdx.x >> 5; row < rows_valid; row += kCombineThreads / 32) {
+    float M = -INFINITY, L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int base = 0; base < n_part; base += 32) {
+      // one round of loads for up to 32 partials: every lane reads one (max, sum) pair
+      float m_i = -INFINITY, l_i = 0.f;
+      size_t rr_i = 0;
+      if (base + lane < n_part) {
+        const int c = c_first + (base + lane) / F, pp = (base + lane) % F;
+        const int slot = c * 2 + (((long long)c * per >= p0) ? 0 : 1);
+        rr_i = (size_t)slot * 128 + pp * RG + row;
+        const float2 ml = *reinterpret_cast<const float2*>(P.part_ml + rr_i * 2);
+        m_i = ml.x;
+        l_i = ml.y;
+      }
+      float Mn = m_i;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) Mn = fmaxf(Mn, __shfl_xor_sync(0xffffffffu, Mn, off));
+      Mn = fmaxf(Mn, M);
+      const float keep = (M == -INFINITY) ? 0.f : ex2f(M - Mn);
+      L *= keep;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[i] *= keep;
+      M = Mn;
+      const float w_i = (m_i == -INFINITY) ? 0.f : ex2f(m_i - M);
+      const int cnt = min(32, n_part - base);
+      for (int i = 0; i < cnt; i += 4) {  // four independent loads in flight
+        float4 o[4];
+        float w[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int ii = min(i + u, cnt - 1);
+          const float wu = __shfl_sync(0xffffffffu, w_i, ii);
+          const float lu = __shfl_sync(0xffffffffu, l_i, ii);
+          const size_t rr = __shfl_sync(0xffffffffu, (unsigned long long)rr_i, ii);
+          w[u] = (i + u < cnt) ? wu : 0.f;
+          L += lu * w[u];
+          o[u] = *reinterpret_cast<const float4*>(P.part_o + rr * 128 + lane * 4);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          acc[0] += o[u].x * w[u]; acc[1] += o[u].y * w[u]; acc[2] += o[u].z * w[u]; acc[3] += o[u].w * w[u];
+        }
       }
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
@@ -1063,7 +1101,7 @@ int isd_launch_attn_tc(isd_ctx* ctx, const isd_batch_state* st, const void* q, c
   if (ctx->ev_attn0) cudaEventRecord(ctx->ev_attn0, stream);
   attn_tc_kernel<<<ctx->attn_ctas, kThreads, kSmemBytes, stream>>>(P, h->map_k, h->map_v);
   if (ctx->ev_attn1) cudaEventRecord(ctx->ev_attn1, stream);
-  attn_combine_kernel<<<ctx->attn_ctas, 256, 0, stream>>>(P);
+  attn_combine_kernel<<<ctx->attn_ctas, kCombineThreads, 0, stream>>>(P);
   ctx->launches += 2 + (c.batch > kMaxSmemPrefixSlots ? 1 : 0);
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }
