@@ -98,9 +98,14 @@ def algorithmic_bytes(w, ctx_len, q_len, rejecting: int):
     return attn, verify
 
 
-def rank_workload(config_index: int, rank: int):
+def rank_workload(config_index: int, rank: int, sweep: str | None = None):
     """Workload of one rank: ranks own disjoint slots with their own pools, so each gets its own seed."""
+    from dataclasses import replace
     from paper_2604_11035_b200 import workloads as wl
+    if sweep:
+        stride, batch = (int(x) for x in sweep.split(","))
+        base = wl.sweep_point(stride, batch)
+        return replace(base, seed=base.seed + 1000 * rank)
     base = wl.config(config_index)
     return wl.config(config_index, seed=base.seed + 1000 * rank)
 
@@ -130,7 +135,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     # weak scaling: every rank owns its own slots, pools and free stack (slots never interact)
-    w = rank_workload(args.config, rank)
+    w = rank_workload(args.config, rank, args.sweep)
     if args.propose_mode is not None:
         from dataclasses import replace
         w = replace(w, propose_mode=args.propose_mode)
@@ -397,6 +402,8 @@ def main():
     ap.add_argument("--cpu-slots", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (smaller captures under ncu)")
+    ap.add_argument("--sweep", default=None, metavar="STRIDE,BATCH",
+                    help="one point of the sweep workload (stride in 2,4,8,16; batch in 1,8,64,256,512) instead of --config")
     ap.add_argument("--sequential-pages", action="store_true", help="identity page order instead of a shuffled pool")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
