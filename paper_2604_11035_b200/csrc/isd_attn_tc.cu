@@ -35,6 +35,10 @@ namespace {
 constexpr int kTile = 128;                 // keys per tile
 constexpr int kStageBytes = 32768;         // one K or V tile: [half(2)][page(8)][tok(16)][128 B]
 constexpr int kStages = 6;
+#ifndef ISD_SEG_COST
+#define ISD_SEG_COST 4
+#endif
+constexpr int kSegCost = ISD_SEG_COST;  // fixed cost of a segment in units of one tile's time (split axis)
 constexpr int kThreads = 256;
 constexpr int kProducerWarps = 3;        // warps 4..6 issue the TMA copies round-robin, warp 7 issues the MMAs
 constexpr int kSmRing = 0;
@@ -69,7 +73,7 @@ struct TcParams {
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
   float* lse;
-  int* tile_prefix;  // [B + 1] tiles per kv head, exclusive prefix over slots
+  int* tile_prefix;  // [B + 1] split-axis length (tiles + kSegCost) per kv head, exclusive prefix over slots
   float* part_o;     // [ctas * 2][128][128]
   float* part_ml;    // [ctas * 2][128][2]
   int num_ctas;
@@ -250,39 +254,51 @@ struct WorkIter {
     b = lo;
   }
   __device__ bool next(const TcParams& P, int cta, Segment& s) {
-    if (t >= t_end) return false;
-    while (b < B && (long long)prefix[b + 1] * Hkv <= t) ++b;
-    if (b >= B) return false;
-    const int T = prefix[b + 1] - prefix[b];
-    const long long off = t - (long long)prefix[b] * Hkv;
-    s.b = b; s.T = T;
-    s.g = (int)(off / T);
-    s.j0 = (int)(off % T);
-    const long long room = t_end - t;
-    s.j1 = (long long)(T - s.j0) <= room ? T : s.j0 + (int)room;
-    if (slot_info) {
-      const int w = slot_info[b];
-      s.ctx = w & 0xFFFFFF;
-      s.q_len = (int)((unsigned)w >> 24);
-    } else {
-      s.ctx = P.ctx_len[b];
-      s.q_len = P.n_ver[b] + P.N;
+    for (;;) {
+      if (t >= t_end) return false;
+      while (b < B && (long long)prefix[b + 1] * Hkv <= t) ++b;
+      if (b >= B) return false;
+      // positions of a pair on the split axis: kSegCost units of fixed cost, then its tiles
+      const int Tv = prefix[b + 1] - prefix[b];
+      const long long off = t - (long long)prefix[b] * Hkv;
+      const int v0 = (int)(off % Tv);
+      const long long room = t_end - t;
+      const int v1 = (long long)(Tv - v0) <= room ? Tv : v0 + (int)room;
+      const bool first = (t == t_begin);
+      t += v1 - v0;
+      const int T = Tv - kSegCost;
+      s.j0 = v0 > kSegCost ? v0 - kSegCost : 0;
+      s.j1 = v1 > kSegCost ? v1 - kSegCost : 0;
+      if (s.j1 <= s.j0) continue;  // only (part of) the fixed-cost units of the pair fell into this share
+      s.b = b; s.T = T;
+      s.g = (int)(off / Tv);
+      if (slot_info) {
+        const int w = slot_info[b];
+        s.ctx = w & 0xFFFFFF;
+        s.q_len = (int)((unsigned)w >> 24);
+      } else {
+        s.ctx = P.ctx_len[b];
+        s.q_len = P.n_ver[b] + P.N;
+      }
+      s.kv_len = s.ctx + s.q_len;
+      const bool whole = (s.j0 == 0 && s.j1 == T);
+      s.part_slot = whole ? -1 : cta * 2 + (first ? 0 : 1);
+      return true;
     }
-    s.kv_len = s.ctx + s.q_len;
-    const bool whole = (s.j0 == 0 && s.j1 == T);
-    s.part_slot = whole ? -1 : cta * 2 + (t == t_begin ? 0 : 1);
-    t += s.j1 - s.j0;
-    return true;
   }
 };
 
+// Length of a slot's (slot, kv head) pairs on the split axis: its 128-key tiles plus kSegCost units for the
+// fixed cost of a segment (Q staging, pipeline fill and drain, epilogue: measured at about the time of four
+// tiles).  Shares of equal length on this axis take equal time whether they hold a few long pairs or many
+// short ones; with tiles alone the CTAs with the most segments finished 10 % after the average.
 __device__ __forceinline__ int slot_tiles(const TcParams& P, int b) {
   if (b >= P.B || !P.active[b]) return 0;
   const int nv = P.n_ver[b];
   const int ctx = P.ctx_len[b];
   const bool ok = nv >= 0 && nv <= P.N - 1 && ctx >= 0 &&
                   (P.slot_status[b] & (ISD_ST_BAD_PAGE_ID | ISD_ST_SLOT_CAPACITY)) == 0;
-  return ok ? (ctx + nv + P.N + kTile - 1) / kTile : 0;
+  return ok ? (ctx + nv + P.N + kTile - 1) / kTile + kSegCost : 0;
 }
 
 // Exclusive prefix of tiles per slot, computed by the 256 threads of a main-kernel CTA into shared
@@ -938,10 +954,10 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const TcP
   }
   __syncthreads();
   const int b = sm_cnt;
-  const int T = P.tile_prefix[b + 1] - P.tile_prefix[b];
+  const int T = P.tile_prefix[b + 1] - P.tile_prefix[b];  // on the split axis: kSegCost units, then the tiles
   const int g = (int)((t_last - (long long)P.tile_prefix[b] * P.Hkv) / T);
   const long long p0 = (long long)P.tile_prefix[b] * P.Hkv + (long long)g * T, p1 = p0 + T;
-  const int c_first = (int)(p0 / per), c_last = (int)((p1 - 1) / per);
+  const int c_first = (int)((p0 + kSegCost) / per), c_last = (int)((p1 - 1) / per);  // shares that hold tiles of the pair
   if (c_first != c0 || c_last == c0) return;  // merged by an earlier share, or written directly
   const int q_len = P.n_ver[b] + P.N;
   const int rows_valid = q_len * P.G;
