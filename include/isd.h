@@ -202,6 +202,42 @@ int isd_commit(isd_ctx* ctx, isd_batch_state* st, const isd_verify_out* out, voi
 int isd_step(isd_ctx* ctx, isd_batch_state* st, const isd_step_args* args, uint64_t step,
              void* cuda_stream);
 
+/* One transformer layer's share of a step: its queries, the block's keys / values, its KV pools and its
+ * output (same shapes and meaning as the fields of isd_step_args). */
+typedef struct isd_layer_args {
+  const void* q;
+  const void* k_new;
+  const void* v_new;
+  void* k_pool;
+  void* v_pool;
+  void* attn_out;
+  float* attn_lse; /* or NULL */
+} isd_layer_args;
+
+/*
+ * A whole model step (Sec. 3.3: the 2N-1 row block goes through every layer of the model in one
+ * forward pass, then verify -> trim -> prepare): isd_attn for each of the n_layers layers in order,
+ * all through the same state (one page table and one set of lengths shared by the layers, each
+ * layer with its own pools), then isd_verify on the logits and isd_commit.  `layers` is a host array
+ * of n_layers >= 1 entries; everything else as in isd_step.  No host synchronisation and no
+ * allocation happen inside, so the call (like isd_step) may be recorded into a CUDA graph by stream
+ * capture on `cuda_stream`; see isd_set_step_counter for the step number of a replayed graph.
+ */
+int isd_step_layers(isd_ctx* ctx, isd_batch_state* st, const isd_layer_args* layers, int32_t n_layers,
+                    const void* logits_cur, const void* q_prev_logits, const isd_verify_out* out,
+                    uint64_t step, void* cuda_stream);
+
+/*
+ * Step number for CUDA-graph replay (Sec. 3.3 (2): the captured extend graph is replayed with its
+ * metadata updated in place).  The `step` argument of isd_verify / isd_step is a host value that a
+ * captured graph would freeze, and every replay would draw the same random numbers.  With a
+ * device counter set (device pointer to one uint32, owned by the caller, initialised by the
+ * caller), isd_verify reads the step number from it and ignores its `step` argument, and
+ * isd_commit adds one to it after committing, so that replay k of a captured step runs as step
+ * counter0 + k.  NULL (the default) switches back to the host argument.
+ */
+int isd_set_step_counter(isd_ctx* ctx, uint32_t* device_counter);
+
 /* Off the hot path: return the pages of finished slots (device array `slots`
  * of n ids) to the free stack and mark them inactive. */
 int isd_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t n,

@@ -19,7 +19,7 @@ ST_BAD_PAGE_ID, ST_NONFINITE_LOGIT, ST_EMPTY_RESIDUAL = 8, 16, 32
 
 EXPORTS = ["isd_create", "isd_destroy", "isd_attn", "isd_verify", "isd_commit", "isd_step",
            "isd_release", "isd_read_status", "isd_set_profile_events", "isd_launch_count", "isd_strerror",
-           "isd_verify_static"]
+           "isd_verify_static", "isd_step_layers", "isd_set_step_counter"]
 
 
 class IsdConfig(C.Structure):
@@ -47,6 +47,10 @@ class IsdStepArgs(C.Structure):
         [("out", IsdVerifyOut)]
 
 
+class IsdLayerArgs(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("q", "k_new", "v_new", "k_pool", "v_pool", "attn_out", "attn_lse")]
+
+
 _lib = None
 
 
@@ -72,6 +76,11 @@ def load():
         lib.isd_verify_static.argtypes = [C.POINTER(IsdConfig), C.POINTER(IsdBatchState), vp, vp, C.c_uint64,
                                           C.POINTER(IsdVerifyOut), vp]
         lib.isd_verify_static.restype = C.c_int
+        lib.isd_step_layers.argtypes = [vp, C.POINTER(IsdBatchState), C.POINTER(IsdLayerArgs), C.c_int32, vp, vp,
+                                        C.POINTER(IsdVerifyOut), C.c_uint64, vp]
+        lib.isd_step_layers.restype = C.c_int
+        lib.isd_set_step_counter.argtypes = [vp, vp]
+        lib.isd_set_step_counter.restype = C.c_int
         lib.isd_launch_count.argtypes = [vp]
         lib.isd_launch_count.restype = C.c_int64
         lib.isd_strerror.argtypes = [C.c_int]
@@ -181,6 +190,26 @@ class Isd:
     def isd_step(self, st, args: IsdStepArgs, step: int, st_struct: IsdBatchState | None = None):
         s = st_struct if st_struct is not None else self.state_struct(st)
         _check(self.lib.isd_step(self.ctx, C.byref(s), C.byref(args), step, _stream()), "isd_step")
+
+    def layer_args(self, layers):
+        """Host array of isd_layer_args from dicts with q, k_new, v_new, k_pool, v_pool, attn_out[, attn_lse]."""
+        arr = (IsdLayerArgs * len(layers))()
+        for i, a in enumerate(layers):
+            arr[i] = IsdLayerArgs(_ptr(a["q"]), _ptr(a["k_new"]), _ptr(a["v_new"]), _ptr(a["k_pool"]), _ptr(a["v_pool"]),
+                                  _ptr(a["attn_out"]), _ptr(a.get("attn_lse")))
+        return arr
+
+    def isd_step_layers(self, st, layers, logits_cur, q_prev_logits, out, step: int,
+                        st_struct: IsdBatchState | None = None):
+        """`layers`: what layer_args returned (keep it alive across calls that reuse it)."""
+        s = st_struct if st_struct is not None else self.state_struct(st)
+        o = self.out_struct(out)
+        _check(self.lib.isd_step_layers(self.ctx, C.byref(s), layers, len(layers), _ptr(logits_cur),
+                                        _ptr(q_prev_logits), C.byref(o), step, _stream()), "isd_step_layers")
+
+    def isd_set_step_counter(self, counter):
+        """`counter`: a CUDA uint32 / int32 tensor of one element, or None."""
+        _check(self.lib.isd_set_step_counter(self.ctx, _ptr(counter)), "isd_set_step_counter")
 
     def isd_release(self, st, slots):
         s = self.state_struct(st)

@@ -181,6 +181,27 @@ int isd_step(isd_ctx* ctx, isd_batch_state* st, const isd_step_args* a, uint64_t
   return isd_commit(ctx, st, &a->out, cuda_stream);
 }
 
+int isd_step_layers(isd_ctx* ctx, isd_batch_state* st, const isd_layer_args* layers, int32_t n_layers,
+                    const void* logits_cur, const void* q_prev_logits, const isd_verify_out* out, uint64_t step,
+                    void* cuda_stream) {
+  if (!ctx || !layers || n_layers < 1 || !out) return ISD_ERR_INVALID_ARG;
+  // every layer attends through the same page table and lengths: the state changes only in the commit
+  for (int32_t l = 0; l < n_layers; ++l) {
+    const isd_layer_args& a = layers[l];
+    const int rc = isd_attn(ctx, st, a.q, a.k_new, a.v_new, a.k_pool, a.v_pool, a.attn_out, a.attn_lse, cuda_stream);
+    if (rc != ISD_OK) return rc;
+  }
+  int rc = isd_verify(ctx, st, logits_cur, q_prev_logits, step, out, cuda_stream);
+  if (rc != ISD_OK) return rc;
+  return isd_commit(ctx, st, out, cuda_stream);
+}
+
+int isd_set_step_counter(isd_ctx* ctx, uint32_t* device_counter) {
+  if (!ctx) return ISD_ERR_INVALID_ARG;
+  ctx->step_counter = device_counter;
+  return ISD_OK;
+}
+
 int isd_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t n, void* cuda_stream) {
   if (!ctx || !slots || n < 0) return ISD_ERR_INVALID_ARG;
   int rc = check_state(st);

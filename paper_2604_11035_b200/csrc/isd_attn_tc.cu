@@ -1051,8 +1051,17 @@ int encode_pool_map(CUtensorMap* map, const void* pool, int num_pages, int Hkv) 
   return r == CUDA_SUCCESS ? ISD_OK : ISD_ERR_CUDA;
 }
 
-struct TcHost {
+// Tensor maps are encoded once per (k_pool, v_pool) pair and kept: a multi-layer step walks through one pair
+// per layer at every call.
+constexpr int kMapCacheSize = 128;
+struct PoolMaps {
+  const void* k_base;
+  const void* v_base;
   CUtensorMap map_k, map_v;
+};
+struct TcHost {
+  PoolMaps maps[kMapCacheSize];
+  int n_maps, next_victim;
   int* tile_prefix;
 };
 
@@ -1068,8 +1077,9 @@ int isd_attn_tc_create(isd_ctx* ctx) {
   TcHost* h = new (std::nothrow) TcHost();
   if (!h) return ISD_ERR_NO_MEMORY;
   h->tile_prefix = nullptr;
+  h->n_maps = 0;
+  h->next_victim = 0;
   ctx->tmap_k = h;
-  ctx->tmap_k_base = ctx->tmap_v_base = nullptr;
   ctx->attn_ctas = ctx->num_sms;
   if (cudaMalloc(&h->tile_prefix, sizeof(int) * (ctx->cfg.batch + 1)) != cudaSuccess) return ISD_ERR_NO_MEMORY;
   if (cudaMalloc(&ctx->attn_part_o, sizeof(float) * (size_t)ctx->attn_ctas * 2 * 128 * 128) != cudaSuccess) return ISD_ERR_NO_MEMORY;
@@ -1097,12 +1107,21 @@ int isd_launch_attn_tc(isd_ctx* ctx, const isd_batch_state* st, const void* q, c
   TcHost* h = reinterpret_cast<TcHost*>(ctx->tmap_k);
   if (!h) return ISD_ERR_INVALID_ARG;
   const isd_config& c = ctx->cfg;
-  if (ctx->tmap_k_base != k_pool || ctx->tmap_v_base != v_pool) {
-    int rc = encode_pool_map(&h->map_k, k_pool, c.num_pages, c.n_kv_heads);
-    if (rc == ISD_OK) rc = encode_pool_map(&h->map_v, v_pool, c.num_pages, c.n_kv_heads);
-    if (rc != ISD_OK) return rc;
-    ctx->tmap_k_base = k_pool;
-    ctx->tmap_v_base = v_pool;
+  PoolMaps* pm = nullptr;
+  for (int i = 0; i < h->n_maps && !pm; ++i)
+    if (h->maps[i].k_base == k_pool && h->maps[i].v_base == v_pool) pm = &h->maps[i];
+  if (!pm) {
+    pm = h->n_maps < kMapCacheSize ? &h->maps[h->n_maps] : &h->maps[h->next_victim];
+    int rc = encode_pool_map(&pm->map_k, k_pool, c.num_pages, c.n_kv_heads);
+    if (rc == ISD_OK) rc = encode_pool_map(&pm->map_v, v_pool, c.num_pages, c.n_kv_heads);
+    if (rc != ISD_OK) {
+      pm->k_base = pm->v_base = nullptr;
+      return rc;
+    }
+    pm->k_base = k_pool;
+    pm->v_base = v_pool;
+    if (h->n_maps < kMapCacheSize) ++h->n_maps;
+    else h->next_victim = (h->next_victim + 1) % kMapCacheSize;
   }
   TcParams P;
   P.B = c.batch; P.Q = ctx->Q; P.N = c.stride; P.Hq = c.n_q_heads; P.Hkv = c.n_kv_heads; P.G = ctx->G;
@@ -1115,7 +1134,7 @@ int isd_launch_attn_tc(isd_ctx* ctx, const isd_batch_state* st, const void* q, c
   P.num_ctas = ctx->attn_ctas;
   if (c.batch > kMaxSmemPrefixSlots) attn_plan_kernel<<<1, 1024, 0, stream>>>(P);
   if (ctx->ev_attn0) cudaEventRecord(ctx->ev_attn0, stream);
-  attn_tc_kernel<<<ctx->attn_ctas, kThreads, kSmemBytes, stream>>>(P, h->map_k, h->map_v);
+  attn_tc_kernel<<<ctx->attn_ctas, kThreads, kSmemBytes, stream>>>(P, pm->map_k, pm->map_v);
   if (ctx->ev_attn1) cudaEventRecord(ctx->ev_attn1, stream);
   attn_combine_kernel<<<ctx->attn_ctas, kCombineThreads, 0, stream>>>(P);
   ctx->launches += 2 + (c.batch > kMaxSmemPrefixSlots ? 1 : 0);

@@ -29,6 +29,7 @@ struct CommitParams {
   const int32_t* repl_tok;
   const int32_t* new_prop_tok;
   const float* new_q_stats;
+  uint32_t* step_counter;  // advanced by one after the commit when set
 };
 
 // exclusive prefix sum over the block; returns the block total through `total`
@@ -120,7 +121,10 @@ __global__ void __launch_bounds__(kCommitThreads) commit_kernel(const CommitPara
     }
   }
   __syncthreads();
-  if (threadIdx.x == 0) *P.free_top = top0 - sm_popped;
+  if (threadIdx.x == 0) {
+    *P.free_top = top0 - sm_popped;
+    if (P.step_counter) *P.step_counter += 1u;  // the next replay of a captured step draws fresh noise
+  }
 }
 
 __global__ void release_kernel(int B, int Q, int max_pages, int32_t* ctx_len, int32_t* n_ver,
@@ -154,6 +158,7 @@ int isd_launch_commit(isd_ctx* ctx, isd_batch_state* st, const isd_verify_out* o
   P.active = st->active; P.slot_status = st->slot_status; P.global_status = ctx->global_status;
   P.accept_len = out->accept_len; P.repl_tok = out->repl_tok; P.new_prop_tok = out->new_prop_tok;
   P.new_q_stats = out->new_q_stats;
+  P.step_counter = ctx->step_counter;
   commit_kernel<<<1, kCommitThreads, 0, stream>>>(P);
   ctx->launches++;
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;

@@ -62,12 +62,11 @@ struct isd_ctx {
   int attn_ctas;         // persistent CTAs of the tensor-core kernel
   float* attn_part_o;    // [attn_ctas * 2, 128, 128] un-normalised partial outputs
   float* attn_part_ml;   // [attn_ctas * 2, 128, 2]   running max / sum of each partial row
-  void* tmap_k;          // CUtensorMap for k_pool (device-usable copy lives in constant/param space)
-  void* tmap_v;
-  const void* tmap_k_base;  // pool pointers the tensor maps were encoded for
-  const void* tmap_v_base;
+  void* tmap_k;          // host-side state of the tensor-core attention (tensor maps of the pools seen so far)
   // ---- optional instrumentation events (owned by the caller)
   cudaEvent_t ev_attn0, ev_attn1, ev_verify0, ev_verify1;
+  // ---- optional device-resident step counter (CUDA-graph replay), owned by the caller
+  uint32_t* step_counter;
   // ---- status
   uint32_t* global_status;  // [1]
   int64_t launches;

@@ -51,6 +51,7 @@ struct VerifyParams {
   int logits_dtype, q_mode, propose_mode;
   float inv_t, tau;
   uint32_t seed_lo, seed_hi, step;
+  const uint32_t* step_dev;  // when set, the step number is read from here (CUDA-graph replay) instead of `step`
   int row_splits, sample_splits;
   const int32_t* n_ver;
   const uint8_t* active;
@@ -73,6 +74,7 @@ struct VerifyParams {
 
 // rows nv .. nv + rows_sampled - 1 of a slot are drawn by the sampling pass
 __device__ __forceinline__ int rows_sampled(const VerifyParams& P) { return P.propose_mode == 0 ? P.N : 1; }
+__device__ __forceinline__ uint32_t step_of(const VerifyParams& P) { return P.step_dev ? *P.step_dev : P.step; }
 
 __device__ __forceinline__ float ex2f(float x) {
   float y;
@@ -225,8 +227,8 @@ __device__ __forceinline__ void block_merge_top2(Top2& t, float* sm_s1, int* sm_
 }
 
 // fp64 score of vocabulary index i of a Gumbel row: logit * invT + g
-__device__ double noisy_score_f64(const VerifyParams& P, const void* row, int i, uint32_t slot, uint32_t tagpos) {
-  const uint4 r = philox4x32_10((uint32_t)i >> 2, P.step, slot, tagpos, P.seed_lo, P.seed_hi);
+__device__ double noisy_score_f64(const VerifyParams& P, const void* row, int i, uint32_t step, uint32_t slot, uint32_t tagpos) {
+  const uint4 r = philox4x32_10((uint32_t)i >> 2, step, slot, tagpos, P.seed_lo, P.seed_hi);
   const double l = (double)load_logit(row, P.logits_dtype, (size_t)i) * (double)P.inv_t;
   return l + gumbel_f64(philox_word(r, i & 3));
 }
@@ -554,7 +556,7 @@ __global__ void __launch_bounds__(kThreads + 32) verify_rows_kernel(const Verify
     float al = (1.f + P.tau) * expf(logp - logq);
     al = fminf(al, 1.f);
     if (al != al) al = 0.f;
-    const uint4 rnd = philox4x32_10(0u, P.step, (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)j, P.seed_lo, P.seed_hi);
+    const uint4 rnd = philox4x32_10(0u, step_of(P), (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)j, P.seed_lo, P.seed_hi);
     const float u = (float)(rnd.x >> 8) * 0x1p-24f;
     P.out.alpha[(size_t)b * NP + j - 1] = al;
     if (u < al) {
@@ -589,14 +591,14 @@ __global__ void __launch_bounds__(kThreads + 32) verify_rows_kernel(const Verify
 // ------------------------------------------------------------------------------------------------
 // fp64 score of vocabulary index i of the residual law: ln max(0, p_i - q_i) + g
 __device__ double resid_score_f64(const VerifyParams& P, const void* prow, const void* qrow, int i, int x,
-                                  double lse_p, double lse_q, uint32_t slot, uint32_t tagpos) {
+                                  double lse_p, double lse_q, uint32_t step, uint32_t slot, uint32_t tagpos) {
   const double pi = exp((double)load_logit(prow, P.logits_dtype, (size_t)i) * (double)P.inv_t - lse_p);
   double qi;
   if (P.q_mode == 0) qi = exp((double)load_logit(qrow, P.logits_dtype, (size_t)i) * (double)P.inv_t - lse_q);
   else qi = (i == x) ? 1.0 : 0.0;
   const double rres = pi - qi;
   if (!(rres > 0.0)) return -INFINITY;
-  const uint4 r = philox4x32_10((uint32_t)i >> 2, P.step, slot, tagpos, P.seed_lo, P.seed_hi);
+  const uint4 r = philox4x32_10((uint32_t)i >> 2, step, slot, tagpos, P.seed_lo, P.seed_hi);
   return log(rres) + gumbel_f64(philox_word(r, i & 3));
 }
 
@@ -607,6 +609,7 @@ struct SampleJob {
   int x;             // residual only: the rejected token
   float lse_p, lse_q;
   uint32_t tagpos;
+  uint32_t step;     // Philox counter word of this step
   bool resid;
 };
 
@@ -654,7 +657,7 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
     const int idx = qi[pos & (kQueueCap - 1)];
     const float4 v = ql[pos & (kQueueCap - 1)];
     const float l4[4] = {v.x, v.y, v.z, v.w};
-    const uint4 rnd = philox4x32_10((uint32_t)idx >> 2, P.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
+    const uint4 rnd = philox4x32_10((uint32_t)idx >> 2, J.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
     const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
     DBG_COUNT(J.resid ? 1 : 0, 1);
     // -ln u' >= 1 - u' >= nf 2^-24 with nf = floor(2^24 (1 - u')), so g_i <= -ln(nf 2^-24): the element
@@ -745,6 +748,7 @@ __global__ void __launch_bounds__(kThreads) verify_sample_kernel(const VerifyPar
   // ---- what this (slot, k) draws
   SampleJob J;
   J.qrow = nullptr; J.x = -1; J.lse_p = 0.f; J.lse_q = 0.f;
+  J.step = step_of(P);
   int r;  // row of this step's logits that is sampled
   if (k == 0 && rej > 0) {
     // replacement for the first rejected proposal, from normalize(max(0, p - q))
@@ -770,7 +774,7 @@ __global__ void __launch_bounds__(kThreads) verify_sample_kernel(const VerifyPar
     float seed = -INFINITY;
     const int i0 = P.row_arg[(size_t)b * P.Q + r];
     if (i0 >= 0 && i0 < P.V) {
-      const uint4 rnd = philox4x32_10((uint32_t)i0 >> 2, P.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
+      const uint4 rnd = philox4x32_10((uint32_t)i0 >> 2, J.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
       seed = job_score(P, J, load_logit(J.prow, P.logits_dtype, (size_t)i0), i0, philox_word(rnd, i0 & 3));
     }
     sm_best = seed > -INFINITY ? enc_ordered(seed) : 0u;
@@ -812,11 +816,11 @@ __global__ void __launch_bounds__(kThreads) verify_sample_kernel(const VerifyPar
     if (t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
       double s1, s2;
       if (J.resid) {
-        s1 = resid_score_f64(P, J.prow, J.qrow, t.i1, J.x, J.lse_p, J.lse_q, (uint32_t)b, J.tagpos);
-        s2 = resid_score_f64(P, J.prow, J.qrow, t.i2, J.x, J.lse_p, J.lse_q, (uint32_t)b, J.tagpos);
+        s1 = resid_score_f64(P, J.prow, J.qrow, t.i1, J.x, J.lse_p, J.lse_q, J.step, (uint32_t)b, J.tagpos);
+        s2 = resid_score_f64(P, J.prow, J.qrow, t.i2, J.x, J.lse_p, J.lse_q, J.step, (uint32_t)b, J.tagpos);
       } else {
-        s1 = noisy_score_f64(P, J.prow, t.i1, (uint32_t)b, J.tagpos);
-        s2 = noisy_score_f64(P, J.prow, t.i2, (uint32_t)b, J.tagpos);
+        s1 = noisy_score_f64(P, J.prow, t.i1, J.step, (uint32_t)b, J.tagpos);
+        s2 = noisy_score_f64(P, J.prow, t.i2, J.step, (uint32_t)b, J.tagpos);
       }
       if (s2 > s1 || (s2 == s1 && t.i2 < t.i1)) y = t.i2;
     }
@@ -836,8 +840,8 @@ __global__ void __launch_bounds__(kThreads) verify_sample_kernel(const VerifyPar
     if (threadIdx.x == 0) {
       y = t.i1;
       if (t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
-        const double s1 = noisy_score_f64(P, J.prow, t.i1, (uint32_t)b, J.tagpos);
-        const double s2 = noisy_score_f64(P, J.prow, t.i2, (uint32_t)b, J.tagpos);
+        const double s1 = noisy_score_f64(P, J.prow, t.i1, J.step, (uint32_t)b, J.tagpos);
+        const double s2 = noisy_score_f64(P, J.prow, t.i2, J.step, (uint32_t)b, J.tagpos);
         if (s2 > s1 || (s2 == s1 && t.i2 < t.i1)) y = t.i2;
       }
       atomicOr(&P.slot_status[b], ISD_ST_EMPTY_RESIDUAL);
@@ -867,6 +871,7 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   P.logits_dtype = c.logits_dtype; P.q_mode = c.q_mode; P.propose_mode = c.propose_mode;
   P.inv_t = c.inv_temperature; P.tau = c.tau;
   P.seed_lo = (uint32_t)c.seed; P.seed_hi = (uint32_t)(c.seed >> 32); P.step = step;
+  P.step_dev = ctx->step_counter;
   P.row_splits = ctx->row_splits; P.sample_splits = ctx->sample_splits;
   P.n_ver = st->n_ver; P.active = st->active; P.block_tok = st->block_tok; P.q_row0 = st->q_row0;
   P.q_stats = st->q_stats; P.slot_status = st->slot_status; P.global_status = ctx->global_status;
