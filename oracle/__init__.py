@@ -112,9 +112,20 @@ class VerifyResult:
     prop_margin: np.ndarray   # [B, N-1] f64
 
 
+def filter_row(row, top_k, top_p):
+    """Top-k then top-p filtered law of a scaled fp64 row: a copy with -inf outside the support."""
+    r = np.ascontiguousarray(np.array(row, dtype=np.float64))
+    f = lib().orc_filter_row
+    f.restype = None
+    f.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_double]
+    f(_p(r), r.shape[0], int(top_k), float(top_p))
+    return r
+
+
 def verify(*, N, V, logits_dtype, q_mode, propose_mode, inv_temperature, tau, seed, step,
-           n_ver, active, block_tok, q_row0, logits_cur, q_prev, slot_status) -> VerifyResult:
-    """Algorithm 1's introspection loop, bonus branch and stride loop for every slot."""
+           n_ver, active, block_tok, q_row0, logits_cur, q_prev, slot_status, top_k=0, top_p=1.0) -> VerifyResult:
+    """Algorithm 1's introspection loop, bonus branch and stride loop for every slot (top_k > 0: on the
+    top-k / top-p filtered laws)."""
     B = n_ver.shape[0]
     Q, NP = 2 * N - 1, N - 1
     ldt = np.float32 if logits_dtype == 0 else np.uint16
@@ -127,10 +138,10 @@ def verify(*, N, V, logits_dtype, q_mode, propose_mode, inv_temperature, tau, se
         accept_len=np.zeros(B, np.int32), n_emit=np.zeros(B, np.int32), repl_tok=np.zeros(B, np.int32),
         out_tok=np.zeros((B, N), np.int32), new_prop_tok=np.zeros((B, NP), np.int32),
         new_q_stats=np.zeros((B, NP, 2)), final_margin=np.zeros(B), prop_margin=np.zeros((B, NP)))
-    f = lib().orc_verify
+    f = lib().orc_verify_filtered
     f.restype = C.c_int
-    f.argtypes = [C.c_int] * 6 + [C.c_double, C.c_double, C.c_uint64, C.c_uint32] + [C.c_void_p] * 18
-    rc = f(B, N, V, logits_dtype, q_mode, propose_mode, float(np.float32(inv_temperature)),
+    f.argtypes = [C.c_int, C.c_double] + [C.c_int] * 6 + [C.c_double, C.c_double, C.c_uint64, C.c_uint32] + [C.c_void_p] * 18
+    rc = f(int(top_k), float(np.float32(top_p)), B, N, V, logits_dtype, q_mode, propose_mode, float(np.float32(inv_temperature)),
            float(np.float32(tau)), seed, step,
            _p(n_ver), _p(active), _p(block_tok), _p(q_row0), _p(logits_cur), _p(q_prev),
            _p(r.accept), _p(r.alpha), _p(r.u), _p(r.accept_len), _p(r.n_emit), _p(r.repl_tok),

@@ -162,6 +162,51 @@ double orc_logsumexp(const double* row, int V) {
   return m + log(s);
 }
 
+/* Top-k / top-p filtered law of a scaled row (the serving configuration of the paper's appendix:
+ * temperature, then top-k, then top-p on what top-k kept).  In place: entries outside the support
+ * become -inf, so that softmax(row) afterwards IS the filtered, renormalised law and every routine
+ * below (log-sum-exp, Gumbel-max, residual) applies unchanged.
+ *   1. S_k = the top_k entries in the order (value descending, index ascending);
+ *   2. w_i = exp(row_i - max) over S_k in that order, Z = sum w_i;
+ *   3. the support is the shortest prefix of S_k whose cumulated w reaches top_p * Z
+ *      (all of S_k when it is never reached, e.g. top_p = 1 with rounding).
+ * top_k <= 0 leaves the row alone.  NaN entries are never selected. */
+void orc_filter_row(double* row, int V, int top_k, double top_p) {
+  if (top_k <= 0) return;
+  if (top_k > V) top_k = V;
+  int* sel = (int*)malloc(sizeof(int) * (size_t)top_k);
+  char* taken = (char*)calloc((size_t)V, 1);
+  if (!sel || !taken) { free(sel); free(taken); return; }
+  int n = 0;
+  for (int r = 0; r < top_k; ++r) {  /* selection, one maximum at a time */
+    int best = -1;
+    for (int i = 0; i < V; ++i) {
+      if (taken[i] || isnan(row[i])) continue;
+      if (best < 0 || row[i] > row[best]) best = i;  /* strict >: the lowest index wins ties */
+    }
+    if (best < 0) break;
+    taken[best] = 1;
+    sel[n++] = best;
+  }
+  int keep = n;
+  if (n > 0 && !(isinf(row[sel[0]]) && row[sel[0]] < 0)) {
+    const double m = row[sel[0]];
+    double Z = 0.0;
+    for (int r = 0; r < n; ++r) Z += exp(row[sel[r]] - m);
+    double cum = 0.0;
+    for (int r = 0; r < n; ++r) {
+      cum += exp(row[sel[r]] - m);
+      if (cum >= top_p * Z) { keep = r + 1; break; }
+    }
+  }
+  memset(taken, 0, (size_t)V);
+  for (int r = 0; r < keep; ++r) taken[sel[r]] = 1;
+  for (int i = 0; i < V; ++i)
+    if (!taken[i] && !isnan(row[i])) row[i] = -INFINITY;
+  free(sel);
+  free(taken);
+}
+
 /* argmax_i (score_i) with the lowest index winning ties; also reports the gap
  * between the best and the second-best score (for "fragile sample" reporting). */
 typedef struct {
@@ -233,6 +278,8 @@ typedef struct {
   double* final_margin;     /* [B] top-2 gap of y's score */
   double* prop_margin;      /* [B, N-1] top-2 gap of each proposal's score */
   uint32_t* slot_status;    /* [B] OR-ed status bits */
+  int top_k;                /* 0 = unfiltered laws */
+  double top_p;
 } verify_args;
 
 static void verify_slot(const verify_args* A, int b, double* lp, double* lq) {
@@ -278,11 +325,13 @@ static void verify_slot(const verify_args* A, int b, double* lp, double* lq) {
     }
     if (load_row(A->logits_cur, A->logits_dtype, cur_base + (size_t)(j - 1) * V, V, A->invT, lp))
       status |= ORC_ST_NONFINITE_LOGIT;
+    orc_filter_row(lp, V, A->top_k, A->top_p);
     const double lse_p = orc_logsumexp(lp, V);
     double lse_q = 0.0, logq_x = 0.0;
     if (A->q_mode == 0) {
       const size_t qoff = ((size_t)b * Q + (size_t)(A->q_row0[b] + j - 1)) * V;
       if (load_row(A->q_prev, A->logits_dtype, qoff, V, A->invT, lq)) status |= ORC_ST_NONFINITE_LOGIT;
+      orc_filter_row(lq, V, A->top_k, A->top_p);
       lse_q = orc_logsumexp(lq, V);
       logq_x = lq[x] - lse_q;
     }
@@ -331,6 +380,7 @@ static void verify_slot(const verify_args* A, int b, double* lp, double* lq) {
      * this is the quality-guaranteed AR token). */
     if (load_row(A->logits_cur, A->logits_dtype, cur_base + (size_t)nv * V, V, A->invT, lp))
       status |= ORC_ST_NONFINITE_LOGIT;
+    orc_filter_row(lp, V, A->top_k, A->top_p);
     y = sample_row(lp, V, A->seed, A->step, (uint32_t)b, ORC_TAG_FINAL, (uint32_t)(nv + 1), &y_margin);
   }
   A->accept_len[b] = a;
@@ -344,6 +394,7 @@ static void verify_slot(const verify_args* A, int b, double* lp, double* lq) {
   for (int m = 1; m <= NP; ++m) {
     if (load_row(A->logits_cur, A->logits_dtype, cur_base + (size_t)(nv + m) * V, V, A->invT, lp))
       status |= ORC_ST_NONFINITE_LOGIT;
+    orc_filter_row(lp, V, A->top_k, A->top_p);
     double margin;
     int xh;
     if (A->propose_mode == 0)
@@ -358,7 +409,8 @@ static void verify_slot(const verify_args* A, int b, double* lp, double* lq) {
   A->slot_status[b] |= status;
 }
 
-int orc_verify(int B, int N, int V, int logits_dtype, int q_mode, int propose_mode, double invT,
+/* The same with every law (anchor p, proposal q, bonus, MASK rows) filtered by top-k then top-p first. */
+int orc_verify_filtered(int top_k, double top_p, int B, int N, int V, int logits_dtype, int q_mode, int propose_mode, double invT,
                double tau, uint64_t seed, uint32_t step, const int32_t* n_ver, const uint8_t* active,
                const int32_t* block_tok, const int32_t* q_row0, const void* logits_cur,
                const void* q_prev, int8_t* accept, double* alpha, double* u_draw, int32_t* accept_len,
@@ -367,7 +419,8 @@ int orc_verify(int B, int N, int V, int logits_dtype, int q_mode, int propose_mo
   if (B < 0 || N < 1 || V < 1) return -1;
   verify_args A = {B, N, V, logits_dtype, q_mode, propose_mode, invT, tau, seed, step, n_ver, active,
                    block_tok, q_row0, logits_cur, q_prev, accept, alpha, u_draw, accept_len, n_emit,
-                   repl_tok, out_tok, new_prop_tok, new_q_stats, final_margin, prop_margin, slot_status};
+                   repl_tok, out_tok, new_prop_tok, new_q_stats, final_margin, prop_margin, slot_status,
+                   top_k, top_p};
   int fail = 0;
 #pragma omp parallel num_threads(g_threads)
   {
@@ -384,6 +437,17 @@ int orc_verify(int B, int N, int V, int logits_dtype, int q_mode, int propose_mo
     free(lq);
   }
   return fail ? -2 : 0;
+}
+
+int orc_verify(int B, int N, int V, int logits_dtype, int q_mode, int propose_mode, double invT,
+               double tau, uint64_t seed, uint32_t step, const int32_t* n_ver, const uint8_t* active,
+               const int32_t* block_tok, const int32_t* q_row0, const void* logits_cur,
+               const void* q_prev, int8_t* accept, double* alpha, double* u_draw, int32_t* accept_len,
+               int32_t* n_emit, int32_t* repl_tok, int32_t* out_tok, int32_t* new_prop_tok,
+               double* new_q_stats, double* final_margin, double* prop_margin, uint32_t* slot_status) {
+  return orc_verify_filtered(0, 1.0, B, N, V, logits_dtype, q_mode, propose_mode, invT, tau, seed, step, n_ver, active,
+                             block_tok, q_row0, logits_cur, q_prev, accept, alpha, u_draw, accept_len, n_emit,
+                             repl_tok, out_tok, new_prop_tok, new_q_stats, final_margin, prop_margin, slot_status);
 }
 
 /* ------------------------------------------------------------------------- */

@@ -36,7 +36,7 @@ def state_to_np(st: dict) -> dict:
 
 
 def oracle_step(w: wl.Workload, s: dict, q, k_new, v_new, logits_cur, q_prev, step, *,
-                inv_temperature=1.0, tau=0.0, mask_token=None, do_attn=True, sm_scale=None):
+                inv_temperature=1.0, tau=0.0, mask_token=None, do_attn=True, sm_scale=None, top_k=0, top_p=1.0):
     """One full oracle step (attention, verify, commit) on numpy state `s`, in place.
 
     Returns (attn_out, attn_lse, VerifyResult, q_len_before).
@@ -55,7 +55,7 @@ def oracle_step(w: wl.Workload, s: dict, q, k_new, v_new, logits_cur, q_prev, st
         N=N, V=w.vocab, logits_dtype=ldt, q_mode=w.q_mode, propose_mode=w.propose_mode,
         inv_temperature=inv_temperature, tau=tau, seed=w.seed, step=step, n_ver=s["n_ver"],
         active=s["active"], block_tok=s["block_tok"], q_row0=s["q_row0"], logits_cur=logits_cur,
-        q_prev=q_prev, slot_status=s["slot_status"])
+        q_prev=q_prev, slot_status=s["slot_status"], top_k=top_k, top_p=top_p)
     oracle.commit(
         N=N, page_size=wl.PAGE, mask_token=(w.vocab - 1 if mask_token is None else mask_token),
         ctx_len=s["ctx_len"], n_ver=s["n_ver"], block_tok=s["block_tok"], q_row0=s["q_row0"],
