@@ -98,16 +98,17 @@ def algorithmic_bytes(w, ctx_len, q_len, rejecting: int):
     return attn, verify
 
 
-def rank_workload(config_index: int, rank: int, sweep: str | None = None):
+def rank_workload(config_index: int, rank: int, sweep: str | None = None, top_k: int = 0, top_p: float = 1.0):
     """Workload of one rank: ranks own disjoint slots with their own pools, so each gets its own seed."""
     from dataclasses import replace
     from paper_2604_11035_b200 import workloads as wl
     if sweep:
         stride, batch = (int(x) for x in sweep.split(","))
         base = wl.sweep_point(stride, batch)
-        return replace(base, seed=base.seed + 1000 * rank)
-    base = wl.config(config_index)
-    return wl.config(config_index, seed=base.seed + 1000 * rank)
+    else:
+        base = wl.config(config_index)
+    return replace(base, seed=base.seed + 1000 * rank, top_k=top_k, top_p=top_p,
+                   name=base.name + (f"[top-k {top_k}, top-p {top_p}]" if top_k else ""))
 
 
 def reduce_over_ranks(dist, device, times, counts):
@@ -131,7 +132,7 @@ def run_model_step(args):
 
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
-    w = rank_workload(args.config, 0, args.sweep)
+    w = rank_workload(args.config, 0, args.sweep, args.top_k, args.top_p)
     K, W, L = args.steps, args.warmup, args.layers
     w = replace(w, steps=max(w.steps, K + W + 2))
     if args.batch:
@@ -237,7 +238,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     # weak scaling: every rank owns its own slots, pools and free stack (slots never interact)
-    w = rank_workload(args.config, rank, args.sweep)
+    w = rank_workload(args.config, rank, args.sweep, args.top_k, args.top_p)
     if args.propose_mode is not None:
         from dataclasses import replace
         w = replace(w, propose_mode=args.propose_mode)
@@ -407,7 +408,7 @@ def run_ours(args):
         "roofline": {"kernel": "attn_tc_kernel", "bound": "hbm", "achieved": attn_gbs, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": attn_gbs / peak, "frac_of_8TBs": attn_gbs / HBM_NOMINAL_GBS,
                      "traffic": None, "ms_per_launch": sum(attn_ms) / K, "bytes_per_launch": attn_bytes / K},
-        "verify_kernels": {"kernels": "verify_rows_kernel + verify_sample_kernel", "achieved_gbs": ver_gbs, "ms_per_launch": sum(ver_ms) / max(1, len(ver_ms)),
+        "verify_kernels": {"kernels": "topk_rows_kernel + topk_decide_kernel" if w.top_k else "verify_rows_kernel + verify_sample_kernel", "achieved_gbs": ver_gbs, "ms_per_launch": sum(ver_ms) / max(1, len(ver_ms)),
                            "timed_on": "%d extra steps after the timed region" % len(ver_ms),
                                "frac_of_measured_copy": (ver_gbs / peak) if ver_gbs else None},
         "gpu_launches": launches, "status_word": status, "clocks": clocks, "wall_s": wall,
@@ -519,6 +520,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (smaller captures under ncu)")
     ap.add_argument("--sweep", default=None, metavar="STRIDE,BATCH",
                     help="one point of the sweep workload (stride in 2,4,8,16; batch in 1,8,64,256,512) instead of --config")
+    ap.add_argument("--top-k", type=int, default=0, help="verify on top-k / top-p filtered laws (0 = plain softmax laws)")
+    ap.add_argument("--top-p", type=float, default=1.0)
     ap.add_argument("--layers", type=int, default=0, help="model-step mode: this many attention layers per step (isd_step_layers)")
     ap.add_argument("--graph", action="store_true", help="model-step mode: replay the step from a CUDA graph")
     ap.add_argument("--sequential-pages", action="store_true", help="identity page order instead of a shuffled pool")

@@ -71,6 +71,8 @@ extern "C" {
 
 typedef struct isd_ctx isd_ctx; /* opaque; owns scratch only */
 
+#define ISD_MAX_TOP_K 64
+
 typedef struct isd_config {
   int32_t batch;              /* B, number of fixed slots (>= 1)                      */
   int32_t stride;             /* N >= 1 (Q = 2N-1 <= 31)                              */
@@ -92,6 +94,13 @@ typedef struct isd_config {
   float inv_temperature;      /* logits are multiplied by this (1.0 = paper default)  */
   float tau;                  /* relaxed acceptance: ratio * (1 + tau), Sec. 4.3      */
   uint64_t seed;              /* Philox key                                           */
+  int32_t top_k;              /* 0: plain softmax laws (Algorithm 1).  1..ISD_MAX_TOP_K:
+                                 every law (anchor p, proposal q, bonus, MASK rows) is
+                                 first cut to its top_k tokens (value descending, lower
+                                 index on ties) and then to the shortest prefix of those
+                                 whose mass reaches top_p, and renormalised (the serving
+                                 sampling configuration of the paper's appendix)       */
+  float top_p;                /* in (0, 1]; read only when top_k > 0                  */
 } isd_config;
 
 /* Stationary-batch state (Sec. 3.3 (2)); all arrays on the device, in place. */

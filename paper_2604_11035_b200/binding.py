@@ -27,7 +27,7 @@ class IsdConfig(C.Structure):
         "batch", "stride", "n_q_heads", "n_kv_heads", "head_dim", "page_size", "vocab",
         "max_pages_per_slot", "num_pages", "logits_dtype", "q_mode", "propose_mode", "mask_token_id",
         "attn_impl")] + [("sm_scale", C.c_float), ("inv_temperature", C.c_float), ("tau", C.c_float),
-                         ("seed", C.c_uint64)]
+                         ("seed", C.c_uint64), ("top_k", C.c_int32), ("top_p", C.c_float)]
 
 
 class IsdBatchState(C.Structure):
@@ -135,7 +135,7 @@ class Isd:
 
     def __init__(self, *, batch, stride, n_q_heads, n_kv_heads, vocab, max_pages_per_slot, num_pages,
                  logits_dtype, head_dim=128, page_size=16, q_mode=0, propose_mode=1, mask_token_id=None,
-                 attn_impl=0, sm_scale=0.0, inv_temperature=1.0, tau=0.0, seed=0):
+                 attn_impl=0, sm_scale=0.0, inv_temperature=1.0, tau=0.0, seed=0, top_k=0, top_p=1.0):
         if not torch.cuda.is_available():
             raise IsdError("a CUDA device is required (there is no CPU path)")
         self.lib = load()
@@ -143,7 +143,7 @@ class Isd:
         self.cfg = IsdConfig(batch, stride, n_q_heads, n_kv_heads, head_dim, page_size, vocab,
                              max_pages_per_slot, num_pages, ld, q_mode, propose_mode,
                              vocab - 1 if mask_token_id is None else mask_token_id, attn_impl,
-                             sm_scale, inv_temperature, tau, seed)
+                             sm_scale, inv_temperature, tau, seed, top_k, top_p)
         self.ctx = C.c_void_p()
         _check(self.lib.isd_create(C.byref(self.cfg), C.byref(self.ctx)), "isd_create")
         self.N, self.B = stride, batch

@@ -52,6 +52,8 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   if (c.q_mode < 0 || c.q_mode > 1 || c.propose_mode < 0 || c.propose_mode > 1) return ISD_ERR_INVALID_ARG;
   if (c.attn_impl < 0 || c.attn_impl > 1) return ISD_ERR_INVALID_ARG;
   if (!(c.inv_temperature > 0.f) || !(c.tau >= 0.f)) return ISD_ERR_INVALID_ARG;
+  if (c.top_k < 0 || (c.top_k > 0 && !(c.top_p > 0.f && c.top_p <= 1.f))) return ISD_ERR_INVALID_ARG;
+  if (c.top_k > ISD_MAX_TOP_K) return ISD_ERR_UNSUPPORTED;
   const int Q = 2 * c.stride - 1;
   const int G = c.n_q_heads / c.n_kv_heads;
   if (c.head_dim != ISD_HEAD_DIM || c.page_size != ISD_PAGE || Q > ISD_MAX_Q || G * Q > 128 || c.vocab % 8 != 0)
@@ -106,6 +108,7 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
     cudaMemset(ctx->row_arg, 0xFF, sizeof(int) * rows);
     cudaMemset(ctx->global_status, 0, sizeof(uint32_t));
   }
+  if (rc == ISD_OK && c.top_k > 0) rc = isd_verify_topk_create(ctx);
   if (rc == ISD_OK && c.attn_impl == 0) rc = isd_attn_tc_create(ctx);
   if (rc == ISD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ISD_ERR_CUDA;
   if (rc != ISD_OK) {
@@ -120,6 +123,7 @@ int isd_destroy(isd_ctx* ctx) {
   if (!ctx) return ISD_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
   isd_attn_tc_destroy(ctx);
+  isd_verify_topk_destroy(ctx);
   cudaFree(ctx->row_part);
   cudaFree(ctx->samp_part);
   cudaFree(ctx->row_ticket);
@@ -159,6 +163,9 @@ int isd_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur, 
   if (!logits_cur || step > 0xFFFFFFFFull) return ISD_ERR_INVALID_ARG;
   if (ctx->cfg.stride > 1 && !st->q_stats) return ISD_ERR_INVALID_ARG;
   if (!aligned16(logits_cur) || (q_prev_logits && !aligned16(q_prev_logits))) return ISD_ERR_ALIGNMENT;
+  if (ctx->cfg.top_k > 0)
+    return isd_launch_verify_topk(ctx, st, logits_cur, q_prev_logits, (uint32_t)step, out,
+                                  reinterpret_cast<cudaStream_t>(cuda_stream));
   return isd_launch_verify(ctx, st, logits_cur, q_prev_logits, (uint32_t)step, out,
                            reinterpret_cast<cudaStream_t>(cuda_stream));
 }
@@ -234,7 +241,7 @@ const char* isd_strerror(int code) {
   switch (code) {
     case ISD_OK: return "ok";
     case ISD_ERR_INVALID_ARG: return "invalid argument";
-    case ISD_ERR_UNSUPPORTED: return "unsupported configuration (head_dim must be 128, page_size 16, (Hq/Hkv)*(2N-1) <= 128, vocab % 8 == 0)";
+    case ISD_ERR_UNSUPPORTED: return "unsupported configuration (head_dim must be 128, page_size 16, (Hq/Hkv)*(2N-1) <= 128, vocab % 8 == 0, top_k <= 64; isd_verify_static: top_k = 0)";
     case ISD_ERR_CUDA: return "CUDA runtime error";
     case ISD_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
     case ISD_ERR_NO_MEMORY: return "out of memory";

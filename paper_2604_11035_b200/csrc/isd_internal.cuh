@@ -65,6 +65,10 @@ struct isd_ctx {
   void* tmap_k;          // host-side state of the tensor-core attention (tensor maps of the pools seen so far)
   // ---- optional instrumentation events (owned by the caller)
   cudaEvent_t ev_attn0, ev_attn1, ev_verify0, ev_verify1;
+  // ---- scratch of the top-k / top-p filtered verification (cfg.top_k > 0)
+  float* topk_val;       // [B, Q, ISD_MAX_TOP_K]
+  int* topk_idx;         // [B, Q, ISD_MAX_TOP_K]
+  int* topk_n;           // [B, Q]
   // ---- optional device-resident step counter (CUDA-graph replay), owned by the caller
   uint32_t* step_counter;
   // ---- status
@@ -294,6 +298,11 @@ __device__ __forceinline__ void lse_merge(float& m, float& s, float om, float os
 int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
                       const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
                       cudaStream_t stream);
+int isd_verify_topk_create(isd_ctx* ctx);
+void isd_verify_topk_destroy(isd_ctx* ctx);
+int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
+                           const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
+                           cudaStream_t stream);
 int isd_launch_commit(isd_ctx* ctx, isd_batch_state* st, const isd_verify_out* out, cudaStream_t stream);
 int isd_launch_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t n,
                        cudaStream_t stream);

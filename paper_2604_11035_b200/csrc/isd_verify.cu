@@ -26,6 +26,7 @@
 // The two best candidates of a row are re-judged in fp64 when their fp32 scores are closer than
 // ISD_TIE_EPS.
 #include "isd_internal.cuh"
+#include "isd_stream.cuh"
 
 #ifdef EXP_COUNT
 __device__ unsigned long long g_dbg[8];
@@ -42,7 +43,6 @@ extern "C" int isd_debug_counters(unsigned long long* out) {
 
 namespace {
 
-constexpr int kThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kGumbelMax = 17.34f;  // > 25 ln 2, the largest variate of the 24-bit lattice
 
@@ -90,34 +90,6 @@ __device__ __forceinline__ unsigned enc_ordered(float f) {
 }
 __device__ __forceinline__ float dec_ordered(unsigned u) {
   return __uint_as_float((u & 0x80000000u) ? (u ^ 0x80000000u) : ~u);
-}
-
-// Eight consecutive logits as fp32 from their raw 16-byte vectors (bf16: byte permutes and masks, which
-// run on the ALU pipe; shifts would be issued as integer multiplies on the busier FMA pipe).
-template <int DT>
-__device__ __forceinline__ void unpack8(const uint4& a, const uint4& b, float (&l)[8]) {
-  if (DT == ISD_LOGITS_BF16) {
-    l[0] = __uint_as_float(__byte_perm(a.x, 0u, 0x1044)); l[1] = __uint_as_float(a.x & 0xFFFF0000u);
-    l[2] = __uint_as_float(__byte_perm(a.y, 0u, 0x1044)); l[3] = __uint_as_float(a.y & 0xFFFF0000u);
-    l[4] = __uint_as_float(__byte_perm(a.z, 0u, 0x1044)); l[5] = __uint_as_float(a.z & 0xFFFF0000u);
-    l[6] = __uint_as_float(__byte_perm(a.w, 0u, 0x1044)); l[7] = __uint_as_float(a.w & 0xFFFF0000u);
-  } else {
-    l[0] = __uint_as_float(a.x); l[1] = __uint_as_float(a.y); l[2] = __uint_as_float(a.z); l[3] = __uint_as_float(a.w);
-    l[4] = __uint_as_float(b.x); l[5] = __uint_as_float(b.y); l[6] = __uint_as_float(b.z); l[7] = __uint_as_float(b.w);
-  }
-}
-
-// Eight consecutive logits starting at element e (e % 8 == 0), straight from global memory.
-template <int DT>
-__device__ __forceinline__ void load8(const void* row, int e, float (&l)[8]) {
-  uint4 a, b = make_uint4(0u, 0u, 0u, 0u);
-  if (DT == ISD_LOGITS_BF16) {
-    a = ld_stream_16B(reinterpret_cast<const uint16_t*>(row) + e);
-  } else {
-    a = ld_stream_16B(reinterpret_cast<const float*>(row) + e);
-    b = ld_stream_16B(reinterpret_cast<const float*>(row) + e + 4);
-  }
-  unpack8<DT>(a, b, l);
 }
 
 // A row piece streamed through shared memory with per-thread asynchronous copies.  Every thread
@@ -184,8 +156,6 @@ struct RowStream {
   }
   __device__ __forceinline__ void finish() const { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 };
-constexpr int kRowStages = 4;            // row pass: bulk-copy ring of kRowStages x kRowStageBytes
-constexpr int kRowStageBytes = 8192;
 constexpr int kSampleRingBytes = 16384;  // sampling pass: one group per iteration
 
 __device__ __forceinline__ void chunk_range(int V, int splits, int split, int& lo, int& hi) {
@@ -194,9 +164,6 @@ __device__ __forceinline__ void chunk_range(int V, int splits, int split, int& l
   lo = split * per;
   hi = min(V, lo + per);
 }
-
-// Barrier of the kThreads worker threads (a producer warp, where a kernel has one, stays out of it).
-__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 
 // Block-wide merge helpers (8 worker warps) -------------------------------------------------------
 __device__ __forceinline__ void block_merge_lse(float& m, float& s, float* sm_m, float* sm_s) {
@@ -232,14 +199,6 @@ __device__ double noisy_score_f64(const VerifyParams& P, const void* row, int i,
   const double l = (double)load_logit(row, P.logits_dtype, (size_t)i) * (double)P.inv_t;
   return l + gumbel_f64(philox_word(r, i & 3));
 }
-
-// Order-preserving map float <-> signed int (an involution), so that a warp can agree on a maximum with
-// one integer reduction.
-__device__ __forceinline__ int ord_key(float f) {
-  const int b = __float_as_int(f);
-  return b ^ ((b >> 31) & 0x7FFFFFFF);
-}
-__device__ __forceinline__ float ord_val(int k) { return __int_as_float(k ^ ((k >> 31) & 0x7FFFFFFF)); }
 
 // Online softmax of a thread's share of a row: S = sum exp((l - M) * invT) in the log2 domain, plain
 // scalar FFMA / ex2 / FADD with four independent partial sums (the packed fp32x2 forms cost more in
@@ -277,34 +236,6 @@ struct OnlineSoftmax {
   }
   __device__ __forceinline__ float sum() const { return (S0 + S1) + (S2 + S3); }
 };
-
-__device__ __forceinline__ float max8(const float (&l)[8]) {
-  return fmaxf(max3(l[0], l[1], l[2]), max3(max3(l[3], l[4], l[5]), l[6], l[7]));
-}
-
-// Shared memory of the row pass: the ring and its barriers.
-struct RowRing {
-  __align__(128) unsigned char stage[kRowStages][kRowStageBytes];
-  __align__(8) uint64_t full[kRowStages];   // a stage's bytes have landed (one arrival + transaction bytes)
-  __align__(8) uint64_t empty[kRowStages];  // every worker warp has read the stage (one arrival per warp)
-};
-
-// Producer (one thread): streams bytes [byte_lo, byte_hi) of a row into the ring, one contiguous bulk copy
-// per stage.  Returns false when a wait ran out.
-__device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t byte_lo, size_t byte_hi) {
-  const uint32_t full0 = ring_smem_u32(R.full), empty0 = ring_smem_u32(R.empty), st0 = ring_smem_u32(R.stage);
-  int c = 0;
-  for (size_t off = byte_lo; off < byte_hi; off += kRowStageBytes, ++c) {
-    const int s = c & (kRowStages - 1);
-    const uint32_t ph = (c / kRowStages) & 1;
-    if (!ring_mbar_wait(empty0 + 8 * s, ph ^ 1)) return false;
-    const size_t left = byte_hi - off;
-    const uint32_t bytes = left < (size_t)kRowStageBytes ? (uint32_t)left : (uint32_t)kRowStageBytes;
-    ring_mbar_expect_tx(full0 + 8 * s, bytes);
-    ring_bulk_g2s(st0 + s * kRowStageBytes, row + off, bytes, full0 + 8 * s);
-  }
-  return true;
-}
 
 // Worker side of one streaming pass over elements [lo, hi) of a logits row: online softmax (m_nat, S
 // relative to the warp's maximum) and this thread's argmax candidate of the raw logits.  A thread
@@ -948,7 +879,7 @@ extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* s
   if (c.batch < 1 || c.stride < 1 || c.vocab < 8 || c.inv_temperature <= 0.f || c.tau < 0.f) return ISD_ERR_INVALID_ARG;
   if (c.logits_dtype != ISD_LOGITS_F32 && c.logits_dtype != ISD_LOGITS_BF16) return ISD_ERR_INVALID_ARG;
   if (c.q_mode < 0 || c.q_mode > 1 || c.propose_mode < 0 || c.propose_mode > 1) return ISD_ERR_INVALID_ARG;
-  if (2 * c.stride - 1 > ISD_MAX_Q || c.vocab % 8 != 0) return ISD_ERR_UNSUPPORTED;
+  if (2 * c.stride - 1 > ISD_MAX_Q || c.vocab % 8 != 0 || c.top_k != 0) return ISD_ERR_UNSUPPORTED;
   if (c.batch > kStaticMaxBatch) return ISD_ERR_TOO_LARGE;
   if (!st->n_ver || !st->active || !st->block_tok || !st->q_row0 || !st->slot_status) return ISD_ERR_INVALID_ARG;
   if (c.stride > 1 && (!st->q_stats || !out->accept || !out->alpha || !out->new_prop_tok || !out->new_q_stats))

@@ -1,0 +1,525 @@
+// isd_verify on top-k / top-p filtered laws (the serving sampling configuration of the paper's
+// appendix: temperature, top-k = 50, top-p = 0.95).  Algorithm 1 is applied to the filtered,
+// renormalised laws: F(row) keeps the top_k entries in the order (value descending, index
+// ascending) and of those the shortest prefix whose probability mass reaches top_p.
+//
+// With at most ISD_MAX_TOP_K tokens of support per law, everything after the selection is tiny, and
+// no vocabulary-wide exponentials are needed at all:
+//   1. topk_rows_kernel    one CTA per (slot, block row): a streaming pass that selects the exact
+//      top-k of the row.  Candidates above a rising threshold go to a shared-memory buffer that is
+//      sorted and cut back to k whenever it has grown by a few hundred entries; the threshold is the
+//      k-th best so far.  Per logit: unpack, one 8-way maximum per thread, one compare.
+//   2. topk_decide_kernel  one CTA per slot: nucleus cut and log-normaliser of every row in fp64
+//      (the oracle's arithmetic, so the cut agrees), sequential accept test, and the Gumbel-max
+//      draws (residual, bonus, proposals) over the supports in fp64 with the same per-index Philox
+//      noise as the unfiltered path.  Only a rejection costs another stream: the proposal-law row
+//      of the previous step is selected again by the same routine.
+#include "isd_internal.cuh"
+#include "isd_stream.cuh"
+
+namespace {
+
+constexpr int kMaxTopK = ISD_MAX_TOP_K;
+constexpr int kCandCap = 8192;     // candidate keys: < kCompactAt left over + at most one stage (4096) of new ones
+constexpr int kCompactAt = 256;    // sort and cut back to k when the buffer holds this many
+constexpr unsigned kKeyNegInf = 0x007FFFFFu;  // value part of the key of -inf: every finite value is above it
+
+struct TopkParams {
+  int B, N, Q, V;
+  int logits_dtype, q_mode, propose_mode, top_k;
+  float inv_t, tau, top_p;
+  uint32_t seed_lo, seed_hi, step;
+  const uint32_t* step_dev;
+  const int32_t* n_ver;
+  const uint8_t* active;
+  const int32_t* block_tok;
+  const int32_t* q_row0;
+  const float* q_stats;
+  uint32_t* slot_status;
+  uint32_t* global_status;
+  const void* logits_cur;
+  const void* q_prev;
+  isd_verify_out out;
+  float* list_val;  // [B, Q, kMaxTopK] raw logits of the row's top-k, best first
+  int* list_idx;    // [B, Q, kMaxTopK]
+  int* list_n;      // [B, Q] entries of the list; -1 - n when the row holds a NaN or +inf
+};
+
+struct TopkShared {
+  RowRing ring;
+  unsigned long long key[kCandCap];
+  int count, bad;
+  unsigned thr;  // value part of the k-th best key so far (candidates of later stages must beat it strictly)
+  float list_val[kMaxTopK];
+  int list_idx[kMaxTopK];
+  int list_n;
+};
+
+// Larger key = better candidate: higher value first, lower index on equal values.
+__device__ __forceinline__ unsigned value_key(float v) { return (unsigned)ord_key(v) ^ 0x80000000u; }
+__device__ __forceinline__ unsigned long long cand_key(float v, int idx) {
+  return ((unsigned long long)value_key(v) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)idx);
+}
+__device__ __forceinline__ float key_value(unsigned long long k) { return ord_val((int)((unsigned)(k >> 32) ^ 0x80000000u)); }
+__device__ __forceinline__ int key_index(unsigned long long k) { return (int)(0xFFFFFFFFu - (unsigned)k); }
+
+__device__ __forceinline__ float max_nan(float a, float b) {  // NaN if either is NaN
+  float d;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
+
+// Sorts the candidate buffer (descending) and keeps the best k; sets the threshold.  Worker threads only.
+__device__ void compact(TopkShared& sh, int k) {
+  worker_sync();  // every append of the stage is visible
+  const int n = sh.count;
+  int m = 2;
+  while (m < n) m <<= 1;
+  for (int i = n + threadIdx.x; i < m; i += kThreads) sh.key[i] = 0ull;  // padding sorts last
+  worker_sync();
+  for (int size = 2; size <= m; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = threadIdx.x; t < (m >> 1); t += kThreads) {
+        const int lo = 2 * t - (t & (stride - 1));
+        const int hi = lo + stride;
+        const bool desc = ((lo & size) == 0);
+        const unsigned long long a = sh.key[lo], b = sh.key[hi];
+        if ((a < b) == desc) { sh.key[lo] = b; sh.key[hi] = a; }
+      }
+      worker_sync();
+    }
+  }
+  if (threadIdx.x == 0) {
+    const int keep = n < k ? n : k;
+    sh.count = keep;
+    sh.thr = keep == k ? (unsigned)(sh.key[k - 1] >> 32) : kKeyNegInf;
+  }
+  worker_sync();
+}
+
+// Exact top-k of a whole logits row, by all kThreads + 32 threads of the CTA: leaves the list (best first)
+// in sh.list_* / sh.list_n and the non-finite flag in sh.bad.  Returns false when a wait ran out.
+template <int DT>
+__device__ bool block_topk(TopkShared& sh, const char* row, int V, int k) {
+  constexpr int kElt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  constexpr int U = DT == ISD_LOGITS_BF16 ? 2 : 1;
+  constexpr int kStageElems = kRowStageBytes / kElt;
+  constexpr int kGroupStep = kStageElems / U;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kRowStages; ++i) {
+      ring_mbar_init(ring_smem_u32(&sh.ring.full[i]), 1);
+      ring_mbar_init(ring_smem_u32(&sh.ring.empty[i]), kThreads / 32);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    sh.count = 0;
+    sh.bad = 0;
+    sh.thr = kKeyNegInf;
+  }
+  __syncthreads();
+  if (threadIdx.x >= kThreads) {
+    bool ok = true;
+    if (threadIdx.x == kThreads) ok = row_producer(sh.ring, row, 0, (size_t)V * kElt);
+    __syncthreads();  // matches the workers' barrier at the end
+    return ok;
+  }
+  const uint32_t full0 = ring_smem_u32(sh.ring.full), empty0 = ring_smem_u32(sh.ring.empty);
+  const uint32_t mine = ring_smem_u32(sh.ring.stage) + threadIdx.x * (DT == ISD_LOGITS_BF16 ? 16 : 32);
+  const int lane = threadIdx.x & 31;
+  bool ok = true;
+  const int stages = (V + kStageElems - 1) / kStageElems;
+  int e = threadIdx.x * 8;
+  for (int c = 0; c < stages; ++c, e += kStageElems) {
+    const int s = c & (kRowStages - 1);
+    ok = ok && mbar_wait_likely(full0 + 8 * s, (uint32_t)(c / kRowStages) & 1u);
+    float l[U][8];
+#pragma unroll
+    for (int g = 0; g < U; ++g) {
+      uint4 a, b = make_uint4(0u, 0u, 0u, 0u);
+      const uint32_t addr = mine + s * kRowStageBytes + g * (kRowStageBytes / U);
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "r"(addr) : "memory");
+      if (DT != ISD_LOGITS_BF16)
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "r"(addr + 16) : "memory");
+      unpack8<DT>(a, b, l[g]);
+      if (!(e + g * kGroupStep < V)) {  // beyond the row (only in its last stage)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) l[g][i] = -INFINITY;
+      }
+    }
+    __syncwarp();
+    if (lane == 0) ring_mbar_arrive(empty0 + 8 * s);
+    float gmax[U];
+#pragma unroll
+    for (int g = 0; g < U; ++g) {
+      gmax[g] = max_nan(max_nan(max_nan(l[g][0], l[g][1]), max_nan(l[g][2], l[g][3])),
+                        max_nan(max_nan(l[g][4], l[g][5]), max_nan(l[g][6], l[g][7])));
+      if (gmax[g] != gmax[g] || gmax[g] == INFINITY) sh.bad = 1;  // NaN or +inf somewhere in the eight
+    }
+    if (c == 0) {
+      // Bootstrap: the k-th best of the threads' maxima of the first group is a lower bound of the k-th best
+      // element, and at least k elements reach it.  The maxima themselves are dropped again; the group is
+      // then scanned like any other, except that equal values still count (they are not "later" elements).
+      if (gmax[0] > -INFINITY) {  // false for NaN
+        int imax = 0;
+#pragma unroll
+        for (int i = 7; i >= 0; --i)
+          if (l[0][i] == gmax[0]) imax = i;
+        sh.key[atomicAdd(&sh.count, 1)] = cand_key(gmax[0], e + imax);
+      }
+      compact(sh, k);
+      if (threadIdx.x == 0) sh.count = 0;
+      worker_sync();
+    }
+    const unsigned thr = *reinterpret_cast<volatile unsigned*>(&sh.thr);
+#pragma unroll
+    for (int g = 0; g < U; ++g) {
+      const bool first = (c == 0 && g == 0);
+      const unsigned gk = value_key(gmax[g]);
+      if (gmax[g] == gmax[g] && (first ? gk >= thr : gk > thr) && gmax[g] > -INFINITY) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const unsigned vk = value_key(l[g][i]);
+          if (l[g][i] == l[g][i] && l[g][i] > -INFINITY && (first ? vk >= thr : vk > thr))
+            sh.key[atomicAdd(&sh.count, 1)] = cand_key(l[g][i], e + g * kGroupStep + i);
+        }
+      }
+    }
+    worker_sync();
+    if (*reinterpret_cast<volatile int*>(&sh.count) >= kCompactAt) compact(sh, k);
+  }
+  compact(sh, k);
+  if (threadIdx.x < sh.count) {
+    sh.list_val[threadIdx.x] = key_value(sh.key[threadIdx.x]);
+    sh.list_idx[threadIdx.x] = key_index(sh.key[threadIdx.x]);
+  }
+  if (threadIdx.x == 0) sh.list_n = sh.count;
+  __syncthreads();  // with the producer warp
+  return ok;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pass 1: the top-k list of every valid row
+// ------------------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(kThreads + 32) topk_rows_kernel(const TopkParams P) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
+  const int b = blockIdx.x, r = blockIdx.y;
+  if (!P.active[b]) return;
+  const int nv = P.n_ver[b];
+  if (nv < 0 || nv > P.N - 1) return;  // flagged by the decide kernel
+  if (r >= nv + P.N) return;
+  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
+  if (!block_topk<DT>(sh, row, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  const size_t base = ((size_t)b * P.Q + r) * kMaxTopK;
+  if (threadIdx.x < sh.list_n) {
+    P.list_val[base + threadIdx.x] = sh.list_val[threadIdx.x];
+    P.list_idx[base + threadIdx.x] = sh.list_idx[threadIdx.x];
+  }
+  if (threadIdx.x == 0) P.list_n[(size_t)b * P.Q + r] = sh.bad ? -1 - sh.list_n : sh.list_n;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pass 2: everything else, one CTA per slot
+// ------------------------------------------------------------------------------------------------
+// Nucleus of a sorted top-k list in fp64, in the oracle's order of operations: w_i = exp(l_i invT - l_0 invT),
+// Z = sum w_i, support = shortest prefix whose cumulated w reaches top_p * Z.  Returns the support size and
+// the log-normaliser of the support.
+__device__ int nucleus(const float* val, int n, double inv_t, double top_p, double& lse) {
+  lse = -INFINITY;
+  if (n <= 0) return 0;
+  const double m = (double)val[0] * inv_t;
+  if (isinf(m) && m < 0) return n;
+  double Z = 0.0;
+  for (int i = 0; i < n; ++i) Z += exp((double)val[i] * inv_t - m);
+  double cum = 0.0;
+  int keep = n;
+  for (int i = 0; i < n; ++i) {
+    cum += exp((double)val[i] * inv_t - m);
+    if (cum >= top_p * Z) { keep = i + 1; break; }
+  }
+  double S = 0.0;
+  for (int i = 0; i < keep; ++i) S += exp((double)val[i] * inv_t - m);
+  lse = m + log(S);
+  return keep;
+}
+
+// warp-wide arg max of (score, index): highest score, lowest index on ties (the oracle scans indices upwards
+// and replaces only on a strictly greater score)
+__device__ __forceinline__ void warp_argmax(double& s, int& idx) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const double os = __shfl_xor_sync(0xffffffffu, s, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+    if (oi >= 0 && (idx < 0 || os > s || (os == s && oi < idx))) { s = os; idx = oi; }
+  }
+}
+
+__device__ __forceinline__ double gumbel_at(const TopkParams& P, uint32_t step, int b, uint32_t tagpos, int idx) {
+  const uint4 r = philox4x32_10((uint32_t)idx >> 2, step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
+  return gumbel_f64(philox_word(r, idx & 3));
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkParams P) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
+  __shared__ int s_n[32], s_bad[32], s_rej, s_a;
+  __shared__ double s_lse[32];
+  const int b = blockIdx.x;
+  if (!P.active[b]) return;
+  const int nv = P.n_ver[b];
+  if (nv < 0 || nv > P.N - 1) {
+    if (threadIdx.x == 0) {
+      atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
+      atomicOr(P.global_status, ISD_ST_SLOT_CAPACITY);
+    }
+    return;
+  }
+  const int q_len = nv + P.N, NP = P.N - 1;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const double inv_t = (double)P.inv_t, top_p = (double)P.top_p;
+  const uint32_t step = P.step_dev ? *P.step_dev : P.step;
+  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  const float* LV = P.list_val + (size_t)b * P.Q * kMaxTopK;
+  const int* LI = P.list_idx + (size_t)b * P.Q * kMaxTopK;
+
+  // ---- every row's support and log-normaliser (lane = row)
+  if (warp == 0) {
+    int n = 0, bad = 0;
+    double lse = -INFINITY;
+    if (lane < q_len) {
+      int ln = P.list_n[(size_t)b * P.Q + lane];
+      if (ln < 0) { bad = 1; ln = -1 - ln; }
+      n = nucleus(LV + (size_t)lane * kMaxTopK, ln, inv_t, top_p, lse);
+    }
+    s_n[lane] = n; s_bad[lane] = bad; s_lse[lane] = lse;
+  }
+  __syncthreads();
+
+  // ---- sequential accept test (Algorithm 1, introspection loop) on the filtered laws
+  if (threadIdx.x == 0) {
+    uint32_t status = 0;
+    int a = nv, rej = 0;
+    for (int m = 1; m <= NP; ++m) status |= s_bad[nv + m] ? ISD_ST_NONFINITE_LOGIT : 0u;
+    for (int j = 1; j <= NP; ++j) {
+      P.out.accept[(size_t)b * NP + j - 1] = -1;
+      P.out.alpha[(size_t)b * NP + j - 1] = NAN;
+    }
+    for (int j = 1; j <= nv; ++j) {
+      const int x = P.block_tok[(size_t)b * P.Q + j];
+      if (x < 0 || x >= P.V) { status |= ISD_ST_BAD_TOKEN_ID; a = -1; break; }
+      if (s_bad[j - 1]) status |= ISD_ST_NONFINITE_LOGIT;
+      // p~(x): zero unless x is in the support of the filtered anchor law
+      float logp = -INFINITY;
+      for (int i = 0; i < s_n[j - 1]; ++i)
+        if (LI[(size_t)(j - 1) * kMaxTopK + i] == x) logp = LV[(size_t)(j - 1) * kMaxTopK + i] * P.inv_t - (float)s_lse[j - 1];
+      float logq = 0.f;
+      if (P.q_mode == 0) {
+        const float* qs = P.q_stats + ((size_t)b * NP + j - 1) * 2;
+        logq = qs[1] - qs[0];
+      }
+      float al = (1.f + P.tau) * expf(logp - logq);
+      al = fminf(al, 1.f);
+      if (al != al) al = 0.f;
+      const uint4 rnd = philox4x32_10(0u, step, (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)j, P.seed_lo, P.seed_hi);
+      const float u = (float)(rnd.x >> 8) * 0x1p-24f;
+      P.out.alpha[(size_t)b * NP + j - 1] = al;
+      if (u < al) {
+        P.out.accept[(size_t)b * NP + j - 1] = 1;
+      } else {
+        P.out.accept[(size_t)b * NP + j - 1] = 0;
+        a = j - 1;
+        rej = j;
+        break;
+      }
+    }
+    if (a >= 0 && rej == 0 && s_bad[nv]) status |= ISD_ST_NONFINITE_LOGIT;
+    for (int j = 0; j < P.N; ++j) P.out.out_tok[(size_t)b * P.N + j] = -1;
+    P.out.repl_tok[b] = -1;
+    if (a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL)) {
+      P.out.accept_len[b] = 0;
+      P.out.n_emit[b] = 0;
+      atomicOr(&P.slot_status[b], status);
+      atomicOr(P.global_status, status);
+      a = -1;
+    } else {
+      P.out.accept_len[b] = a;
+      P.out.n_emit[b] = a + 1;
+      for (int j = 1; j <= a; ++j) P.out.out_tok[(size_t)b * P.N + j - 1] = P.block_tok[(size_t)b * P.Q + j];
+    }
+    s_a = a;
+    s_rej = rej;
+  }
+  __syncthreads();
+  const int a = s_a, rej = s_rej;
+
+  // ---- proposals of the MASK rows: Gumbel-max over the support (warp m - 1 draws row nv + m), or its head
+  if (warp >= 1 && warp <= NP && warp < kThreads / 32) {
+    for (int m = warp; m <= NP; m += kThreads / 32 - 1) {
+      const int rr = nv + m, n = s_n[rr];
+      const float* v = LV + (size_t)rr * kMaxTopK;
+      const int* ix = LI + (size_t)rr * kMaxTopK;
+      double best = -INFINITY;
+      int tok = -1;
+      float ltok = NAN;
+      if (P.propose_mode == 1) {
+        if (n > 0) tok = ix[0];
+      } else {
+        const uint32_t tagpos = (ISD_TAG_PROPOSE << 16) | (uint32_t)m;
+        for (int i = lane; i < n; i += 32) {
+          const double lp = (double)v[i] * inv_t;
+          if (isinf(lp) && lp < 0) continue;
+          const double sc = lp + gumbel_at(P, step, b, tagpos, ix[i]);
+          if (tok < 0 || sc > best || (sc == best && ix[i] < tok)) { best = sc; tok = ix[i]; }
+        }
+        warp_argmax(best, tok);
+      }
+      if (lane == 0) {
+        for (int i = 0; i < n; ++i)
+          if (ix[i] == tok) ltok = v[i] * P.inv_t;
+        P.out.new_prop_tok[(size_t)b * NP + m - 1] = tok;
+        P.out.new_q_stats[((size_t)b * NP + m - 1) * 2 + 0] = (float)s_lse[rr];
+        P.out.new_q_stats[((size_t)b * NP + m - 1) * 2 + 1] = tok >= 0 ? ltok : NAN;
+      }
+    }
+  }
+  if (a < 0) return;  // frozen: no emission (uniform over the CTA)
+
+  // ---- the token drawn for the emission
+  if (rej == 0) {
+    // bonus / free token: Gumbel-max over the support of the row of the last clean token
+    if (warp == 0) {
+      const int n = s_n[nv];
+      const float* v = LV + (size_t)nv * kMaxTopK;
+      const int* ix = LI + (size_t)nv * kMaxTopK;
+      const uint32_t tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)(nv + 1);
+      double best = -INFINITY;
+      int tok = -1;
+      for (int i = lane; i < n; i += 32) {
+        const double lp = (double)v[i] * inv_t;
+        if (isinf(lp) && lp < 0) continue;
+        const double sc = lp + gumbel_at(P, step, b, tagpos, ix[i]);
+        if (tok < 0 || sc > best || (sc == best && ix[i] < tok)) { best = sc; tok = ix[i]; }
+      }
+      warp_argmax(best, tok);
+      if (lane == 0) {
+        P.out.repl_tok[b] = tok;
+        P.out.out_tok[(size_t)b * P.N + a] = tok;
+      }
+    }
+    return;
+  }
+  // replacement from normalize(max(0, p~ - q~)) over the anchor's support; q~ needs the filtered proposal law,
+  // whose row (of the previous step's logits) is selected again here
+  int nq = 0;
+  double lse_q = 0.0;
+  const int x = P.block_tok[(size_t)b * P.Q + rej];
+  if (P.q_mode == 0) {
+    if (P.q_prev == nullptr) return;  // the caller gave no proposal-law rows
+    const char* qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + (P.q_row0[b] + rej - 1)) * (size_t)P.V * elt;
+    if (!block_topk<DT>(sh, qrow, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+    if (threadIdx.x == 0) {
+      double l;
+      s_n[31] = nucleus(sh.list_val, sh.list_n, inv_t, top_p, l);  // rows above 30 do not exist (Q <= 31)
+      s_lse[31] = l;
+    }
+    __syncthreads();
+    nq = s_n[31];
+    lse_q = s_lse[31];
+  }
+  if (warp != 0) return;
+  const int r = rej - 1, n = s_n[r];
+  const float* v = LV + (size_t)r * kMaxTopK;
+  const int* ix = LI + (size_t)r * kMaxTopK;
+  const uint32_t tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)rej;
+  double best = -INFINITY, best_p = -INFINITY;
+  int tok = -1, tok_p = -1;  // residual draw; draw from p~ with the same noise (fallback for an empty residual)
+  for (int i = lane; i < n; i += 32) {
+    const double lp = (double)v[i] * inv_t;
+    if (isinf(lp) && lp < 0) continue;
+    const double g = gumbel_at(P, step, b, tagpos, ix[i]);
+    const double pi = exp(lp - s_lse[r]);
+    double qi = 0.0;
+    if (P.q_mode == 0) {
+      for (int t = 0; t < nq; ++t)
+        if (sh.list_idx[t] == ix[i]) qi = exp((double)sh.list_val[t] * inv_t - lse_q);
+    } else {
+      qi = (ix[i] == x) ? 1.0 : 0.0;
+    }
+    const double rr = pi - qi;
+    if (rr > 0.0) {
+      const double sc = log(rr) + g;
+      if (tok < 0 || sc > best || (sc == best && ix[i] < tok)) { best = sc; tok = ix[i]; }
+    }
+    const double scp = lp - s_lse[r] + g;
+    if (tok_p < 0 || scp > best_p || (scp == best_p && ix[i] < tok_p)) { best_p = scp; tok_p = ix[i]; }
+  }
+  warp_argmax(best, tok);
+  warp_argmax(best_p, tok_p);
+  if (lane == 0) {
+    if (tok < 0) {
+      tok = tok_p;
+      atomicOr(&P.slot_status[b], ISD_ST_EMPTY_RESIDUAL);
+      atomicOr(P.global_status, ISD_ST_EMPTY_RESIDUAL);
+    }
+    P.out.repl_tok[b] = tok;
+    P.out.out_tok[(size_t)b * P.N + a] = tok;
+  }
+}
+
+constexpr size_t kTopkSmem = sizeof(TopkShared);
+
+}  // namespace
+
+int isd_verify_topk_create(isd_ctx* ctx) {
+  const isd_config& c = ctx->cfg;
+  const size_t rows = (size_t)c.batch * ctx->Q;
+  if (cudaMalloc(&ctx->topk_val, sizeof(float) * rows * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  if (cudaMalloc(&ctx->topk_idx, sizeof(int) * rows * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  if (cudaMalloc(&ctx->topk_n, sizeof(int) * rows) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  cudaMemset(ctx->topk_n, 0, sizeof(int) * rows);
+  cudaError_t e = cudaSuccess;
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_rows_kernel<ISD_LOGITS_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_rows_kernel<ISD_LOGITS_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_decide_kernel<ISD_LOGITS_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_decide_kernel<ISD_LOGITS_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmem);
+  return e == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}
+
+void isd_verify_topk_destroy(isd_ctx* ctx) {
+  cudaFree(ctx->topk_val);
+  cudaFree(ctx->topk_idx);
+  cudaFree(ctx->topk_n);
+  ctx->topk_val = nullptr;
+  ctx->topk_idx = nullptr;
+  ctx->topk_n = nullptr;
+}
+
+int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
+                           const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
+                           cudaStream_t stream) {
+  const isd_config& c = ctx->cfg;
+  TopkParams P;
+  P.B = c.batch; P.N = c.stride; P.Q = ctx->Q; P.V = c.vocab;
+  P.logits_dtype = c.logits_dtype; P.q_mode = c.q_mode; P.propose_mode = c.propose_mode; P.top_k = c.top_k;
+  P.inv_t = c.inv_temperature; P.tau = c.tau; P.top_p = c.top_p;
+  P.seed_lo = (uint32_t)c.seed; P.seed_hi = (uint32_t)(c.seed >> 32); P.step = step;
+  P.step_dev = ctx->step_counter;
+  P.n_ver = st->n_ver; P.active = st->active; P.block_tok = st->block_tok; P.q_row0 = st->q_row0;
+  P.q_stats = st->q_stats; P.slot_status = st->slot_status; P.global_status = ctx->global_status;
+  P.logits_cur = logits_cur; P.q_prev = q_prev_logits; P.out = *out;
+  P.list_val = ctx->topk_val; P.list_idx = ctx->topk_idx; P.list_n = ctx->topk_n;
+  const dim3 grid1(c.batch, ctx->Q);
+  if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
+  if (c.logits_dtype == ISD_LOGITS_BF16) {
+    topk_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads + 32, kTopkSmem, stream>>>(P);
+    topk_decide_kernel<ISD_LOGITS_BF16><<<c.batch, kThreads + 32, kTopkSmem, stream>>>(P);
+  } else {
+    topk_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads + 32, kTopkSmem, stream>>>(P);
+    topk_decide_kernel<ISD_LOGITS_F32><<<c.batch, kThreads + 32, kTopkSmem, stream>>>(P);
+  }
+  if (ctx->ev_verify1) cudaEventRecord(ctx->ev_verify1, stream);
+  ctx->launches += 2;
+  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}

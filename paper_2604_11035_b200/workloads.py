@@ -44,6 +44,8 @@ class Workload:
     propose_mode: int = 1           # 1 = argmax proposals (paper's serving setting), 0 = sampled
     q_mode: int = 0
     seed: int = 0
+    top_k: int = 0                  # > 0: top-k / top-p filtered laws (the paper's serving sampling configuration)
+    top_p: float = 1.0
 
     @property
     def Q(self) -> int:

@@ -36,13 +36,15 @@ def state_to_np(st: dict) -> dict:
 
 
 def oracle_step(w: wl.Workload, s: dict, q, k_new, v_new, logits_cur, q_prev, step, *,
-                inv_temperature=1.0, tau=0.0, mask_token=None, do_attn=True, sm_scale=None, top_k=0, top_p=1.0):
+                inv_temperature=1.0, tau=0.0, mask_token=None, do_attn=True, sm_scale=None, top_k=None, top_p=None):
     """One full oracle step (attention, verify, commit) on numpy state `s`, in place.
 
     Returns (attn_out, attn_lse, VerifyResult, q_len_before).
     """
     N = w.stride
     ldt = 0 if w.logits_dtype == "f32" else 1
+    top_k = w.top_k if top_k is None else top_k       # the workload's sampling configuration unless overridden
+    top_p = w.top_p if top_p is None else top_p
     q_len = np.where(s["active"] != 0, s["n_ver"] + N, 0).astype(np.int32)
     out = lse = None
     if do_attn:

@@ -42,6 +42,30 @@ def test_ragged_multi_tile_chain(attn_impl, dtype, propose_mode, q_mode, N):
     assert rep["rejections"] > 0 and rep["tpf"] > 1.0
 
 
+@pytest.mark.parametrize("dtype,propose_mode,q_mode,N,top_k,top_p", [
+    ("bf16", 0, 0, 4, 50, 0.95), ("f32", 0, 0, 4, 8, 0.7), ("bf16", 1, 0, 8, 50, 0.95), ("bf16", 1, 1, 3, 20, 1.0),
+    ("bf16", 0, 0, 2, 1, 1.0), ("f32", 0, 0, 3, 64, 0.5)])
+def test_filtered_laws_chain(dtype, propose_mode, q_mode, N, top_k, top_p):
+    # top-k / top-p filtered verification: ragged rows, ties (bf16 logits repeat values), mixed P / NP steps
+    w = Workload("filtered", batch=6, stride=N, n_q_heads=8, n_kv_heads=2, vocab=8192 + 8 * 29, ctx_min=3,
+                 ctx_max=300, logits_dtype=dtype, logit_sigma=2.0, peaked_frac=0.5, steps=8,
+                 propose_mode=propose_mode, q_mode=q_mode, seed=60 + N + top_k, top_k=top_k, top_p=top_p)
+    rep = run_chain_parity(w, steps=8, device=DEV)
+    assert_clean(rep)
+    assert rep["tpf"] >= 1.0
+    if top_k > 1:
+        assert rep["rejections"] > 0
+
+
+def test_filtered_laws_full_vocab_and_batch():
+    # the serving configuration at the benchmark's vocabulary and a batch that fills the machine several times
+    w = Workload("filtered_big", batch=96, stride=8, vocab=151936, ctx_min=64, ctx_max=512, logits_dtype="bf16",
+                 peaked_frac=0.9, steps=4, propose_mode=0, seed=71, top_k=50, top_p=0.95)
+    rep = run_chain_parity(w, steps=3, device=DEV, attn_slots=[0, 95])
+    assert_clean(rep)
+    assert rep["rejections"] > 0
+
+
 def test_temperature_and_relaxed_acceptance():
     w = Workload("temp", batch=6, stride=4, n_q_heads=8, n_kv_heads=2, vocab=2048, ctx_min=20, ctx_max=200,
                  logits_dtype="f32", logit_sigma=2.0, peaked_frac=0.5, steps=6, propose_mode=0, seed=77)
