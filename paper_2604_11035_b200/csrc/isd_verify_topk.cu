@@ -20,9 +20,7 @@
 namespace {
 
 constexpr int kMaxTopK = ISD_MAX_TOP_K;
-constexpr int kCandCap = 8192;     // candidate keys: < kCompactAt left over + at most one stage (4096) of new ones
-constexpr int kCompactAt = 256;    // sort and cut back to k when the buffer holds this many
-constexpr unsigned kKeyNegInf = 0x007FFFFFu;  // value part of the key of -inf: every finite value is above it
+constexpr int kCandCap = 1024;  // candidate keys in shared memory
 
 struct TopkParams {
   int B, N, Q, V;
@@ -48,8 +46,9 @@ struct TopkParams {
 struct TopkShared {
   RowRing ring;
   unsigned long long key[kCandCap];
-  int count, bad;
-  unsigned thr;  // value part of the k-th best key so far (candidates of later stages must beat it strictly)
+  unsigned long long sorted[kMaxTopK];
+  unsigned offer[kThreads / 32];
+  int count, bad, again, have;
   float list_val[kMaxTopK];
   int list_idx[kMaxTopK];
   int list_n;
@@ -69,13 +68,29 @@ __device__ __forceinline__ float max_nan(float a, float b) {  // NaN if either i
   return d;
 }
 
-// Sorts the candidate buffer (descending) and keeps the best k; sets the threshold.  Worker threads only.
-__device__ void compact(TopkShared& sh, int k) {
-  worker_sync();  // every append of the stage is visible
-  const int n = sh.count;
+// Appends the elements of a group of eight that reach the bound.  Deliberately not inlined: the call keeps this
+// rare path (about one group in three hundred) behind a real branch; inlined, the compiler predicates it and
+// every group pays for its instructions.
+__device__ __noinline__ void collect_group(TopkShared* sh, float x0, float x1, float x2, float x3, float x4, float x5,
+                                           float x6, float x7, int e, unsigned long long bound) {
+  const float x[8] = {x0, x1, x2, x3, x4, x5, x6, x7};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if (x[i] > -INFINITY) {
+      const unsigned long long kk = cand_key(x[i], e + i);
+      if (kk >= bound) {
+        const int pos = atomicAdd(&sh->count, 1);
+        if (pos < kCandCap) sh->key[pos] = kk;
+      }
+    }
+  }
+}
+
+// Sorts key[0, n) descending (bitonic, padded with zeros to a power of two <= kCandCap).  Worker threads only.
+__device__ void sort_keys(unsigned long long* key, int n) {
   int m = 2;
   while (m < n) m <<= 1;
-  for (int i = n + threadIdx.x; i < m; i += kThreads) sh.key[i] = 0ull;  // padding sorts last
+  for (int i = n + threadIdx.x; i < m; i += kThreads) key[i] = 0ull;  // padding sorts last
   worker_sync();
   for (int size = 2; size <= m; size <<= 1) {
     for (int stride = size >> 1; stride > 0; stride >>= 1) {
@@ -83,116 +98,158 @@ __device__ void compact(TopkShared& sh, int k) {
         const int lo = 2 * t - (t & (stride - 1));
         const int hi = lo + stride;
         const bool desc = ((lo & size) == 0);
-        const unsigned long long a = sh.key[lo], b = sh.key[hi];
-        if ((a < b) == desc) { sh.key[lo] = b; sh.key[hi] = a; }
+        const unsigned long long a = key[lo], b = key[hi];
+        if ((a < b) == desc) { key[lo] = b; key[hi] = a; }
       }
       worker_sync();
     }
   }
-  if (threadIdx.x == 0) {
-    const int keep = n < k ? n : k;
-    sh.count = keep;
-    sh.thr = keep == k ? (unsigned)(sh.key[k - 1] >> 32) : kKeyNegInf;
+}
+
+// The best k of n <= kThreads distinct non-zero keys, best first, by counting: thread t ranks key t among all of
+// them (no barriers inside, unlike a sorting network).  Result in out[0, return value).  Worker threads only.
+__device__ int rank_select(const unsigned long long* key, int n, int k, unsigned long long* out) {
+  if (threadIdx.x < n) {
+    const unsigned long long mine = key[threadIdx.x];
+    int rank = 0;
+    for (int j = 0; j < n; ++j) rank += key[j] > mine ? 1 : 0;
+    if (rank < k) out[rank] = mine;
   }
   worker_sync();
+  return n < k ? n : k;
+}
+
+// A value that at least k elements reach, from the threads' maxima, without a block-wide sort: every warp sorts
+// its 32 maxima with shuffles and offers its ceil(k / warps)-th best; the smallest offer is reached by that many
+// maxima in every warp, k or more in all.  0 when some warp has too few finite maxima (then everything finite is
+// collected).  Worker threads only.
+__device__ unsigned bound_from_maxima(unsigned vkey, int k, unsigned* sm_offer) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned v = vkey;
+#pragma unroll
+  for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      const unsigned o = __shfl_xor_sync(0xffffffffu, v, stride);
+      const bool up = ((lane & size) == 0), lower = ((lane & stride) == 0);
+      v = (lower == up) ? (v > o ? v : o) : (v < o ? v : o);
+    }
+  }
+  const int per_warp = (k + kThreads / 32 - 1) / (kThreads / 32);
+  if (lane == per_warp - 1) sm_offer[warp] = v;  // descending: lane r - 1 holds the r-th best
+  worker_sync();
+  unsigned b = sm_offer[0];
+#pragma unroll
+  for (int w = 1; w < kThreads / 32; ++w) b = b < sm_offer[w] ? b : sm_offer[w];
+  return b;
 }
 
 // Exact top-k of a whole logits row, by all kThreads + 32 threads of the CTA: leaves the list (best first)
 // in sh.list_* / sh.list_n and the non-finite flag in sh.bad.  Returns false when a wait ran out.
+//
+// The row is streamed twice.  First stream: every thread keeps the best value it sees, and from those maxima
+// comes a value that at least k elements of the row reach, i.e. a lower bound of the row's k-th best (a tight
+// one: the top-k fall into mostly distinct threads).  Second stream: every element that reaches the bound is
+// collected, about k plus a few dozen, and ranked by (value, index).  Should the collected set overflow the
+// buffer (many equal values), the k-th best of what was collected is a strictly better bound and the second
+// stream is repeated.
 template <int DT>
 __device__ bool block_topk(TopkShared& sh, const char* row, int V, int k) {
   constexpr int kElt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   constexpr int U = DT == ISD_LOGITS_BF16 ? 2 : 1;
   constexpr int kStageElems = kRowStageBytes / kElt;
   constexpr int kGroupStep = kStageElems / U;
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < kRowStages; ++i) {
-      ring_mbar_init(ring_smem_u32(&sh.ring.full[i]), 1);
-      ring_mbar_init(ring_smem_u32(&sh.ring.empty[i]), kThreads / 32);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    sh.count = 0;
-    sh.bad = 0;
-    sh.thr = kKeyNegInf;
-  }
-  __syncthreads();
-  if (threadIdx.x >= kThreads) {
-    bool ok = true;
-    if (threadIdx.x == kThreads) ok = row_producer(sh.ring, row, 0, (size_t)V * kElt);
-    __syncthreads();  // matches the workers' barrier at the end
-    return ok;
-  }
+  const bool worker = threadIdx.x < kThreads;
   const uint32_t full0 = ring_smem_u32(sh.ring.full), empty0 = ring_smem_u32(sh.ring.empty);
   const uint32_t mine = ring_smem_u32(sh.ring.stage) + threadIdx.x * (DT == ISD_LOGITS_BF16 ? 16 : 32);
   const int lane = threadIdx.x & 31;
-  bool ok = true;
   const int stages = (V + kStageElems - 1) / kStageElems;
-  int e = threadIdx.x * 8;
-  for (int c = 0; c < stages; ++c, e += kStageElems) {
-    const int s = c & (kRowStages - 1);
-    ok = ok && mbar_wait_likely(full0 + 8 * s, (uint32_t)(c / kRowStages) & 1u);
-    float l[U][8];
-#pragma unroll
-    for (int g = 0; g < U; ++g) {
-      uint4 a, b = make_uint4(0u, 0u, 0u, 0u);
-      const uint32_t addr = mine + s * kRowStageBytes + g * (kRowStageBytes / U);
-      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "r"(addr) : "memory");
-      if (DT != ISD_LOGITS_BF16)
-        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "r"(addr + 16) : "memory");
-      unpack8<DT>(a, b, l[g]);
-      if (!(e + g * kGroupStep < V)) {  // beyond the row (only in its last stage)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) l[g][i] = -INFINITY;
+  bool ok = true;
+  unsigned long long bound = 0ull;
+  if (threadIdx.x == 0) sh.bad = 0;
+  for (int pass = 0;; ++pass) {
+    if (threadIdx.x == 0) {
+      for (int i = 0; i < kRowStages; ++i) {
+        ring_mbar_init(ring_smem_u32(&sh.ring.full[i]), 1);
+        ring_mbar_init(ring_smem_u32(&sh.ring.empty[i]), kThreads / 32);
       }
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      sh.count = 0;
+      sh.again = 0;
     }
-    __syncwarp();
-    if (lane == 0) ring_mbar_arrive(empty0 + 8 * s);
-    float gmax[U];
+    __syncthreads();
+    if (!worker) {
+      if (threadIdx.x == kThreads) ok = row_producer(sh.ring, row, 0, (size_t)V * kElt) && ok;
+    } else {
+      float tmax = -INFINITY;  // first stream: the best value this thread has seen
+      int e = threadIdx.x * 8;
+      for (int c = 0; c < stages; ++c, e += kStageElems) {
+        const int s = c & (kRowStages - 1);
+        ok = mbar_wait_likely(full0 + 8 * s, (uint32_t)(c / kRowStages) & 1u) && ok;
+        float l[U][8];
 #pragma unroll
-    for (int g = 0; g < U; ++g) {
-      gmax[g] = max_nan(max_nan(max_nan(l[g][0], l[g][1]), max_nan(l[g][2], l[g][3])),
-                        max_nan(max_nan(l[g][4], l[g][5]), max_nan(l[g][6], l[g][7])));
-      if (gmax[g] != gmax[g] || gmax[g] == INFINITY) sh.bad = 1;  // NaN or +inf somewhere in the eight
-    }
-    if (c == 0) {
-      // Bootstrap: the k-th best of the threads' maxima of the first group is a lower bound of the k-th best
-      // element, and at least k elements reach it.  The maxima themselves are dropped again; the group is
-      // then scanned like any other, except that equal values still count (they are not "later" elements).
-      if (gmax[0] > -INFINITY) {  // false for NaN
-        int imax = 0;
+        for (int g = 0; g < U; ++g) {
+          uint4 a, b = make_uint4(0u, 0u, 0u, 0u);
+          const uint32_t addr = mine + s * kRowStageBytes + g * (kRowStageBytes / U);
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "r"(addr) : "memory");
+          if (DT != ISD_LOGITS_BF16)
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "r"(addr + 16) : "memory");
+          unpack8<DT>(a, b, l[g]);
+          if (c == stages - 1 && !(e + g * kGroupStep < V)) {  // beyond the row
 #pragma unroll
-        for (int i = 7; i >= 0; --i)
-          if (l[0][i] == gmax[0]) imax = i;
-        sh.key[atomicAdd(&sh.count, 1)] = cand_key(gmax[0], e + imax);
-      }
-      compact(sh, k);
-      if (threadIdx.x == 0) sh.count = 0;
-      worker_sync();
-    }
-    const unsigned thr = *reinterpret_cast<volatile unsigned*>(&sh.thr);
+            for (int i = 0; i < 8; ++i) l[g][i] = -INFINITY;
+          }
+        }
+        __syncwarp();
+        if (lane == 0) ring_mbar_arrive(empty0 + 8 * s);
 #pragma unroll
-    for (int g = 0; g < U; ++g) {
-      const bool first = (c == 0 && g == 0);
-      const unsigned gk = value_key(gmax[g]);
-      if (gmax[g] == gmax[g] && (first ? gk >= thr : gk > thr) && gmax[g] > -INFINITY) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const unsigned vk = value_key(l[g][i]);
-          if (l[g][i] == l[g][i] && l[g][i] > -INFINITY && (first ? vk >= thr : vk > thr))
-            sh.key[atomicAdd(&sh.count, 1)] = cand_key(l[g][i], e + g * kGroupStep + i);
+        for (int g = 0; g < U; ++g) {
+          const float gmax = max_nan(max_nan(max_nan(l[g][0], l[g][1]), max_nan(l[g][2], l[g][3])),
+                                     max_nan(max_nan(l[g][4], l[g][5]), max_nan(l[g][6], l[g][7])));
+          if (gmax != gmax || gmax == INFINITY) {
+            sh.bad = 1;  // NaN or +inf somewhere in the eight: the slot will be frozen, the list does not matter
+            continue;
+          }
+          if (pass == 0) {
+            tmax = fmaxf(tmax, gmax);  // value only: which element it was does not matter for a bound
+          } else if (gmax > -INFINITY && value_key(gmax) >= (unsigned)(bound >> 32)) {
+            collect_group(&sh, l[g][0], l[g][1], l[g][2], l[g][3], l[g][4], l[g][5], l[g][6], l[g][7],
+                          e + g * kGroupStep, bound);
+          }
         }
       }
+      if (pass == 0) {
+        bound = (unsigned long long)bound_from_maxima(tmax > -INFINITY ? value_key(tmax) : 0u, k, sh.offer) << 32;
+        if (threadIdx.x == 0) sh.again = 1;
+      } else {
+        worker_sync();
+        const int total = sh.count;
+        worker_sync();  // everybody has read the count
+        int n;
+        if (total <= kThreads) {  // the usual case
+          n = rank_select(sh.key, total, k, sh.sorted);
+        } else {
+          const int collected = total < kCandCap ? total : kCandCap;
+          sort_keys(sh.key, collected);
+          n = collected < k ? collected : k;
+          if (threadIdx.x < n) sh.sorted[threadIdx.x] = sh.key[threadIdx.x];
+          if (total > kCandCap && pass < 4096) {  // overflow (many equal values): a strictly better bound, once more
+            bound = sh.key[k - 1];
+            if (threadIdx.x == 0) sh.again = 1;
+          }
+          worker_sync();
+        }
+        if (threadIdx.x < n) {
+          sh.list_val[threadIdx.x] = key_value(sh.sorted[threadIdx.x]);
+          sh.list_idx[threadIdx.x] = key_index(sh.sorted[threadIdx.x]);
+        }
+        if (threadIdx.x == 0) sh.list_n = n;
+      }
     }
-    worker_sync();
-    if (*reinterpret_cast<volatile int*>(&sh.count) >= kCompactAt) compact(sh, k);
+    __syncthreads();  // producer warp and workers meet; sh.again is final
+    if (!sh.again) break;
+    __syncthreads();  // everybody has read the flag before thread 0 clears it for the next pass
   }
-  compact(sh, k);
-  if (threadIdx.x < sh.count) {
-    sh.list_val[threadIdx.x] = key_value(sh.key[threadIdx.x]);
-    sh.list_idx[threadIdx.x] = key_index(sh.key[threadIdx.x]);
-  }
-  if (threadIdx.x == 0) sh.list_n = sh.count;
-  __syncthreads();  // with the producer warp
   return ok;
 }
 
