@@ -165,39 +165,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
-// 2^x for a pair of non-positive arguments without the transcendental unit, which both streaming kernels
-// saturate: round to the nearest integer with the 1.5 * 2^23 trick, evaluate a polynomial of the
-// remainder f in [-0.5, 0.5] with packed FMAs, and add the integer to the exponent field.
-// DEG = 5: relative error < 3e-7 (as good as ex2.approx); DEG = 3: < 1.1e-4 (enough for bf16 results).
-// Arguments below -125 (including -inf) give a value below 2^-124, i.e. zero for every use here.
-template <int DEG>
-__device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& r0, float& r1) {
-  const float c0 = fmaxf(x0, -125.f), c1 = fmaxf(x1, -125.f);
-  const uint64_t xc = pack2(c0, c1);
-  const uint64_t magic = pack2(12582912.f, 12582912.f), nmagic = pack2(-12582912.f, -12582912.f);
-  const uint64_t t = add2(xc, magic);                       // magic + round(x)
-  const uint64_t f = fma2(add2(t, nmagic), pack2(-1.f, -1.f), xc);  // x - round(x)
-  uint64_t p;
-  if (DEG == 5) {
-    p = pack2(0.0013400432653725147f, 0.0013400432653725147f);
-    p = fma2(p, f, pack2(0.009676037356257439f, 0.009676037356257439f));
-    p = fma2(p, f, pack2(0.05550327152013779f, 0.05550327152013779f));
-    p = fma2(p, f, pack2(0.2402210682630539f, 0.2402210682630539f));
-    p = fma2(p, f, pack2(0.6931471824645996f, 0.6931471824645996f));
-    p = fma2(p, f, pack2(1.0000001192092896f, 1.0000001192092896f));
-  } else {
-    p = pack2(0.05592203512787819f, 0.05592203512787819f);
-    p = fma2(p, f, pack2(0.24264007806777954f, 0.24264007806777954f));
-    p = fma2(p, f, pack2(0.6931210160255432f, 0.6931210160255432f));
-    p = fma2(p, f, pack2(0.9999244809150696f, 0.9999244809150696f));
-  }
-  float t0, t1, p0, p1;
-  unpack2(t, t0, t1);
-  unpack2(p, p0, p1);
-  r0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
-  r1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
-}
-
 // -------------------------------------------------------------------------------------------------
 // mbarrier / bulk-copy helpers for shared-memory rings (one producer thread, many consumers)
 // -------------------------------------------------------------------------------------------------

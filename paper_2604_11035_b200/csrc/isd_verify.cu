@@ -28,19 +28,6 @@
 #include "isd_internal.cuh"
 #include "isd_stream.cuh"
 
-#ifdef EXP_COUNT
-__device__ unsigned long long g_dbg[8];
-extern "C" int isd_debug_counters(unsigned long long* out) {
-  cudaMemcpyFromSymbol(out, g_dbg, sizeof(g_dbg));
-  unsigned long long z[8] = {};
-  cudaMemcpyToSymbol(g_dbg, z, sizeof(z));
-  return 0;
-}
-#define DBG_COUNT(i, v) atomicAdd(&g_dbg[i], (unsigned long long)(v))
-#else
-#define DBG_COUNT(i, v)
-#endif
-
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
@@ -590,7 +577,6 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
     const float l4[4] = {v.x, v.y, v.z, v.w};
     const uint4 rnd = philox4x32_10((uint32_t)idx >> 2, J.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
     const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-    DBG_COUNT(J.resid ? 1 : 0, 1);
     // -ln u' >= 1 - u' >= nf 2^-24 with nf = floor(2^24 (1 - u')), so g_i <= -ln(nf 2^-24): the element
     // cannot come within 2e-3 of the running best when nf >= 1.002 * 2^24 * exp(l_i invT - shift - best)
     float K2 = 24.0028853901f - (shift + best) * kLog2e;  // log2 of the factor; +inf while there is no best
@@ -600,7 +586,6 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
       const float nf = (float)((~w[i]) >> 8);
       const float bound = ex2f(fmaf(l4[i], scale2, K2));
       if (!(nf >= bound)) {
-        DBG_COUNT(J.resid ? 3 : 2, 1);
         const float sc = job_score(P, J, l4[i], idx + i, w[i]);
         if (sc > -INFINITY) {
           top.push(sc, idx + i);
@@ -715,7 +700,6 @@ __global__ void __launch_bounds__(kThreads) verify_sample_kernel(const VerifyPar
 
   int lo, hi;
   chunk_range(P.V, P.sample_splits, split, lo, hi);
-  if (threadIdx.x == 0) { DBG_COUNT(J.resid ? 5 : 4, (hi - lo) / 4); if (J.resid && !(best0 > -INFINITY)) DBG_COUNT(6, 1); }
   Top2 top;
   sample_pass<DT>(P, J, lo, hi, b, fmaxf(-INFINITY, best0), top, sm_queue, &sm_best, sm_ring);
 
