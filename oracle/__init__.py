@@ -205,3 +205,13 @@ def release(*, N, page_size, ctx_len, n_ver, page_table, free_stack, free_top, a
     rc = f(B, N, page_size, page_table.shape[1], _p(ctx_len), _p(n_ver), _p(page_table),
            _p(free_stack), _p(free_top), _p(active), _p(slots), slots.shape[0])
     assert rc == 0, rc
+
+
+def lora_linear(x, w, a, b, gate, scale):
+    """Segment-gated LoRA linear layer of the lossless R-ISD variant (Eq. 5 and the R-ISD paragraph of Sec. 3.2):
+    row j of the output is W x_j, plus scale * B A x_j only where gate[j] is set (the [MASK] rows); clean rows see
+    the base weights alone, which is what makes their verification lossless.  Plain fp64 definition:
+    x [M, K], w [N, K], a [R, K], b [N, R], gate [M] -> y [M, N]."""
+    x, w, a, b = (np.asarray(t, np.float64) for t in (x, w, a, b))
+    g = (np.asarray(gate) != 0).astype(np.float64)[:, None]
+    return x @ w.T + g * float(scale) * ((x @ a.T) @ b.T)
