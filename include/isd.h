@@ -247,6 +247,30 @@ int isd_step_layers(isd_ctx* ctx, isd_batch_state* st, const isd_layer_args* lay
  */
 int isd_set_step_counter(isd_ctx* ctx, uint32_t* device_counter);
 
+/* Arguments of isd_lora_linear: device pointers, row-major bf16 matrices. */
+typedef struct isd_lora_args {
+  const void* x;       /* [m, k]    activations of the step's token rows (m = B * Q)          */
+  const void* w;       /* [n, k]    base weight: y = x w^T                                     */
+  const void* a;       /* [rank, k] LoRA down-projection                                      */
+  const void* b;       /* [n, rank] LoRA up-projection                                        */
+  const uint8_t* gate; /* [m]       1 = [MASK] row (LoRA residual applied), 0 = clean row     */
+  void* t;             /* [m, rank] scratch of the caller: gated down-projection              */
+  void* y;             /* [m, n]    output                                                    */
+  int32_t m, n, k, rank;
+  float scale;         /* LoRA scaling (alpha / rank)                                         */
+} isd_lora_args;
+
+/*
+ * Segment-gated LoRA linear layer of the lossless R-ISD variant (Sec. 3.2, R-ISD paragraph, Eq. 5):
+ *   y[j, :] = w x[j, :] + gate[j] * scale * b (a x[j, :])
+ * so that clean rows are computed with the base weights alone (their verification is lossless) and
+ * only [MASK] rows see the adapter.  bf16 operands, fp32 accumulation on the tensor cores, bf16
+ * results; the intermediate t = gate * scale * (x a^T) is rounded to bf16 once.  Requirements
+ * (else ISD_ERR_UNSUPPORTED / ISD_ERR_ALIGNMENT): k and rank multiples of 64, n a multiple of 32,
+ * 16-byte aligned pointers.  Two kernels on `cuda_stream`, no allocation, no synchronisation.
+ */
+int isd_lora_linear(isd_ctx* ctx, const isd_lora_args* args, void* cuda_stream);
+
 /* Off the hot path: return the pages of finished slots (device array `slots`
  * of n ids) to the free stack and mark them inactive. */
 int isd_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t n,

@@ -19,7 +19,7 @@ ST_BAD_PAGE_ID, ST_NONFINITE_LOGIT, ST_EMPTY_RESIDUAL = 8, 16, 32
 
 EXPORTS = ["isd_create", "isd_destroy", "isd_attn", "isd_verify", "isd_commit", "isd_step",
            "isd_release", "isd_read_status", "isd_set_profile_events", "isd_launch_count", "isd_strerror",
-           "isd_verify_static", "isd_step_layers", "isd_set_step_counter"]
+           "isd_verify_static", "isd_step_layers", "isd_set_step_counter", "isd_lora_linear"]
 
 
 class IsdConfig(C.Structure):
@@ -49,6 +49,11 @@ class IsdStepArgs(C.Structure):
 
 class IsdLayerArgs(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("q", "k_new", "v_new", "k_pool", "v_pool", "attn_out", "attn_lse")]
+
+
+class IsdLoraArgs(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("x", "w", "a", "b", "gate", "t", "y")] + \
+        [(n, C.c_int32) for n in ("m", "n", "k", "rank")] + [("scale", C.c_float)]
 
 
 _lib = None
@@ -81,6 +86,8 @@ def load():
         lib.isd_step_layers.restype = C.c_int
         lib.isd_set_step_counter.argtypes = [vp, vp]
         lib.isd_set_step_counter.restype = C.c_int
+        lib.isd_lora_linear.argtypes = [vp, C.POINTER(IsdLoraArgs), vp]
+        lib.isd_lora_linear.restype = C.c_int
         lib.isd_launch_count.argtypes = [vp]
         lib.isd_launch_count.restype = C.c_int64
         lib.isd_strerror.argtypes = [C.c_int]
@@ -206,6 +213,16 @@ class Isd:
         o = self.out_struct(out)
         _check(self.lib.isd_step_layers(self.ctx, C.byref(s), layers, len(layers), _ptr(logits_cur),
                                         _ptr(q_prev_logits), C.byref(o), step, _stream()), "isd_step_layers")
+
+    def isd_lora_linear(self, x, w, a, b, gate, scale: float, t=None, y=None):
+        """y = x w^T + gate * scale * (x a^T) b^T on bf16 CUDA tensors; allocates t / y when not given."""
+        m, k = x.shape
+        n, rank = b.shape
+        t = torch.empty(m, rank, dtype=torch.bfloat16, device=x.device) if t is None else t
+        y = torch.empty(m, n, dtype=torch.bfloat16, device=x.device) if y is None else y
+        args = IsdLoraArgs(_ptr(x), _ptr(w), _ptr(a), _ptr(b), _ptr(gate), _ptr(t), _ptr(y), m, n, k, rank, scale)
+        _check(self.lib.isd_lora_linear(self.ctx, C.byref(args), _stream()), "isd_lora_linear")
+        return y
 
     def isd_set_step_counter(self, counter):
         """`counter`: a CUDA uint32 / int32 tensor of one element, or None."""

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libisd.so")
-SOURCES = ["isd_api.cu", "isd_verify.cu", "isd_verify_topk.cu", "isd_commit.cu", "isd_attn_plain.cu", "isd_attn_tc.cu"]
+SOURCES = ["isd_api.cu", "isd_verify.cu", "isd_verify_topk.cu", "isd_commit.cu", "isd_attn_plain.cu", "isd_attn_tc.cu", "isd_lora_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

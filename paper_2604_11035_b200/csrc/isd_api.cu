@@ -203,6 +203,15 @@ int isd_step_layers(isd_ctx* ctx, isd_batch_state* st, const isd_layer_args* lay
   return isd_commit(ctx, st, out, cuda_stream);
 }
 
+int isd_lora_linear(isd_ctx* ctx, const isd_lora_args* a, void* cuda_stream) {
+  if (!ctx || !a || !a->x || !a->w || !a->a || !a->b || !a->gate || !a->t || !a->y) return ISD_ERR_INVALID_ARG;
+  if (a->m < 1 || a->n < 1 || a->k < 1 || a->rank < 1) return ISD_ERR_INVALID_ARG;
+  if (a->k % 64 != 0 || a->rank % 64 != 0 || a->n % 32 != 0) return ISD_ERR_UNSUPPORTED;
+  if (!aligned16(a->x) || !aligned16(a->w) || !aligned16(a->a) || !aligned16(a->b) || !aligned16(a->t) || !aligned16(a->y))
+    return ISD_ERR_ALIGNMENT;
+  return isd_launch_lora_linear(ctx, a, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
 int isd_set_step_counter(isd_ctx* ctx, uint32_t* device_counter) {
   if (!ctx) return ISD_ERR_INVALID_ARG;
   ctx->step_counter = device_counter;

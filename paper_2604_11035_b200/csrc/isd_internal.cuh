@@ -270,6 +270,7 @@ void isd_verify_topk_destroy(isd_ctx* ctx);
 int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
                            const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
                            cudaStream_t stream);
+int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t stream);
 int isd_launch_commit(isd_ctx* ctx, isd_batch_state* st, const isd_verify_out* out, cudaStream_t stream);
 int isd_launch_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t n,
                        cudaStream_t stream);

@@ -1,0 +1,316 @@
+// isd_lora_linear: segment-gated LoRA linear layer of the lossless R-ISD variant (Sec. 3.2, the R-ISD
+// paragraph and Eq. 5): y_j = W x_j + 1[j in MASK] * s * B A x_j over the M = B * Q token rows of a step.
+//
+// Two launches of one tcgen05 GEMM kernel (C = A1 B1^T (+ A2 B2^T), bf16 operands, fp32 accumulation in
+// tensor memory):
+//   1. t = gate * s * (x A^T)            [M, R]  the gated, scaled down-projection (bf16)
+//   2. y = x W^T + t B^T                 [M, N]  one GEMM over the two K segments (K, then R)
+// so the gate costs nothing in the large GEMM and clean rows provably see the base weights only (their t is 0).
+//
+// Kernel: persistent CTAs, one 128 x BN output tile at a time.  Warp 4 streams the operands with TMA
+// (2-D maps, 64-element K slices = 128-byte rows, SWIZZLE_128B, no multicast) into a 4-stage ring; warp 5
+// issues tcgen05.mma (M = 128, N = BN, K = 16, both operands from shared memory) into one of two TMEM
+// accumulators; warps 0-3 read the other accumulator back (tcgen05.ld, one lane = one row), apply gate and
+// scale, and store bf16, so the epilogue of a tile overlaps the main loop of the next.  Every mbarrier wait is
+// bounded (status bit 0x80000000, then the CTA drains and frees its tensor memory).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "isd_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kBM = 128;
+constexpr int kBK = 64;                       // bf16 elements per K slice = one 128-byte swizzled row
+constexpr int kStages = 4;
+constexpr uint32_t kSpinLimit = 1u << 24;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false (and the abort flag raised) when the limit is reached or somebody else gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile(
+      "{\n.reg .b32 rx;\n.reg .pred px;\n"
+      "elect.sync rx|px, 0xffffffff;\n"
+      "selp.u32 %0, 1, 0, px;\n}"
+      : "=r"(pred));
+  return pred != 0;
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
+}
+// K-major shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1: rows of 128 bytes, groups of
+// eight rows 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr) {
+  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | ((16u >> 4) << 16);
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  return ((uint64_t)hi << 32) | lo;
+}
+#define TMEM_LD32(taddr, v)                                                                             \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                         \
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25," \
+      "%26,%27,%28,%29,%30,%31}, [%32];"                                                                \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),        \
+        "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),      \
+        "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),      \
+        "=r"(v[29]), "=r"(v[30]), "=r"(v[31])                                                           \
+      : "r"(taddr))
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+struct GemmParams {
+  int M, N, K1, K2;           // C[M, N] = A1[M, K1] B1[N, K1]^T + A2[M, K2] B2[N, K2]^T   (K2 = 0: one segment)
+  __nv_bfloat16* c;           // row-major, leading dimension N
+  const uint8_t* gate;        // [M] or nullptr: rows with gate 0 are written as zeros
+  float scale;
+  uint32_t* global_status;
+};
+
+enum { BAR_FULL = 0, BAR_EMPTY = kStages, BAR_ACC_FULL = 2 * kStages, BAR_ACC_FREE = 2 * kStages + 2,
+       BAR_COUNT = 2 * kStages + 4 };
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_b1,
+               const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b2) {
+  constexpr int kStageA = kBM * kBK * 2, kStageB = BN * kBK * 2, kStageBytes = kStageA + kStageB;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sm_base = smem_u32(smem);
+  const uint32_t bar_base = sm_base + kStages * kStageBytes;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kStages * kStageBytes + BAR_COUNT * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kStages * kStageBytes + BAR_COUNT * 8 + 8);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  auto bar = [&](int i) { return bar_base + 8u * (uint32_t)i; };
+  if (sm_base & 1023u) {  // the swizzled layout assumes a 1 KiB aligned window
+    if (threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+    return;
+  }
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kStages; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_ACC_FULL + i), 1); mbar_init(bar(BAR_ACC_FREE + i), 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  const int tiles_m = (P.M + kBM - 1) / kBM, tiles_n = (P.N + BN - 1) / BN;
+  const int n_tiles = tiles_m * tiles_n;
+  const int ks1 = P.K1 / kBK, ks2 = P.K2 / kBK, ks = ks1 + ks2;  // K slices per tile
+
+  if (warp == 4) {
+    // ============================================================================ TMA producer
+    uint32_t fill = 0;
+    for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
+      const int m0 = (tile % tiles_m) * kBM, n0 = (tile / tiles_m) * BN;  // neighbouring CTAs share a B panel
+      bool ok = true;
+      for (int i = 0; i < ks && ok; ++i, ++fill) {
+        const uint32_t s = fill % kStages, ph = (fill / kStages) & 1u;
+        ok = mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag);
+        if (!ok) break;
+        if (elect_one()) {
+          mbar_arrive_expect_tx(bar(BAR_FULL + s), (uint32_t)kStageBytes);  // out-of-range rows are zero-filled, still counted
+          const uint32_t dst = sm_base + s * kStageBytes;
+          const bool seg2 = i >= ks1;
+          const int k0 = (seg2 ? i - ks1 : i) * kBK;
+          tma_load_2d(dst, seg2 ? &map_a2 : &map_a1, k0, m0, bar(BAR_FULL + s));
+          tma_load_2d(dst + kStageA, seg2 ? &map_b2 : &map_b1, k0, n0, bar(BAR_FULL + s));
+        }
+        __syncwarp();
+      }
+      if (!ok) break;
+    }
+    if (*abort_flag) {  // every issued copy must land before the CTA may leave
+      for (uint32_t f = (fill > kStages ? fill - kStages : 0); f < fill; ++f)
+        mbar_wait(bar(BAR_FULL + f % kStages), (f / kStages) & 1u, abort_flag);
+    }
+  } else if (warp == 5) {
+    // ============================================================================ MMA issuer
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+    uint32_t cons = 0, t_local = 0;
+    for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x, ++t_local) {
+      const uint32_t acc = t_local & 1u;
+      // the epilogue warps must have read this accumulator's previous tile
+      if (t_local >= 2 && !mbar_wait(bar(BAR_ACC_FREE + acc), ((t_local >> 1) - 1u) & 1u, abort_flag)) break;
+      tc_fence_after();
+      bool ok = true;
+      for (int i = 0; i < ks && ok; ++i, ++cons) {
+        const uint32_t s = cons % kStages, ph = (cons / kStages) & 1u;
+        ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        if (elect_one()) {
+          const uint32_t a0 = sm_base + s * kStageBytes, b0 = a0 + kStageA;
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)
+            tc_mma(tmem + acc * (uint32_t)BN, smem_desc_kmajor(a0 + k * 32), smem_desc_kmajor(b0 + k * 32), idesc,
+                   (i > 0 || k > 0) ? 1u : 0u);
+          tc_commit(bar(BAR_EMPTY + s));
+          if (i == ks - 1) tc_commit(bar(BAR_ACC_FULL + acc));
+        }
+        __syncwarp();
+      }
+      if (!ok) break;
+    }
+  } else {
+    // ============================================================================ epilogue (warps 0-3)
+    uint32_t t_local = 0;
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x, ++t_local) {
+      const int m0 = (tile % tiles_m) * kBM, n0 = (tile / tiles_m) * BN;
+      const uint32_t acc = t_local & 1u;
+      if (!mbar_wait(bar(BAR_ACC_FULL + acc), (t_local >> 1) & 1u, abort_flag)) break;
+      tc_fence_after();
+      const int row = m0 + warp * 32 + lane;
+      const bool row_ok = row < P.M;
+      const float f = (P.gate == nullptr || (row_ok && P.gate[row])) ? P.scale : 0.f;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t v[32];
+        TMEM_LD32(tmem + lane_base + acc * (uint32_t)BN + (uint32_t)c0, v);
+        tmem_wait_ld();
+        if (row_ok && n0 + c0 < P.N) {  // N is a multiple of 32 here (checked by the launcher)
+          uint4* dst = reinterpret_cast<uint4*>(P.c + (size_t)row * P.N + n0 + c0);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            dst[q] = make_uint4(pack_bf16(__uint_as_float(v[8 * q]) * f, __uint_as_float(v[8 * q + 1]) * f),
+                                pack_bf16(__uint_as_float(v[8 * q + 2]) * f, __uint_as_float(v[8 * q + 3]) * f),
+                                pack_bf16(__uint_as_float(v[8 * q + 4]) * f, __uint_as_float(v[8 * q + 5]) * f),
+                                pack_bf16(__uint_as_float(v[8 * q + 6]) * f, __uint_as_float(v[8 * q + 7]) * f));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_ACC_FREE + acc));
+    }
+  }
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// row-major bf16 matrix [rows, cols] viewed in boxes of 64 columns x box_rows rows
+int encode_matrix(CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return ISD_ERR_CUDA;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ISD_OK : ISD_ERR_CUDA;
+}
+
+template <int BN>
+int launch_gemm(isd_ctx* ctx, const GemmParams& P, const void* a1, const void* b1, const void* a2, const void* b2,
+                cudaStream_t stream) {
+  constexpr int kSmem = kStages * (kBM * kBK * 2 + BN * kBK * 2) + BAR_COUNT * 8 + 64;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+      return ISD_ERR_CUDA;
+    attr_set = true;
+  }
+  CUtensorMap ma1, mb1, ma2, mb2;
+  int rc = encode_matrix(&ma1, a1, P.M, P.K1, kBM);
+  if (rc == ISD_OK) rc = encode_matrix(&mb1, b1, P.N, P.K1, BN);
+  if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&ma2, a2, P.M, P.K2, kBM) : encode_matrix(&ma2, a1, P.M, P.K1, kBM);
+  if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&mb2, b2, P.N, P.K2, BN) : encode_matrix(&mb2, b1, P.N, P.K1, BN);
+  if (rc != ISD_OK) return rc;
+  const int tiles = ((P.M + kBM - 1) / kBM) * ((P.N + BN - 1) / BN);
+  const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
+  gemm_tc_kernel<BN><<<grid, kThreads, kSmem, stream>>>(P, ma1, mb1, ma2, mb2);
+  ctx->launches++;
+  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}
+
+}  // namespace
+
+int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t stream) {
+  // 1. t = gate * scale * (x A^T): N = rank, one K segment
+  GemmParams P1;
+  P1.M = a->m; P1.N = a->rank; P1.K1 = a->k; P1.K2 = 0;
+  P1.c = reinterpret_cast<__nv_bfloat16*>(a->t); P1.gate = a->gate; P1.scale = a->scale;
+  P1.global_status = ctx->global_status;
+  int rc = launch_gemm<128>(ctx, P1, a->x, a->a, nullptr, nullptr, stream);
+  if (rc != ISD_OK) return rc;
+  // 2. y = x W^T + t B^T: two K segments, no gate (it is already in t)
+  GemmParams P2;
+  P2.M = a->m; P2.N = a->n; P2.K1 = a->k; P2.K2 = a->rank;
+  P2.c = reinterpret_cast<__nv_bfloat16*>(a->y); P2.gate = nullptr; P2.scale = 1.f;
+  P2.global_status = ctx->global_status;
+  return launch_gemm<256>(ctx, P2, a->x, a->w, a->t, a->b, stream);
+}
