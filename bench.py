@@ -223,6 +223,57 @@ def run_model_step(args):
     print(json.dumps(line))
 
 
+def run_lora(args):
+    """`--lora N,K,R`: the segment-gated LoRA linear layer (isd_lora_linear) on the token rows of one step of the
+    workload (M = batch x (2 stride - 1)), timed by CUDA events; roofline against the measured dense bf16 peak."""
+    import torch
+    import paper_2604_11035_b200 as pkg
+    from paper_2604_11035_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = rank_workload(args.config, 0, args.sweep)
+    N, K, R = (int(v) for v in args.lora.split(","))
+    M = (args.batch or w.batch) * w.Q
+    small = wl.Workload("lora_ctx", batch=1, stride=2, n_q_heads=8, n_kv_heads=2, vocab=1024, ctx_min=16, ctx_max=16, steps=1)
+    eng = pkg.isd_for_workload(small, wl.make_state(small, dev))
+    g = torch.Generator(device=dev)
+    g.manual_seed(w.seed)
+    bf = lambda *shape, s=1.0: (torch.randn(*shape, generator=g, device=dev) * s).to(torch.bfloat16)
+    x, wt, a, b = bf(M, K), bf(N, K, s=K ** -0.5), bf(R, K, s=K ** -0.5), bf(N, R, s=R ** -0.5)
+    # MASK rows of a P step: rows n_ver + 1 .. of every slot (here: the last stride - 1 rows of each block)
+    gate = (torch.arange(M, device=dev) % w.Q >= w.stride).to(torch.uint8)
+    t = torch.empty(M, R, dtype=torch.bfloat16, device=dev)
+    y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+    flush = wl.l2_flush_buffer(dev, 512)
+    Kn, W = args.steps, args.warmup
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(W + Kn)]
+    sampler = ClockSampler(0)
+    for i in range(W + Kn):
+        if i == W:
+            torch.cuda.synchronize()
+            sampler.start()
+        flush.zero_()
+        ev[i][0].record()
+        eng.isd_lora_linear(x, wt, a, b, gate, 0.5, t=t, y=y)
+        ev[i][1].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = [a_.elapsed_time(b_) for a_, b_ in ev[W:]]
+    t_total = sum(ms) / 1e3
+    flops = 2.0 * M * (N * (K + R) + R * K)
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    peak = float(peaks.get("bf16_tflops", 1590.0))
+    tf = flops * Kn / t_total / 1e12
+    print(json.dumps({
+        "metric": "isd_lora_linear_positions_per_s", "value": M * Kn / t_total, "unit": UNIT, "n_gpus": 1, "steps": Kn,
+        "warmup": W, "ms_per_step": sum(ms) / Kn, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"lora_linear m{M} n{N} k{K} rank{R} (token rows of {w.name})", "l2": "flushed before every call"},
+        "roofline": {"kernel": "gemm_tc_kernel (2 launches)", "bound": "tensor", "achieved": tf, "peak": peak,
+                     "peak_kind": "measured (burst)" if peaks else "fallback", "unit": "TFLOP/s", "frac": tf / peak, "traffic": None},
+        "gpu_launches": 2 * Kn, "status_word": eng.isd_read_status(), "clocks": clocks}))
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -522,6 +573,7 @@ def main():
                     help="one point of the sweep workload (stride in 2,4,8,16; batch in 1,8,64,256,512) instead of --config")
     ap.add_argument("--top-k", type=int, default=0, help="verify on top-k / top-p filtered laws (0 = plain softmax laws)")
     ap.add_argument("--top-p", type=float, default=1.0)
+    ap.add_argument("--lora", default=None, metavar="N,K,RANK", help="time the segment-gated LoRA linear layer on the step's token rows")
     ap.add_argument("--layers", type=int, default=0, help="model-step mode: this many attention layers per step (isd_step_layers)")
     ap.add_argument("--graph", action="store_true", help="model-step mode: replay the step from a CUDA graph")
     ap.add_argument("--sequential-pages", action="store_true", help="identity page order instead of a shuffled pool")
@@ -529,6 +581,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.lora:
+        run_lora(args)
     elif args.layers > 0 or args.graph:
         args.layers = max(1, args.layers)
         run_model_step(args)

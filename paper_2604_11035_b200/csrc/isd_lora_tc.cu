@@ -23,7 +23,10 @@ namespace {
 constexpr int kThreads = 192;
 constexpr int kBM = 128;
 constexpr int kBK = 64;                       // bf16 elements per K slice = one 128-byte swizzled row
-constexpr int kStages = 4;
+#ifndef ISD_LORA_STAGES
+#define ISD_LORA_STAGES 4
+#endif
+constexpr int kStages = ISD_LORA_STAGES;
 constexpr uint32_t kSpinLimit = 1u << 24;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -312,5 +315,8 @@ int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t st
   P2.M = a->m; P2.N = a->n; P2.K1 = a->k; P2.K2 = a->rank;
   P2.c = reinterpret_cast<__nv_bfloat16*>(a->y); P2.gate = nullptr; P2.scale = 1.f;
   P2.global_status = ctx->global_status;
-  return launch_gemm<256>(ctx, P2, a->x, a->w, a->t, a->b, stream);
+#ifndef ISD_LORA_BN
+#define ISD_LORA_BN 256
+#endif
+  return launch_gemm<ISD_LORA_BN>(ctx, P2, a->x, a->w, a->t, a->b, stream);
 }
