@@ -63,10 +63,10 @@ struct RowRing {
 };
 
 // Producer (one thread): streams bytes [byte_lo, byte_hi) of a row into the ring, one contiguous bulk copy
-// per stage.  Returns false when a wait ran out.
-__device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t byte_lo, size_t byte_hi) {
+// per stage.  c is the ring's running stage counter: it carries on over consecutive ranges, so that several
+// ranges can go through one ring without re-initialising its barriers.  Returns false when a wait ran out.
+__device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t byte_lo, size_t byte_hi, int& c) {
   const uint32_t full0 = ring_smem_u32(R.full), empty0 = ring_smem_u32(R.empty), st0 = ring_smem_u32(R.stage);
-  int c = 0;
   for (size_t off = byte_lo; off < byte_hi; off += kRowStageBytes, ++c) {
     const int s = c & (kRowStages - 1);
     const uint32_t ph = (c / kRowStages) & 1;
@@ -77,6 +77,11 @@ __device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t
     ring_bulk_g2s(st0 + s * kRowStageBytes, row + off, bytes, full0 + 8 * s);
   }
   return true;
+}
+
+__device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t byte_lo, size_t byte_hi) {
+  int c = 0;
+  return row_producer(R, row, byte_lo, byte_hi, c);
 }
 
 

@@ -21,6 +21,7 @@ namespace {
 
 constexpr int kMaxTopK = ISD_MAX_TOP_K;
 constexpr int kCandCap = 1024;  // candidate keys in shared memory
+constexpr int kGroupCap = 512;  // queued groups in shared memory
 
 struct TopkParams {
   int B, N, Q, V;
@@ -45,10 +46,11 @@ struct TopkParams {
 
 struct TopkShared {
   RowRing ring;
-  unsigned long long key[kCandCap];
+  __align__(16) unsigned long long key[kCandCap];
   unsigned long long sorted[kMaxTopK];
   unsigned offer[kThreads / 32];
-  int count, bad, again, have;
+  int group[kGroupCap];  // first element of every group of eight that may hold a candidate
+  int count, gcount, bad, again, have, over;
   float list_val[kMaxTopK];
   int list_idx[kMaxTopK];
   int list_n;
@@ -86,6 +88,23 @@ __device__ __noinline__ void collect_group(TopkShared* sh, float x0, float x1, f
   }
 }
 
+// The largest of the eight logits of a group, NaN if one of them is NaN.  bf16 pairs are compared packed: three
+// two-lane maxima, then the two halves of the last word.  (Which of -0 and +0 wins is irrelevant to the callers:
+// they use the result in float comparisons, or as a lower bound.)
+template <int DT>
+__device__ __forceinline__ float group_max(const uint4& a, const uint4& b) {
+  if (DT == ISD_LOGITS_BF16) {
+    uint32_t m0, m1, m;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(m0) : "r"(a.x), "r"(a.y));
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(m1) : "r"(a.z), "r"(a.w));
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(m0), "r"(m1));
+    return max_nan(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+  }
+  const float m0 = max_nan(max_nan(__uint_as_float(a.x), __uint_as_float(a.y)), max_nan(__uint_as_float(a.z), __uint_as_float(a.w)));
+  const float m1 = max_nan(max_nan(__uint_as_float(b.x), __uint_as_float(b.y)), max_nan(__uint_as_float(b.z), __uint_as_float(b.w)));
+  return max_nan(m0, m1);
+}
+
 // Sorts key[0, n) descending (bitonic, padded with zeros to a power of two <= kCandCap).  Worker threads only.
 __device__ void sort_keys(unsigned long long* key, int n) {
   int m = 2;
@@ -111,9 +130,16 @@ __device__ void sort_keys(unsigned long long* key, int n) {
 __device__ int rank_select(const unsigned long long* key, int n, int k, unsigned long long* out) {
   if (threadIdx.x < n) {
     const unsigned long long mine = key[threadIdx.x];
-    int rank = 0;
-    for (int j = 0; j < n; ++j) rank += key[j] > mine ? 1 : 0;
-    if (rank < k) out[rank] = mine;
+    int r0 = 0, r1 = 0;
+    int j = 0;
+    for (; j + 4 <= n; j += 4) {  // key is 16-byte aligned: two keys per load
+      const ulonglong2 p = *reinterpret_cast<const ulonglong2*>(key + j);
+      const ulonglong2 q = *reinterpret_cast<const ulonglong2*>(key + j + 2);
+      r0 += (p.x > mine ? 1 : 0) + (q.x > mine ? 1 : 0);
+      r1 += (p.y > mine ? 1 : 0) + (q.y > mine ? 1 : 0);
+    }
+    for (; j < n; ++j) r0 += key[j] > mine ? 1 : 0;
+    if (r0 + r1 < k) out[r0 + r1] = mine;
   }
   worker_sync();
   return n < k ? n : k;
@@ -154,7 +180,7 @@ __device__ unsigned bound_from_maxima(unsigned vkey, int k, unsigned* sm_offer) 
 // buffer (many equal values), the k-th best of what was collected is a strictly better bound and the second
 // stream is repeated.
 template <int DT>
-__device__ bool block_topk(TopkShared& sh, const char* row, int V, int k) {
+__device__ bool block_topk_two_stream(TopkShared& sh, const char* row, int e_lo, int e_hi, int k) {
   constexpr int kElt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   constexpr int U = DT == ISD_LOGITS_BF16 ? 2 : 1;
   constexpr int kStageElems = kRowStageBytes / kElt;
@@ -163,7 +189,7 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int V, int k) {
   const uint32_t full0 = ring_smem_u32(sh.ring.full), empty0 = ring_smem_u32(sh.ring.empty);
   const uint32_t mine = ring_smem_u32(sh.ring.stage) + threadIdx.x * (DT == ISD_LOGITS_BF16 ? 16 : 32);
   const int lane = threadIdx.x & 31;
-  const int stages = (V + kStageElems - 1) / kStageElems;
+  const int stages = (e_hi - e_lo + kStageElems - 1) / kStageElems;
   bool ok = true;
   unsigned long long bound = 0ull;
   if (threadIdx.x == 0) sh.bad = 0;
@@ -179,10 +205,10 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int V, int k) {
     }
     __syncthreads();
     if (!worker) {
-      if (threadIdx.x == kThreads) ok = row_producer(sh.ring, row, 0, (size_t)V * kElt) && ok;
+      if (threadIdx.x == kThreads) ok = row_producer(sh.ring, row, (size_t)e_lo * kElt, (size_t)e_hi * kElt) && ok;
     } else {
       float tmax = -INFINITY;  // first stream: the best value this thread has seen
-      int e = threadIdx.x * 8;
+      int e = e_lo + threadIdx.x * 8;
       for (int c = 0; c < stages; ++c, e += kStageElems) {
         const int s = c & (kRowStages - 1);
         ok = mbar_wait_likely(full0 + 8 * s, (uint32_t)(c / kRowStages) & 1u) && ok;
@@ -195,7 +221,7 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int V, int k) {
           if (DT != ISD_LOGITS_BF16)
             asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "r"(addr + 16) : "memory");
           unpack8<DT>(a, b, l[g]);
-          if (c == stages - 1 && !(e + g * kGroupStep < V)) {  // beyond the row
+          if (c == stages - 1 && !(e + g * kGroupStep < e_hi)) {  // beyond the range
 #pragma unroll
             for (int i = 0; i < 8; ++i) l[g][i] = -INFINITY;
           }
@@ -253,6 +279,183 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int V, int k) {
   return ok;
 }
 
+constexpr int kHeadStages = 8;  // stages of the head, read twice to find a first bound
+constexpr int kCheckEvery = 4;  // stages between two looks at the queue of noted groups (a power of two)
+constexpr int kExpandAt = 48;   // noted groups from which a look turns them into candidates
+constexpr int kCompactAt = 96;  // candidates from which they are cut back to the best k and the bound rises
+
+// One stage of the ring: waits for it, takes this thread's groups of eight as packed words, releases the stage.
+template <int DT, int U>
+__device__ __forceinline__ bool take_stage(uint32_t full0, uint32_t empty0, uint32_t mine, int cc, uint4 (&a)[U], uint4 (&b)[U]) {
+  const int s = cc & (kRowStages - 1);
+  const bool ok = mbar_wait_likely(full0 + 8 * s, (uint32_t)(cc / kRowStages) & 1u);
+#pragma unroll
+  for (int g = 0; g < U; ++g) {
+    b[g] = make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t addr = mine + s * kRowStageBytes + g * (kRowStageBytes / U);
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a[g].x), "=r"(a[g].y), "=r"(a[g].z), "=r"(a[g].w) : "r"(addr) : "memory");
+    if (DT != ISD_LOGITS_BF16)
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b[g].x), "=r"(b[g].y), "=r"(b[g].z), "=r"(b[g].w) : "r"(addr + 16) : "memory");
+  }
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) ring_mbar_arrive(empty0 + 8 * s);
+  return ok;
+}
+
+// Exact top-k of elements [e_lo, e_hi) of a logits row (e_lo a multiple of 8) in ONE stream of them (plus their
+// head a second time), by all kThreads + 32 threads of the CTA; same result as block_topk_two_stream: the list
+// (best first) in sh.list_* / sh.list_n and the non-finite flag in sh.bad.  Returns false when a wait ran out.
+//
+// The head (kHeadStages stages) goes through the ring first: the threads' maxima over it give a value that k of
+// its elements reach.  Then the whole range follows through the same ring, head included (those bytes come from
+// L2).  The common path per group of eight is its packed maximum and one compare.  A group whose maximum reaches
+// the bound is only noted (its element index goes to a queue).  At the end of the head, and then every
+// kCheckEvery stages, the workers look at the queue; when it is long enough they expand it densely, one group
+// per thread, re-reading the eight logits from global memory (L2): the elements that reach the bound become
+// candidates, and from kCompactAt candidates on the best k are kept and the bound rises to the k-th best so
+// far, so that fewer and fewer groups are noted (about k ln(n / head) after the head).  When more arrives
+// between two looks than the buffers hold (a row sorted upwards, long runs of equal values), nothing more is
+// noted, the stream is drained and the two-stream routine, which handles any input, starts over.
+template <int DT>
+__device__ bool block_topk(TopkShared& sh, const char* row, int e_lo, int e_hi, int k) {
+  constexpr int kElt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  constexpr int U = DT == ISD_LOGITS_BF16 ? 2 : 1;
+  constexpr int kStageElems = kRowStageBytes / kElt;
+  constexpr int kGroupStep = kStageElems / U;
+  const bool worker = threadIdx.x < kThreads;
+  const int stages = (e_hi - e_lo + kStageElems - 1) / kStageElems;
+  const int head = stages < kHeadStages ? stages : kHeadStages;
+  bool ok = true;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kRowStages; ++i) {
+      ring_mbar_init(ring_smem_u32(&sh.ring.full[i]), 1);
+      ring_mbar_init(ring_smem_u32(&sh.ring.empty[i]), kThreads / 32);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    sh.count = 0;
+    sh.gcount = 0;
+    sh.bad = 0;
+    sh.over = 0;
+    sh.list_n = 0;
+  }
+  __syncthreads();
+  if (!worker) {
+    if (threadIdx.x == kThreads) {
+      const size_t lo = (size_t)e_lo * kElt, hi = (size_t)e_hi * kElt, head_hi = lo + (size_t)head * kRowStageBytes;
+      int c = 0;
+      ok = row_producer(sh.ring, row, lo, head_hi < hi ? head_hi : hi, c);
+      ok = ok && row_producer(sh.ring, row, lo, hi, c);
+    }
+  } else {
+    const uint32_t full0 = ring_smem_u32(sh.ring.full), empty0 = ring_smem_u32(sh.ring.empty);
+    const uint32_t mine = ring_smem_u32(sh.ring.stage) + threadIdx.x * (DT == ISD_LOGITS_BF16 ? 16 : 32);
+    uint4 a[U], b[U];
+    // ---- the head: the best value this thread sees
+    float tmax = -INFINITY;
+    for (int c = 0; c < head; ++c) {
+      ok = take_stage<DT, U>(full0, empty0, mine, c, a, b) && ok;
+      const int e = e_lo + c * kStageElems + threadIdx.x * 8;
+#pragma unroll
+      for (int g = 0; g < U; ++g) {
+        if (c == stages - 1 && !(e + g * kGroupStep < e_hi)) continue;  // beyond the range
+        const float gmax = group_max<DT>(a[g], b[g]);
+        if (gmax < INFINITY) tmax = fmaxf(tmax, gmax);  // value only: which element it was does not matter for a bound
+      }
+    }
+    // candidates are the keys >= bound; a group is noted when its maximum reaches the bound's value
+    unsigned long long bound = (unsigned long long)bound_from_maxima(tmax > -INFINITY ? value_key(tmax) : 0u, k, sh.offer) << 32;
+    float bound_f = bound ? key_value(bound) : -INFINITY;
+    bool over = false;
+    // ---- the range
+    for (int c = 0; c < stages; ++c) {
+      ok = take_stage<DT, U>(full0, empty0, mine, head + c, a, b) && ok;
+      const int e = e_lo + c * kStageElems + threadIdx.x * 8;
+      const bool last = c == stages - 1;
+#pragma unroll
+      for (int g = 0; g < U; ++g) {
+        const bool valid = !last || e + g * kGroupStep < e_hi;
+        const float gmax = group_max<DT>(a[g], b[g]);
+        const bool finite = gmax < INFINITY;  // false for NaN too
+        if (__any_sync(0xffffffffu, valid && (!finite || gmax >= bound_f))) {  // rare for the warp as a whole
+          if (valid && !finite) {
+            sh.bad = 1;  // NaN or +inf somewhere in the eight: the slot will be frozen, the list does not matter
+          } else if (valid && gmax >= bound_f) {
+            const int pos = atomicAdd(&sh.gcount, 1);
+            if (pos < kGroupCap) sh.group[pos] = e + g * kGroupStep;
+          }
+        }
+      }
+      const bool head_end = c == head - 1;
+      if (!last && !head_end && (c & (kCheckEvery - 1)) != kCheckEvery - 1) continue;
+      // ---- a look at the queue
+      worker_sync();
+      const int groups = sh.gcount;
+      if (groups > kGroupCap) {  // too much between two looks: note nothing more, start over below
+        over = true;
+        bound_f = INFINITY;
+        continue;  // (the count stays above the capacity, so every later look ends here as well)
+      }
+      if (!last && !head_end && groups < kExpandAt) {
+        worker_sync();  // everybody has read the count before anybody adds to it
+        continue;
+      }
+      for (int i = threadIdx.x; i < groups; i += kThreads) {  // one group per thread, re-read from global memory
+        const int ge = sh.group[i];
+        float x[8];
+        load8<DT>(row, ge, x);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (x[j] > -INFINITY) {
+            const unsigned long long kk = cand_key(x[j], ge + j);
+            if (kk >= bound) {
+              const int pos = atomicAdd(&sh.count, 1);
+              if (pos < kCandCap) sh.key[pos] = kk;
+            }
+          }
+        }
+      }
+      worker_sync();
+      const int total = sh.count;
+      if (threadIdx.x == 0) sh.gcount = total > kCandCap ? kGroupCap + 1 : 0;  // overflow: as above
+      worker_sync();  // everybody has read the counts; the queue is empty again
+      if (total > kCandCap) {
+        over = true;
+        bound_f = INFINITY;
+        continue;
+      }
+      if (!last && !head_end && total < kCompactAt) continue;
+      int n;
+      if (total <= kThreads) {  // the usual case
+        n = rank_select(sh.key, total, k, sh.sorted);
+      } else {
+        sort_keys(sh.key, total);
+        n = total < k ? total : k;
+        if (threadIdx.x < n) sh.sorted[threadIdx.x] = sh.key[threadIdx.x];
+        worker_sync();
+      }
+      if (last) {
+        if (threadIdx.x < n) {
+          sh.list_val[threadIdx.x] = key_value(sh.sorted[threadIdx.x]);
+          sh.list_idx[threadIdx.x] = key_index(sh.sorted[threadIdx.x]);
+        }
+        if (threadIdx.x == 0) sh.list_n = n;
+      } else {
+        if (threadIdx.x < n) sh.key[threadIdx.x] = sh.sorted[threadIdx.x];
+        if (threadIdx.x == 0) sh.count = n;
+        if (n == k) {
+          bound = sh.sorted[k - 1];
+          bound_f = key_value(bound);
+        }
+        worker_sync();  // the cut-back buffer and its count are in place before the next look
+      }
+    }
+    if (over && threadIdx.x == 0) sh.over = 1;
+  }
+  __syncthreads();  // producer warp and workers meet
+  if (sh.over) return block_topk_two_stream<DT>(sh, row, e_lo, e_hi, k) && ok;
+  return ok;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Pass 1: the top-k list of every valid row
 // ------------------------------------------------------------------------------------------------
@@ -267,7 +470,7 @@ __global__ void __launch_bounds__(kThreads + 32) topk_rows_kernel(const TopkPara
   if (r >= nv + P.N) return;
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
-  if (!block_topk<DT>(sh, row, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  if (!block_topk<DT>(sh, row, 0, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
   const size_t base = ((size_t)b * P.Q + r) * kMaxTopK;
   if (threadIdx.x < sh.list_n) {
     P.list_val[base + threadIdx.x] = sh.list_val[threadIdx.x];
@@ -281,23 +484,33 @@ __global__ void __launch_bounds__(kThreads + 32) topk_rows_kernel(const TopkPara
 // ------------------------------------------------------------------------------------------------
 // Nucleus of a sorted top-k list in fp64, in the oracle's order of operations: w_i = exp(l_i invT - l_0 invT),
 // Z = sum w_i, support = shortest prefix whose cumulated w reaches top_p * Z.  Returns the support size and
-// the log-normaliser of the support.
-__device__ int nucleus(const float* val, int n, double inv_t, double top_p, double& lse) {
+// the log-normaliser of the support.  By one warp: the lanes compute the exponentials (w: n doubles of shared
+// memory), lane 0 adds them up in index order; every lane gets the result.
+__device__ int warp_nucleus(const float* val, int n, double inv_t, double top_p, double* w, double& lse) {
+  const int lane = threadIdx.x & 31;
   lse = -INFINITY;
   if (n <= 0) return 0;
   const double m = (double)val[0] * inv_t;
   if (isinf(m) && m < 0) return n;
-  double Z = 0.0;
-  for (int i = 0; i < n; ++i) Z += exp((double)val[i] * inv_t - m);
-  double cum = 0.0;
+  for (int i = lane; i < n; i += 32) w[i] = exp((double)val[i] * inv_t - m);
+  __syncwarp();
   int keep = n;
-  for (int i = 0; i < n; ++i) {
-    cum += exp((double)val[i] * inv_t - m);
-    if (cum >= top_p * Z) { keep = i + 1; break; }
+  double l = 0.0;
+  if (lane == 0) {
+    double Z = 0.0;
+    for (int i = 0; i < n; ++i) Z += w[i];
+    double cum = 0.0;
+    for (int i = 0; i < n; ++i) {
+      cum += w[i];
+      if (cum >= top_p * Z) { keep = i + 1; break; }
+    }
+    double S = 0.0;
+    for (int i = 0; i < keep; ++i) S += w[i];
+    l = m + log(S);
   }
-  double S = 0.0;
-  for (int i = 0; i < keep; ++i) S += exp((double)val[i] * inv_t - m);
-  lse = m + log(S);
+  keep = __shfl_sync(0xffffffffu, keep, 0);
+  lse = __shfl_sync(0xffffffffu, l, 0);
+  __syncwarp();
   return keep;
 }
 
@@ -323,6 +536,7 @@ __global__ void __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkPa
   TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
   __shared__ int s_n[32], s_bad[32], s_rej, s_a;
   __shared__ double s_lse[32];
+  __shared__ double s_w[kThreads / 32][kMaxTopK];
   const int b = blockIdx.x;
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
@@ -341,16 +555,15 @@ __global__ void __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkPa
   const float* LV = P.list_val + (size_t)b * P.Q * kMaxTopK;
   const int* LI = P.list_idx + (size_t)b * P.Q * kMaxTopK;
 
-  // ---- every row's support and log-normaliser (lane = row)
-  if (warp == 0) {
-    int n = 0, bad = 0;
-    double lse = -INFINITY;
-    if (lane < q_len) {
-      int ln = P.list_n[(size_t)b * P.Q + lane];
+  // ---- every row's support and log-normaliser (one warp per row, rows dealt round-robin)
+  if (warp < kThreads / 32) {
+    for (int rr = warp; rr < q_len; rr += kThreads / 32) {
+      int ln = P.list_n[(size_t)b * P.Q + rr], bad = 0;
       if (ln < 0) { bad = 1; ln = -1 - ln; }
-      n = nucleus(LV + (size_t)lane * kMaxTopK, ln, inv_t, top_p, lse);
+      double lse;
+      const int n = warp_nucleus(LV + (size_t)rr * kMaxTopK, ln, inv_t, top_p, s_w[warp], lse);
+      if (lane == 0) { s_n[rr] = n; s_bad[rr] = bad; s_lse[rr] = lse; }
     }
-    s_n[lane] = n; s_bad[lane] = bad; s_lse[lane] = lse;
   }
   __syncthreads();
 
@@ -475,11 +688,11 @@ __global__ void __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkPa
   if (P.q_mode == 0) {
     if (P.q_prev == nullptr) return;  // the caller gave no proposal-law rows
     const char* qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + (P.q_row0[b] + rej - 1)) * (size_t)P.V * elt;
-    if (!block_topk<DT>(sh, qrow, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
-    if (threadIdx.x == 0) {
+    if (!block_topk<DT>(sh, qrow, 0, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+    if (warp == 0) {
       double l;
-      s_n[31] = nucleus(sh.list_val, sh.list_n, inv_t, top_p, l);  // rows above 30 do not exist (Q <= 31)
-      s_lse[31] = l;
+      const int n = warp_nucleus(sh.list_val, sh.list_n, inv_t, top_p, s_w[0], l);
+      if (lane == 0) { s_n[31] = n; s_lse[31] = l; }  // rows above 30 do not exist (Q <= 31)
     }
     __syncthreads();
     nq = s_n[31];

@@ -87,3 +87,30 @@ def tiny_state(B, N, V, *, n_ver=0, ctx=32, pages_per_slot=8, seed=0):
         q_stats=np.zeros((B, NP, 2)), page_table=pt, free_stack=fs,
         free_top=np.array([nfree], np.int32), active=np.ones(B, np.uint8),
         slot_status=np.zeros(B, np.uint32), num_pages=num_pages)
+
+
+def compare_verify_and_state(w, t, out, st, vr, s, n_ver_before):
+    """Bit-exact comparison of the verification outputs and the committed state of every slot."""
+    N, Q = w.stride, w.Q
+    g = {k: v.cpu().numpy() for k, v in out.items()}
+    gst = {k: st[k].cpu().numpy() for k in STATE_KEYS}
+    for b in range(w.batch):
+        evaluated = vr.accept[b] >= 0
+        near = evaluated & (np.abs(vr.alpha[b] - vr.u[b]) < 1e-4)
+        assert not near.any(), "pick another seed: an acceptance test sits within 1e-4 of its uniform draw"
+        assert np.array_equal(g["accept"][b], vr.accept[b]), (t, b, g["accept"][b], vr.accept[b])
+        for name in ("accept_len", "n_emit", "repl_tok", "out_tok", "new_prop_tok"):
+            assert np.array_equal(g[name][b], getattr(vr, name)[b]), (t, b, name, g[name][b], getattr(vr, name)[b])
+        ev = np.where(evaluated)[0]
+        if len(ev):
+            assert np.abs(g["alpha"][b][ev] - vr.alpha[b][ev]).max() < 2e-2
+        if N > 1:
+            assert np.abs(g["new_q_stats"][b] - vr.new_q_stats[b]).max() < 2e-2
+        for name in ("ctx_len", "n_ver", "q_row0"):
+            assert gst[name][b] == s[name][b], (t, b, name)
+        assert np.array_equal(gst["block_tok"][b], s["block_tok"][b]), (t, b)
+        own = (int(s["ctx_len"][b]) + Q + 15) // 16
+        assert np.array_equal(gst["page_table"][b, :own], s["page_table"][b, :own]), (t, b)
+    top = int(s["free_top"][0])
+    assert gst["free_top"][0] == top and np.array_equal(gst["free_stack"][:top], s["free_stack"][:top])
+    assert np.array_equal(gst["slot_status"].view(np.uint32), s["slot_status"])

@@ -5,7 +5,7 @@ import torch
 
 import oracle
 import paper_2604_11035_b200 as isd_pkg
-from helpers import STATE_KEYS, bits16, logits_np, oracle_step, state_to_np
+from helpers import STATE_KEYS, bits16, compare_verify_and_state, logits_np, oracle_step, state_to_np
 from paper_2604_11035_b200 import workloads as wl
 from paper_2604_11035_b200.workloads import Workload
 from parity import run_chain_parity
@@ -64,6 +64,50 @@ def test_filtered_laws_full_vocab_and_batch():
     rep = run_chain_parity(w, steps=3, device=DEV, attn_slots=[0, 95])
     assert_clean(rep)
     assert rep["rejections"] > 0
+
+
+def _structured_logits(w, t, dtype):
+    """Rows that stress the top-k selection: monotone in the index, constant, long runs of equal values, the
+    best entries at the very end, almost everything masked out; slots 6 and 7 are ordinary random rows."""
+    V, Q = w.vocab, w.Q
+    g = torch.Generator(device="cpu")
+    g.manual_seed(1000 + t)
+    lg = torch.randn(w.batch, Q, V, generator=g) * 2.0
+    i = torch.arange(V, dtype=torch.float32)
+    shift = torch.arange(Q, dtype=torch.float32)[:, None]
+    lg[0] = i[None, :] * 2e-4 + 0.01 * shift                        # upwards: every element beats the ones before it
+    lg[1] = -i[None, :] * 2e-4 - 0.01 * shift                       # downwards
+    lg[2] = 0.25 + 0.0 * shift                                      # one value everywhere
+    lg[3] = torch.floor((i[None, :] + 37 * shift + 11 * t) / 3000.0) * 0.5   # runs of 3000 equal values, rising
+    lg[4, :, V - 200:] += 6.0                                       # the top of the row sits in its last stage
+    mask = torch.rand(Q, V, generator=g) < 0.9995
+    lg[5][mask] = float("-inf")                                     # fewer finite entries than top_k
+    return lg.to(dtype).to(DEV)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_filtered_selection_on_structured_rows(dtype):
+    # rows on which the single-stream selection has to give up and start over (upward rows, runs of equal values),
+    # next to rows it handles directly; every output and the committed state must equal the oracle's
+    steps = 3
+    w = Workload("structured", batch=8, stride=4, n_q_heads=8, n_kv_heads=2, vocab=40000 + 8 * 3, ctx_min=5,
+                 ctx_max=200, logits_dtype=dtype, steps=steps, propose_mode=0, seed=33, top_k=50, top_p=0.95)
+    oracle.set_threads(oracle.max_threads())
+    st, eng, out = _fresh(w)
+    s = state_to_np(st)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    prev = prev_np = None
+    for t in range(steps):
+        lg = _structured_logits(w, t, tdt)
+        q, k, v = wl.make_qkv(w, t, DEV)
+        n_ver_before = s["n_ver"].copy()
+        _step(w, st, eng, out, t, prev, logits=lg)
+        lg_np = logits_np(lg)
+        _, _, vr, _ = oracle_step(w, s, bits16(q), bits16(k), bits16(v), lg_np, prev_np, t)
+        compare_verify_and_state(w, t, out, st, vr, s, n_ver_before)
+        prev, prev_np = lg, lg_np
+    assert eng.isd_read_status() == 0
+    eng.close()
 
 
 def test_temperature_and_relaxed_acceptance():
