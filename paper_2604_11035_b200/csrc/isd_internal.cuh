@@ -69,6 +69,8 @@ struct isd_ctx {
   float* topk_val;       // [B, Q, ISD_MAX_TOP_K]
   int* topk_idx;         // [B, Q, ISD_MAX_TOP_K]
   int* topk_n;           // [B, Q]
+  unsigned long long* topk_q_key;  // [B, pieces, ISD_MAX_TOP_K] piece lists of a proposal-law row (as sort keys)
+  int* topk_q_n;         // [B, pieces], then [B, 2] (decision of a cluster's first CTA)
   // ---- optional device-resident step counter (CUDA-graph replay), owned by the caller
   uint32_t* step_counter;
   // ---- status

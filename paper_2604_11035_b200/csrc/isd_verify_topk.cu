@@ -5,23 +5,26 @@
 //
 // With at most ISD_MAX_TOP_K tokens of support per law, everything after the selection is tiny, and
 // no vocabulary-wide exponentials are needed at all:
-//   1. topk_rows_kernel    one CTA per (slot, block row): a streaming pass that selects the exact
-//      top-k of the row.  Candidates above a rising threshold go to a shared-memory buffer that is
-//      sorted and cut back to k whenever it has grown by a few hundred entries; the threshold is the
-//      k-th best so far.  Per logit: unpack, one 8-way maximum per thread, one compare.
-//   2. topk_decide_kernel  one CTA per slot: nucleus cut and log-normaliser of every row in fp64
-//      (the oracle's arithmetic, so the cut agrees), sequential accept test, and the Gumbel-max
-//      draws (residual, bonus, proposals) over the supports in fp64 with the same per-index Philox
-//      noise as the unfiltered path.  Only a rejection costs another stream: the proposal-law row
-//      of the previous step is selected again by the same routine.
+//   1. topk_rows_kernel    one CTA per (slot, block row): the exact top-k of the row in one stream of
+//      it (block_topk).  Per logit: a packed maximum over groups of eight and one compare against a
+//      rising bound; the few groups that reach it are re-read from L2 and ranked.
+//   2. topk_decide_kernel  one cluster of kQSplit CTAs per slot.  The first CTA: nucleus cut and
+//      log-normaliser of every row in fp64 (the oracle's arithmetic, so the cut agrees), sequential
+//      accept test, and the Gumbel-max draws (residual, bonus, proposals) over the supports in fp64
+//      with the same per-index Philox noise as the unfiltered path.  Only a rejection costs another
+//      stream: the proposal-law row of the previous step is selected again by the same routine, one
+//      piece of it per CTA of the cluster, and the first CTA merges the piece lists.
 #include "isd_internal.cuh"
 #include "isd_stream.cuh"
+
+#include <cooperative_groups.h>
 
 namespace {
 
 constexpr int kMaxTopK = ISD_MAX_TOP_K;
 constexpr int kCandCap = 1024;  // candidate keys in shared memory
 constexpr int kGroupCap = 512;  // queued groups in shared memory
+constexpr int kQSplit = 2;      // CTAs (one cluster) per slot in the decide kernel: pieces of a proposal-law row
 
 struct TopkParams {
   int B, N, Q, V;
@@ -42,6 +45,9 @@ struct TopkParams {
   float* list_val;  // [B, Q, kMaxTopK] raw logits of the row's top-k, best first
   int* list_idx;    // [B, Q, kMaxTopK]
   int* list_n;      // [B, Q] entries of the list; -1 - n when the row holds a NaN or +inf
+  unsigned long long* q_key;  // [B, kQSplit, kMaxTopK] piece lists of the proposal-law row of a rejection
+  int* q_n;                   // [B, kQSplit]
+  int* q_dec;                 // [B, 2] accept length and rejected position, from a cluster's first CTA to the others
 };
 
 struct TopkShared {
@@ -324,7 +330,8 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int e_lo, int e_hi, 
   constexpr int kGroupStep = kStageElems / U;
   const bool worker = threadIdx.x < kThreads;
   const int stages = (e_hi - e_lo + kStageElems - 1) / kStageElems;
-  const int head = stages < kHeadStages ? stages : kHeadStages;
+  // the head: kHeadStages stages of a long range, a quarter of a short one (it is read twice)
+  const int head = stages >= 4 * kHeadStages ? kHeadStages : stages >= 4 ? stages / 4 : stages > 0 ? 1 : 0;
   bool ok = true;
   if (threadIdx.x == 0) {
     for (int i = 0; i < kRowStages; ++i) {
@@ -494,23 +501,25 @@ __device__ int warp_nucleus(const float* val, int n, double inv_t, double top_p,
   if (isinf(m) && m < 0) return n;
   for (int i = lane; i < n; i += 32) w[i] = exp((double)val[i] * inv_t - m);
   __syncwarp();
-  int keep = n;
-  double l = 0.0;
+  // lane 0 adds in index order, once: w[i] becomes the sum of the first i + 1 (the oracle's three loops - the
+  // normaliser, the cumulated mass, the mass of the support - add the same numbers in the same order)
   if (lane == 0) {
-    double Z = 0.0;
-    for (int i = 0; i < n; ++i) Z += w[i];
     double cum = 0.0;
     for (int i = 0; i < n; ++i) {
       cum += w[i];
-      if (cum >= top_p * Z) { keep = i + 1; break; }
+      w[i] = cum;
     }
-    double S = 0.0;
-    for (int i = 0; i < keep; ++i) S += w[i];
-    l = m + log(S);
   }
-  keep = __shfl_sync(0xffffffffu, keep, 0);
-  lse = __shfl_sync(0xffffffffu, l, 0);
   __syncwarp();
+  const double Z = w[n - 1];
+  int keep = n;
+  for (int i0 = 0; i0 < n; i0 += 32) {
+    const unsigned hit = __ballot_sync(0xffffffffu, i0 + lane < n && w[i0 + lane] >= top_p * Z);
+    if (hit) { keep = i0 + __ffs(hit); break; }
+  }
+  const double l = m + log(w[keep - 1]);
+  lse = l;
+  __syncwarp();  // w may be reused
   return keep;
 }
 
@@ -531,17 +540,21 @@ __device__ __forceinline__ double gumbel_at(const TopkParams& P, uint32_t step, 
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkParams P) {
+__global__ void __cluster_dims__(kQSplit, 1, 1) __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkParams P) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
-  __shared__ int s_n[32], s_bad[32], s_rej, s_a;
+  __shared__ int s_n[32], s_bad[32], s_x[32], s_rej, s_a;
+  __shared__ float s_logp[32], s_logq[32];
   __shared__ double s_lse[32];
   __shared__ double s_w[kThreads / 32][kMaxTopK];
-  const int b = blockIdx.x;
+  // A cluster of kQSplit CTAs per slot.  All of them run the accept test (it is short); the first one writes the
+  // outputs and draws; the others only help when a rejection needs the proposal-law row, one piece of it each.
+  const int b = blockIdx.x / kQSplit, piece = blockIdx.x % kQSplit;
+  const bool lead = piece == 0;
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
   if (nv < 0 || nv > P.N - 1) {
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0 && lead) {
       atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
       atomicOr(P.global_status, ISD_ST_SLOT_CAPACITY);
     }
@@ -555,77 +568,99 @@ __global__ void __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkPa
   const float* LV = P.list_val + (size_t)b * P.Q * kMaxTopK;
   const int* LI = P.list_idx + (size_t)b * P.Q * kMaxTopK;
 
-  // ---- every row's support and log-normaliser (one warp per row, rows dealt round-robin)
-  if (warp < kThreads / 32) {
+  // ---- every row's support and log-normaliser (one warp per row, rows dealt round-robin); first CTA only
+  if (lead && warp < kThreads / 32) {
     for (int rr = warp; rr < q_len; rr += kThreads / 32) {
       int ln = P.list_n[(size_t)b * P.Q + rr], bad = 0;
       if (ln < 0) { bad = 1; ln = -1 - ln; }
       double lse;
       const int n = warp_nucleus(LV + (size_t)rr * kMaxTopK, ln, inv_t, top_p, s_w[warp], lse);
       if (lane == 0) { s_n[rr] = n; s_bad[rr] = bad; s_lse[rr] = lse; }
+      // the inputs of the accept test at position rr + 1, whose anchor law this row is: the proposal, log p~ of it
+      // (-inf unless it is in the support) and log q~ of it
+      const int j = rr + 1;
+      if (j <= nv) {
+        const int x = P.block_tok[(size_t)b * P.Q + j];
+        float logp = -INFINITY;
+        for (int i = lane; i < n; i += 32)
+          if (LI[(size_t)rr * kMaxTopK + i] == x) logp = LV[(size_t)rr * kMaxTopK + i] * P.inv_t - (float)lse;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) logp = fmaxf(logp, __shfl_xor_sync(0xffffffffu, logp, off));  // at most one lane found it
+        if (lane == 0) {
+          s_x[j] = x;
+          s_logp[j] = logp;
+          float logq = 0.f;
+          if (P.q_mode == 0) {
+            const float* qs = P.q_stats + ((size_t)b * NP + j - 1) * 2;
+            logq = qs[1] - qs[0];
+          }
+          s_logq[j] = logq;
+        }
+      }
     }
   }
   __syncthreads();
-
-  // ---- sequential accept test (Algorithm 1, introspection loop) on the filtered laws
-  if (threadIdx.x == 0) {
+  // ---- sequential accept test (Algorithm 1, introspection loop) on the filtered laws; first CTA only
+  if (lead && threadIdx.x == 0) {
     uint32_t status = 0;
     int a = nv, rej = 0;
     for (int m = 1; m <= NP; ++m) status |= s_bad[nv + m] ? ISD_ST_NONFINITE_LOGIT : 0u;
     for (int j = 1; j <= NP; ++j) {
-      P.out.accept[(size_t)b * NP + j - 1] = -1;
-      P.out.alpha[(size_t)b * NP + j - 1] = NAN;
+      if (lead) P.out.accept[(size_t)b * NP + j - 1] = -1;
+      if (lead) P.out.alpha[(size_t)b * NP + j - 1] = NAN;
     }
     for (int j = 1; j <= nv; ++j) {
-      const int x = P.block_tok[(size_t)b * P.Q + j];
+      const int x = s_x[j];
       if (x < 0 || x >= P.V) { status |= ISD_ST_BAD_TOKEN_ID; a = -1; break; }
       if (s_bad[j - 1]) status |= ISD_ST_NONFINITE_LOGIT;
-      // p~(x): zero unless x is in the support of the filtered anchor law
-      float logp = -INFINITY;
-      for (int i = 0; i < s_n[j - 1]; ++i)
-        if (LI[(size_t)(j - 1) * kMaxTopK + i] == x) logp = LV[(size_t)(j - 1) * kMaxTopK + i] * P.inv_t - (float)s_lse[j - 1];
-      float logq = 0.f;
-      if (P.q_mode == 0) {
-        const float* qs = P.q_stats + ((size_t)b * NP + j - 1) * 2;
-        logq = qs[1] - qs[0];
-      }
+      const float logp = s_logp[j], logq = s_logq[j];
       float al = (1.f + P.tau) * expf(logp - logq);
       al = fminf(al, 1.f);
       if (al != al) al = 0.f;
       const uint4 rnd = philox4x32_10(0u, step, (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)j, P.seed_lo, P.seed_hi);
       const float u = (float)(rnd.x >> 8) * 0x1p-24f;
-      P.out.alpha[(size_t)b * NP + j - 1] = al;
+      if (lead) P.out.alpha[(size_t)b * NP + j - 1] = al;
       if (u < al) {
-        P.out.accept[(size_t)b * NP + j - 1] = 1;
+        if (lead) P.out.accept[(size_t)b * NP + j - 1] = 1;
       } else {
-        P.out.accept[(size_t)b * NP + j - 1] = 0;
+        if (lead) P.out.accept[(size_t)b * NP + j - 1] = 0;
         a = j - 1;
         rej = j;
         break;
       }
     }
     if (a >= 0 && rej == 0 && s_bad[nv]) status |= ISD_ST_NONFINITE_LOGIT;
-    for (int j = 0; j < P.N; ++j) P.out.out_tok[(size_t)b * P.N + j] = -1;
-    P.out.repl_tok[b] = -1;
+    for (int j = 0; j < P.N; ++j) if (lead) P.out.out_tok[(size_t)b * P.N + j] = -1;
+    if (lead) P.out.repl_tok[b] = -1;
     if (a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL)) {
-      P.out.accept_len[b] = 0;
-      P.out.n_emit[b] = 0;
-      atomicOr(&P.slot_status[b], status);
-      atomicOr(P.global_status, status);
+      if (lead) P.out.accept_len[b] = 0;
+      if (lead) P.out.n_emit[b] = 0;
+      if (lead) atomicOr(&P.slot_status[b], status);
+      if (lead) atomicOr(P.global_status, status);
       a = -1;
     } else {
-      P.out.accept_len[b] = a;
-      P.out.n_emit[b] = a + 1;
-      for (int j = 1; j <= a; ++j) P.out.out_tok[(size_t)b * P.N + j - 1] = P.block_tok[(size_t)b * P.Q + j];
+      if (lead) P.out.accept_len[b] = a;
+      if (lead) P.out.n_emit[b] = a + 1;
+      for (int j = 1; j <= a; ++j) if (lead) P.out.out_tok[(size_t)b * P.N + j - 1] = P.block_tok[(size_t)b * P.Q + j];
     }
     s_a = a;
     s_rej = rej;
+    P.q_dec[2 * b] = a;  // for the other CTAs of the cluster
+    P.q_dec[2 * b + 1] = rej;
+    __threadfence();
+  }
+  cooperative_groups::this_cluster().sync();  // every CTA of an active slot's cluster passes here once
+  if (!lead && threadIdx.x == 0) {
+    s_a = P.q_dec[2 * b];
+    s_rej = P.q_dec[2 * b + 1];
   }
   __syncthreads();
   const int a = s_a, rej = s_rej;
+  // the helpers are needed only for the proposal-law row of a rejection (the same decision in all CTAs of the cluster)
+  if (!lead && (a < 0 || rej == 0 || P.q_mode != 0 || P.q_prev == nullptr)) return;
 
   // ---- proposals of the MASK rows: Gumbel-max over the support (warp m - 1 draws row nv + m), or its head
-  if (warp >= 1 && warp <= NP && warp < kThreads / 32) {
+  if (lead && warp >= 1 && warp <= NP && warp < kThreads / 32) {
     for (int m = warp; m <= NP; m += kThreads / 32 - 1) {
       const int rr = nv + m, n = s_n[rr];
       const float* v = LV + (size_t)rr * kMaxTopK;
@@ -688,7 +723,34 @@ __global__ void __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkPa
   if (P.q_mode == 0) {
     if (P.q_prev == nullptr) return;  // the caller gave no proposal-law rows
     const char* qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + (P.q_row0[b] + rej - 1)) * (size_t)P.V * elt;
-    if (!block_topk<DT>(sh, qrow, 0, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+    // every CTA of the cluster selects the top-k of its piece of the row (whole stages); their union holds the row's
+    const int stage_elems = kRowStageBytes / (int)elt;
+    const int per = ((P.V + stage_elems - 1) / stage_elems + kQSplit - 1) / kQSplit * stage_elems;
+    const int e_lo = piece * per < P.V ? piece * per : P.V;
+    const int e_hi = e_lo + per < P.V ? e_lo + per : P.V;
+    if (!block_topk<DT>(sh, qrow, e_lo, e_hi, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+    if (threadIdx.x < sh.list_n)
+      P.q_key[((size_t)b * kQSplit + piece) * kMaxTopK + threadIdx.x] = cand_key(sh.list_val[threadIdx.x], sh.list_idx[threadIdx.x]);
+    if (threadIdx.x == 0) P.q_n[(size_t)b * kQSplit + piece] = sh.list_n;
+    __threadfence();
+    cooperative_groups::this_cluster().sync();  // every CTA of the cluster is here: the early returns above are the same for all
+    if (!lead) return;
+    if (threadIdx.x < kThreads) {
+      int total = 0;
+      for (int r = 0; r < kQSplit; ++r) {
+        const int n_r = P.q_n[(size_t)b * kQSplit + r];
+        if (threadIdx.x < n_r) sh.key[total + threadIdx.x] = P.q_key[((size_t)b * kQSplit + r) * kMaxTopK + threadIdx.x];
+        total += n_r;
+      }
+      worker_sync();
+      const int n = rank_select(sh.key, total, P.top_k, sh.sorted);  // total <= kQSplit * kMaxTopK = kThreads
+      if (threadIdx.x < n) {
+        sh.list_val[threadIdx.x] = key_value(sh.sorted[threadIdx.x]);
+        sh.list_idx[threadIdx.x] = key_index(sh.sorted[threadIdx.x]);
+      }
+      if (threadIdx.x == 0) sh.list_n = n;
+    }
+    __syncthreads();
     if (warp == 0) {
       double l;
       const int n = warp_nucleus(sh.list_val, sh.list_n, inv_t, top_p, s_w[0], l);
@@ -739,6 +801,7 @@ __global__ void __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkPa
 }
 
 constexpr size_t kTopkSmem = sizeof(TopkShared);
+static_assert(kQSplit * kMaxTopK <= kThreads, "the merge of the piece lists ranks one key per thread");
 
 }  // namespace
 
@@ -749,6 +812,9 @@ int isd_verify_topk_create(isd_ctx* ctx) {
   if (cudaMalloc(&ctx->topk_idx, sizeof(int) * rows * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
   if (cudaMalloc(&ctx->topk_n, sizeof(int) * rows) != cudaSuccess) return ISD_ERR_NO_MEMORY;
   cudaMemset(ctx->topk_n, 0, sizeof(int) * rows);
+  if (cudaMalloc(&ctx->topk_q_key, sizeof(unsigned long long) * (size_t)c.batch * kQSplit * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  if (cudaMalloc(&ctx->topk_q_n, sizeof(int) * (size_t)c.batch * (kQSplit + 2)) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  cudaMemset(ctx->topk_q_n, 0, sizeof(int) * (size_t)c.batch * (kQSplit + 2));
   cudaError_t e = cudaSuccess;
   if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_rows_kernel<ISD_LOGITS_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_rows_kernel<ISD_LOGITS_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmem);
@@ -761,9 +827,13 @@ void isd_verify_topk_destroy(isd_ctx* ctx) {
   cudaFree(ctx->topk_val);
   cudaFree(ctx->topk_idx);
   cudaFree(ctx->topk_n);
+  cudaFree(ctx->topk_q_key);
+  cudaFree(ctx->topk_q_n);
   ctx->topk_val = nullptr;
   ctx->topk_idx = nullptr;
   ctx->topk_n = nullptr;
+  ctx->topk_q_key = nullptr;
+  ctx->topk_q_n = nullptr;
 }
 
 int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
@@ -780,14 +850,15 @@ int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* 
   P.q_stats = st->q_stats; P.slot_status = st->slot_status; P.global_status = ctx->global_status;
   P.logits_cur = logits_cur; P.q_prev = q_prev_logits; P.out = *out;
   P.list_val = ctx->topk_val; P.list_idx = ctx->topk_idx; P.list_n = ctx->topk_n;
+  P.q_key = ctx->topk_q_key; P.q_n = ctx->topk_q_n; P.q_dec = ctx->topk_q_n + (size_t)c.batch * kQSplit;
   const dim3 grid1(c.batch, ctx->Q);
   if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
   if (c.logits_dtype == ISD_LOGITS_BF16) {
     topk_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads + 32, kTopkSmem, stream>>>(P);
-    topk_decide_kernel<ISD_LOGITS_BF16><<<c.batch, kThreads + 32, kTopkSmem, stream>>>(P);
+    topk_decide_kernel<ISD_LOGITS_BF16><<<c.batch * kQSplit, kThreads + 32, kTopkSmem, stream>>>(P);
   } else {
     topk_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads + 32, kTopkSmem, stream>>>(P);
-    topk_decide_kernel<ISD_LOGITS_F32><<<c.batch, kThreads + 32, kTopkSmem, stream>>>(P);
+    topk_decide_kernel<ISD_LOGITS_F32><<<c.batch * kQSplit, kThreads + 32, kTopkSmem, stream>>>(P);
   }
   if (ctx->ev_verify1) cudaEventRecord(ctx->ev_verify1, stream);
   ctx->launches += 2;
