@@ -109,6 +109,7 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
     cudaMemset(ctx->global_status, 0, sizeof(uint32_t));
   }
   if (rc == ISD_OK && c.top_k > 0) rc = isd_verify_topk_create(ctx);
+  if (rc == ISD_OK) rc = isd_lora_create(ctx);
   if (rc == ISD_OK && c.attn_impl == 0) rc = isd_attn_tc_create(ctx);
   if (rc == ISD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ISD_ERR_CUDA;
   if (rc != ISD_OK) {
@@ -124,6 +125,7 @@ int isd_destroy(isd_ctx* ctx) {
   cudaDeviceSynchronize();
   isd_attn_tc_destroy(ctx);
   isd_verify_topk_destroy(ctx);
+  isd_lora_destroy(ctx);
   cudaFree(ctx->row_part);
   cudaFree(ctx->samp_part);
   cudaFree(ctx->row_ticket);

@@ -71,6 +71,8 @@ struct isd_ctx {
   int* topk_n;           // [B, Q]
   unsigned long long* topk_q_key;  // [B, pieces, ISD_MAX_TOP_K] piece lists of a proposal-law row (as sort keys)
   int* topk_q_n;         // [B, pieces], then [B, 2] (decision of a cluster's first CTA)
+  // ---- isd_lora_linear: readiness flags of the row blocks of t, then one counter (all zero between launches)
+  uint32_t* lora_flags;
   // ---- optional device-resident step counter (CUDA-graph replay), owned by the caller
   uint32_t* step_counter;
   // ---- status
@@ -273,6 +275,8 @@ int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* 
                            const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
                            cudaStream_t stream);
 int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t stream);
+int isd_lora_create(isd_ctx* ctx);
+void isd_lora_destroy(isd_ctx* ctx);
 int isd_launch_commit(isd_ctx* ctx, isd_batch_state* st, const isd_verify_out* out, cudaStream_t stream);
 int isd_launch_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t n,
                        cudaStream_t stream);

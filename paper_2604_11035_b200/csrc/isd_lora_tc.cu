@@ -1,11 +1,14 @@
 // isd_lora_linear: segment-gated LoRA linear layer of the lossless R-ISD variant (Sec. 3.2, the R-ISD
 // paragraph and Eq. 5): y_j = W x_j + 1[j in MASK] * s * B A x_j over the M = B * Q token rows of a step.
 //
-// Two launches of one tcgen05 GEMM kernel (C = A1 B1^T (+ A2 B2^T), bf16 operands, fp32 accumulation in
-// tensor memory):
-//   1. t = gate * s * (x A^T)            [M, R]  the gated, scaled down-projection (bf16)
-//   2. y = x W^T + t B^T                 [M, N]  one GEMM over the two K segments (K, then R)
+// One tcgen05 GEMM kernel (C = A1 B1^T (+ A2 B2^T), bf16 operands, fp32 accumulation in tensor memory) computes
+//   t = gate * s * (x A^T)            [M, R]  the gated, scaled down-projection (bf16), and
+//   y = x W^T + t B^T                 [M, N]  one GEMM over the two K segments (K, then R)
 // so the gate costs nothing in the large GEMM and clean rows provably see the base weights only (their t is 0).
+// In one launch when rank <= 256: the last ceil(M / 128) CTAs first compute one 128-row block of t each and
+// publish it (release store of a flag after a proxy fence: t is read back by TMA); the producer of an output
+// tile waits (bounded) for the flag of its row block before it loads the second K segment, which comes last.
+// The last CTA to finish clears the flags.  Otherwise two launches of the same kernel, t first.
 //
 // Kernel: persistent CTAs, one 128 x BN output tile at a time.  Warp 4 streams the operands with TMA
 // (2-D maps, 64-element K slices = 128-byte rows, SWIZZLE_128B, no multicast) into a 4-stage ring; warp 5
@@ -112,7 +115,26 @@ struct GemmParams {
   const uint8_t* gate;        // [M] or nullptr: rows with gate 0 are written as zeros
   float scale;
   uint32_t* global_status;
+  // fused down-projection (fuse != 0): the last tiles_m CTAs first compute one 128-row block each of
+  // t[M, R] = t_gate * t_scale * (A1 Bt^T), Bt[R, K1], and publish it; the second K segment of C (A2 = t) waits for it
+  int fuse, R;
+  __nv_bfloat16* t;
+  const uint8_t* t_gate;
+  float t_scale;
+  uint32_t* flags;            // [tiles_m] 1 = that block of t is written (all zero between launches)
+  uint32_t* done;             // [1] CTAs that have finished (zero between launches)
 };
+
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// orders accesses through the generic proxy (ordinary loads and stores) with those of the async proxy (TMA)
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 enum { BAR_FULL = 0, BAR_EMPTY = kStages, BAR_ACC_FULL = 2 * kStages, BAR_ACC_FREE = 2 * kStages + 2,
        BAR_COUNT = 2 * kStages + 4 };
@@ -120,7 +142,8 @@ enum { BAR_FULL = 0, BAR_EMPTY = kStages, BAR_ACC_FULL = 2 * kStages, BAR_ACC_FR
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_b1,
-               const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b2) {
+               const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b2,
+               const __grid_constant__ CUtensorMap map_bt) {
   constexpr int kStageA = kBM * kBK * 2, kStageB = BN * kBK * 2, kStageBytes = kStageA + kStageB;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sm_base = smem_u32(smem);
@@ -151,24 +174,45 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
   const int tiles_m = (P.M + kBM - 1) / kBM, tiles_n = (P.N + BN - 1) / BN;
   const int n_tiles = tiles_m * tiles_n;
   const int ks1 = P.K1 / kBK, ks2 = P.K2 / kBK, ks = ks1 + ks2;  // K slices per tile
+  // Work items of this CTA: with the fused down-projection, the last tiles_m CTAs (the ones with the fewest
+  // output tiles) start with one block of t; then the output tiles blockIdx.x, blockIdx.x + grid, ...
+  const int t_block = P.fuse ? (int)blockIdx.x - ((int)gridDim.x - tiles_m) : -1;  // >= 0: this CTA computes that block of t
+  const int n_pre = t_block >= 0 ? 1 : 0;
+  const int n_main = (int)blockIdx.x < n_tiles ? (n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  const int n_items = n_pre + n_main;
+  auto item_tile = [&](int it) { return (int)blockIdx.x + (it - n_pre) * (int)gridDim.x; };
 
   if (warp == 4) {
     // ============================================================================ TMA producer
     uint32_t fill = 0;
-    for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
-      const int m0 = (tile % tiles_m) * kBM, n0 = (tile / tiles_m) * BN;  // neighbouring CTAs share a B panel
+    for (int it = 0; it < n_items && !*abort_flag; ++it) {
+      const bool pre = it < n_pre;
+      const int tile = pre ? 0 : item_tile(it);
+      const int m0 = pre ? t_block * kBM : (tile % tiles_m) * kBM;  // neighbouring CTAs share a B panel
+      const int n0 = pre ? 0 : (tile / tiles_m) * BN;
+      const int n_slices = pre ? ks1 : ks;
+      const uint32_t bytes = pre ? (uint32_t)(kStageA + P.R * kBK * 2) : (uint32_t)kStageBytes;
       bool ok = true;
-      for (int i = 0; i < ks && ok; ++i, ++fill) {
+      for (int i = 0; i < n_slices && ok; ++i, ++fill) {
         const uint32_t s = fill % kStages, ph = (fill / kStages) & 1u;
         ok = mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag);
         if (!ok) break;
+        const bool seg2 = !pre && i >= ks1;
+        if (P.fuse && seg2 && i == ks1) {
+          // the second segment reads t: wait until this row block of it has been published
+          uint32_t spins = 0;
+          while (ld_acquire(P.flags + m0 / kBM) == 0u) {
+            if (++spins >= kSpinLimit || ((spins & 1023u) == 0u && *abort_flag)) { *abort_flag = 1; ok = false; break; }
+          }
+          if (!ok) break;
+          fence_proxy_async();
+        }
         if (elect_one()) {
-          mbar_arrive_expect_tx(bar(BAR_FULL + s), (uint32_t)kStageBytes);  // out-of-range rows are zero-filled, still counted
+          mbar_arrive_expect_tx(bar(BAR_FULL + s), bytes);  // out-of-range rows are zero-filled, still counted
           const uint32_t dst = sm_base + s * kStageBytes;
-          const bool seg2 = i >= ks1;
           const int k0 = (seg2 ? i - ks1 : i) * kBK;
           tma_load_2d(dst, seg2 ? &map_a2 : &map_a1, k0, m0, bar(BAR_FULL + s));
-          tma_load_2d(dst + kStageA, seg2 ? &map_b2 : &map_b1, k0, n0, bar(BAR_FULL + s));
+          tma_load_2d(dst + kStageA, pre ? &map_bt : (seg2 ? &map_b2 : &map_b1), k0, n0, bar(BAR_FULL + s));
         }
         __syncwarp();
       }
@@ -181,14 +225,17 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
   } else if (warp == 5) {
     // ============================================================================ MMA issuer
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+    const uint32_t idesc_t = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.R >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
     uint32_t cons = 0, t_local = 0;
-    for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x, ++t_local) {
+    for (int it = 0; it < n_items && !*abort_flag; ++it, ++t_local) {
+      const bool pre = it < n_pre;
+      const int n_slices = pre ? ks1 : ks;
       const uint32_t acc = t_local & 1u;
       // the epilogue warps must have read this accumulator's previous tile
       if (t_local >= 2 && !mbar_wait(bar(BAR_ACC_FREE + acc), ((t_local >> 1) - 1u) & 1u, abort_flag)) break;
       tc_fence_after();
       bool ok = true;
-      for (int i = 0; i < ks && ok; ++i, ++cons) {
+      for (int i = 0; i < n_slices && ok; ++i, ++cons) {
         const uint32_t s = cons % kStages, ph = (cons / kStages) & 1u;
         ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag);
         if (!ok) break;
@@ -197,10 +244,10 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
           const uint32_t a0 = sm_base + s * kStageBytes, b0 = a0 + kStageA;
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k)
-            tc_mma(tmem + acc * (uint32_t)BN, smem_desc_kmajor(a0 + k * 32), smem_desc_kmajor(b0 + k * 32), idesc,
-                   (i > 0 || k > 0) ? 1u : 0u);
+            tc_mma(tmem + acc * (uint32_t)BN, smem_desc_kmajor(a0 + k * 32), smem_desc_kmajor(b0 + k * 32),
+                   pre ? idesc_t : idesc, (i > 0 || k > 0) ? 1u : 0u);
           tc_commit(bar(BAR_EMPTY + s));
-          if (i == ks - 1) tc_commit(bar(BAR_ACC_FULL + acc));
+          if (i == n_slices - 1) tc_commit(bar(BAR_ACC_FULL + acc));
         }
         __syncwarp();
       }
@@ -210,21 +257,27 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
     // ============================================================================ epilogue (warps 0-3)
     uint32_t t_local = 0;
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-    for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x, ++t_local) {
-      const int m0 = (tile % tiles_m) * kBM, n0 = (tile / tiles_m) * BN;
+    for (int it = 0; it < n_items && !*abort_flag; ++it, ++t_local) {
+      const bool pre = it < n_pre;
+      const int tile = pre ? 0 : item_tile(it);
+      const int m0 = pre ? t_block * kBM : (tile % tiles_m) * kBM;
+      const int n0 = pre ? 0 : (tile / tiles_m) * BN;
+      const int n_cols = pre ? P.R : BN, ld_c = pre ? P.R : P.N, n_lim = pre ? P.R : P.N;
+      __nv_bfloat16* c = pre ? P.t : P.c;
+      const uint8_t* gate = pre ? P.t_gate : P.gate;
       const uint32_t acc = t_local & 1u;
       if (!mbar_wait(bar(BAR_ACC_FULL + acc), (t_local >> 1) & 1u, abort_flag)) break;
       tc_fence_after();
       const int row = m0 + warp * 32 + lane;
       const bool row_ok = row < P.M;
-      const float f = (P.gate == nullptr || (row_ok && P.gate[row])) ? P.scale : 0.f;
+      const float f = (gate == nullptr || (row_ok && gate[row])) ? (pre ? P.t_scale : P.scale) : 0.f;
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = 0; c0 < n_cols; c0 += 32) {
         uint32_t v[32];
         TMEM_LD32(tmem + lane_base + acc * (uint32_t)BN + (uint32_t)c0, v);
         tmem_wait_ld();
-        if (row_ok && n0 + c0 < P.N) {  // N is a multiple of 32 here (checked by the launcher)
-          uint4* dst = reinterpret_cast<uint4*>(P.c + (size_t)row * P.N + n0 + c0);
+        if (row_ok && n0 + c0 < n_lim) {  // the column counts are multiples of 32 here (checked by the launcher)
+          uint4* dst = reinterpret_cast<uint4*>(c + (size_t)row * ld_c + n0 + c0);
 #pragma unroll
           for (int q = 0; q < 4; ++q)
             dst[q] = make_uint4(pack_bf16(__uint_as_float(v[8 * q]) * f, __uint_as_float(v[8 * q + 1]) * f),
@@ -236,12 +289,26 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_ACC_FREE + acc));
+      if (pre) {
+        // publish the block of t: every epilogue thread's stores, made visible to the TMA reads of other CTAs
+        fence_proxy_async();
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (threadIdx.x == 0) st_release(P.flags + t_block, 1u);
+      }
     }
   }
   // ---- teardown
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  if (P.fuse && threadIdx.x == 0) {  // the CTA that finishes last leaves the flags as it found them
+    __threadfence();
+    if (atomicAdd(P.done, 1u) == gridDim.x - 1) {
+      for (int m = 0; m < tiles_m; ++m) P.flags[m] = 0u;
+      *P.done = 0u;
+    }
+  }
   if (warp == 4) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
@@ -277,9 +344,11 @@ int encode_matrix(CUtensorMap* map, const void* base, int rows, int cols, int bo
   return r == CUDA_SUCCESS ? ISD_OK : ISD_ERR_CUDA;
 }
 
+constexpr int kMaxFlags = 4096;  // row blocks of t that the fused kernel can track
+
 template <int BN>
-int launch_gemm(isd_ctx* ctx, const GemmParams& P, const void* a1, const void* b1, const void* a2, const void* b2,
-                cudaStream_t stream) {
+int launch_gemm(isd_ctx* ctx, GemmParams P, const void* a1, const void* b1, const void* a2, const void* b2,
+                const void* bt, cudaStream_t stream) {
   constexpr int kSmem = kStages * (kBM * kBK * 2 + BN * kBK * 2) + BAR_COUNT * 8 + 64;
   static bool attr_set = false;
   if (!attr_set) {
@@ -287,36 +356,58 @@ int launch_gemm(isd_ctx* ctx, const GemmParams& P, const void* a1, const void* b
       return ISD_ERR_CUDA;
     attr_set = true;
   }
-  CUtensorMap ma1, mb1, ma2, mb2;
+  CUtensorMap ma1, mb1, ma2, mb2, mbt;
   int rc = encode_matrix(&ma1, a1, P.M, P.K1, kBM);
   if (rc == ISD_OK) rc = encode_matrix(&mb1, b1, P.N, P.K1, BN);
   if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&ma2, a2, P.M, P.K2, kBM) : encode_matrix(&ma2, a1, P.M, P.K1, kBM);
   if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&mb2, b2, P.N, P.K2, BN) : encode_matrix(&mb2, b1, P.N, P.K1, BN);
+  if (rc == ISD_OK) rc = P.fuse ? encode_matrix(&mbt, bt, P.R, P.K1, P.R) : encode_matrix(&mbt, b1, P.N, P.K1, BN);
   if (rc != ISD_OK) return rc;
-  const int tiles = ((P.M + kBM - 1) / kBM) * ((P.N + BN - 1) / BN);
+  const int tiles_m = (P.M + kBM - 1) / kBM;
+  int tiles = tiles_m * ((P.N + BN - 1) / BN);
+  if (P.fuse && tiles < tiles_m) tiles = tiles_m;  // every block of t needs a CTA
   const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
-  gemm_tc_kernel<BN><<<grid, kThreads, kSmem, stream>>>(P, ma1, mb1, ma2, mb2);
+  gemm_tc_kernel<BN><<<grid, kThreads, kSmem, stream>>>(P, ma1, mb1, ma2, mb2, mbt);
   ctx->launches++;
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }
 
 }  // namespace
 
+int isd_lora_create(isd_ctx* ctx) {
+  if (cudaMalloc(&ctx->lora_flags, sizeof(uint32_t) * (kMaxFlags + 1)) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  return cudaMemset(ctx->lora_flags, 0, sizeof(uint32_t) * (kMaxFlags + 1)) == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}
+
+void isd_lora_destroy(isd_ctx* ctx) {
+  cudaFree(ctx->lora_flags);
+  ctx->lora_flags = nullptr;
+}
+
+#ifndef ISD_LORA_BN
+#define ISD_LORA_BN 256
+#endif
+
 int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t stream) {
-  // 1. t = gate * scale * (x A^T): N = rank, one K segment
-  GemmParams P1;
-  P1.M = a->m; P1.N = a->rank; P1.K1 = a->k; P1.K2 = 0;
-  P1.c = reinterpret_cast<__nv_bfloat16*>(a->t); P1.gate = a->gate; P1.scale = a->scale;
-  P1.global_status = ctx->global_status;
-  int rc = launch_gemm<128>(ctx, P1, a->x, a->a, nullptr, nullptr, stream);
-  if (rc != ISD_OK) return rc;
-  // 2. y = x W^T + t B^T: two K segments, no gate (it is already in t)
+  const int tiles_m = (a->m + kBM - 1) / kBM;
   GemmParams P2;
   P2.M = a->m; P2.N = a->n; P2.K1 = a->k; P2.K2 = a->rank;
   P2.c = reinterpret_cast<__nv_bfloat16*>(a->y); P2.gate = nullptr; P2.scale = 1.f;
   P2.global_status = ctx->global_status;
-#ifndef ISD_LORA_BN
-#define ISD_LORA_BN 256
-#endif
-  return launch_gemm<ISD_LORA_BN>(ctx, P2, a->x, a->w, a->t, a->b, stream);
+  P2.fuse = 0; P2.R = a->rank; P2.t = reinterpret_cast<__nv_bfloat16*>(a->t); P2.t_gate = a->gate; P2.t_scale = a->scale;
+  P2.flags = ctx->lora_flags; P2.done = ctx->lora_flags + kMaxFlags;
+  // One launch when a block of t fits one MMA (rank <= the tile width) and every block gets its own CTA: the
+  // last tiles_m CTAs compute t = gate * scale * (x A^T) block by block before their output tiles, and the second
+  // K segment of y = x W^T + t B^T waits for the block it reads.
+  if (a->rank <= ISD_LORA_BN && tiles_m <= ctx->num_sms && tiles_m <= kMaxFlags) {
+    P2.fuse = 1;
+    return launch_gemm<ISD_LORA_BN>(ctx, P2, a->x, a->w, a->t, a->b, a->a, stream);
+  }
+  // Otherwise two launches.  1. t = gate * scale * (x A^T): N = rank, one K segment
+  GemmParams P1 = P2;
+  P1.N = a->rank; P1.K2 = 0; P1.c = reinterpret_cast<__nv_bfloat16*>(a->t); P1.gate = a->gate; P1.scale = a->scale;
+  int rc = launch_gemm<128>(ctx, P1, a->x, a->a, nullptr, nullptr, nullptr, stream);
+  if (rc != ISD_OK) return rc;
+  // 2. y = x W^T + t B^T: two K segments, no gate (it is already in t)
+  return launch_gemm<ISD_LORA_BN>(ctx, P2, a->x, a->w, a->t, a->b, nullptr, stream);
 }

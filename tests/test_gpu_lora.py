@@ -74,3 +74,26 @@ def test_model_sized_layer_sampled_rows():
     assert (err <= tol).all(), float(err.max())
     assert eng.isd_read_status() == 0
     eng.close()
+
+
+def test_repeated_calls_reuse_the_scratch_and_big_ranks_take_two_launches():
+    # The one-launch form hands t from CTA to CTA through readiness flags that every launch must leave cleared:
+    # with a stale flag the second K segment would read the previous call's t.  Same buffers, the gate flipped
+    # between calls; every call is checked in full.  Rank 320 exceeds one MMA's width: two launches.
+    eng = _engine()
+    for (M, N, K, R), launches in (((300, 288, 256, 128), 1), ((260, 160, 128, 320), 2)):
+        x, w, a, b, gate = _inputs(M, N, K, R, seed=3 * M + R)
+        t = torch.empty(M, R, dtype=torch.bfloat16, device=DEV)
+        y = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+        for call in range(3):
+            g = gate if call % 2 == 0 else 1 - gate
+            n0 = eng.isd_launch_count()
+            eng.isd_lora_linear(x, w, a, b, g, 1.25, t=t, y=y)
+            torch.cuda.synchronize()
+            assert eng.isd_launch_count() - n0 == launches
+            ref = oracle.lora_linear(_f64(x), _f64(w), _f64(a), _f64(b), g.cpu().numpy(), 1.25)
+            tol = _tolerance(ref, _f64(x), _f64(a), _f64(b), g.cpu().numpy(), 1.25)
+            err = np.abs(_f64(y) - ref)
+            assert (err <= tol).all(), (M, R, call, float(err.max()))
+    assert eng.isd_read_status() == 0
+    eng.close()
