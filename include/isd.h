@@ -267,8 +267,8 @@ typedef struct isd_lora_args {
  * only [MASK] rows see the adapter.  bf16 operands, fp32 accumulation on the tensor cores, bf16
  * results; the intermediate t = gate * scale * (x a^T) is rounded to bf16 once.  Requirements
  * (else ISD_ERR_UNSUPPORTED / ISD_ERR_ALIGNMENT): k and rank multiples of 64, n a multiple of 32,
- * 16-byte aligned pointers.  One kernel on `cuda_stream` (two when rank > 256 or m > 128 x the number
- * of SMs), no allocation, no synchronisation.
+ * 16-byte aligned pointers.  One kernel on `cuda_stream` (two when rank > 256 is not a multiple of
+ * 256, or when t has more 128 x 256 blocks than the GPU has SMs), no allocation, no synchronisation.
  */
 int isd_lora_linear(isd_ctx* ctx, const isd_lora_args* args, void* cuda_stream);
 

@@ -4,8 +4,8 @@
 //
 //   * GQA packing: the G = Hq/Hkv query heads that share a KV head and the q_len block rows form one
 //     M = 128 row tile (row m = r * G + head-in-group), so each KV byte is read once per step.
-//   * KV pages (16 tokens x 128 dims, 4 KiB per head) are staged by TMA (cp.async.bulk.tensor, no
-//     multicast) into a 6-deep shared-memory ring in the 128-byte-swizzled layout tcgen05 consumes;
+//   * KV pages (16 tokens x 128 dims, 4 KiB per head) are staged by TMA (cp.async.bulk.tensor, every
+//     CTA loads for itself) into a 6-deep shared-memory ring in the 128-byte-swizzled layout tcgen05 consumes;
 //     one 128-key tile = 8 pages.
 //   * S = Q K^T and O += P V run on the 5th-gen tensor cores (tcgen05.mma, cta_group::1, M=128,
 //     N=128, K=16, bf16 -> fp32) with accumulators in TMEM; S is double-buffered so that the

@@ -5,13 +5,14 @@
 //   t = gate * s * (x A^T)            [M, R]  the gated, scaled down-projection (bf16), and
 //   y = x W^T + t B^T                 [M, N]  one GEMM over the two K segments (K, then R)
 // so the gate costs nothing in the large GEMM and clean rows provably see the base weights only (their t is 0).
-// In one launch when rank <= 256: the last ceil(M / 128) CTAs first compute one 128-row block of t each and
-// publish it (release store of a flag after a proxy fence: t is read back by TMA); the producer of an output
-// tile waits (bounded) for the flag of its row block before it loads the second K segment, which comes last.
+// In one launch when rank <= 256 or a multiple of 256: the last CTAs first compute one 128-row x (<= 256)-column
+// block of t each and publish it (a counter per row block, raised after a proxy fence: t is read back by TMA);
+// the producer of an output tile waits (bounded) until the counter of its row block is complete before it loads
+// the second K segment, which comes last.
 // The last CTA to finish clears the flags.  Otherwise two launches of the same kernel, t first.
 //
 // Kernel: persistent CTAs, one 128 x BN output tile at a time.  Warp 4 streams the operands with TMA
-// (2-D maps, 64-element K slices = 128-byte rows, SWIZZLE_128B, no multicast) into a 4-stage ring; warp 5
+// (2-D maps, 64-element K slices = 128-byte rows, SWIZZLE_128B, every CTA loads for itself) into a 4-stage ring; warp 5
 // issues tcgen05.mma (M = 128, N = BN, K = 16, both operands from shared memory) into one of two TMEM
 // accumulators; warps 0-3 read the other accumulator back (tcgen05.ld, one lane = one row), apply gate and
 // scale, and store bf16, so the epilogue of a tile overlaps the main loop of the next.  Every mbarrier wait is
@@ -115,13 +116,14 @@ struct GemmParams {
   const uint8_t* gate;        // [M] or nullptr: rows with gate 0 are written as zeros
   float scale;
   uint32_t* global_status;
-  // fused down-projection (fuse != 0): the last tiles_m CTAs first compute one 128-row block each of
-  // t[M, R] = t_gate * t_scale * (A1 Bt^T), Bt[R, K1], and publish it; the second K segment of C (A2 = t) waits for it
-  int fuse, R;
+  // fused down-projection (fuse != 0): the last tiles_m * t_chunks CTAs first compute one 128-row x Rc-column
+  // block each of t[M, R] = t_gate * t_scale * (A1 Bt^T), Bt[R, K1], and publish it; the second K segment of C
+  // (A2 = t) waits until all t_chunks blocks of its rows are there
+  int fuse, R, Rc, t_chunks;  // Rc = columns of a block of t (R = t_chunks * Rc)
   __nv_bfloat16* t;
   const uint8_t* t_gate;
   float t_scale;
-  uint32_t* flags;            // [tiles_m] 1 = that block of t is written (all zero between launches)
+  uint32_t* flags;            // [tiles_m] blocks of t written for that row block (all zero between launches)
   uint32_t* done;             // [1] CTAs that have finished (zero between launches)
 };
 
@@ -129,9 +131,6 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
   uint32_t v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
-}
-__device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
-  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 // orders accesses through the generic proxy (ordinary loads and stores) with those of the async proxy (TMA)
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
@@ -174,10 +173,11 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
   const int tiles_m = (P.M + kBM - 1) / kBM, tiles_n = (P.N + BN - 1) / BN;
   const int n_tiles = tiles_m * tiles_n;
   const int ks1 = P.K1 / kBK, ks2 = P.K2 / kBK, ks = ks1 + ks2;  // K slices per tile
-  // Work items of this CTA: with the fused down-projection, the last tiles_m CTAs (the ones with the fewest
-  // output tiles) start with one block of t; then the output tiles blockIdx.x, blockIdx.x + grid, ...
-  const int t_block = P.fuse ? (int)blockIdx.x - ((int)gridDim.x - tiles_m) : -1;  // >= 0: this CTA computes that block of t
-  const int n_pre = t_block >= 0 ? 1 : 0;
+  // Work items of this CTA: with the fused down-projection, the last tiles_m * t_chunks CTAs (the ones with the
+  // fewest output tiles) start with one block of t; then the output tiles blockIdx.x, blockIdx.x + grid, ...
+  const int t_item = P.fuse ? (int)blockIdx.x - ((int)gridDim.x - tiles_m * P.t_chunks) : -1;  // >= 0: this CTA computes a block of t
+  const int t_block = t_item >= 0 ? t_item % tiles_m : 0, t_chunk = t_item >= 0 ? t_item / tiles_m : 0;
+  const int n_pre = t_item >= 0 ? 1 : 0;
   const int n_main = (int)blockIdx.x < n_tiles ? (n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
   const int n_items = n_pre + n_main;
   auto item_tile = [&](int it) { return (int)blockIdx.x + (it - n_pre) * (int)gridDim.x; };
@@ -189,9 +189,9 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
       const bool pre = it < n_pre;
       const int tile = pre ? 0 : item_tile(it);
       const int m0 = pre ? t_block * kBM : (tile % tiles_m) * kBM;  // neighbouring CTAs share a B panel
-      const int n0 = pre ? 0 : (tile / tiles_m) * BN;
+      const int n0 = pre ? t_chunk * P.Rc : (tile / tiles_m) * BN;
       const int n_slices = pre ? ks1 : ks;
-      const uint32_t bytes = pre ? (uint32_t)(kStageA + P.R * kBK * 2) : (uint32_t)kStageBytes;
+      const uint32_t bytes = pre ? (uint32_t)(kStageA + P.Rc * kBK * 2) : (uint32_t)kStageBytes;
       bool ok = true;
       for (int i = 0; i < n_slices && ok; ++i, ++fill) {
         const uint32_t s = fill % kStages, ph = (fill / kStages) & 1u;
@@ -201,7 +201,7 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
         if (P.fuse && seg2 && i == ks1) {
           // the second segment reads t: wait until this row block of it has been published
           uint32_t spins = 0;
-          while (ld_acquire(P.flags + m0 / kBM) == 0u) {
+          while (ld_acquire(P.flags + m0 / kBM) != (uint32_t)P.t_chunks) {
             if (++spins >= kSpinLimit || ((spins & 1023u) == 0u && *abort_flag)) { *abort_flag = 1; ok = false; break; }
           }
           if (!ok) break;
@@ -225,7 +225,7 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
   } else if (warp == 5) {
     // ============================================================================ MMA issuer
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
-    const uint32_t idesc_t = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.R >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+    const uint32_t idesc_t = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.Rc >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
     uint32_t cons = 0, t_local = 0;
     for (int it = 0; it < n_items && !*abort_flag; ++it, ++t_local) {
       const bool pre = it < n_pre;
@@ -261,8 +261,8 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
       const bool pre = it < n_pre;
       const int tile = pre ? 0 : item_tile(it);
       const int m0 = pre ? t_block * kBM : (tile % tiles_m) * kBM;
-      const int n0 = pre ? 0 : (tile / tiles_m) * BN;
-      const int n_cols = pre ? P.R : BN, ld_c = pre ? P.R : P.N, n_lim = pre ? P.R : P.N;
+      const int n0 = pre ? t_chunk * P.Rc : (tile / tiles_m) * BN;
+      const int n_cols = pre ? P.Rc : BN, ld_c = pre ? P.R : P.N, n_lim = pre ? P.R : P.N;
       __nv_bfloat16* c = pre ? P.t : P.c;
       const uint8_t* gate = pre ? P.t_gate : P.gate;
       const uint32_t acc = t_local & 1u;
@@ -294,7 +294,7 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
         fence_proxy_async();
         __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (threadIdx.x == 0) st_release(P.flags + t_block, 1u);
+        if (threadIdx.x == 0) atomicAdd(P.flags + t_block, 1u);  // after the fence above: a release
       }
     }
   }
@@ -361,11 +361,11 @@ int launch_gemm(isd_ctx* ctx, GemmParams P, const void* a1, const void* b1, cons
   if (rc == ISD_OK) rc = encode_matrix(&mb1, b1, P.N, P.K1, BN);
   if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&ma2, a2, P.M, P.K2, kBM) : encode_matrix(&ma2, a1, P.M, P.K1, kBM);
   if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&mb2, b2, P.N, P.K2, BN) : encode_matrix(&mb2, b1, P.N, P.K1, BN);
-  if (rc == ISD_OK) rc = P.fuse ? encode_matrix(&mbt, bt, P.R, P.K1, P.R) : encode_matrix(&mbt, b1, P.N, P.K1, BN);
+  if (rc == ISD_OK) rc = P.fuse ? encode_matrix(&mbt, bt, P.R, P.K1, P.Rc) : encode_matrix(&mbt, b1, P.N, P.K1, BN);
   if (rc != ISD_OK) return rc;
   const int tiles_m = (P.M + kBM - 1) / kBM;
   int tiles = tiles_m * ((P.N + BN - 1) / BN);
-  if (P.fuse && tiles < tiles_m) tiles = tiles_m;  // every block of t needs a CTA
+  if (P.fuse && tiles < tiles_m * P.t_chunks) tiles = tiles_m * P.t_chunks;  // every block of t needs a CTA
   const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
   gemm_tc_kernel<BN><<<grid, kThreads, kSmem, stream>>>(P, ma1, mb1, ma2, mb2, mbt);
   ctx->launches++;
@@ -394,13 +394,16 @@ int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t st
   P2.M = a->m; P2.N = a->n; P2.K1 = a->k; P2.K2 = a->rank;
   P2.c = reinterpret_cast<__nv_bfloat16*>(a->y); P2.gate = nullptr; P2.scale = 1.f;
   P2.global_status = ctx->global_status;
-  P2.fuse = 0; P2.R = a->rank; P2.t = reinterpret_cast<__nv_bfloat16*>(a->t); P2.t_gate = a->gate; P2.t_scale = a->scale;
+  P2.fuse = 0; P2.R = a->rank; P2.Rc = a->rank; P2.t_chunks = 1; P2.t = reinterpret_cast<__nv_bfloat16*>(a->t); P2.t_gate = a->gate; P2.t_scale = a->scale;
   P2.flags = ctx->lora_flags; P2.done = ctx->lora_flags + kMaxFlags;
-  // One launch when a block of t fits one MMA (rank <= the tile width) and every block gets its own CTA: the
-  // last tiles_m CTAs compute t = gate * scale * (x A^T) block by block before their output tiles, and the second
-  // K segment of y = x W^T + t B^T waits for the block it reads.
-  if (a->rank <= ISD_LORA_BN && tiles_m <= ctx->num_sms && tiles_m <= kMaxFlags) {
+  // One launch when t divides into blocks of one MMA's width (rank <= the tile width, or a multiple of it) and
+  // every block gets its own CTA: the last CTAs compute t = gate * scale * (x A^T) block by block before their
+  // output tiles, and the second K segment of y = x W^T + t B^T waits for the blocks of the rows it reads.
+  const int chunks = a->rank <= ISD_LORA_BN ? 1 : (a->rank % ISD_LORA_BN == 0 ? a->rank / ISD_LORA_BN : 0);
+  if (chunks > 0 && tiles_m * chunks <= ctx->num_sms && tiles_m <= kMaxFlags) {
     P2.fuse = 1;
+    P2.t_chunks = chunks;
+    P2.Rc = a->rank / chunks;
     return launch_gemm<ISD_LORA_BN>(ctx, P2, a->x, a->w, a->t, a->b, a->a, stream);
   }
   // Otherwise two launches.  1. t = gate * scale * (x A^T): N = rank, one K segment

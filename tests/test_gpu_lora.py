@@ -79,9 +79,10 @@ def test_model_sized_layer_sampled_rows():
 def test_repeated_calls_reuse_the_scratch_and_big_ranks_take_two_launches():
     # The one-launch form hands t from CTA to CTA through readiness flags that every launch must leave cleared:
     # with a stale flag the second K segment would read the previous call's t.  Same buffers, the gate flipped
-    # between calls; every call is checked in full.  Rank 320 exceeds one MMA's width: two launches.
+    # between calls; every call is checked in full.  Rank 512 = two blocks of t per row block, still one launch;
+    # rank 320 is neither below one MMA's width nor a multiple of it: two launches.
     eng = _engine()
-    for (M, N, K, R), launches in (((300, 288, 256, 128), 1), ((260, 160, 128, 320), 2)):
+    for (M, N, K, R), launches in (((300, 288, 256, 128), 1), ((300, 544, 192, 512), 1), ((260, 160, 128, 320), 2)):
         x, w, a, b, gate = _inputs(M, N, K, R, seed=3 * M + R)
         t = torch.empty(M, R, dtype=torch.bfloat16, device=DEV)
         y = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
