@@ -9,7 +9,8 @@
 // block of t each and publish it (a counter per row block, raised after a proxy fence: t is read back by TMA);
 // the producer of an output tile waits (bounded) until the counter of its row block is complete before it loads
 // the second K segment, which comes last.
-// The last CTA to finish clears the flags.  Otherwise two launches of the same kernel, t first.
+// The last CTA to finish clears the flags.  Otherwise two launches of the same kernel, t first.  The output tiles
+// of the last, partial round of the grid are cut into column strips, one per CTA.
 //
 // Kernel: persistent CTAs, one 128 x BN output tile at a time.  Warp 4 streams the operands with TMA
 // (2-D maps, 64-element K slices = 128-byte rows, SWIZZLE_128B, every CTA loads for itself) into a 4-stage ring; warp 5
@@ -120,6 +121,7 @@ struct GemmParams {
   // block each of t[M, R] = t_gate * t_scale * (A1 Bt^T), Bt[R, K1], and publish it; the second K segment of C
   // (A2 = t) waits until all t_chunks blocks of its rows are there
   int fuse, R, Rc, t_chunks;  // Rc = columns of a block of t (R = t_chunks * Rc)
+  int tail_split;             // the tiles of the last, partial round are cut into this many column strips (1, 2 or 4)
   __nv_bfloat16* t;
   const uint8_t* t_gate;
   float t_scale;
@@ -142,7 +144,8 @@ template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_b1,
                const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b2,
-               const __grid_constant__ CUtensorMap map_bt) {
+               const __grid_constant__ CUtensorMap map_bt, const __grid_constant__ CUtensorMap map_b1n,
+               const __grid_constant__ CUtensorMap map_b2n) {
   constexpr int kStageA = kBM * kBK * 2, kStageB = BN * kBK * 2, kStageBytes = kStageA + kStageB;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sm_base = smem_u32(smem);
@@ -178,20 +181,37 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
   const int t_item = P.fuse ? (int)blockIdx.x - ((int)gridDim.x - tiles_m * P.t_chunks) : -1;  // >= 0: this CTA computes a block of t
   const int t_block = t_item >= 0 ? t_item % tiles_m : 0, t_chunk = t_item >= 0 ? t_item / tiles_m : 0;
   const int n_pre = t_item >= 0 ? 1 : 0;
-  const int n_main = (int)blockIdx.x < n_tiles ? (n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-  const int n_items = n_pre + n_main;
-  auto item_tile = [&](int it) { return (int)blockIdx.x + (it - n_pre) * (int)gridDim.x; };
+  // The output tiles: whole rounds of the grid as 128 x BN tiles; the tiles of the last, partial round are cut
+  // into tail_split column strips each, one strip per CTA, so that more CTAs share that round (strip u: tile
+  // tail0 + u / tail_split, columns (u % tail_split) * BN / tail_split ...).  No CTA gets a strip and a block of t.
+  const int rounds = n_tiles / (int)gridDim.x, tail0 = rounds * (int)gridDim.x;
+  const int n_strips = (n_tiles - tail0) * P.tail_split, strip_cols = BN / P.tail_split;
+  const int n_items = n_pre + rounds + ((int)blockIdx.x < n_strips ? 1 : 0);
+  struct Item { bool pre; int m0, n0, cols; };
+  auto item = [&](int it) {
+    Item w;
+    w.pre = it < n_pre;
+    if (w.pre) {
+      w.m0 = t_block * kBM; w.n0 = t_chunk * P.Rc; w.cols = P.Rc;
+    } else if (it - n_pre < rounds) {
+      const int tile = (int)blockIdx.x + (it - n_pre) * (int)gridDim.x;
+      w.m0 = (tile % tiles_m) * kBM; w.n0 = (tile / tiles_m) * BN; w.cols = BN;  // neighbouring CTAs share a B panel
+    } else {
+      const int tile = tail0 + (int)blockIdx.x / P.tail_split;
+      w.m0 = (tile % tiles_m) * kBM; w.n0 = (tile / tiles_m) * BN + ((int)blockIdx.x % P.tail_split) * strip_cols; w.cols = strip_cols;
+    }
+    return w;
+  };
 
   if (warp == 4) {
     // ============================================================================ TMA producer
     uint32_t fill = 0;
     for (int it = 0; it < n_items && !*abort_flag; ++it) {
-      const bool pre = it < n_pre;
-      const int tile = pre ? 0 : item_tile(it);
-      const int m0 = pre ? t_block * kBM : (tile % tiles_m) * kBM;  // neighbouring CTAs share a B panel
-      const int n0 = pre ? t_chunk * P.Rc : (tile / tiles_m) * BN;
+      const Item w = item(it);
+      const bool pre = w.pre, narrow = !pre && w.cols != BN;
+      const int m0 = w.m0, n0 = w.n0;
       const int n_slices = pre ? ks1 : ks;
-      const uint32_t bytes = pre ? (uint32_t)(kStageA + P.Rc * kBK * 2) : (uint32_t)kStageBytes;
+      const uint32_t bytes = (uint32_t)(kStageA + w.cols * kBK * 2);
       bool ok = true;
       for (int i = 0; i < n_slices && ok; ++i, ++fill) {
         const uint32_t s = fill % kStages, ph = (fill / kStages) & 1u;
@@ -212,7 +232,8 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
           const uint32_t dst = sm_base + s * kStageBytes;
           const int k0 = (seg2 ? i - ks1 : i) * kBK;
           tma_load_2d(dst, seg2 ? &map_a2 : &map_a1, k0, m0, bar(BAR_FULL + s));
-          tma_load_2d(dst + kStageA, pre ? &map_bt : (seg2 ? &map_b2 : &map_b1), k0, n0, bar(BAR_FULL + s));
+          tma_load_2d(dst + kStageA, pre ? &map_bt : (seg2 ? (narrow ? &map_b2n : &map_b2) : (narrow ? &map_b1n : &map_b1)), k0, n0,
+                      bar(BAR_FULL + s));
         }
         __syncwarp();
       }
@@ -224,12 +245,13 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
     }
   } else if (warp == 5) {
     // ============================================================================ MMA issuer
-    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
-    const uint32_t idesc_t = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.Rc >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+    auto idesc_for = [](int n) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24); };
     uint32_t cons = 0, t_local = 0;
     for (int it = 0; it < n_items && !*abort_flag; ++it, ++t_local) {
-      const bool pre = it < n_pre;
+      const Item w = item(it);
+      const bool pre = w.pre;
       const int n_slices = pre ? ks1 : ks;
+      const uint32_t idesc = idesc_for(w.cols);
       const uint32_t acc = t_local & 1u;
       // the epilogue warps must have read this accumulator's previous tile
       if (t_local >= 2 && !mbar_wait(bar(BAR_ACC_FREE + acc), ((t_local >> 1) - 1u) & 1u, abort_flag)) break;
@@ -245,7 +267,7 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k)
             tc_mma(tmem + acc * (uint32_t)BN, smem_desc_kmajor(a0 + k * 32), smem_desc_kmajor(b0 + k * 32),
-                   pre ? idesc_t : idesc, (i > 0 || k > 0) ? 1u : 0u);
+                   idesc, (i > 0 || k > 0) ? 1u : 0u);
           tc_commit(bar(BAR_EMPTY + s));
           if (i == n_slices - 1) tc_commit(bar(BAR_ACC_FULL + acc));
         }
@@ -258,11 +280,10 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
     uint32_t t_local = 0;
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     for (int it = 0; it < n_items && !*abort_flag; ++it, ++t_local) {
-      const bool pre = it < n_pre;
-      const int tile = pre ? 0 : item_tile(it);
-      const int m0 = pre ? t_block * kBM : (tile % tiles_m) * kBM;
-      const int n0 = pre ? t_chunk * P.Rc : (tile / tiles_m) * BN;
-      const int n_cols = pre ? P.Rc : BN, ld_c = pre ? P.R : P.N, n_lim = pre ? P.R : P.N;
+      const Item w = item(it);
+      const bool pre = w.pre;
+      const int m0 = w.m0, n0 = w.n0;
+      const int n_cols = w.cols, ld_c = pre ? P.R : P.N, n_lim = pre ? P.R : P.N;
       __nv_bfloat16* c = pre ? P.t : P.c;
       const uint8_t* gate = pre ? P.t_gate : P.gate;
       const uint32_t acc = t_local & 1u;
@@ -356,7 +377,7 @@ int launch_gemm(isd_ctx* ctx, GemmParams P, const void* a1, const void* b1, cons
       return ISD_ERR_CUDA;
     attr_set = true;
   }
-  CUtensorMap ma1, mb1, ma2, mb2, mbt;
+  CUtensorMap ma1, mb1, ma2, mb2, mbt, mb1n, mb2n;
   int rc = encode_matrix(&ma1, a1, P.M, P.K1, kBM);
   if (rc == ISD_OK) rc = encode_matrix(&mb1, b1, P.N, P.K1, BN);
   if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&ma2, a2, P.M, P.K2, kBM) : encode_matrix(&ma2, a1, P.M, P.K1, kBM);
@@ -364,10 +385,19 @@ int launch_gemm(isd_ctx* ctx, GemmParams P, const void* a1, const void* b1, cons
   if (rc == ISD_OK) rc = P.fuse ? encode_matrix(&mbt, bt, P.R, P.K1, P.Rc) : encode_matrix(&mbt, b1, P.N, P.K1, BN);
   if (rc != ISD_OK) return rc;
   const int tiles_m = (P.M + kBM - 1) / kBM;
-  int tiles = tiles_m * ((P.N + BN - 1) / BN);
-  if (P.fuse && tiles < tiles_m * P.t_chunks) tiles = tiles_m * P.t_chunks;  // every block of t needs a CTA
+  const int n_tiles = tiles_m * ((P.N + BN - 1) / BN), n_t = P.fuse ? tiles_m * P.t_chunks : 0;
+  int tiles = n_tiles;
+  if (tiles < n_t) tiles = n_t;  // every block of t needs a CTA
   const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
-  gemm_tc_kernel<BN><<<grid, kThreads, kSmem, stream>>>(P, ma1, mb1, ma2, mb2, mbt);
+  // column strips for the last, partial round of tiles: as many as the CTAs without a block of t can take
+  const int tail = n_tiles % grid;
+  P.tail_split = 1;
+  for (int sp = 4; sp > 1; sp >>= 1)
+    if (tail > 0 && tail * sp <= grid - n_t && (BN / sp) % 32 == 0) { P.tail_split = sp; break; }
+  rc = encode_matrix(&mb1n, b1, P.N, P.K1, BN / P.tail_split);
+  if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&mb2n, b2, P.N, P.K2, BN / P.tail_split) : encode_matrix(&mb2n, b1, P.N, P.K1, BN / P.tail_split);
+  if (rc != ISD_OK) return rc;
+  gemm_tc_kernel<BN><<<grid, kThreads, kSmem, stream>>>(P, ma1, mb1, ma2, mb2, mbt, mb1n, mb2n);
   ctx->launches++;
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }
