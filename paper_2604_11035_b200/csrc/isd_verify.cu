@@ -543,6 +543,11 @@ __device__ __forceinline__ float job_score(const VerifyParams& P, const SampleJo
   return rr > 0.f ? logf(rr) + gumbel_f32(w) : -INFINITY;
 }
 
+// resident CTAs per SM the sampling kernel is compiled for: three keep it at 80 registers (without the bound
+// the compiler takes 89 and only two CTAs fit)
+#ifndef ISD_SAMPLE_MINB
+#define ISD_SAMPLE_MINB 3
+#endif
 // Per-warp queue of groups of four logits that survived the first skip test.
 constexpr int kQueueCap = 128;  // < 32 left over + at most 64 new per iteration
 struct SampleQueue {
@@ -641,7 +646,7 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads) verify_sample_kernel(const VerifyParams P) {
+__global__ void __launch_bounds__(kThreads, ISD_SAMPLE_MINB) verify_sample_kernel(const VerifyParams P) {
   const int split = blockIdx.x, k = blockIdx.y, b = blockIdx.z;
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
