@@ -286,8 +286,8 @@ __device__ bool block_topk_two_stream(TopkShared& sh, const char* row, int e_lo,
 }
 
 constexpr int kHeadStages = 8;  // stages of the head, read twice to find a first bound
-constexpr int kCheckEvery = 4;  // stages between two looks at the queue of noted groups (a power of two)
-constexpr int kExpandAt = 48;   // noted groups from which a look turns them into candidates
+constexpr int kCheckEvery = 8;  // stages between two looks at the queue of noted groups (a power of two)
+constexpr int kExpandAt = 64;   // noted groups from which a look turns them into candidates
 constexpr int kCompactAt = 96;  // candidates from which they are cut back to the best k and the bound rises
 
 // One stage of the ring: waits for it, takes this thread's groups of eight as packed words, releases the stage.
