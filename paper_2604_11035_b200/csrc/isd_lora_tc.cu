@@ -12,7 +12,11 @@
 // The last CTA to finish clears the flags.  Otherwise two launches of the same kernel, t first.  The output tiles
 // of the last, partial round of the grid are cut into column strips, one per CTA.
 //
-// Kernel: persistent CTAs, one 128 x BN output tile at a time.  Warp 4 streams the operands with TMA
+// Two forms of the kernel.  gemm_tc2_kernel (further down, the one normally used) works on CTA pairs; the one-CTA
+// form below serves shapes the pairs cannot take (ranks above 256 that are not multiples of 256, more blocks of t
+// than CTA pairs) and comparison runs.
+//
+// One-CTA kernel: persistent CTAs, one 128 x BN output tile at a time.  Warp 4 streams the operands with TMA
 // (2-D maps, 64-element K slices = 128-byte rows, SWIZZLE_128B, every CTA loads for itself) into a 4-stage ring; warp 5
 // issues tcgen05.mma (M = 128, N = BN, K = 16, both operands from shared memory) into one of two TMEM
 // accumulators; warps 0-3 read the other accumulator back (tcgen05.ld, one lane = one row), apply gate and
@@ -20,6 +24,8 @@
 // bounded (status bit 0x80000000, then the CTA drains and frees its tensor memory).
 #include <cuda.h>
 #include <cuda_bf16.h>
+
+#include <cstdlib>
 
 #include "isd_internal.cuh"
 
@@ -336,6 +342,249 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same GEMM on CTA pairs (tcgen05 cta_group::2): a cluster of two CTAs owns a 256 x 256 output tile.  Each CTA
+// stages its own 128 rows of A and 128 of the tile's 256 rows of B (half the shared-memory traffic per flop of the
+// one-CTA form), the first CTA of the pair issues M = 256 MMAs that read both CTAs' shared memory and write both
+// CTAs' tensor memory (rows 0-127 into its own, 128-255 into its partner's), and each CTA's epilogue warps store
+// their 128 rows.  Barriers: TMA of both CTAs reports to the first CTA's `full` barrier; the MMA thread's commits
+// arrive on the `empty` and `accumulator full` barriers of both CTAs; the epilogue warps of both CTAs arrive on
+// the first CTA's `accumulator free` barrier.  Every wait is bounded.
+// ------------------------------------------------------------------------------------------------
+constexpr int kStages2 = 6;
+constexpr int kStage2A = kBM * kBK * 2, kStage2B = 128 * kBK * 2, kStage2Bytes = kStage2A + kStage2B;
+constexpr int kBN2 = 256;
+enum { B2_FULL = 0, B2_EMPTY = kStages2, B2_ACC_FULL = 2 * kStages2, B2_ACC_FREE = 2 * kStages2 + 2,
+       B2_COUNT = 2 * kStages2 + 4 };
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// the address, in the cluster's shared window, of this CTA's shared-memory address `addr` in CTA `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load of a CTA pair: the bytes land in this CTA's shared memory and are reported to the barrier at `bar`,
+// an address in the cluster's shared window (the first CTA's barrier)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tc2_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_b1,
+                const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b2,
+                const __grid_constant__ CUtensorMap map_bt, const __grid_constant__ CUtensorMap map_b1n,
+                const __grid_constant__ CUtensorMap map_b2n) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sm_base = smem_u32(smem);
+  const uint32_t bar_base = sm_base + kStages2 * kStage2Bytes;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kStages2 * kStage2Bytes + B2_COUNT * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kStages2 * kStage2Bytes + B2_COUNT * 8 + 8);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();
+  const bool leader = rank == 0;
+  auto bar = [&](int i) { return bar_base + 8u * (uint32_t)i; };
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kStages2; ++i) { mbar_init(bar(B2_FULL + i), 1); mbar_init(bar(B2_EMPTY + i), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar(B2_ACC_FULL + i), 1); mbar_init(bar(B2_ACC_FREE + i), 8); }
+    *abort_flag = (sm_base & 1023u) ? 1 : 0;  // the swizzled layout assumes a 1 KiB aligned window
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) {  // the same warp in both CTAs
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the partner's barriers exist before anything is reported to them
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  const int tiles_m = (P.M + 2 * kBM - 1) / (2 * kBM), tiles_n = (P.N + kBN2 - 1) / kBN2;
+  const int n_tiles = tiles_m * tiles_n;
+  const int ks1 = P.K1 / kBK, ks2 = P.K2 / kBK, ks = ks1 + ks2;
+  const int pr = (int)blockIdx.x >> 1, n_pairs = (int)gridDim.x >> 1;
+  // work items of the pair, as in the one-CTA kernel: a block of t first (last pairs), whole tiles, one column strip
+  const int t_item = P.fuse ? pr - (n_pairs - tiles_m * P.t_chunks) : -1;
+  const int t_block = t_item >= 0 ? t_item % tiles_m : 0, t_chunk = t_item >= 0 ? t_item / tiles_m : 0;
+  const int n_pre = t_item >= 0 ? 1 : 0;
+  const int rounds = n_tiles / n_pairs, tail0 = rounds * n_pairs;
+  const int n_strips = (n_tiles - tail0) * P.tail_split, strip_cols = kBN2 / P.tail_split;
+  const int n_items = n_pre + rounds + (pr < n_strips ? 1 : 0);
+  struct Item { bool pre; int m0, n0, cols; };
+  auto item = [&](int it) {
+    Item w;
+    w.pre = it < n_pre;
+    if (w.pre) {
+      w.m0 = t_block * 2 * kBM; w.n0 = t_chunk * P.Rc; w.cols = P.Rc;
+    } else if (it - n_pre < rounds) {
+      const int tile = pr + (it - n_pre) * n_pairs;
+      w.m0 = (tile % tiles_m) * 2 * kBM; w.n0 = (tile / tiles_m) * kBN2; w.cols = kBN2;
+    } else {
+      const int tile = tail0 + pr / P.tail_split;
+      w.m0 = (tile % tiles_m) * 2 * kBM; w.n0 = (tile / tiles_m) * kBN2 + (pr % P.tail_split) * strip_cols; w.cols = strip_cols;
+    }
+    return w;
+  };
+
+  if (warp == 4) {
+    // ============================================================================ TMA producer (both CTAs)
+    uint32_t fill = 0;
+    for (int it = 0; it < n_items && !*abort_flag; ++it) {
+      const Item w = item(it);
+      const bool pre = w.pre, narrow = !pre && w.cols != kBN2;
+      const int m0 = w.m0 + (int)rank * kBM;          // this CTA's rows of A
+      const int half = w.cols / 2, n0 = w.n0 + (int)rank * half;  // this CTA's rows of B
+      const int n_slices = pre ? ks1 : ks;
+      const uint32_t bytes = 2u * (uint32_t)(kStage2A + half * kBK * 2);  // of both CTAs
+      bool ok = true;
+      for (int i = 0; i < n_slices && ok; ++i, ++fill) {
+        const uint32_t s = fill % kStages2, ph = (fill / kStages2) & 1u;
+        ok = mbar_wait(bar(B2_EMPTY + s), ph ^ 1u, abort_flag);
+        if (!ok) break;
+        const bool seg2 = !pre && i >= ks1;
+        if (P.fuse && seg2 && i == ks1) {
+          uint32_t spins = 0;
+          while (ld_acquire(P.flags + w.m0 / (2 * kBM)) != 2u * (uint32_t)P.t_chunks) {
+            if (++spins >= kSpinLimit || ((spins & 1023u) == 0u && *abort_flag)) { *abort_flag = 1; ok = false; break; }
+          }
+          if (!ok) break;
+          fence_proxy_async();
+        }
+        if (elect_one()) {
+          const uint32_t full = map_to_cta(bar(B2_FULL + s), 0u);
+          if (leader) mbar_arrive_expect_tx(bar(B2_FULL + s), bytes);
+          const uint32_t dst = sm_base + s * kStage2Bytes;
+          const int k0 = (seg2 ? i - ks1 : i) * kBK;
+          tma_load_2d_pair(dst, seg2 ? &map_a2 : &map_a1, k0, m0, full);
+          tma_load_2d_pair(dst + kStage2A, pre ? &map_bt : (seg2 ? (narrow ? &map_b2n : &map_b2) : (narrow ? &map_b1n : &map_b1)), k0, n0, full);
+        }
+        __syncwarp();
+      }
+      if (!ok) break;
+    }
+    if (*abort_flag && leader) {  // every issued copy must land before the CTAs may leave
+      for (uint32_t f = (fill > kStages2 ? fill - kStages2 : 0); f < fill; ++f)
+        mbar_wait(bar(B2_FULL + f % kStages2), (f / kStages2) & 1u, abort_flag);
+    }
+  } else if (warp == 5) {
+    // ============================================================================ MMA issuer (first CTA only)
+    if (leader) {
+      auto idesc_for = [](int n) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)((2 * kBM) >> 4) << 24); };
+      uint32_t cons = 0, t_local = 0;
+      for (int it = 0; it < n_items && !*abort_flag; ++it, ++t_local) {
+        const Item w = item(it);
+        const int n_slices = w.pre ? ks1 : ks;
+        const uint32_t idesc = idesc_for(w.cols);
+        const uint32_t acc = t_local & 1u;
+        if (t_local >= 2 && !mbar_wait(bar(B2_ACC_FREE + acc), ((t_local >> 1) - 1u) & 1u, abort_flag)) break;
+        tc_fence_after();
+        bool ok = true;
+        for (int i = 0; i < n_slices && ok; ++i, ++cons) {
+          const uint32_t s = cons % kStages2, ph = (cons / kStages2) & 1u;
+          ok = mbar_wait(bar(B2_FULL + s), ph, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          if (elect_one()) {
+            const uint32_t a0 = sm_base + s * kStage2Bytes, b0 = a0 + kStage2A;
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k)
+              tc_mma_pair(tmem + acc * (uint32_t)kBN2, smem_desc_kmajor(a0 + k * 32), smem_desc_kmajor(b0 + k * 32), idesc,
+                          (i > 0 || k > 0) ? 1u : 0u);
+            tc_commit_pair(map_to_cta(bar(B2_EMPTY + s), 0u));
+            tc_commit_pair(map_to_cta(bar(B2_EMPTY + s), 1u));
+            if (i == n_slices - 1) {
+              tc_commit_pair(map_to_cta(bar(B2_ACC_FULL + acc), 0u));
+              tc_commit_pair(map_to_cta(bar(B2_ACC_FULL + acc), 1u));
+            }
+          }
+          __syncwarp();
+        }
+        if (!ok) break;
+      }
+    }
+  } else {
+    // ============================================================================ epilogue (warps 0-3, both CTAs)
+    uint32_t t_local = 0;
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    for (int it = 0; it < n_items && !*abort_flag; ++it, ++t_local) {
+      const Item w = item(it);
+      const bool pre = w.pre;
+      const int m0 = w.m0 + (int)rank * kBM, n0 = w.n0;
+      const int n_cols = w.cols, ld_c = pre ? P.R : P.N, n_lim = pre ? P.R : P.N;
+      __nv_bfloat16* c = pre ? P.t : P.c;
+      const uint8_t* gate = pre ? P.t_gate : P.gate;
+      const uint32_t acc = t_local & 1u;
+      if (!mbar_wait(bar(B2_ACC_FULL + acc), (t_local >> 1) & 1u, abort_flag)) break;
+      tc_fence_after();
+      const int row = m0 + warp * 32 + lane;
+      const bool row_ok = row < P.M;
+      const float f = (gate == nullptr || (row_ok && gate[row])) ? (pre ? P.t_scale : P.scale) : 0.f;
+#pragma unroll 1
+      for (int c0 = 0; c0 < n_cols; c0 += 32) {
+        uint32_t v[32];
+        TMEM_LD32(tmem + lane_base + acc * (uint32_t)kBN2 + (uint32_t)c0, v);
+        tmem_wait_ld();
+        if (row_ok && n0 + c0 < n_lim) {
+          uint4* dst = reinterpret_cast<uint4*>(c + (size_t)row * ld_c + n0 + c0);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            dst[q] = make_uint4(pack_bf16(__uint_as_float(v[8 * q]) * f, __uint_as_float(v[8 * q + 1]) * f),
+                                pack_bf16(__uint_as_float(v[8 * q + 2]) * f, __uint_as_float(v[8 * q + 3]) * f),
+                                pack_bf16(__uint_as_float(v[8 * q + 4]) * f, __uint_as_float(v[8 * q + 5]) * f),
+                                pack_bf16(__uint_as_float(v[8 * q + 6]) * f, __uint_as_float(v[8 * q + 7]) * f));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(bar(B2_ACC_FREE + acc), 0u));
+      if (pre) {
+        fence_proxy_async();
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (threadIdx.x == 0) atomicAdd(P.flags + t_block, 1u);  // after the fence above: a release
+      }
+    }
+  }
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  if (P.fuse && threadIdx.x == 0) {  // the CTA that finishes last leaves the flags as it found them
+    __threadfence();
+    if (atomicAdd(P.done, 1u) == gridDim.x - 1) {
+      for (int m = 0; m < tiles_m; ++m) P.flags[m] = 0u;
+      *P.done = 0u;
+    }
+  }
+  cluster_sync_all();  // nobody frees tensor memory or leaves while the partner may still use this CTA's
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -402,6 +651,39 @@ int launch_gemm(isd_ctx* ctx, GemmParams P, const void* a1, const void* b1, cons
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }
 
+// The CTA-pair form: same arguments; fuse, R, Rc, t_chunks as prepared by the caller (blocks of t are 256 rows here).
+int launch_gemm_pair(isd_ctx* ctx, GemmParams P, const void* a1, const void* b1, const void* a2, const void* b2,
+                     const void* bt, cudaStream_t stream) {
+  constexpr int kSmem = kStages2 * kStage2Bytes + B2_COUNT * 8 + 64;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+      return ISD_ERR_CUDA;
+    attr_set = true;
+  }
+  const int tiles_m = (P.M + 2 * kBM - 1) / (2 * kBM);
+  const int n_tiles = tiles_m * ((P.N + kBN2 - 1) / kBN2), n_t = P.fuse ? tiles_m * P.t_chunks : 0;
+  int pairs = n_tiles < n_t ? n_t : n_tiles;
+  if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;
+  const int tail = n_tiles % pairs;
+  P.tail_split = 1;
+  for (int sp = 4; sp > 1; sp >>= 1)
+    if (tail > 0 && tail * sp <= pairs - n_t) { P.tail_split = sp; break; }
+  const int strip_half = kBN2 / P.tail_split / 2;
+  CUtensorMap ma1, mb1, ma2, mb2, mbt, mb1n, mb2n;
+  int rc = encode_matrix(&ma1, a1, P.M, P.K1, kBM);
+  if (rc == ISD_OK) rc = encode_matrix(&mb1, b1, P.N, P.K1, kBN2 / 2);
+  if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&ma2, a2, P.M, P.K2, kBM) : encode_matrix(&ma2, a1, P.M, P.K1, kBM);
+  if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&mb2, b2, P.N, P.K2, kBN2 / 2) : encode_matrix(&mb2, b1, P.N, P.K1, kBN2 / 2);
+  if (rc == ISD_OK) rc = P.fuse ? encode_matrix(&mbt, bt, P.R, P.K1, P.Rc / 2) : encode_matrix(&mbt, b1, P.N, P.K1, kBN2 / 2);
+  if (rc == ISD_OK) rc = encode_matrix(&mb1n, b1, P.N, P.K1, strip_half);
+  if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&mb2n, b2, P.N, P.K2, strip_half) : encode_matrix(&mb2n, b1, P.N, P.K1, strip_half);
+  if (rc != ISD_OK) return rc;
+  gemm_tc2_kernel<<<2 * pairs, kThreads, kSmem, stream>>>(P, ma1, mb1, ma2, mb2, mbt, mb1n, mb2n);
+  ctx->launches++;
+  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}
+
 }  // namespace
 
 int isd_lora_create(isd_ctx* ctx) {
@@ -430,6 +712,17 @@ int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t st
   // every block gets its own CTA: the last CTAs compute t = gate * scale * (x A^T) block by block before their
   // output tiles, and the second K segment of y = x W^T + t B^T waits for the blocks of the rows it reads.
   const int chunks = a->rank <= ISD_LORA_BN ? 1 : (a->rank % ISD_LORA_BN == 0 ? a->rank / ISD_LORA_BN : 0);
+  // ISD_LORA_PAIR=0 in the environment keeps the CTA-pair kernel out (comparison runs, tests of the one-CTA form)
+  const char* env_pair = getenv("ISD_LORA_PAIR");
+  const bool use_pairs = !(env_pair && env_pair[0] == '0');
+  const int blocks2 = (a->m + 2 * kBM - 1) / (2 * kBM);  // 256-row blocks
+  if (use_pairs && chunks > 0 && blocks2 * chunks <= ctx->num_sms / 2 && blocks2 <= kMaxFlags) {
+    // CTA pairs: 256 x 256 tiles, blocks of t of 256 rows
+    P2.fuse = 1;
+    P2.t_chunks = chunks;
+    P2.Rc = a->rank / chunks;
+    return launch_gemm_pair(ctx, P2, a->x, a->w, a->t, a->b, a->a, stream);
+  }
   if (chunks > 0 && tiles_m * chunks <= ctx->num_sms && tiles_m <= kMaxFlags) {
     P2.fuse = 1;
     P2.t_chunks = chunks;

@@ -98,3 +98,20 @@ def test_repeated_calls_reuse_the_scratch_and_big_ranks_take_two_launches():
             assert (err <= tol).all(), (M, R, call, float(err.max()))
     assert eng.isd_read_status() == 0
     eng.close()
+
+
+@pytest.mark.parametrize("M,N,K,R", [(517, 544, 448, 192), (300, 544, 192, 512), (700, 1120, 128, 64)])
+def test_one_cta_form_of_the_kernel(M, N, K, R, monkeypatch):
+    # ISD_LORA_PAIR=0 keeps the CTA-pair kernel out: the one-CTA kernel with the fused down-projection and the
+    # column strips of the last round takes the same shapes (the library reads the variable at every call)
+    monkeypatch.setenv("ISD_LORA_PAIR", "0")
+    eng = _engine()
+    x, w, a, b, gate = _inputs(M, N, K, R, seed=7 * M + R)
+    y = eng.isd_lora_linear(x, w, a, b, gate, 0.6)
+    torch.cuda.synchronize()
+    ref = oracle.lora_linear(_f64(x), _f64(w), _f64(a), _f64(b), gate.cpu().numpy(), 0.6)
+    tol = _tolerance(ref, _f64(x), _f64(a), _f64(b), gate.cpu().numpy(), 0.6)
+    err = np.abs(_f64(y) - ref)
+    assert (err <= tol).all(), float(err.max())
+    assert eng.isd_read_status() == 0
+    eng.close()
