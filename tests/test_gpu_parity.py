@@ -184,9 +184,10 @@ def test_run_to_run_determinism():
                                y.view(torch.uint8) if y.dtype.is_floating_point else y)
 
 
-def test_inactive_slots_and_empty_batch():
+@pytest.mark.parametrize("top_k,top_p", [(0, 1.0), (20, 0.9)], ids=["plain", "filtered"])
+def test_inactive_slots_and_empty_batch(top_k, top_p):
     w = Workload("inact", batch=4, stride=3, n_q_heads=8, n_kv_heads=2, vocab=1024, ctx_min=10, ctx_max=90,
-                 logits_dtype="f32", steps=3, propose_mode=0, seed=8)
+                 logits_dtype="f32", steps=3, propose_mode=0, seed=8, top_k=top_k, top_p=top_p)
     st, eng, out = _fresh(w)
     st["active"][1] = 0
     before = {k: st[k].clone() for k in STATE_KEYS}
@@ -205,9 +206,11 @@ def test_inactive_slots_and_empty_batch():
     eng.close()
 
 
-def test_faults_set_status_bits_and_freeze_the_slot():
+@pytest.mark.parametrize("top_k,top_p", [(0, 1.0), (20, 0.9)], ids=["plain", "filtered"])
+def test_faults_set_status_bits_and_freeze_the_slot(top_k, top_p):
+    # (filtered: the decide kernel runs as clusters of two CTAs; frozen and inactive slots leave before its barriers)
     w = Workload("fault", batch=5, stride=3, n_q_heads=8, n_kv_heads=2, vocab=1024, ctx_min=30, ctx_max=60,
-                 logits_dtype="f32", steps=4, propose_mode=0, seed=9)
+                 logits_dtype="f32", steps=4, propose_mode=0, seed=9, top_k=top_k, top_p=top_p)
     st, eng, out = _fresh(w)
     s_np = state_to_np(st)                              # oracle starts from the same generated state
     lg0 = wl.make_logits(w, 0, torch.from_numpy(s_np["ctx_len"]).to(DEV))
