@@ -60,9 +60,10 @@ def test_small_and_ragged_shapes(M, N, K, R):
     eng.close()
 
 
-def test_model_sized_layer_sampled_rows():
-    # token rows of the benchmark batch (256 slots x 15 rows), hidden size 4096, rank 128
-    M, N, K, R = 3840, 4096, 4096, 128
+@pytest.mark.parametrize("R", [128, 1024])
+def test_model_sized_layer_sampled_rows(R):
+    # token rows of the benchmark batch (256 slots x 15 rows), hidden size 4096, the two adapter ranks of the paper
+    M, N, K = 3840, 4096, 4096
     eng = _engine()
     x, w, a, b, gate = _inputs(M, N, K, R, seed=9)
     y = eng.isd_lora_linear(x, w, a, b, gate, 0.5)
