@@ -70,7 +70,8 @@ struct isd_ctx {
   int* topk_idx;         // [B, Q, ISD_MAX_TOP_K]
   int* topk_n;           // [B, Q]
   unsigned long long* topk_q_key;  // [B, pieces, ISD_MAX_TOP_K] piece lists of a proposal-law row (as sort keys)
-  int* topk_q_n;         // [B, pieces], then [B, 2] (decision of a cluster's first CTA)
+  int* topk_q_n;         // [B, pieces], then the slot decisions, supports and row tickets of the accept phase
+  double* topk_nuc_lse;  // [B, Q] log-normaliser of every row's filtered law
   // ---- isd_lora_linear: readiness flags of the row blocks of t, then one counter (all zero between launches)
   uint32_t* lora_flags;
   // ---- optional device-resident step counter (CUDA-graph replay), owned by the caller

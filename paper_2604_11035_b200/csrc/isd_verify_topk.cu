@@ -7,13 +7,14 @@
 // no vocabulary-wide exponentials are needed at all:
 //   1. topk_rows_kernel    one CTA per (slot, block row): the exact top-k of the row in one stream of
 //      it (block_topk).  Per logit: a packed maximum over groups of eight and one compare against a
-//      rising bound; the few groups that reach it are re-read from L2 and ranked.
-//   2. topk_decide_kernel  one cluster of kQSplit CTAs per slot.  The first CTA: nucleus cut and
-//      log-normaliser of every row in fp64 (the oracle's arithmetic, so the cut agrees), sequential
-//      accept test, and the Gumbel-max draws (residual, bonus, proposals) over the supports in fp64
-//      with the same per-index Philox noise as the unfiltered path.  Only a rejection costs another
-//      stream: the proposal-law row of the previous step is selected again by the same routine, one
-//      piece of it per CTA of the cluster, and the first CTA merges the piece lists.
+//      rising bound; the few groups that reach it are re-read from L2 and ranked.  The CTA that
+//      finishes a slot's last row runs the slot's accept phase: nucleus cut and log-normaliser of
+//      every row in fp64 (the oracle's arithmetic, so the cut agrees) and the sequential accept test.
+//   2. topk_decide_kernel  one cluster of kQSplit CTAs per slot.  The first CTA: the Gumbel-max draws
+//      (residual, bonus, proposals) over the supports in fp64 with the same per-index Philox noise as
+//      the unfiltered path.  Only a rejection costs another stream: the proposal-law row of the
+//      previous step is selected again by the same routine, one piece of it per CTA of the cluster,
+//      and the first CTA merges the piece lists.
 #include "isd_internal.cuh"
 #include "isd_stream.cuh"
 
@@ -47,7 +48,11 @@ struct TopkParams {
   int* list_n;      // [B, Q] entries of the list; -1 - n when the row holds a NaN or +inf
   unsigned long long* q_key;  // [B, kQSplit, kMaxTopK] piece lists of the proposal-law row of a rejection
   int* q_n;                   // [B, kQSplit]
-  int* q_dec;                 // [B, 2] accept length and rejected position, from a cluster's first CTA to the others
+  int* q_dec;                 // [B, 2] accept length (-1: frozen) and rejected position, from the row kernel to the decide kernel
+  int* nuc_n;                 // [B, Q] support size of every row's filtered law
+  int* nuc_bad;               // [B, Q] 1 = the row holds a NaN or +inf
+  double* nuc_lse;            // [B, Q] log-normaliser of the support
+  int* row_ticket;            // [B] rows of the slot that are done (zero between launches)
 };
 
 struct TopkShared {
@@ -463,43 +468,31 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int e_lo, int e_hi, 
   return ok;
 }
 
-// ------------------------------------------------------------------------------------------------
-// Pass 1: the top-k list of every valid row
-// ------------------------------------------------------------------------------------------------
-template <int DT>
-__global__ void __launch_bounds__(kThreads + 32) topk_rows_kernel(const TopkParams P) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
-  const int b = blockIdx.x, r = blockIdx.y;
-  if (!P.active[b]) return;
-  const int nv = P.n_ver[b];
-  if (nv < 0 || nv > P.N - 1) return;  // flagged by the decide kernel
-  if (r >= nv + P.N) return;
-  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
-  const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
-  if (!block_topk<DT>(sh, row, 0, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
-  const size_t base = ((size_t)b * P.Q + r) * kMaxTopK;
-  if (threadIdx.x < sh.list_n) {
-    P.list_val[base + threadIdx.x] = sh.list_val[threadIdx.x];
-    P.list_idx[base + threadIdx.x] = sh.list_idx[threadIdx.x];
-  }
-  if (threadIdx.x == 0) P.list_n[(size_t)b * P.Q + r] = sh.bad ? -1 - sh.list_n : sh.list_n;
-}
+// Shared memory of the accept phase (it reuses the ring of a CTA whose row is done).
+struct SlotScratch {
+  int n[32], bad[32], x[32];
+  float logp[32], logq[32];
+  double lse[32];
+  double w[kThreads / 32][kMaxTopK];
+};
+static_assert(sizeof(SlotScratch) <= sizeof(RowRing::stage), "the accept phase lives in the ring's stages");
 
-// ------------------------------------------------------------------------------------------------
-// Pass 2: everything else, one CTA per slot
-// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float ldcg_f(const float* p) { return __ldcg(p); }
+__device__ __forceinline__ int ldcg_i(const int* p) { return __ldcg(p); }
+
 // Nucleus of a sorted top-k list in fp64, in the oracle's order of operations: w_i = exp(l_i invT - l_0 invT),
 // Z = sum w_i, support = shortest prefix whose cumulated w reaches top_p * Z.  Returns the support size and
 // the log-normaliser of the support.  By one warp: the lanes compute the exponentials (w: n doubles of shared
-// memory), lane 0 adds them up in index order; every lane gets the result.
+// memory), lane 0 adds them up in index order; every lane gets the result.  FROM_L2: the list is in global memory
+// and is read from L2 (other CTAs of this launch may have written it).
+template <bool FROM_L2>
 __device__ int warp_nucleus(const float* val, int n, double inv_t, double top_p, double* w, double& lse) {
   const int lane = threadIdx.x & 31;
   lse = -INFINITY;
   if (n <= 0) return 0;
-  const double m = (double)val[0] * inv_t;
+  const double m = (double)(FROM_L2 ? ldcg_f(val) : val[0]) * inv_t;
   if (isinf(m) && m < 0) return n;
-  for (int i = lane; i < n; i += 32) w[i] = exp((double)val[i] * inv_t - m);
+  for (int i = lane; i < n; i += 32) w[i] = exp((double)(FROM_L2 ? ldcg_f(val + i) : val[i]) * inv_t - m);
   __syncwarp();
   // lane 0 adds in index order, once: w[i] becomes the sum of the first i + 1 (the oracle's three loops - the
   // normaliser, the cumulated mass, the mass of the support - add the same numbers in the same order)
@@ -523,6 +516,137 @@ __device__ int warp_nucleus(const float* val, int n, double inv_t, double top_p,
   return keep;
 }
 
+// The accept phase of one slot, by the CTA that finished the slot's last row (all its threads): support and
+// log-normaliser of every row, then the sequential accept test (Algorithm 1, introspection loop) on the filtered
+// laws.  Leaves the supports, the decision and the outputs that need no random draw in global memory.
+__device__ void slot_accept(const TopkParams& P, SlotScratch& S, int b, int nv) {
+  const int q_len = nv + P.N, NP = P.N - 1;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const double inv_t = (double)P.inv_t, top_p = (double)P.top_p;
+  const uint32_t step = P.step_dev ? *P.step_dev : P.step;
+  const float* LV = P.list_val + (size_t)b * P.Q * kMaxTopK;
+  const int* LI = P.list_idx + (size_t)b * P.Q * kMaxTopK;
+  // ---- every row's support and log-normaliser (one warp per row, rows dealt round-robin)
+  if (warp < kThreads / 32) {
+    for (int rr = warp; rr < q_len; rr += kThreads / 32) {
+      int ln = ldcg_i(P.list_n + (size_t)b * P.Q + rr), bad = 0;
+      if (ln < 0) { bad = 1; ln = -1 - ln; }
+      double lse;
+      const int n = warp_nucleus<true>(LV + (size_t)rr * kMaxTopK, ln, inv_t, top_p, S.w[warp], lse);
+      if (lane == 0) {
+        S.n[rr] = n; S.bad[rr] = bad; S.lse[rr] = lse;
+        P.nuc_n[(size_t)b * P.Q + rr] = n; P.nuc_bad[(size_t)b * P.Q + rr] = bad; P.nuc_lse[(size_t)b * P.Q + rr] = lse;
+      }
+      // the inputs of the accept test at position rr + 1, whose anchor law this row is: the proposal, log p~ of it
+      // (-inf unless it is in the support) and log q~ of it
+      const int j = rr + 1;
+      if (j <= nv) {
+        const int x = P.block_tok[(size_t)b * P.Q + j];
+        float logp = -INFINITY;
+        for (int i = lane; i < n; i += 32)
+          if (ldcg_i(LI + (size_t)rr * kMaxTopK + i) == x) logp = ldcg_f(LV + (size_t)rr * kMaxTopK + i) * P.inv_t - (float)lse;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) logp = fmaxf(logp, __shfl_xor_sync(0xffffffffu, logp, off));  // at most one lane found it
+        if (lane == 0) {
+          S.x[j] = x;
+          S.logp[j] = logp;
+          float logq = 0.f;
+          if (P.q_mode == 0) {
+            const float* qs = P.q_stats + ((size_t)b * NP + j - 1) * 2;
+            logq = qs[1] - qs[0];
+          }
+          S.logq[j] = logq;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  // ---- sequential accept test
+  if (threadIdx.x == 0) {
+    uint32_t status = 0;
+    int a = nv, rej = 0;
+    for (int m = 1; m <= NP; ++m) status |= S.bad[nv + m] ? ISD_ST_NONFINITE_LOGIT : 0u;
+    for (int j = 1; j <= NP; ++j) {
+      P.out.accept[(size_t)b * NP + j - 1] = -1;
+      P.out.alpha[(size_t)b * NP + j - 1] = NAN;
+    }
+    for (int j = 1; j <= nv; ++j) {
+      const int x = S.x[j];
+      if (x < 0 || x >= P.V) { status |= ISD_ST_BAD_TOKEN_ID; a = -1; break; }
+      if (S.bad[j - 1]) status |= ISD_ST_NONFINITE_LOGIT;
+      const float logp = S.logp[j], logq = S.logq[j];
+      float al = (1.f + P.tau) * expf(logp - logq);
+      al = fminf(al, 1.f);
+      if (al != al) al = 0.f;
+      const uint4 rnd = philox4x32_10(0u, step, (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)j, P.seed_lo, P.seed_hi);
+      const float u = (float)(rnd.x >> 8) * 0x1p-24f;
+      P.out.alpha[(size_t)b * NP + j - 1] = al;
+      if (u < al) {
+        P.out.accept[(size_t)b * NP + j - 1] = 1;
+      } else {
+        P.out.accept[(size_t)b * NP + j - 1] = 0;
+        a = j - 1;
+        rej = j;
+        break;
+      }
+    }
+    if (a >= 0 && rej == 0 && S.bad[nv]) status |= ISD_ST_NONFINITE_LOGIT;
+    for (int j = 0; j < P.N; ++j) P.out.out_tok[(size_t)b * P.N + j] = -1;
+    P.out.repl_tok[b] = -1;
+    if (a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL)) {
+      P.out.accept_len[b] = 0;
+      P.out.n_emit[b] = 0;
+      atomicOr(&P.slot_status[b], status);
+      atomicOr(P.global_status, status);
+      a = -1;
+    } else {
+      P.out.accept_len[b] = a;
+      P.out.n_emit[b] = a + 1;
+      for (int j = 1; j <= a; ++j) P.out.out_tok[(size_t)b * P.N + j - 1] = P.block_tok[(size_t)b * P.Q + j];
+    }
+    P.q_dec[2 * b] = a;
+    P.q_dec[2 * b + 1] = rej;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pass 1: the top-k list of every valid row
+// ------------------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(kThreads + 32) topk_rows_kernel(const TopkParams P) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
+  const int b = blockIdx.x, r = blockIdx.y;
+  if (!P.active[b]) return;
+  const int nv = P.n_ver[b];
+  if (nv < 0 || nv > P.N - 1) return;  // flagged by the decide kernel
+  if (r >= nv + P.N) return;
+  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
+  if (!block_topk<DT>(sh, row, 0, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  const size_t base = ((size_t)b * P.Q + r) * kMaxTopK;
+  if (threadIdx.x < sh.list_n) {
+    P.list_val[base + threadIdx.x] = sh.list_val[threadIdx.x];
+    P.list_idx[base + threadIdx.x] = sh.list_idx[threadIdx.x];
+  }
+  if (threadIdx.x == 0) P.list_n[(size_t)b * P.Q + r] = sh.bad ? -1 - sh.list_n : sh.list_n;
+  // ---- the CTA that finishes the slot's last row runs the slot's accept phase (nobody waits for anybody)
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int done = atomicAdd(&P.row_ticket[b], 1);
+    sh.have = done == nv + P.N - 1;
+    if (sh.have) P.row_ticket[b] = 0;  // ready for the next launch
+  }
+  __syncthreads();
+  if (!sh.have) return;
+  __threadfence();
+  slot_accept(P, *reinterpret_cast<SlotScratch*>(sh.ring.stage), b, nv);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pass 2: everything else, one CTA per slot
+// ------------------------------------------------------------------------------------------------
 // warp-wide arg max of (score, index): highest score, lowest index on ties (the oracle scans indices upwards
 // and replaces only on a strictly greater score)
 __device__ __forceinline__ void warp_argmax(double& s, int& idx) {
@@ -543,12 +667,11 @@ template <int DT>
 __global__ void __cluster_dims__(kQSplit, 1, 1) __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkParams P) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
-  __shared__ int s_n[32], s_bad[32], s_x[32], s_rej, s_a;
-  __shared__ float s_logp[32], s_logq[32];
+  __shared__ int s_n[32], s_bad[32], s_rej, s_a;
   __shared__ double s_lse[32];
-  __shared__ double s_w[kThreads / 32][kMaxTopK];
-  // A cluster of kQSplit CTAs per slot.  All of them run the accept test (it is short); the first one writes the
-  // outputs and draws; the others only help when a rejection needs the proposal-law row, one piece of it each.
+  __shared__ double s_w[1][kMaxTopK];
+  // A cluster of kQSplit CTAs per slot.  The first one draws and writes; the others only help when a rejection
+  // needs the proposal-law row, one piece of it each.
   const int b = blockIdx.x / kQSplit, piece = blockIdx.x % kQSplit;
   const bool lead = piece == 0;
   if (!P.active[b]) return;
@@ -568,95 +691,19 @@ __global__ void __cluster_dims__(kQSplit, 1, 1) __launch_bounds__(kThreads + 32)
   const float* LV = P.list_val + (size_t)b * P.Q * kMaxTopK;
   const int* LI = P.list_idx + (size_t)b * P.Q * kMaxTopK;
 
-  // ---- every row's support and log-normaliser (one warp per row, rows dealt round-robin); first CTA only
-  if (lead && warp < kThreads / 32) {
-    for (int rr = warp; rr < q_len; rr += kThreads / 32) {
-      int ln = P.list_n[(size_t)b * P.Q + rr], bad = 0;
-      if (ln < 0) { bad = 1; ln = -1 - ln; }
-      double lse;
-      const int n = warp_nucleus(LV + (size_t)rr * kMaxTopK, ln, inv_t, top_p, s_w[warp], lse);
-      if (lane == 0) { s_n[rr] = n; s_bad[rr] = bad; s_lse[rr] = lse; }
-      // the inputs of the accept test at position rr + 1, whose anchor law this row is: the proposal, log p~ of it
-      // (-inf unless it is in the support) and log q~ of it
-      const int j = rr + 1;
-      if (j <= nv) {
-        const int x = P.block_tok[(size_t)b * P.Q + j];
-        float logp = -INFINITY;
-        for (int i = lane; i < n; i += 32)
-          if (LI[(size_t)rr * kMaxTopK + i] == x) logp = LV[(size_t)rr * kMaxTopK + i] * P.inv_t - (float)lse;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) logp = fmaxf(logp, __shfl_xor_sync(0xffffffffu, logp, off));  // at most one lane found it
-        if (lane == 0) {
-          s_x[j] = x;
-          s_logp[j] = logp;
-          float logq = 0.f;
-          if (P.q_mode == 0) {
-            const float* qs = P.q_stats + ((size_t)b * NP + j - 1) * 2;
-            logq = qs[1] - qs[0];
-          }
-          s_logq[j] = logq;
-        }
-      }
-    }
+  // ---- the row kernel has left the supports and the accept decision of the slot in global memory
+  if (threadIdx.x < q_len) {
+    s_n[threadIdx.x] = P.nuc_n[(size_t)b * P.Q + threadIdx.x];
+    s_bad[threadIdx.x] = P.nuc_bad[(size_t)b * P.Q + threadIdx.x];
+    s_lse[threadIdx.x] = P.nuc_lse[(size_t)b * P.Q + threadIdx.x];
   }
-  __syncthreads();
-  // ---- sequential accept test (Algorithm 1, introspection loop) on the filtered laws; first CTA only
-  if (lead && threadIdx.x == 0) {
-    uint32_t status = 0;
-    int a = nv, rej = 0;
-    for (int m = 1; m <= NP; ++m) status |= s_bad[nv + m] ? ISD_ST_NONFINITE_LOGIT : 0u;
-    for (int j = 1; j <= NP; ++j) {
-      if (lead) P.out.accept[(size_t)b * NP + j - 1] = -1;
-      if (lead) P.out.alpha[(size_t)b * NP + j - 1] = NAN;
-    }
-    for (int j = 1; j <= nv; ++j) {
-      const int x = s_x[j];
-      if (x < 0 || x >= P.V) { status |= ISD_ST_BAD_TOKEN_ID; a = -1; break; }
-      if (s_bad[j - 1]) status |= ISD_ST_NONFINITE_LOGIT;
-      const float logp = s_logp[j], logq = s_logq[j];
-      float al = (1.f + P.tau) * expf(logp - logq);
-      al = fminf(al, 1.f);
-      if (al != al) al = 0.f;
-      const uint4 rnd = philox4x32_10(0u, step, (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)j, P.seed_lo, P.seed_hi);
-      const float u = (float)(rnd.x >> 8) * 0x1p-24f;
-      if (lead) P.out.alpha[(size_t)b * NP + j - 1] = al;
-      if (u < al) {
-        if (lead) P.out.accept[(size_t)b * NP + j - 1] = 1;
-      } else {
-        if (lead) P.out.accept[(size_t)b * NP + j - 1] = 0;
-        a = j - 1;
-        rej = j;
-        break;
-      }
-    }
-    if (a >= 0 && rej == 0 && s_bad[nv]) status |= ISD_ST_NONFINITE_LOGIT;
-    for (int j = 0; j < P.N; ++j) if (lead) P.out.out_tok[(size_t)b * P.N + j] = -1;
-    if (lead) P.out.repl_tok[b] = -1;
-    if (a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL)) {
-      if (lead) P.out.accept_len[b] = 0;
-      if (lead) P.out.n_emit[b] = 0;
-      if (lead) atomicOr(&P.slot_status[b], status);
-      if (lead) atomicOr(P.global_status, status);
-      a = -1;
-    } else {
-      if (lead) P.out.accept_len[b] = a;
-      if (lead) P.out.n_emit[b] = a + 1;
-      for (int j = 1; j <= a; ++j) if (lead) P.out.out_tok[(size_t)b * P.N + j - 1] = P.block_tok[(size_t)b * P.Q + j];
-    }
-    s_a = a;
-    s_rej = rej;
-    P.q_dec[2 * b] = a;  // for the other CTAs of the cluster
-    P.q_dec[2 * b + 1] = rej;
-    __threadfence();
-  }
-  cooperative_groups::this_cluster().sync();  // every CTA of an active slot's cluster passes here once
-  if (!lead && threadIdx.x == 0) {
+  if (threadIdx.x == 0) {
     s_a = P.q_dec[2 * b];
     s_rej = P.q_dec[2 * b + 1];
   }
   __syncthreads();
   const int a = s_a, rej = s_rej;
-  // the helpers are needed only for the proposal-law row of a rejection (the same decision in all CTAs of the cluster)
+  // the helpers are needed only for the proposal-law row of a rejection (all CTAs of the cluster read the same decision)
   if (!lead && (a < 0 || rej == 0 || P.q_mode != 0 || P.q_prev == nullptr)) return;
 
   // ---- proposals of the MASK rows: Gumbel-max over the support (warp m - 1 draws row nv + m), or its head
@@ -753,7 +800,7 @@ __global__ void __cluster_dims__(kQSplit, 1, 1) __launch_bounds__(kThreads + 32)
     __syncthreads();
     if (warp == 0) {
       double l;
-      const int n = warp_nucleus(sh.list_val, sh.list_n, inv_t, top_p, s_w[0], l);
+      const int n = warp_nucleus<false>(sh.list_val, sh.list_n, inv_t, top_p, s_w[0], l);
       if (lane == 0) { s_n[31] = n; s_lse[31] = l; }  // rows above 30 do not exist (Q <= 31)
     }
     __syncthreads();
@@ -813,8 +860,11 @@ int isd_verify_topk_create(isd_ctx* ctx) {
   if (cudaMalloc(&ctx->topk_n, sizeof(int) * rows) != cudaSuccess) return ISD_ERR_NO_MEMORY;
   cudaMemset(ctx->topk_n, 0, sizeof(int) * rows);
   if (cudaMalloc(&ctx->topk_q_key, sizeof(unsigned long long) * (size_t)c.batch * kQSplit * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
-  if (cudaMalloc(&ctx->topk_q_n, sizeof(int) * (size_t)c.batch * (kQSplit + 2)) != cudaSuccess) return ISD_ERR_NO_MEMORY;
-  cudaMemset(ctx->topk_q_n, 0, sizeof(int) * (size_t)c.batch * (kQSplit + 2));
+  // ints: piece counts [B, kQSplit], decisions [B, 2], supports and flags [B, Q] each, row tickets [B]
+  const size_t n_ints = (size_t)c.batch * (kQSplit + 2 + 2 * ctx->Q + 1);
+  if (cudaMalloc(&ctx->topk_q_n, sizeof(int) * n_ints) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  cudaMemset(ctx->topk_q_n, 0, sizeof(int) * n_ints);
+  if (cudaMalloc(&ctx->topk_nuc_lse, sizeof(double) * rows) != cudaSuccess) return ISD_ERR_NO_MEMORY;
   cudaError_t e = cudaSuccess;
   if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_rows_kernel<ISD_LOGITS_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_rows_kernel<ISD_LOGITS_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmem);
@@ -829,11 +879,13 @@ void isd_verify_topk_destroy(isd_ctx* ctx) {
   cudaFree(ctx->topk_n);
   cudaFree(ctx->topk_q_key);
   cudaFree(ctx->topk_q_n);
+  cudaFree(ctx->topk_nuc_lse);
   ctx->topk_val = nullptr;
   ctx->topk_idx = nullptr;
   ctx->topk_n = nullptr;
   ctx->topk_q_key = nullptr;
   ctx->topk_q_n = nullptr;
+  ctx->topk_nuc_lse = nullptr;
 }
 
 int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
@@ -851,6 +903,8 @@ int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* 
   P.logits_cur = logits_cur; P.q_prev = q_prev_logits; P.out = *out;
   P.list_val = ctx->topk_val; P.list_idx = ctx->topk_idx; P.list_n = ctx->topk_n;
   P.q_key = ctx->topk_q_key; P.q_n = ctx->topk_q_n; P.q_dec = ctx->topk_q_n + (size_t)c.batch * kQSplit;
+  P.nuc_n = P.q_dec + 2 * (size_t)c.batch; P.nuc_bad = P.nuc_n + (size_t)c.batch * ctx->Q;
+  P.row_ticket = P.nuc_bad + (size_t)c.batch * ctx->Q; P.nuc_lse = ctx->topk_nuc_lse;
   const dim3 grid1(c.batch, ctx->Q);
   if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
   if (c.logits_dtype == ISD_LOGITS_BF16) {
