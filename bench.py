@@ -94,7 +94,8 @@ def algorithmic_bytes(w, ctx_len, q_len, rejecting: int):
     q_sum = int(q_len.sum().item())
     attn = int((ctx_len.to(torch.int64) + q_len).sum().item()) * kv_tok + q_sum * kv_tok \
         + q_sum * w.n_q_heads * w.head_dim * 2 * 2
-    verify = q_sum * w.vocab * lb + rejecting * 2 * w.vocab * lb
+    # a rejection re-reads the anchor row and the proposal-law row; with filtered laws both are short lists
+    verify = q_sum * w.vocab * lb + (0 if w.top_k else rejecting * 2 * w.vocab * lb)
     return attn, verify
 
 
@@ -387,7 +388,8 @@ def run_ours(args):
     rejecting = int(rej_acc[W:W + K].sum().item())
     lb = 2 if w.logits_dtype == "bf16" else 4
     attn_bytes = int(attn_bytes_acc[W:W + K].sum().item())
-    verify_bytes = positions * w.vocab * lb + rejecting * 2 * w.vocab * lb
+    rej_rows = 0 if w.top_k else 2      # full rows a rejection reads again (filtered laws: short lists instead)
+    verify_bytes = positions * w.vocab * lb + rejecting * rej_rows * w.vocab * lb
 
     # ---- end to end through the C ABI with HOST buffers: H2D of the step's inputs and D2H of its
     # results inside the timed window (fewer steps: the logits alone are > 1 GB per step)
@@ -443,7 +445,7 @@ def run_ours(args):
 
     peak, peak_kind = measured_peaks()
     attn_gbs = attn_bytes / (sum(attn_ms) / 1e3) / 1e9
-    ver_bytes_timed = ver_positions * w.vocab * lb + ver_rejecting * 2 * w.vocab * lb   # of the steps that carry the events
+    ver_bytes_timed = ver_positions * w.vocab * lb + ver_rejecting * rej_rows * w.vocab * lb   # of the steps that carry the events
     ver_gbs = ver_bytes_timed / (sum(ver_ms) / 1e3) / 1e9 if sum(ver_ms) > 0 else None
     step_bytes = attn_bytes + positions * kv_tok + verify_bytes      # + K/V append writes
     line = {

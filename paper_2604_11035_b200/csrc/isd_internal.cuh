@@ -68,7 +68,9 @@ struct isd_ctx {
   // ---- scratch of the top-k / top-p filtered verification (cfg.top_k > 0)
   float* topk_val;       // [B, Q, ISD_MAX_TOP_K]
   int* topk_idx;         // [B, Q, ISD_MAX_TOP_K]
-  int* topk_n;           // [B, Q]
+  int* topk_n;           // [B, Q]   (each of the three twice: this call's lists and the previous call's)
+  int topk_cur;          // which half the next call writes
+  const void* topk_prev_rows;  // logits_cur of the previous filtered call (whose lists the other half holds)
   unsigned long long* topk_q_key;  // [B, pieces, ISD_MAX_TOP_K] piece lists of a proposal-law row (as sort keys)
   int* topk_q_n;         // [B, pieces], then the slot decisions, supports and row tickets of the accept phase
   double* topk_nuc_lse;  // [B, Q] log-normaliser of every row's filtered law

@@ -46,6 +46,11 @@ struct TopkParams {
   float* list_val;  // [B, Q, kMaxTopK] raw logits of the row's top-k, best first
   int* list_idx;    // [B, Q, kMaxTopK]
   int* list_n;      // [B, Q] entries of the list; -1 - n when the row holds a NaN or +inf
+  // the same three of the previous call (read only), valid when q_prev is the row buffer that call selected from
+  const float* prev_val;
+  const int* prev_idx;
+  const int* prev_n;
+  int prev_valid;
   unsigned long long* q_key;  // [B, kQSplit, kMaxTopK] piece lists of the proposal-law row of a rejection
   int* q_n;                   // [B, kQSplit]
   int* q_dec;                 // [B, 2] accept length (-1: frozen) and rejected position, from the row kernel to the decide kernel
@@ -704,7 +709,7 @@ __global__ void __cluster_dims__(kQSplit, 1, 1) __launch_bounds__(kThreads + 32)
   __syncthreads();
   const int a = s_a, rej = s_rej;
   // the helpers are needed only for the proposal-law row of a rejection (all CTAs of the cluster read the same decision)
-  if (!lead && (a < 0 || rej == 0 || P.q_mode != 0 || P.q_prev == nullptr)) return;
+  if (!lead && (a < 0 || rej == 0 || P.q_mode != 0 || P.q_prev == nullptr || P.prev_valid)) return;
 
   // ---- proposals of the MASK rows: Gumbel-max over the support (warp m - 1 draws row nv + m), or its head
   if (lead && warp >= 1 && warp <= NP && warp < kThreads / 32) {
@@ -769,33 +774,46 @@ __global__ void __cluster_dims__(kQSplit, 1, 1) __launch_bounds__(kThreads + 32)
   const int x = P.block_tok[(size_t)b * P.Q + rej];
   if (P.q_mode == 0) {
     if (P.q_prev == nullptr) return;  // the caller gave no proposal-law rows
-    const char* qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + (P.q_row0[b] + rej - 1)) * (size_t)P.V * elt;
-    // every CTA of the cluster selects the top-k of its piece of the row (whole stages); their union holds the row's
-    const int stage_elems = kRowStageBytes / (int)elt;
-    const int per = ((P.V + stage_elems - 1) / stage_elems + kQSplit - 1) / kQSplit * stage_elems;
-    const int e_lo = piece * per < P.V ? piece * per : P.V;
-    const int e_hi = e_lo + per < P.V ? e_lo + per : P.V;
-    if (!block_topk<DT>(sh, qrow, e_lo, e_hi, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
-    if (threadIdx.x < sh.list_n)
-      P.q_key[((size_t)b * kQSplit + piece) * kMaxTopK + threadIdx.x] = cand_key(sh.list_val[threadIdx.x], sh.list_idx[threadIdx.x]);
-    if (threadIdx.x == 0) P.q_n[(size_t)b * kQSplit + piece] = sh.list_n;
-    __threadfence();
-    cooperative_groups::this_cluster().sync();  // every CTA of the cluster is here: the early returns above are the same for all
-    if (!lead) return;
-    if (threadIdx.x < kThreads) {
-      int total = 0;
-      for (int r = 0; r < kQSplit; ++r) {
-        const int n_r = P.q_n[(size_t)b * kQSplit + r];
-        if (threadIdx.x < n_r) sh.key[total + threadIdx.x] = P.q_key[((size_t)b * kQSplit + r) * kMaxTopK + threadIdx.x];
-        total += n_r;
+    const int q_row = P.q_row0[b] + rej - 1;
+    if (P.prev_valid) {
+      // the row was a [MASK] row of the previous call, which selected its top-k already: no second stream
+      const size_t pbase = ((size_t)b * P.Q + q_row) * kMaxTopK;
+      int pn = P.prev_n[(size_t)b * P.Q + q_row];
+      if (pn < 0) pn = -1 - pn;
+      if (threadIdx.x < pn) {
+        sh.list_val[threadIdx.x] = P.prev_val[pbase + threadIdx.x];
+        sh.list_idx[threadIdx.x] = P.prev_idx[pbase + threadIdx.x];
       }
-      worker_sync();
-      const int n = rank_select(sh.key, total, P.top_k, sh.sorted);  // total <= kQSplit * kMaxTopK = kThreads
-      if (threadIdx.x < n) {
-        sh.list_val[threadIdx.x] = key_value(sh.sorted[threadIdx.x]);
-        sh.list_idx[threadIdx.x] = key_index(sh.sorted[threadIdx.x]);
+      if (threadIdx.x == 0) sh.list_n = pn;
+    } else {
+      const char* qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + q_row) * (size_t)P.V * elt;
+      // every CTA of the cluster selects the top-k of its piece of the row (whole stages); their union holds the row's
+      const int stage_elems = kRowStageBytes / (int)elt;
+      const int per = ((P.V + stage_elems - 1) / stage_elems + kQSplit - 1) / kQSplit * stage_elems;
+      const int e_lo = piece * per < P.V ? piece * per : P.V;
+      const int e_hi = e_lo + per < P.V ? e_lo + per : P.V;
+      if (!block_topk<DT>(sh, qrow, e_lo, e_hi, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+      if (threadIdx.x < sh.list_n)
+        P.q_key[((size_t)b * kQSplit + piece) * kMaxTopK + threadIdx.x] = cand_key(sh.list_val[threadIdx.x], sh.list_idx[threadIdx.x]);
+      if (threadIdx.x == 0) P.q_n[(size_t)b * kQSplit + piece] = sh.list_n;
+      __threadfence();
+      cooperative_groups::this_cluster().sync();  // every CTA of the cluster is here: the early returns above are the same for all
+      if (!lead) return;
+      if (threadIdx.x < kThreads) {
+        int total = 0;
+        for (int r = 0; r < kQSplit; ++r) {
+          const int n_r = P.q_n[(size_t)b * kQSplit + r];
+          if (threadIdx.x < n_r) sh.key[total + threadIdx.x] = P.q_key[((size_t)b * kQSplit + r) * kMaxTopK + threadIdx.x];
+          total += n_r;
+        }
+        worker_sync();
+        const int n = rank_select(sh.key, total, P.top_k, sh.sorted);  // total <= kQSplit * kMaxTopK = kThreads
+        if (threadIdx.x < n) {
+          sh.list_val[threadIdx.x] = key_value(sh.sorted[threadIdx.x]);
+          sh.list_idx[threadIdx.x] = key_index(sh.sorted[threadIdx.x]);
+        }
+        if (threadIdx.x == 0) sh.list_n = n;
       }
-      if (threadIdx.x == 0) sh.list_n = n;
     }
     __syncthreads();
     if (warp == 0) {
@@ -855,10 +873,13 @@ static_assert(kQSplit * kMaxTopK <= kThreads, "the merge of the piece lists rank
 int isd_verify_topk_create(isd_ctx* ctx) {
   const isd_config& c = ctx->cfg;
   const size_t rows = (size_t)c.batch * ctx->Q;
-  if (cudaMalloc(&ctx->topk_val, sizeof(float) * rows * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
-  if (cudaMalloc(&ctx->topk_idx, sizeof(int) * rows * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
-  if (cudaMalloc(&ctx->topk_n, sizeof(int) * rows) != cudaSuccess) return ISD_ERR_NO_MEMORY;
-  cudaMemset(ctx->topk_n, 0, sizeof(int) * rows);
+  // two sets of lists: this call's and the previous call's
+  if (cudaMalloc(&ctx->topk_val, 2 * sizeof(float) * rows * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  if (cudaMalloc(&ctx->topk_idx, 2 * sizeof(int) * rows * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  if (cudaMalloc(&ctx->topk_n, 2 * sizeof(int) * rows) != cudaSuccess) return ISD_ERR_NO_MEMORY;
+  cudaMemset(ctx->topk_n, 0, 2 * sizeof(int) * rows);
+  ctx->topk_cur = 0;
+  ctx->topk_prev_rows = nullptr;
   if (cudaMalloc(&ctx->topk_q_key, sizeof(unsigned long long) * (size_t)c.batch * kQSplit * kMaxTopK) != cudaSuccess) return ISD_ERR_NO_MEMORY;
   // ints: piece counts [B, kQSplit], decisions [B, 2], supports and flags [B, Q] each, row tickets [B]
   const size_t n_ints = (size_t)c.batch * (kQSplit + 2 + 2 * ctx->Q + 1);
@@ -901,7 +922,17 @@ int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* 
   P.n_ver = st->n_ver; P.active = st->active; P.block_tok = st->block_tok; P.q_row0 = st->q_row0;
   P.q_stats = st->q_stats; P.slot_status = st->slot_status; P.global_status = ctx->global_status;
   P.logits_cur = logits_cur; P.q_prev = q_prev_logits; P.out = *out;
-  P.list_val = ctx->topk_val; P.list_idx = ctx->topk_idx; P.list_n = ctx->topk_n;
+  const size_t rows = (size_t)c.batch * ctx->Q;
+  const int cur = ctx->topk_cur, prv = cur ^ 1;
+  P.list_val = ctx->topk_val + cur * rows * kMaxTopK; P.list_idx = ctx->topk_idx + cur * rows * kMaxTopK;
+  P.list_n = ctx->topk_n + cur * rows;
+  P.prev_val = ctx->topk_val + prv * rows * kMaxTopK; P.prev_idx = ctx->topk_idx + prv * rows * kMaxTopK;
+  P.prev_n = ctx->topk_n + prv * rows;
+  // the proposal-law rows are the [MASK] rows of the previous step's logits: when that buffer is the one the previous
+  // call selected from, its lists are reused instead of streaming the rows again
+  P.prev_valid = (q_prev_logits != nullptr && q_prev_logits == ctx->topk_prev_rows) ? 1 : 0;
+  ctx->topk_cur = prv;
+  ctx->topk_prev_rows = logits_cur;
   P.q_key = ctx->topk_q_key; P.q_n = ctx->topk_q_n; P.q_dec = ctx->topk_q_n + (size_t)c.batch * kQSplit;
   P.nuc_n = P.q_dec + 2 * (size_t)c.batch; P.nuc_bad = P.nuc_n + (size_t)c.batch * ctx->Q;
   P.row_ticket = P.nuc_bad + (size_t)c.batch * ctx->Q; P.nuc_lse = ctx->topk_nuc_lse;

@@ -110,6 +110,33 @@ def test_filtered_selection_on_structured_rows(dtype):
     eng.close()
 
 
+def test_filtered_proposal_law_rows_cached_or_streamed():
+    # On a rejection the filtered proposal law of the rejected position is needed.  When q_prev_logits is the very
+    # buffer the previous call selected from, the lists of that call are reused; any other buffer (here: a copy)
+    # is streamed and selected again.  Both routes must give the same step, bit for bit.
+    w = Workload("qcache", batch=6, stride=4, n_q_heads=8, n_kv_heads=2, vocab=8192 + 8 * 5, ctx_min=3, ctx_max=200,
+                 logits_dtype="bf16", logit_sigma=2.0, peaked_frac=0.5, steps=6, propose_mode=0, seed=44,
+                 top_k=50, top_p=0.95)
+    runs = []
+    for copy_prev in (False, True):
+        st, eng, out = _fresh(w)
+        prev, acc, rejections = None, [], 0
+        for t in range(6):
+            n_ver_before = st["n_ver"].clone()
+            fed = prev.clone() if (copy_prev and prev is not None) else prev
+            prev, _ = _step(w, st, eng, out, t, fed)
+            rejections += int((out["accept_len"] < n_ver_before).sum())
+            acc.append([x.clone() for x in out.values()] + [st[k].clone() for k in STATE_KEYS])
+        assert eng.isd_read_status() & ~isd_pkg.binding.ST_EMPTY_RESIDUAL == 0
+        eng.close()
+        runs.append(acc)
+        assert rejections > 0
+    for a, b in zip(*runs):
+        for x, y in zip(a, b):
+            assert torch.equal(x.view(torch.uint8) if x.dtype.is_floating_point else x,
+                               y.view(torch.uint8) if y.dtype.is_floating_point else y)
+
+
 def test_temperature_and_relaxed_acceptance():
     w = Workload("temp", batch=6, stride=4, n_q_heads=8, n_kv_heads=2, vocab=2048, ctx_min=20, ctx_max=200,
                  logits_dtype="f32", logit_sigma=2.0, peaked_frac=0.5, steps=6, propose_mode=0, seed=77)
