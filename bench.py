@@ -464,7 +464,7 @@ def run_ours(args):
         "roofline": {"kernel": "attn_tc_kernel", "bound": "hbm", "achieved": attn_gbs, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": attn_gbs / peak, "frac_of_8TBs": attn_gbs / HBM_NOMINAL_GBS,
                      "traffic": None, "ms_per_launch": sum(attn_ms) / K, "bytes_per_launch": attn_bytes / K},
-        "verify_kernels": {"kernels": "topk_rows_kernel + topk_decide_kernel" if w.top_k else "verify_rows_kernel + verify_sample_kernel", "achieved_gbs": ver_gbs, "ms_per_launch": sum(ver_ms) / max(1, len(ver_ms)),
+        "verify_kernels": {"kernels": "topk_rows_kernel (+ topk_decide_kernel when proposal-law rows are streamed)" if w.top_k else "verify_rows_kernel + verify_sample_kernel", "achieved_gbs": ver_gbs, "ms_per_launch": sum(ver_ms) / max(1, len(ver_ms)),
                            "timed_on": "%d extra steps after the timed region" % len(ver_ms),
                                "frac_of_measured_copy": (ver_gbs / peak) if ver_gbs else None},
         "gpu_launches": launches, "status_word": status, "clocks": clocks, "wall_s": wall,

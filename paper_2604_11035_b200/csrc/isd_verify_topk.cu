@@ -8,13 +8,15 @@
 //   1. topk_rows_kernel    one CTA per (slot, block row): the exact top-k of the row in one stream of
 //      it (block_topk).  Per logit: a packed maximum over groups of eight and one compare against a
 //      rising bound; the few groups that reach it are re-read from L2 and ranked.  The CTA that
-//      finishes a slot's last row runs the slot's accept phase: nucleus cut and log-normaliser of
-//      every row in fp64 (the oracle's arithmetic, so the cut agrees) and the sequential accept test.
-//   2. topk_decide_kernel  one cluster of kQSplit CTAs per slot.  The first CTA: the Gumbel-max draws
-//      (residual, bonus, proposals) over the supports in fp64 with the same per-index Philox noise as
-//      the unfiltered path.  Only a rejection costs another stream: the proposal-law row of the
-//      previous step is selected again by the same routine, one piece of it per CTA of the cluster,
-//      and the first CTA merges the piece lists.
+//      finishes a slot's last row runs the rest of the slot: nucleus cut and log-normaliser of every
+//      row in fp64 (the oracle's arithmetic, so the cut agrees), the sequential accept test, and the
+//      Gumbel-max draws (residual, bonus, proposals) over the supports in fp64 with the same
+//      per-index Philox noise as the unfiltered path.  The filtered proposal law a rejection needs
+//      is a list of the previous call (kept by the context) whenever q_prev_logits is that call's
+//      buffer: then this is the only kernel.
+//   2. topk_decide_kernel  otherwise: one cluster of kQSplit CTAs per slot with a rejection selects
+//      the top-k of the proposal-law row again, one piece per CTA, and the first CTA merges the
+//      pieces and draws the replacement.
 #include "isd_internal.cuh"
 #include "isd_stream.cuh"
 
@@ -479,6 +481,7 @@ struct SlotScratch {
   float logp[32], logq[32];
   double lse[32];
   double w[kThreads / 32][kMaxTopK];
+  int a, rej;  // accept length (-1: frozen) and rejected position (0: none)
 };
 static_assert(sizeof(SlotScratch) <= sizeof(RowRing::stage), "the accept phase lives in the ring's stages");
 
@@ -611,6 +614,138 @@ __device__ void slot_accept(const TopkParams& P, SlotScratch& S, int b, int nv) 
     }
     P.q_dec[2 * b] = a;
     P.q_dec[2 * b + 1] = rej;
+    S.a = a;
+    S.rej = rej;
+  }
+  __syncthreads();
+}
+
+// warp-wide arg max of (score, index): highest score, lowest index on ties (the oracle scans indices upwards
+// and replaces only on a strictly greater score)
+__device__ __forceinline__ void warp_argmax(double& s, int& idx) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const double os = __shfl_xor_sync(0xffffffffu, s, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+    if (oi >= 0 && (idx < 0 || os > s || (os == s && oi < idx))) { s = os; idx = oi; }
+  }
+}
+
+__device__ __forceinline__ double gumbel_at(const TopkParams& P, uint32_t step, int b, uint32_t tagpos, int idx) {
+  const uint4 r = philox4x32_10((uint32_t)idx >> 2, step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
+  return gumbel_f64(philox_word(r, idx & 3));
+}
+
+// The draws of a slot, once its supports (s_n, s_lse) and its accept decision are known.  The lists are read from
+// L2: in the row kernel other CTAs of the same launch have written them.
+//
+// Proposals of the MASK rows: Gumbel-max over the support (warp m - 1 draws row nv + m), or its head.
+__device__ void draw_proposals(const TopkParams& P, const int* s_n, const double* s_lse, int b, int nv, uint32_t step) {
+  const int NP = P.N - 1, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const double inv_t = (double)P.inv_t;
+  const float* LV = P.list_val + (size_t)b * P.Q * kMaxTopK;
+  const int* LI = P.list_idx + (size_t)b * P.Q * kMaxTopK;
+  if (warp < 1 || warp >= kThreads / 32) return;
+  for (int m = warp; m <= NP; m += kThreads / 32 - 1) {
+    const int rr = nv + m, n = s_n[rr];
+    const float* v = LV + (size_t)rr * kMaxTopK;
+    const int* ix = LI + (size_t)rr * kMaxTopK;
+    double best = -INFINITY;
+    int tok = -1;
+    float ltok = NAN;
+    if (P.propose_mode == 1) {
+      if (n > 0) tok = ldcg_i(ix);
+    } else {
+      const uint32_t tagpos = (ISD_TAG_PROPOSE << 16) | (uint32_t)m;
+      for (int i = lane; i < n; i += 32) {
+        const double lp = (double)ldcg_f(v + i) * inv_t;
+        if (isinf(lp) && lp < 0) continue;
+        const int id = ldcg_i(ix + i);
+        const double sc = lp + gumbel_at(P, step, b, tagpos, id);
+        if (tok < 0 || sc > best || (sc == best && id < tok)) { best = sc; tok = id; }
+      }
+      warp_argmax(best, tok);
+    }
+    if (lane == 0) {
+      for (int i = 0; i < n; ++i)
+        if (ldcg_i(ix + i) == tok) ltok = ldcg_f(v + i) * P.inv_t;
+      P.out.new_prop_tok[(size_t)b * NP + m - 1] = tok;
+      P.out.new_q_stats[((size_t)b * NP + m - 1) * 2 + 0] = (float)s_lse[rr];
+      P.out.new_q_stats[((size_t)b * NP + m - 1) * 2 + 1] = tok >= 0 ? ltok : NAN;
+    }
+  }
+}
+
+// Bonus / free token: Gumbel-max over the support of the row of the last clean token (warp 0).
+__device__ void draw_bonus(const TopkParams& P, const int* s_n, int b, int nv, int a, uint32_t step) {
+  const int lane = threadIdx.x & 31;
+  if (threadIdx.x >= 32) return;
+  const double inv_t = (double)P.inv_t;
+  const int n = s_n[nv];
+  const float* v = P.list_val + ((size_t)b * P.Q + nv) * kMaxTopK;
+  const int* ix = P.list_idx + ((size_t)b * P.Q + nv) * kMaxTopK;
+  const uint32_t tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)(nv + 1);
+  double best = -INFINITY;
+  int tok = -1;
+  for (int i = lane; i < n; i += 32) {
+    const double lp = (double)ldcg_f(v + i) * inv_t;
+    if (isinf(lp) && lp < 0) continue;
+    const int id = ldcg_i(ix + i);
+    const double sc = lp + gumbel_at(P, step, b, tagpos, id);
+    if (tok < 0 || sc > best || (sc == best && id < tok)) { best = sc; tok = id; }
+  }
+  warp_argmax(best, tok);
+  if (lane == 0) {
+    P.out.repl_tok[b] = tok;
+    P.out.out_tok[(size_t)b * P.N + a] = tok;
+  }
+}
+
+// Replacement from normalize(max(0, p~ - q~)) over the anchor's support (warp 0).  q~: the first nq entries of
+// sh.list_* with log-normaliser lse_q (softmax q), or the point mass at the rejected token.
+__device__ void draw_residual(const TopkParams& P, const TopkShared& sh, const int* s_n, const double* s_lse, int b, int rej,
+                              int a, int nq, double lse_q, uint32_t step) {
+  const int lane = threadIdx.x & 31;
+  if (threadIdx.x >= 32) return;
+  const double inv_t = (double)P.inv_t;
+  const int x = P.block_tok[(size_t)b * P.Q + rej];
+  const int r = rej - 1, n = s_n[r];
+  const float* v = P.list_val + ((size_t)b * P.Q + r) * kMaxTopK;
+  const int* ix = P.list_idx + ((size_t)b * P.Q + r) * kMaxTopK;
+  const uint32_t tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)rej;
+  double best = -INFINITY, best_p = -INFINITY;
+  int tok = -1, tok_p = -1;  // residual draw; draw from p~ with the same noise (fallback for an empty residual)
+  for (int i = lane; i < n; i += 32) {
+    const double lp = (double)ldcg_f(v + i) * inv_t;
+    if (isinf(lp) && lp < 0) continue;
+    const int id = ldcg_i(ix + i);
+    const double g = gumbel_at(P, step, b, tagpos, id);
+    const double pi = exp(lp - s_lse[r]);
+    double qi = 0.0;
+    if (P.q_mode == 0) {
+      for (int t = 0; t < nq; ++t)
+        if (sh.list_idx[t] == id) qi = exp((double)sh.list_val[t] * inv_t - lse_q);
+    } else {
+      qi = (id == x) ? 1.0 : 0.0;
+    }
+    const double rr = pi - qi;
+    if (rr > 0.0) {
+      const double sc = log(rr) + g;
+      if (tok < 0 || sc > best || (sc == best && id < tok)) { best = sc; tok = id; }
+    }
+    const double scp = lp - s_lse[r] + g;
+    if (tok_p < 0 || scp > best_p || (scp == best_p && id < tok_p)) { best_p = scp; tok_p = id; }
+  }
+  warp_argmax(best, tok);
+  warp_argmax(best_p, tok_p);
+  if (lane == 0) {
+    if (tok < 0) {
+      tok = tok_p;
+      atomicOr(&P.slot_status[b], ISD_ST_EMPTY_RESIDUAL);
+      atomicOr(P.global_status, ISD_ST_EMPTY_RESIDUAL);
+    }
+    P.out.repl_tok[b] = tok;
+    P.out.out_tok[(size_t)b * P.N + a] = tok;
   }
 }
 
@@ -618,13 +753,19 @@ __device__ void slot_accept(const TopkParams& P, SlotScratch& S, int b, int nv) 
 // Pass 1: the top-k list of every valid row
 // ------------------------------------------------------------------------------------------------
 template <int DT>
-__global__ void __launch_bounds__(kThreads + 32) topk_rows_kernel(const TopkParams P) {
+__global__ void __launch_bounds__(kThreads + 32, 5) topk_rows_kernel(const TopkParams P) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
   const int b = blockIdx.x, r = blockIdx.y;
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
-  if (nv < 0 || nv > P.N - 1) return;  // flagged by the decide kernel
+  if (nv < 0 || nv > P.N - 1) {
+    if (r == 0 && threadIdx.x == 0) {
+      atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
+      atomicOr(P.global_status, ISD_ST_SLOT_CAPACITY);
+    }
+    return;
+  }
   if (r >= nv + P.N) return;
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
@@ -646,223 +787,101 @@ __global__ void __launch_bounds__(kThreads + 32) topk_rows_kernel(const TopkPara
   __syncthreads();
   if (!sh.have) return;
   __threadfence();
-  slot_accept(P, *reinterpret_cast<SlotScratch*>(sh.ring.stage), b, nv);
+  SlotScratch& S = *reinterpret_cast<SlotScratch*>(sh.ring.stage);
+  slot_accept(P, S, b, nv);
+  // ---- and the slot's draws, unless the proposal-law row of a rejection has to be streamed (decide kernel)
+  const uint32_t step = P.step_dev ? *P.step_dev : P.step;
+  const int a = S.a, rej = S.rej;
+  draw_proposals(P, S.n, S.lse, b, nv, step);
+  if (a < 0) return;  // frozen: no emission
+  if (rej == 0) {
+    draw_bonus(P, S.n, b, nv, a, step);
+  } else if (P.q_mode != 0) {
+    draw_residual(P, sh, S.n, S.lse, b, rej, a, 0, 0.0, step);
+  } else if (P.q_prev != nullptr && P.prev_valid) {
+    // the row was a [MASK] row of the previous call, which selected its top-k already: no second stream
+    const int q_row = P.q_row0[b] + rej - 1;
+    const size_t pbase = ((size_t)b * P.Q + q_row) * kMaxTopK;
+    int pn = P.prev_n[(size_t)b * P.Q + q_row];
+    if (pn < 0) pn = -1 - pn;
+    if (threadIdx.x < pn) {
+      sh.list_val[threadIdx.x] = P.prev_val[pbase + threadIdx.x];
+      sh.list_idx[threadIdx.x] = P.prev_idx[pbase + threadIdx.x];
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      double lse_q;
+      const int nq = warp_nucleus<false>(sh.list_val, pn, (double)P.inv_t, (double)P.top_p, S.w[0], lse_q);
+      draw_residual(P, sh, S.n, S.lse, b, rej, a, nq, lse_q, step);
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
 // Pass 2: everything else, one CTA per slot
 // ------------------------------------------------------------------------------------------------
-// warp-wide arg max of (score, index): highest score, lowest index on ties (the oracle scans indices upwards
-// and replaces only on a strictly greater score)
-__device__ __forceinline__ void warp_argmax(double& s, int& idx) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    const double os = __shfl_xor_sync(0xffffffffu, s, off);
-    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-    if (oi >= 0 && (idx < 0 || os > s || (os == s && oi < idx))) { s = os; idx = oi; }
-  }
-}
-
-__device__ __forceinline__ double gumbel_at(const TopkParams& P, uint32_t step, int b, uint32_t tagpos, int idx) {
-  const uint4 r = philox4x32_10((uint32_t)idx >> 2, step, (uint32_t)b, tagpos, P.seed_lo, P.seed_hi);
-  return gumbel_f64(philox_word(r, idx & 3));
-}
-
 template <int DT>
 __global__ void __cluster_dims__(kQSplit, 1, 1) __launch_bounds__(kThreads + 32) topk_decide_kernel(const TopkParams P) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
-  __shared__ int s_n[32], s_bad[32], s_rej, s_a;
+  __shared__ int s_n[32];
   __shared__ double s_lse[32];
-  __shared__ double s_w[1][kMaxTopK];
-  // A cluster of kQSplit CTAs per slot.  The first one draws and writes; the others only help when a rejection
-  // needs the proposal-law row, one piece of it each.
+  __shared__ double s_w[kMaxTopK];
+  // Launched only when rejections need a proposal-law row that no list of the previous call covers (softmax q,
+  // q_prev given, not the previous call's buffer).  A cluster of kQSplit CTAs per slot: each selects the top-k of
+  // one piece of the row, the first one merges the pieces and draws the replacement.  All CTAs of a cluster read
+  // the same decision, so they leave before the cluster barrier together or not at all.
   const int b = blockIdx.x / kQSplit, piece = blockIdx.x % kQSplit;
   const bool lead = piece == 0;
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
-  if (nv < 0 || nv > P.N - 1) {
-    if (threadIdx.x == 0 && lead) {
-      atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
-      atomicOr(P.global_status, ISD_ST_SLOT_CAPACITY);
-    }
-    return;
-  }
-  const int q_len = nv + P.N, NP = P.N - 1;
+  if (nv < 0 || nv > P.N - 1) return;
+  const int a = P.q_dec[2 * b], rej = P.q_dec[2 * b + 1];
+  if (a < 0 || rej == 0) return;
+  const int q_len = nv + P.N;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const double inv_t = (double)P.inv_t, top_p = (double)P.top_p;
   const uint32_t step = P.step_dev ? *P.step_dev : P.step;
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
-  const float* LV = P.list_val + (size_t)b * P.Q * kMaxTopK;
-  const int* LI = P.list_idx + (size_t)b * P.Q * kMaxTopK;
-
-  // ---- the row kernel has left the supports and the accept decision of the slot in global memory
-  if (threadIdx.x < q_len) {
+  if (lead && threadIdx.x < q_len) {
     s_n[threadIdx.x] = P.nuc_n[(size_t)b * P.Q + threadIdx.x];
-    s_bad[threadIdx.x] = P.nuc_bad[(size_t)b * P.Q + threadIdx.x];
     s_lse[threadIdx.x] = P.nuc_lse[(size_t)b * P.Q + threadIdx.x];
   }
-  if (threadIdx.x == 0) {
-    s_a = P.q_dec[2 * b];
-    s_rej = P.q_dec[2 * b + 1];
+  const int q_row = P.q_row0[b] + rej - 1;
+  const char* qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + q_row) * (size_t)P.V * elt;
+  // every CTA of the cluster selects the top-k of its piece of the row (whole stages); their union holds the row's
+  const int stage_elems = kRowStageBytes / (int)elt;
+  const int per = ((P.V + stage_elems - 1) / stage_elems + kQSplit - 1) / kQSplit * stage_elems;
+  const int e_lo = piece * per < P.V ? piece * per : P.V;
+  const int e_hi = e_lo + per < P.V ? e_lo + per : P.V;
+  if (!block_topk<DT>(sh, qrow, e_lo, e_hi, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  if (threadIdx.x < sh.list_n)
+    P.q_key[((size_t)b * kQSplit + piece) * kMaxTopK + threadIdx.x] = cand_key(sh.list_val[threadIdx.x], sh.list_idx[threadIdx.x]);
+  if (threadIdx.x == 0) P.q_n[(size_t)b * kQSplit + piece] = sh.list_n;
+  __threadfence();
+  cooperative_groups::this_cluster().sync();
+  if (!lead) return;
+  if (threadIdx.x < kThreads) {
+    int total = 0;
+    for (int r = 0; r < kQSplit; ++r) {
+      const int n_r = P.q_n[(size_t)b * kQSplit + r];
+      if (threadIdx.x < n_r) sh.key[total + threadIdx.x] = P.q_key[((size_t)b * kQSplit + r) * kMaxTopK + threadIdx.x];
+      total += n_r;
+    }
+    worker_sync();
+    const int n = rank_select(sh.key, total, P.top_k, sh.sorted);  // total <= kQSplit * kMaxTopK = kThreads
+    if (threadIdx.x < n) {
+      sh.list_val[threadIdx.x] = key_value(sh.sorted[threadIdx.x]);
+      sh.list_idx[threadIdx.x] = key_index(sh.sorted[threadIdx.x]);
+    }
+    if (threadIdx.x == 0) sh.list_n = n;
   }
   __syncthreads();
-  const int a = s_a, rej = s_rej;
-  // the helpers are needed only for the proposal-law row of a rejection (all CTAs of the cluster read the same decision)
-  if (!lead && (a < 0 || rej == 0 || P.q_mode != 0 || P.q_prev == nullptr || P.prev_valid)) return;
-
-  // ---- proposals of the MASK rows: Gumbel-max over the support (warp m - 1 draws row nv + m), or its head
-  if (lead && warp >= 1 && warp <= NP && warp < kThreads / 32) {
-    for (int m = warp; m <= NP; m += kThreads / 32 - 1) {
-      const int rr = nv + m, n = s_n[rr];
-      const float* v = LV + (size_t)rr * kMaxTopK;
-      const int* ix = LI + (size_t)rr * kMaxTopK;
-      double best = -INFINITY;
-      int tok = -1;
-      float ltok = NAN;
-      if (P.propose_mode == 1) {
-        if (n > 0) tok = ix[0];
-      } else {
-        const uint32_t tagpos = (ISD_TAG_PROPOSE << 16) | (uint32_t)m;
-        for (int i = lane; i < n; i += 32) {
-          const double lp = (double)v[i] * inv_t;
-          if (isinf(lp) && lp < 0) continue;
-          const double sc = lp + gumbel_at(P, step, b, tagpos, ix[i]);
-          if (tok < 0 || sc > best || (sc == best && ix[i] < tok)) { best = sc; tok = ix[i]; }
-        }
-        warp_argmax(best, tok);
-      }
-      if (lane == 0) {
-        for (int i = 0; i < n; ++i)
-          if (ix[i] == tok) ltok = v[i] * P.inv_t;
-        P.out.new_prop_tok[(size_t)b * NP + m - 1] = tok;
-        P.out.new_q_stats[((size_t)b * NP + m - 1) * 2 + 0] = (float)s_lse[rr];
-        P.out.new_q_stats[((size_t)b * NP + m - 1) * 2 + 1] = tok >= 0 ? ltok : NAN;
-      }
-    }
+  if (warp == 0) {
+    double lse_q;
+    const int nq = warp_nucleus<false>(sh.list_val, sh.list_n, (double)P.inv_t, (double)P.top_p, s_w, lse_q);
+    draw_residual(P, sh, s_n, s_lse, b, rej, a, nq, lse_q, step);
   }
-  if (a < 0) return;  // frozen: no emission (uniform over the CTA)
-
-  // ---- the token drawn for the emission
-  if (rej == 0) {
-    // bonus / free token: Gumbel-max over the support of the row of the last clean token
-    if (warp == 0) {
-      const int n = s_n[nv];
-      const float* v = LV + (size_t)nv * kMaxTopK;
-      const int* ix = LI + (size_t)nv * kMaxTopK;
-      const uint32_t tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)(nv + 1);
-      double best = -INFINITY;
-      int tok = -1;
-      for (int i = lane; i < n; i += 32) {
-        const double lp = (double)v[i] * inv_t;
-        if (isinf(lp) && lp < 0) continue;
-        const double sc = lp + gumbel_at(P, step, b, tagpos, ix[i]);
-        if (tok < 0 || sc > best || (sc == best && ix[i] < tok)) { best = sc; tok = ix[i]; }
-      }
-      warp_argmax(best, tok);
-      if (lane == 0) {
-        P.out.repl_tok[b] = tok;
-        P.out.out_tok[(size_t)b * P.N + a] = tok;
-      }
-    }
-    return;
-  }
-  // replacement from normalize(max(0, p~ - q~)) over the anchor's support; q~ needs the filtered proposal law,
-  // whose row (of the previous step's logits) is selected again here
-  int nq = 0;
-  double lse_q = 0.0;
-  const int x = P.block_tok[(size_t)b * P.Q + rej];
-  if (P.q_mode == 0) {
-    if (P.q_prev == nullptr) return;  // the caller gave no proposal-law rows
-    const int q_row = P.q_row0[b] + rej - 1;
-    if (P.prev_valid) {
-      // the row was a [MASK] row of the previous call, which selected its top-k already: no second stream
-      const size_t pbase = ((size_t)b * P.Q + q_row) * kMaxTopK;
-      int pn = P.prev_n[(size_t)b * P.Q + q_row];
-      if (pn < 0) pn = -1 - pn;
-      if (threadIdx.x < pn) {
-        sh.list_val[threadIdx.x] = P.prev_val[pbase + threadIdx.x];
-        sh.list_idx[threadIdx.x] = P.prev_idx[pbase + threadIdx.x];
-      }
-      if (threadIdx.x == 0) sh.list_n = pn;
-    } else {
-      const char* qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + q_row) * (size_t)P.V * elt;
-      // every CTA of the cluster selects the top-k of its piece of the row (whole stages); their union holds the row's
-      const int stage_elems = kRowStageBytes / (int)elt;
-      const int per = ((P.V + stage_elems - 1) / stage_elems + kQSplit - 1) / kQSplit * stage_elems;
-      const int e_lo = piece * per < P.V ? piece * per : P.V;
-      const int e_hi = e_lo + per < P.V ? e_lo + per : P.V;
-      if (!block_topk<DT>(sh, qrow, e_lo, e_hi, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
-      if (threadIdx.x < sh.list_n)
-        P.q_key[((size_t)b * kQSplit + piece) * kMaxTopK + threadIdx.x] = cand_key(sh.list_val[threadIdx.x], sh.list_idx[threadIdx.x]);
-      if (threadIdx.x == 0) P.q_n[(size_t)b * kQSplit + piece] = sh.list_n;
-      __threadfence();
-      cooperative_groups::this_cluster().sync();  // every CTA of the cluster is here: the early returns above are the same for all
-      if (!lead) return;
-      if (threadIdx.x < kThreads) {
-        int total = 0;
-        for (int r = 0; r < kQSplit; ++r) {
-          const int n_r = P.q_n[(size_t)b * kQSplit + r];
-          if (threadIdx.x < n_r) sh.key[total + threadIdx.x] = P.q_key[((size_t)b * kQSplit + r) * kMaxTopK + threadIdx.x];
-          total += n_r;
-        }
-        worker_sync();
-        const int n = rank_select(sh.key, total, P.top_k, sh.sorted);  // total <= kQSplit * kMaxTopK = kThreads
-        if (threadIdx.x < n) {
-          sh.list_val[threadIdx.x] = key_value(sh.sorted[threadIdx.x]);
-          sh.list_idx[threadIdx.x] = key_index(sh.sorted[threadIdx.x]);
-        }
-        if (threadIdx.x == 0) sh.list_n = n;
-      }
-    }
-    __syncthreads();
-    if (warp == 0) {
-      double l;
-      const int n = warp_nucleus<false>(sh.list_val, sh.list_n, inv_t, top_p, s_w[0], l);
-      if (lane == 0) { s_n[31] = n; s_lse[31] = l; }  // rows above 30 do not exist (Q <= 31)
-    }
-    __syncthreads();
-    nq = s_n[31];
-    lse_q = s_lse[31];
-  }
-  if (warp != 0) return;
-  const int r = rej - 1, n = s_n[r];
-  const float* v = LV + (size_t)r * kMaxTopK;
-  const int* ix = LI + (size_t)r * kMaxTopK;
-  const uint32_t tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)rej;
-  double best = -INFINITY, best_p = -INFINITY;
-  int tok = -1, tok_p = -1;  // residual draw; draw from p~ with the same noise (fallback for an empty residual)
-  for (int i = lane; i < n; i += 32) {
-    const double lp = (double)v[i] * inv_t;
-    if (isinf(lp) && lp < 0) continue;
-    const double g = gumbel_at(P, step, b, tagpos, ix[i]);
-    const double pi = exp(lp - s_lse[r]);
-    double qi = 0.0;
-    if (P.q_mode == 0) {
-      for (int t = 0; t < nq; ++t)
-        if (sh.list_idx[t] == ix[i]) qi = exp((double)sh.list_val[t] * inv_t - lse_q);
-    } else {
-      qi = (ix[i] == x) ? 1.0 : 0.0;
-    }
-    const double rr = pi - qi;
-    if (rr > 0.0) {
-      const double sc = log(rr) + g;
-      if (tok < 0 || sc > best || (sc == best && ix[i] < tok)) { best = sc; tok = ix[i]; }
-    }
-    const double scp = lp - s_lse[r] + g;
-    if (tok_p < 0 || scp > best_p || (scp == best_p && ix[i] < tok_p)) { best_p = scp; tok_p = ix[i]; }
-  }
-  warp_argmax(best, tok);
-  warp_argmax(best_p, tok_p);
-  if (lane == 0) {
-    if (tok < 0) {
-      tok = tok_p;
-      atomicOr(&P.slot_status[b], ISD_ST_EMPTY_RESIDUAL);
-      atomicOr(P.global_status, ISD_ST_EMPTY_RESIDUAL);
-    }
-    P.out.repl_tok[b] = tok;
-    P.out.out_tok[(size_t)b * P.N + a] = tok;
-  }
+  (void)lane;
 }
 
 constexpr size_t kTopkSmem = sizeof(TopkShared);
@@ -937,15 +956,17 @@ int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* 
   P.nuc_n = P.q_dec + 2 * (size_t)c.batch; P.nuc_bad = P.nuc_n + (size_t)c.batch * ctx->Q;
   P.row_ticket = P.nuc_bad + (size_t)c.batch * ctx->Q; P.nuc_lse = ctx->topk_nuc_lse;
   const dim3 grid1(c.batch, ctx->Q);
+  // a second kernel only when rejections need proposal-law rows that have to be streamed
+  const bool stream_q = c.q_mode == 0 && q_prev_logits != nullptr && !P.prev_valid;
   if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
   if (c.logits_dtype == ISD_LOGITS_BF16) {
     topk_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads + 32, kTopkSmem, stream>>>(P);
-    topk_decide_kernel<ISD_LOGITS_BF16><<<c.batch * kQSplit, kThreads + 32, kTopkSmem, stream>>>(P);
+    if (stream_q) topk_decide_kernel<ISD_LOGITS_BF16><<<c.batch * kQSplit, kThreads + 32, kTopkSmem, stream>>>(P);
   } else {
     topk_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads + 32, kTopkSmem, stream>>>(P);
-    topk_decide_kernel<ISD_LOGITS_F32><<<c.batch * kQSplit, kThreads + 32, kTopkSmem, stream>>>(P);
+    if (stream_q) topk_decide_kernel<ISD_LOGITS_F32><<<c.batch * kQSplit, kThreads + 32, kTopkSmem, stream>>>(P);
   }
   if (ctx->ev_verify1) cudaEventRecord(ctx->ev_verify1, stream);
-  ctx->launches += 2;
+  ctx->launches += stream_q ? 2 : 1;
   return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }
