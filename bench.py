@@ -95,7 +95,7 @@ def algorithmic_bytes(w, ctx_len, q_len, rejecting: int):
     attn = int((ctx_len.to(torch.int64) + q_len).sum().item()) * kv_tok + q_sum * kv_tok \
         + q_sum * w.n_q_heads * w.head_dim * 2 * 2
     # a rejection re-reads the anchor row and the proposal-law row; with filtered laws both are short lists
-    verify = q_sum * w.vocab * lb + (0 if w.top_k else rejecting * 2 * w.vocab * lb)
+    verify = q_sum * w.vocab * lb + (0 if w.top_k else rejecting * (2 if w.q_mode == 0 else 1) * w.vocab * lb)
     return attn, verify
 
 
@@ -297,6 +297,9 @@ def run_ours(args):
     if args.propose_mode is not None:
         from dataclasses import replace
         w = replace(w, propose_mode=args.propose_mode)
+    if args.q_mode is not None:
+        from dataclasses import replace
+        w = replace(w, q_mode=args.q_mode, name=w.name + f"[q_mode {args.q_mode}]")
     K, W = args.steps, args.warmup
     from dataclasses import replace
     VER_STEPS = 3   # extra untimed steps that carry the verification kernels' events
@@ -388,7 +391,8 @@ def run_ours(args):
     rejecting = int(rej_acc[W:W + K].sum().item())
     lb = 2 if w.logits_dtype == "bf16" else 4
     attn_bytes = int(attn_bytes_acc[W:W + K].sum().item())
-    rej_rows = 0 if w.top_k else 2      # full rows a rejection reads again (filtered laws: short lists instead)
+    # full rows a rejection reads again (filtered laws: short lists instead; point-mass q: no proposal-law row)
+    rej_rows = 0 if w.top_k else (2 if w.q_mode == 0 else 1)
     verify_bytes = positions * w.vocab * lb + rejecting * rej_rows * w.vocab * lb
 
     # ---- end to end through the C ABI with HOST buffers: H2D of the step's inputs and D2H of its
@@ -570,6 +574,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="workload index 0..4 (2 = batch 256, stride 8, ctx 1k-8k)")
     ap.add_argument("--propose-mode", type=int, default=None, choices=[0, 1])
+    ap.add_argument("--q-mode", type=int, default=None, choices=[0, 1],
+                    help="1: point-mass q (verification variant for argmax proposals)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-slots", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
