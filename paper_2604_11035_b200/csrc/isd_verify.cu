@@ -335,7 +335,7 @@ __device__ __forceinline__ bool row_pass(const VerifyParams& P, RowRing& R, cons
 // Pass 1: row statistics + decision
 // ------------------------------------------------------------------------------------------------
 template <int DT>
-__global__ void __launch_bounds__(kThreads + 32) verify_rows_kernel(const VerifyParams P) {
+__global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const VerifyParams P) {
   // Launch order = (split, slot, k): the rows that the sampling pass reads again come last, so that
   // they are the most recent lines in L2 when it starts.
   const int split = blockIdx.x, b = blockIdx.y, k = blockIdx.z;
