@@ -287,7 +287,7 @@ int isd_read_status(isd_ctx* ctx, uint32_t* host_status, void* cuda_stream);
 
 /* Optional instrumentation (the paper has no counterpart): cudaEvent_t handles, passed as void*,
  * that later calls record on their stream immediately before / after the attention main kernel
- * (attn_*) and the two kernels of isd_verify together (verify_*).  NULL switches a pair off.
+ * (attn_*) and the kernels of isd_verify together (verify_*).  NULL switches a pair off.
  * The events stay owned by the caller. */
 int isd_set_profile_events(isd_ctx* ctx, void* attn_start, void* attn_stop, void* verify_start,
                            void* verify_stop);
