@@ -191,8 +191,9 @@ int isd_attn(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void*
  * `step` must fit 32 bits.
  * q_prev_logits must hold what the previous step's logits_cur held (the proposals were drawn from
  * its rows).  With filtered laws (top_k > 0) the context remembers the top-k lists of the previous
- * call: when q_prev_logits is the very pointer that call got as logits_cur, the lists are reused and
- * the rows are not read again; with any other pointer the rows are read and selected again.
+ * call: when q_prev_logits is the very pointer that call got as logits_cur and `step` is that call's
+ * step + 1 (and no device step counter is set), the lists are reused and the rows are not read again;
+ * otherwise the rows are read and selected again.
  */
 int isd_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
                const void* q_prev_logits, uint64_t step, const isd_verify_out* out,

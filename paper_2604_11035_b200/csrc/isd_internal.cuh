@@ -71,6 +71,7 @@ struct isd_ctx {
   int* topk_n;           // [B, Q]   (each of the three twice: this call's lists and the previous call's)
   int topk_cur;          // which half the next call writes
   const void* topk_prev_rows;  // logits_cur of the previous filtered call (whose lists the other half holds)
+  uint32_t topk_prev_step;     // and its step number
   unsigned long long* topk_q_key;  // [B, pieces, ISD_MAX_TOP_K] piece lists of a proposal-law row (as sort keys)
   int* topk_q_n;         // [B, pieces], then the slot decisions, supports and row tickets of the accept phase
   double* topk_nuc_lse;  // [B, Q] log-normaliser of every row's filtered law

@@ -949,9 +949,12 @@ int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* 
   P.prev_n = ctx->topk_n + prv * rows;
   // the proposal-law rows are the [MASK] rows of the previous step's logits: when that buffer is the one the previous
   // call selected from, its lists are reused instead of streaming the rows again
-  P.prev_valid = (q_prev_logits != nullptr && q_prev_logits == ctx->topk_prev_rows) ? 1 : 0;
+  // (and when this call is the step right after it; with a device-resident step number the host cannot tell)
+  P.prev_valid = (q_prev_logits != nullptr && q_prev_logits == ctx->topk_prev_rows && ctx->step_counter == nullptr &&
+                  step == ctx->topk_prev_step + 1u) ? 1 : 0;
   ctx->topk_cur = prv;
   ctx->topk_prev_rows = logits_cur;
+  ctx->topk_prev_step = step;
   P.q_key = ctx->topk_q_key; P.q_n = ctx->topk_q_n; P.q_dec = ctx->topk_q_n + (size_t)c.batch * kQSplit;
   P.nuc_n = P.q_dec + 2 * (size_t)c.batch; P.nuc_bad = P.nuc_n + (size_t)c.batch * ctx->Q;
   P.row_ticket = P.nuc_bad + (size_t)c.batch * ctx->Q; P.nuc_lse = ctx->topk_nuc_lse;
