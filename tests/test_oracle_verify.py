@@ -9,6 +9,7 @@ import os
 
 import numpy as np
 import pytest
+import scipy.special
 import scipy.stats
 
 import oracle
@@ -303,3 +304,133 @@ def test_free_running_chain_matches_tpf_closed_form(N, c):
         assert abs(tpf - want) < N / steps + 1e-9
     else:
         assert abs(tpf - want) < 0.035, (tpf, want)
+
+
+# --------------------------------------------------------------------------- temperature
+def _softmax64(x):
+    x = np.asarray(x, np.float64)
+    e = np.exp(x - x.max())
+    return e / e.sum()
+
+
+@pytest.mark.parametrize("inv_t", [0.5, 2.0])
+def test_temperature_scales_both_laws_before_the_ratio_and_the_draws(inv_t):
+    # Sampling configuration of the appendix (temperature T): every law is softmax(logits / T).  The ratio
+    # and the Gumbel-max draws are written out here in numpy from the raw fp32 logits; scaling only one of
+    # the two laws, or dividing where the oracle multiplies by 1/T, changes alpha and the token laws.
+    B, N, V = 60000, 3, 6
+    Q = 2 * N - 1
+    rng = np.random.default_rng(int(inv_t * 10))
+    raw0 = rng.normal(0, 1.5, (Q, V)).astype(np.float32)
+    raw1 = rng.normal(0, 1.5, (Q, V)).astype(np.float32)
+    l0 = np.ascontiguousarray(np.broadcast_to(raw0[None], (B, Q, V)))
+    l1 = np.ascontiguousarray(np.broadcast_to(raw1[None], (B, Q, V)))
+    w = wl_tiny(B, N, V, 55)
+    s = tiny_state(B, N, V)
+    _, _, v0, _ = oracle_step(w, s, None, None, None, l0, None, 0, do_attn=False, inv_temperature=inv_t)
+    cnt = lambda t: np.bincount(t, minlength=V)
+    # NP step: free token from row 0, proposals from MASK rows 1..N-1, all at temperature T
+    assert chi2_p(cnt(v0.repl_tok), _softmax64(raw0[0].astype(np.float64) * inv_t)) > 1e-3
+    for m in range(1, N):
+        assert chi2_p(cnt(v0.new_prop_tok[:, m - 1]), _softmax64(raw0[m].astype(np.float64) * inv_t)) > 1e-3
+    # a wrong exponent would be visible: the same counts do not fit the untempered law
+    assert chi2_p(cnt(v0.repl_tok), _softmax64(raw0[0])) < 1e-6
+    _, _, v1, _ = oracle_step(w, s, None, None, None, l1, l0, 1, do_attn=False, inv_temperature=inv_t)
+    x = v0.new_prop_tok[:, 0]
+    p = _softmax64(raw1[0].astype(np.float64) * inv_t)
+    q = _softmax64(raw0[1].astype(np.float64) * inv_t)
+    assert np.allclose(v1.alpha[:, 0], np.minimum(1.0, p[x] / q[x]), rtol=1e-12)
+    # second position, where it was evaluated
+    ev = v1.accept[:, 1] >= 0
+    x2 = v0.new_prop_tok[:, 1]
+    p2 = _softmax64(raw1[1].astype(np.float64) * inv_t)
+    q2 = _softmax64(raw0[2].astype(np.float64) * inv_t)
+    assert ev.sum() > 1000
+    assert np.allclose(v1.alpha[ev, 1], np.minimum(1.0, p2[x2[ev]] / q2[x2[ev]]), rtol=1e-12)
+    # losslessness at temperature T: the finalised first token follows the tempered anchor law
+    assert chi2_p(cnt(v1.out_tok[:, 0]), p) > 1e-3
+    rej = v1.accept[:, 0] == 0
+    assert chi2_p(cnt(v1.repl_tok[rej]), np.maximum(0.0, p - q)) > 1e-3
+    assert not np.any(s["slot_status"] & oracle.ST_EMPTY_RESIDUAL)
+
+
+# --------------------------------------------------------------------------- cached proposal-law statistics
+@pytest.mark.parametrize("propose_mode", [0, 1])
+@pytest.mark.parametrize("inv_t,top_k,top_p", [(1.0, 0, 1.0), (0.7, 0, 1.0), (1.3, 5, 0.8)])
+def test_proposal_law_statistics_are_lse_and_logit_of_the_mask_rows(propose_mode, inv_t, top_k, top_p):
+    # new_q_stats[b, m-1] = {LSE(row * invT), row[x^] * invT} of MASK row n_ver + m (the two scalars the next
+    # step's accept test uses instead of re-reading the row); with a filter on, of the filtered law's support.
+    B, N, V = 7, 4, 40
+    Q = 2 * N - 1
+    rng = np.random.default_rng(17 + propose_mode)
+    lg = rng.normal(0, 2.0, (B, Q, V)).astype(np.float32)
+    w = wl_tiny(B, N, V, 3, propose_mode=propose_mode)
+    for n_ver in (0, N - 1):
+        s = tiny_state(B, N, V, n_ver=n_ver)
+        s["block_tok"][:, 1:n_ver + 1] = rng.integers(0, V, (B, n_ver))
+        prev = rng.normal(0, 2.0, (B, Q, V)).astype(np.float32)
+        _, _, v, _ = oracle_step(w, s, None, None, None, lg, prev, 4, do_attn=False, inv_temperature=inv_t,
+                                 top_k=top_k, top_p=top_p)
+        for b in range(B):
+            for m in range(1, N):
+                row = lg[b, n_ver + m].astype(np.float64) * float(np.float32(inv_t))
+                if top_k:
+                    order = np.lexsort((np.arange(V), -row))[:top_k]
+                    wgt = np.exp(row[order] - row[order[0]])
+                    reached = np.nonzero(np.cumsum(wgt) >= float(np.float32(top_p)) * wgt.sum())[0]
+                    keep = order[:int(reached[0]) + 1 if len(reached) else len(order)]
+                    support = np.zeros(V, bool)
+                    support[keep] = True
+                    row = np.where(support, row, -np.inf)
+                xh = int(v.new_prop_tok[b, m - 1])
+                assert np.isfinite(row[xh])
+                if propose_mode == 1:
+                    assert xh == int(np.argmax(row))
+                assert abs(v.new_q_stats[b, m - 1, 0] - scipy.special.logsumexp(row)) < 1e-12
+                assert v.new_q_stats[b, m - 1, 1] == row[xh]
+        # and the next step's accept test consumes exactly these two numbers through commit
+        assert np.array_equal(s["q_stats"], v.new_q_stats)
+
+
+# --------------------------------------------------------------------------- data faults
+def test_verify_status_branches_and_frozen_slots():
+    # Data faults never abort: an out-of-range proposal id or a NaN / +inf logit sets its bit on the slot,
+    # the commit leaves that slot where it was, and its neighbours advance.
+    B, N, V = 5, 3, 16
+    Q = 2 * N - 1
+    rng = np.random.default_rng(2)
+    w = wl_tiny(B, N, V, 8)
+    s = tiny_state(B, N, V)
+    l0 = rng.normal(0, 1, (B, Q, V)).astype(np.float32)
+    oracle_step(w, s, None, None, None, l0, None, 0, do_attn=False)
+    assert np.all(s["n_ver"] == N - 1)
+    l1 = rng.normal(0, 1, (B, Q, V)).astype(np.float32)
+    s["block_tok"][1, 1] = V + 2          # proposal id outside the vocabulary
+    s["block_tok"][2, 2] = -1             # negative id (reached only if the first proposal is accepted)
+    l1[3, 0, 5] = np.nan                  # NaN in an anchor row
+    l1[4, N, 0] = np.inf                  # +inf in a MASK row (-inf would be legal)
+    before = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in s.items()}
+    _, _, v, _ = oracle_step(w, s, None, None, None, l1, l0, 1, do_attn=False)
+    st = s["slot_status"]
+    assert st[0] == 0
+    assert st[1] == oracle.ST_BAD_TOKEN_ID
+    # the faulty slot's outputs stay at their defaults
+    assert v.n_emit[1] == 0 and v.accept_len[1] == 0 and v.repl_tok[1] == -1
+    assert np.all(v.out_tok[1] == -1) and np.all(v.new_prop_tok[1] == -1) and np.all(v.accept[1] == -1)
+    if v.accept[2, 0] == 1:
+        assert st[2] == oracle.ST_BAD_TOKEN_ID and v.n_emit[2] == 0
+    else:
+        assert st[2] == 0 and v.n_emit[2] == 1   # the loop stopped at the rejection before the bad id
+    assert st[3] & oracle.ST_NONFINITE_LOGIT and st[4] & oracle.ST_NONFINITE_LOGIT
+    for b in (1, 3, 4):                   # frozen by the commit: lengths, roles, block and pages unchanged
+        for k in ("ctx_len", "n_ver", "q_row0"):
+            assert s[k][b] == before[k][b], (b, k)
+        assert np.array_equal(s["block_tok"][b], before["block_tok"][b])
+        assert np.array_equal(s["page_table"][b], before["page_table"][b])
+    assert s["ctx_len"][0] == before["ctx_len"][0] + v.n_emit[0] and v.n_emit[0] >= 1
+    # -inf is a legal logit (probability zero), not a fault
+    s2 = tiny_state(B, N, V)
+    l2 = rng.normal(0, 1, (B, Q, V)).astype(np.float32)
+    l2[:, :, 3] = -np.inf
+    _, _, v2, _ = oracle_step(w, s2, None, None, None, l2, None, 0, do_attn=False)
+    assert np.all(s2["slot_status"] == 0) and np.all(v2.repl_tok != 3) and np.all(v2.new_prop_tok != 3)
