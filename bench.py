@@ -218,7 +218,7 @@ def run_model_step(args):
                    "ctx": [w.ctx_min, w.ctx_max], "l2": "flushed (512 MB write) before every step"},
         "emitted_tokens_per_s": int(emit_acc[W:].sum().item()) / t_total,
         "step_algorithmic_gbs": gbs, "step_frac_of_8TBs": gbs / HBM_NOMINAL_GBS, "step_frac_of_measured_copy": gbs / peak,
-        "gpu_launches": launches if graph is None else K * (3 * L + 3), "launches_issued_by_host": launches,
+        "gpu_launches": launches if graph is None else K * (3 * L + (3 if w.top_k else 2)), "launches_issued_by_host": launches,
         "status_word": status, "clocks": clocks,
     }
     print(json.dumps(line))
@@ -302,7 +302,10 @@ def run_ours(args):
         w = replace(w, q_mode=args.q_mode, name=w.name + f"[q_mode {args.q_mode}]")
     K, W = args.steps, args.warmup
     from dataclasses import replace
-    VER_STEPS = 3   # extra untimed steps that carry the verification kernels' events
+    VER_STEPS = 6   # instrumented steps after the timed region: 3 carry the events around the attention kernel,
+                    # 3 those around the verification kernels (an event between two kernels serialises launches
+                    # that the timed steps overlap, so the timed steps carry none)
+    ATTN_INSTR = 3
     w = replace(w, steps=max(w.steps, K + W + args.e2e_steps + VER_STEPS + 2))
     if args.sequential_pages:
         w = replace(w, shuffle_pages=False, name=w.name + "[sequential pages]")
@@ -345,9 +348,9 @@ def run_ours(args):
         flush.zero_()                                   # L2 flush: 512 MB > 126 MB L2
         sargs = eng.step_args(q=q, k_new=k, v_new=v, k_pool=st["k_pool"], v_pool=st["v_pool"], attn_out=attn_out,
                               attn_lse=None, logits_cur=cur, q_prev_logits=prev, out=out)
-        # events inside the step cost a few microseconds each: the timed steps carry only the pair around the
-        # dominant kernel (the roofline figure), the verification kernels are timed on extra steps afterwards
         if t < W + K:
+            eng.isd_set_profile_events(None, None, None, None)
+        elif t < W + K + ATTN_INSTR:
             eng.isd_set_profile_events(e_attn[t][0], e_attn[t][1], None, None)
         else:
             eng.isd_set_profile_events(None, None, e_ver[t][0], e_ver[t][1])
@@ -381,16 +384,18 @@ def run_ours(args):
     status = eng.isd_read_status()
 
     step_ms = [a.elapsed_time(b) for a, b in e_step[W:W + K]]
-    attn_ms = [a.elapsed_time(b) for a, b in e_attn[W:W + K]]
-    ver_ms = [a.elapsed_time(b) for a, b in e_ver[W + K:]]
-    ver_positions = int(pos_acc[W + K:].sum().item())
-    ver_rejecting = int(rej_acc[W + K:].sum().item())
+    attn_ms = [a.elapsed_time(b) for a, b in e_attn[W + K:W + K + ATTN_INSTR]]
+    ver_ms = [a.elapsed_time(b) for a, b in e_ver[W + K + ATTN_INSTR:]]
+    instr_step_ms = [a.elapsed_time(b) for a, b in e_step[W + K:]]
+    ver_positions = int(pos_acc[W + K + ATTN_INSTR:].sum().item())
+    ver_rejecting = int(rej_acc[W + K + ATTN_INSTR:].sum().item())
     t_total = sum(step_ms) / 1e3
     positions = int(pos_acc[W:W + K].sum().item())
     emitted = int(emit_acc[W:W + K].sum().item())
     rejecting = int(rej_acc[W:W + K].sum().item())
     lb = 2 if w.logits_dtype == "bf16" else 4
     attn_bytes = int(attn_bytes_acc[W:W + K].sum().item())
+    attn_bytes_instr = int(attn_bytes_acc[W + K:W + K + ATTN_INSTR].sum().item())
     # full rows a rejection reads again (filtered laws: short lists instead; point-mass q: no proposal-law row)
     rej_rows = 0 if w.top_k else (2 if w.q_mode == 0 else 1)
     verify_bytes = positions * w.vocab * lb + rejecting * rej_rows * w.vocab * lb
@@ -406,12 +411,10 @@ def run_ours(args):
                     if k_ in ("n_emit", "out_tok", "accept_len")}
         dq, dk, dv = [torch.empty_like(x) for x in wl.make_qkv(w, 0, dev)]
         e2e_pos, e2e_t = 0, 0.0
-        t_base = W + K
+        t_base = W + K + VER_STEPS          # the chain goes on where the instrumented steps left it
         ee = [(ev(), ev()) for _ in range(e2e_steps)]
         for i in range(e2e_steps):
             t = t_base + i
-            if t >= len(e_step):
-                pass
             q, k, v = wl.make_qkv(w, t, dev)
             cur, prev = logits[t & 1], logits[(t - 1) & 1]
             wl.make_logits(w, t, st["ctx_len"], out=cur)
@@ -448,7 +451,7 @@ def run_ours(args):
         return
 
     peak, peak_kind = measured_peaks()
-    attn_gbs = attn_bytes / (sum(attn_ms) / 1e3) / 1e9
+    attn_gbs = attn_bytes_instr / (sum(attn_ms) / 1e3) / 1e9
     ver_bytes_timed = ver_positions * w.vocab * lb + ver_rejecting * rej_rows * w.vocab * lb   # of the steps that carry the events
     ver_gbs = ver_bytes_timed / (sum(ver_ms) / 1e3) / 1e9 if sum(ver_ms) > 0 else None
     step_bytes = attn_bytes + positions * kv_tok + verify_bytes      # + K/V append writes
@@ -467,9 +470,13 @@ def run_ours(args):
         "step_frac_of_measured_copy": step_bytes / (sum(step_ms) / 1e3) / 1e9 / peak,
         "roofline": {"kernel": "attn_tc_kernel", "bound": "hbm", "achieved": attn_gbs, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": attn_gbs / peak, "frac_of_8TBs": attn_gbs / HBM_NOMINAL_GBS,
-                     "traffic": None, "ms_per_launch": sum(attn_ms) / K, "bytes_per_launch": attn_bytes / K},
+                     "traffic": None, "ms_per_launch": sum(attn_ms) / len(attn_ms),
+                     "bytes_per_launch": attn_bytes_instr / len(attn_ms),
+                     "timed_on": "%d instrumented steps right after the timed region (same chain, L2 flushed; %.3f ms per "
+                                 "instrumented step)" % (len(attn_ms), sum(instr_step_ms) / len(instr_step_ms)),
+                     "share_of_step": (sum(attn_ms) / len(attn_ms)) / (sum(step_ms) / K)},
         "verify_kernels": {"kernels": "topk_rows_kernel (+ topk_decide_kernel when proposal-law rows are streamed)" if w.top_k else "verify_rows_kernel + verify_sample_kernel", "achieved_gbs": ver_gbs, "ms_per_launch": sum(ver_ms) / max(1, len(ver_ms)),
-                           "timed_on": "%d extra steps after the timed region" % len(ver_ms),
+                           "timed_on": "%d instrumented steps after the timed region" % len(ver_ms),
                                "frac_of_measured_copy": (ver_gbs / peak) if ver_gbs else None},
         "gpu_launches": launches, "status_word": status, "clocks": clocks, "wall_s": wall,
     }
@@ -483,7 +490,7 @@ def run_ours(args):
         import re
         m = re.search(r"dram_bytes_per_algorithmic_byte = ([0-9.]+)", open(prof).read())
         if m:
-            line["roofline"]["traffic"] = float(m.group(1)) * attn_bytes / K
+            line["roofline"]["traffic"] = float(m.group(1)) * attn_bytes_instr / len(attn_ms)
             line["roofline"]["traffic_source"] = "ncu capture of B=64 case scaled by algorithmic bytes"
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(args, w)

@@ -65,6 +65,15 @@ extern "C" {
 #define ISD_ST_NONFINITE_LOGIT 16u /* NaN or +inf logit (-inf is legal)               */
 #define ISD_ST_EMPTY_RESIDUAL 32u /* informational: residual max(0,p-q) was empty in
                                      fp32, token drawn from p instead; not an error  */
+#define ISD_ST_KERNEL_TIMEOUT 0x80000000u /* a wait inside a kernel (on a shared-memory
+                                     barrier or on another CTA's readiness counter) outlasted
+                                     its time limit (isd_set_wait_limit): the CTA stopped
+                                     issuing work, drained its copies, freed what it held and
+                                     returned.  The results of that call are incomplete.  In
+                                     the verification kernels the bit is also set in
+                                     slot_status[b], so that isd_commit leaves the slot alone;
+                                     the attention and LoRA kernels report it in the global
+                                     word only (their CTAs serve many slots)               */
 
 #define ISD_LOGITS_F32 0
 #define ISD_LOGITS_BF16 1
@@ -89,7 +98,6 @@ typedef struct isd_config {
   int32_t propose_mode;       /* 0: Gumbel-max sample of the MASK row; 1: argmax
                                  (Sec. 3.3 (3))                                       */
   int32_t mask_token_id;      /* id written into [MASK] rows of the next block        */
-  int32_t attn_impl;          /* 0: default (tensor-core kernel); 1: plain FMA kernel */
   float sm_scale;             /* attention scale; <= 0 selects 1/sqrt(head_dim)       */
   float inv_temperature;      /* logits are multiplied by this (1.0 = paper default)  */
   float tau;                  /* relaxed acceptance: ratio * (1 + tau), Sec. 4.3      */
@@ -285,6 +293,15 @@ int isd_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t
 /* Synchronises the stream and copies the OR of all status bits raised since the
  * last call into *host_status (host pointer), then clears the global word. */
 int isd_read_status(isd_ctx* ctx, uint32_t* host_status, void* cuda_stream);
+
+/*
+ * Time limit of the waits inside the kernels (the paper has no counterpart).  Every device-side wait of the
+ * library -- on a shared-memory barrier of a copy ring, on a readiness counter another CTA raises -- gives up
+ * after this long (default 250 ms) and the kernel reports ISD_ST_KERNEL_TIMEOUT instead of hanging.  The
+ * limit is far above anything a healthy kernel waits for; lower it on hosts that must bound how long a
+ * faulty launch can hold the GPU.  milliseconds >= 1.
+ */
+int isd_set_wait_limit(isd_ctx* ctx, uint32_t milliseconds);
 
 /* Optional instrumentation (the paper has no counterpart): cudaEvent_t handles, passed as void*,
  * that later calls record on their stream immediately before / after the attention main kernel

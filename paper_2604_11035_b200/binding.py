@@ -16,17 +16,17 @@ LIB_PATH = os.path.join(_HERE, "libisd.so")
 
 ST_POOL_EXHAUSTED, ST_SLOT_CAPACITY, ST_BAD_TOKEN_ID = 1, 2, 4
 ST_BAD_PAGE_ID, ST_NONFINITE_LOGIT, ST_EMPTY_RESIDUAL = 8, 16, 32
+ST_KERNEL_TIMEOUT = 0x80000000
 
 EXPORTS = ["isd_create", "isd_destroy", "isd_attn", "isd_verify", "isd_commit", "isd_step",
            "isd_release", "isd_read_status", "isd_set_profile_events", "isd_launch_count", "isd_strerror",
-           "isd_verify_static", "isd_step_layers", "isd_set_step_counter", "isd_lora_linear"]
+           "isd_verify_static", "isd_step_layers", "isd_set_step_counter", "isd_lora_linear", "isd_set_wait_limit"]
 
 
 class IsdConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "batch", "stride", "n_q_heads", "n_kv_heads", "head_dim", "page_size", "vocab",
-        "max_pages_per_slot", "num_pages", "logits_dtype", "q_mode", "propose_mode", "mask_token_id",
-        "attn_impl")] + [("sm_scale", C.c_float), ("inv_temperature", C.c_float), ("tau", C.c_float),
+        "max_pages_per_slot", "num_pages", "logits_dtype", "q_mode", "propose_mode", "mask_token_id")] + [("sm_scale", C.c_float), ("inv_temperature", C.c_float), ("tau", C.c_float),
                          ("seed", C.c_uint64), ("top_k", C.c_int32), ("top_p", C.c_float)]
 
 
@@ -88,6 +88,8 @@ def load():
         lib.isd_set_step_counter.restype = C.c_int
         lib.isd_lora_linear.argtypes = [vp, C.POINTER(IsdLoraArgs), vp]
         lib.isd_lora_linear.restype = C.c_int
+        lib.isd_set_wait_limit.argtypes = [vp, C.c_uint32]
+        lib.isd_set_wait_limit.restype = C.c_int
         lib.isd_launch_count.argtypes = [vp]
         lib.isd_launch_count.restype = C.c_int64
         lib.isd_strerror.argtypes = [C.c_int]
@@ -141,15 +143,15 @@ class Isd:
     """One ISD context (scratch owner).  Methods mirror the C entry points by name."""
 
     def __init__(self, *, batch, stride, n_q_heads, n_kv_heads, vocab, max_pages_per_slot, num_pages,
-                 logits_dtype, head_dim=128, page_size=16, q_mode=0, propose_mode=1, mask_token_id=None,
-                 attn_impl=0, sm_scale=0.0, inv_temperature=1.0, tau=0.0, seed=0, top_k=0, top_p=1.0):
+                 logits_dtype, head_dim=128, page_size=16, q_mode=0, propose_mode=0, mask_token_id=None,
+                 sm_scale=0.0, inv_temperature=1.0, tau=0.0, seed=0, top_k=0, top_p=1.0):
         if not torch.cuda.is_available():
             raise IsdError("a CUDA device is required (there is no CPU path)")
         self.lib = load()
         ld = {"f32": 0, "bf16": 1, torch.float32: 0, torch.bfloat16: 1, 0: 0, 1: 1}[logits_dtype]
         self.cfg = IsdConfig(batch, stride, n_q_heads, n_kv_heads, head_dim, page_size, vocab,
                              max_pages_per_slot, num_pages, ld, q_mode, propose_mode,
-                             vocab - 1 if mask_token_id is None else mask_token_id, attn_impl,
+                             vocab - 1 if mask_token_id is None else mask_token_id,
                              sm_scale, inv_temperature, tau, seed, top_k, top_p)
         self.ctx = C.c_void_p()
         _check(self.lib.isd_create(C.byref(self.cfg), C.byref(self.ctx)), "isd_create")
@@ -227,6 +229,10 @@ class Isd:
     def isd_set_step_counter(self, counter):
         """`counter`: a CUDA uint32 / int32 tensor of one element, or None."""
         _check(self.lib.isd_set_step_counter(self.ctx, _ptr(counter)), "isd_set_step_counter")
+
+    def isd_set_wait_limit(self, milliseconds: int):
+        """Time limit of every wait inside the kernels (default 250 ms); see include/isd.h."""
+        _check(self.lib.isd_set_wait_limit(self.ctx, int(milliseconds)), "isd_set_wait_limit")
 
     def isd_release(self, st, slots):
         s = self.state_struct(st)

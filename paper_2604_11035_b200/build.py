@@ -8,9 +8,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libisd.so")
-SOURCES = ["isd_api.cu", "isd_verify.cu", "isd_verify_topk.cu", "isd_commit.cu", "isd_attn_plain.cu", "isd_attn_tc.cu", "isd_lora_tc.cu"]
+SOURCES = ["isd_api.cu", "isd_verify.cu", "isd_verify_topk.cu", "isd_commit.cu", "isd_kv_append.cu", "isd_attn_tc.cu", "isd_lora_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-              "-Xcompiler", "-fPIC", "--use_fast_math=false"]
+              "-Xcompiler", "-fPIC"]
 
 
 def _stale() -> bool:
@@ -25,13 +25,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
+    flags = list(NVCC_FLAGS)
     if verbose:
         flags += ["-Xptxas", "-v"]
-    if os.environ.get("ISD_DEBUG_TIMING"):
-        flags += ["-DISD_DEBUG_TIMING"]
-    if os.environ.get("ISD_EXTRA_DEFS"):
-        flags += os.environ["ISD_EXTRA_DEFS"].split()
     objs = []
     procs = []
     for src in SOURCES:

@@ -5,8 +5,6 @@
 
 #include "isd_internal.cuh"
 
-int isd_launch_kv_append(isd_ctx* ctx, const isd_batch_state* st, const void* k_new, const void* v_new,
-                         void* k_pool, void* v_pool, cudaStream_t stream);
 int isd_attn_tc_create(isd_ctx* ctx);
 void isd_attn_tc_destroy(isd_ctx* ctx);
 
@@ -50,7 +48,6 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
     return ISD_ERR_INVALID_ARG;
   if (c.logits_dtype != ISD_LOGITS_F32 && c.logits_dtype != ISD_LOGITS_BF16) return ISD_ERR_INVALID_ARG;
   if (c.q_mode < 0 || c.q_mode > 1 || c.propose_mode < 0 || c.propose_mode > 1) return ISD_ERR_INVALID_ARG;
-  if (c.attn_impl < 0 || c.attn_impl > 1) return ISD_ERR_INVALID_ARG;
   if (!(c.inv_temperature > 0.f) || !(c.tau >= 0.f)) return ISD_ERR_INVALID_ARG;
   if (c.top_k < 0 || (c.top_k > 0 && !(c.top_p > 0.f && c.top_p <= 1.f))) return ISD_ERR_INVALID_ARG;
   if (c.top_k > ISD_MAX_TOP_K) return ISD_ERR_UNSUPPORTED;
@@ -66,6 +63,7 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   ctx->G = G;
   ctx->sm_scale = c.sm_scale > 0.f ? c.sm_scale : 1.0f / sqrtf((float)c.head_dim);
   ctx->launches = 0;
+  ctx->wait_ns = ISD_DEFAULT_WAIT_NS;
   if (cudaGetDevice(&ctx->device) != cudaSuccess) { delete ctx; return ISD_ERR_CUDA; }
   int sms = 0;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
@@ -76,19 +74,14 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   const int target = ctx->num_sms * 4;
   int rs = (target + rows - 1) / rows;
   const int max_by_len = (c.vocab + 8191) / 8192;  // keep at least 8k elements per CTA
-#ifdef ISD_ROW_SPLITS_MIN
-  rs = rs < ISD_ROW_SPLITS_MIN ? ISD_ROW_SPLITS_MIN : rs;
-#endif
   rs = rs < 1 ? 1 : rs;
   rs = rs > 16 ? 16 : rs;
   rs = rs > max_by_len ? max_by_len : rs;
   ctx->row_splits = rs;
   // every slot samples one row (bonus token or residual replacement; N rows with sampled proposals)
   // in the second pass; those passes are light, so they are cut as finely as the row length allows
-#ifndef ISD_SAMPLE_SPLITS
-#define ISD_SAMPLE_SPLITS 4
-#endif
-  int ps = ISD_SAMPLE_SPLITS;
+  // (four pieces per row: every further piece re-learns the running best score; eight cost 45 % more)
+  int ps = 4;
   ps = ps > max_by_len ? max_by_len : ps;
   ctx->sample_splits = ps;
 
@@ -101,7 +94,9 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   if (rc == ISD_OK) rc = dev_alloc(&ctx->row_arg, (size_t)rows);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->lse_p_rej, c.batch);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->global_status, 1);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->step_ticket, 1);
   if (rc == ISD_OK) {
+    cudaMemset(ctx->step_ticket, 0, sizeof(int));
     cudaMemset(ctx->row_ticket, 0, sizeof(int) * c.batch);
     cudaMemset(ctx->samp_ticket, 0, sizeof(int) * c.batch * c.stride);
     cudaMemset(ctx->reject_pos, 0xFF, sizeof(int) * c.batch);
@@ -110,7 +105,7 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   }
   if (rc == ISD_OK && c.top_k > 0) rc = isd_verify_topk_create(ctx);
   if (rc == ISD_OK) rc = isd_lora_create(ctx);
-  if (rc == ISD_OK && c.attn_impl == 0) rc = isd_attn_tc_create(ctx);
+  if (rc == ISD_OK) rc = isd_attn_tc_create(ctx);
   if (rc == ISD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ISD_ERR_CUDA;
   if (rc != ISD_OK) {
     isd_destroy(ctx);
@@ -134,6 +129,7 @@ int isd_destroy(isd_ctx* ctx) {
   cudaFree(ctx->row_arg);
   cudaFree(ctx->lse_p_rej);
   cudaFree(ctx->global_status);
+  cudaFree(ctx->step_ticket);
   delete ctx;
   return ISD_OK;
 }
@@ -148,8 +144,6 @@ int isd_attn(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void*
       !aligned16(attn_out))
     return ISD_ERR_ALIGNMENT;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
-  if (ctx->cfg.attn_impl == 1)
-    return isd_launch_attn_plain(ctx, st, q, k_new, v_new, k_pool, v_pool, attn_out, attn_lse, s);
   rc = isd_launch_kv_append(ctx, st, k_new, v_new, k_pool, v_pool, s);
   if (rc != ISD_OK) return rc;
   return isd_launch_attn_tc(ctx, st, q, k_new, v_new, k_pool, v_pool, attn_out, attn_lse, s);
@@ -181,13 +175,31 @@ int isd_commit(isd_ctx* ctx, isd_batch_state* st, const isd_verify_out* out, voi
   return isd_launch_commit(ctx, st, out, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
+// Verification followed by the commit.  With plain softmax laws the last CTA of the sampling kernel commits
+// (no kernel of its own for it); the filtered path keeps the commit kernel.
+static int verify_then_commit(isd_ctx* ctx, isd_batch_state* st, const void* logits_cur, const void* q_prev_logits,
+                              uint64_t step, const isd_verify_out* out, void* cuda_stream) {
+  if (ctx->cfg.top_k > 0) {
+    const int rc = isd_verify(ctx, st, logits_cur, q_prev_logits, step, out, cuda_stream);
+    if (rc != ISD_OK) return rc;
+    return isd_commit(ctx, st, out, cuda_stream);
+  }
+  int rc = check_state(st);
+  if (rc != ISD_OK) return rc;
+  rc = check_out(ctx, out);
+  if (rc != ISD_OK) return rc;
+  if (!logits_cur || step > 0xFFFFFFFFull) return ISD_ERR_INVALID_ARG;
+  if (ctx->cfg.stride > 1 && !st->q_stats) return ISD_ERR_INVALID_ARG;
+  if (!aligned16(logits_cur) || (q_prev_logits && !aligned16(q_prev_logits))) return ISD_ERR_ALIGNMENT;
+  return isd_launch_verify(ctx, st, logits_cur, q_prev_logits, (uint32_t)step, out,
+                           reinterpret_cast<cudaStream_t>(cuda_stream), st);
+}
+
 int isd_step(isd_ctx* ctx, isd_batch_state* st, const isd_step_args* a, uint64_t step, void* cuda_stream) {
   if (!ctx || !a) return ISD_ERR_INVALID_ARG;
   int rc = isd_attn(ctx, st, a->q, a->k_new, a->v_new, a->k_pool, a->v_pool, a->attn_out, a->attn_lse, cuda_stream);
   if (rc != ISD_OK) return rc;
-  rc = isd_verify(ctx, st, a->logits_cur, a->q_prev_logits, step, &a->out, cuda_stream);
-  if (rc != ISD_OK) return rc;
-  return isd_commit(ctx, st, &a->out, cuda_stream);
+  return verify_then_commit(ctx, st, a->logits_cur, a->q_prev_logits, step, &a->out, cuda_stream);
 }
 
 int isd_step_layers(isd_ctx* ctx, isd_batch_state* st, const isd_layer_args* layers, int32_t n_layers,
@@ -200,9 +212,7 @@ int isd_step_layers(isd_ctx* ctx, isd_batch_state* st, const isd_layer_args* lay
     const int rc = isd_attn(ctx, st, a.q, a.k_new, a.v_new, a.k_pool, a.v_pool, a.attn_out, a.attn_lse, cuda_stream);
     if (rc != ISD_OK) return rc;
   }
-  int rc = isd_verify(ctx, st, logits_cur, q_prev_logits, step, out, cuda_stream);
-  if (rc != ISD_OK) return rc;
-  return isd_commit(ctx, st, out, cuda_stream);
+  return verify_then_commit(ctx, st, logits_cur, q_prev_logits, step, out, cuda_stream);
 }
 
 int isd_lora_linear(isd_ctx* ctx, const isd_lora_args* a, void* cuda_stream) {
@@ -212,6 +222,12 @@ int isd_lora_linear(isd_ctx* ctx, const isd_lora_args* a, void* cuda_stream) {
   if (!aligned16(a->x) || !aligned16(a->w) || !aligned16(a->a) || !aligned16(a->b) || !aligned16(a->t) || !aligned16(a->y))
     return ISD_ERR_ALIGNMENT;
   return isd_launch_lora_linear(ctx, a, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int isd_set_wait_limit(isd_ctx* ctx, uint32_t milliseconds) {
+  if (!ctx || milliseconds == 0) return ISD_ERR_INVALID_ARG;
+  ctx->wait_ns = (unsigned long long)milliseconds * 1000000ull;
+  return ISD_OK;
 }
 
 int isd_set_step_counter(isd_ctx* ctx, uint32_t* device_counter) {

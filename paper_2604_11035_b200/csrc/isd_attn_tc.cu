@@ -28,17 +28,12 @@
 
 #include "isd_internal.cuh"
 
-#define ISD_ST_KERNEL_TIMEOUT 0x80000000u
-
 namespace {
 
 constexpr int kTile = 128;                 // keys per tile
 constexpr int kStageBytes = 32768;         // one K or V tile: [half(2)][page(8)][tok(16)][128 B]
 constexpr int kStages = 6;
-#ifndef ISD_SEG_COST
-#define ISD_SEG_COST 4
-#endif
-constexpr int kSegCost = ISD_SEG_COST;  // fixed cost of a segment in units of one tile's time (split axis)
+constexpr int kSegCost = 4;  // fixed cost of a segment in units of one tile's time (split axis), measured
 constexpr int kThreads = 256;
 constexpr int kProducerWarps = 3;        // warps 4..6 issue the TMA copies round-robin, warp 7 issues the MMAs
 constexpr int kSmRing = 0;
@@ -52,7 +47,6 @@ constexpr int kSmPrefix = kSmXchg + 12288;  // tile prefix over slots when the b
 constexpr int kMaxSmemPrefixSlots = 1024;
 constexpr int kSmSlot = kSmPrefix + (kMaxSmemPrefixSlots + 1) * 4 + 12;  // per slot: ctx_len | q_len << 24 (with the prefix)
 constexpr int kSmemBytes = kSmSlot + kMaxSmemPrefixSlots * 4;
-constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -77,6 +71,7 @@ struct TcParams {
   float* part_o;     // [ctas * 2][128][128]
   float* part_ml;    // [ctas * 2][128][2]
   int num_ctas;
+  unsigned long long wait_ns;  // time limit of a device-side wait
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -102,25 +97,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-#ifdef ISD_DEBUG_TIMING
-// cycles spent waiting, per CTA: [0] producer on EMPTY, [1] MMA on K FULL, [2] MMA on V FULL, [3] MMA on
-// S buffer free, [4] MMA on P ready, [5] softmax on S ready, [6] softmax busy, [7] total
-__device__ unsigned long long g_isd_dbg[160 * 12];
-#define DBG_T0() const long long _t0 = clock64()
-#define DBG_ADD(slot) dbg_acc[slot] += clock64() - _t0
-#else
-#define DBG_T0()
-#define DBG_ADD(slot)
-#endif
 
-// Bounded wait: returns false (and raises the abort flag) when the limit is reached.
+// Bounded wait: returns false (and raises the abort flag) when the time limit is reached or another thread of
+// the CTA has given up.  The limit (nanoseconds) sits in shared memory two words behind the abort flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long budget = *reinterpret_cast<const volatile unsigned long long*>(abort_flag + 2);
+  return isd_bounded_wait(budget, abort_flag, [&]() { return mbar_try_wait(bar, parity); });
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
@@ -344,6 +327,8 @@ __device__ void block_tile_prefix(const TcParams& P, int* sm_prefix, int* sm_slo
 // Plan for batches too large for the in-kernel prefix: tiles per slot and their exclusive prefix
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) attn_plan_kernel(const TcParams P) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ int sm_warp[33];
   __shared__ int sm_carry;
   if (threadIdx.x == 0) sm_carry = 0;
@@ -398,9 +383,6 @@ struct SoftmaxCtx {
   volatile int* abort_flag;
   uint32_t tmem_s0, tmem_o, tmem_q;
   uint32_t n, seg;
-#ifdef ISD_DEBUG_TIMING
-  long long* dbg;
-#endif
 };
 
 __device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -456,9 +438,6 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
   const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
   volatile int* abort_flag = sc.abort_flag;
   auto bar = [&](int i) { return sc.bar_base + 8u * (uint32_t)i; };
-#ifdef ISD_DEBUG_TIMING
-  long long* dbg_acc = sc.dbg;
-#endif
   const int cnt = sg.j1 - sg.j0;
   const int rows_valid = sg.q_len * P.G;
   const int r = v / P.G, hg = v % P.G;
@@ -477,13 +456,10 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
     const uint32_t nn = sc.n + i;
     const int j = sg.j0 + i;
     {
-      DBG_T0();
       ok = mbar_wait(bar(BAR_SFULL + (nn & 1u)), (nn >> 1) & 1u, abort_flag);
-      DBG_ADD(5);
     }
     if (!ok) break;
     tc_fence_after();
-    DBG_T0();
     uint32_t sv[C];
     const uint32_t ts = sc.tmem_s0 + (nn & 1u) * 128u + lane_base;
 #pragma unroll
@@ -560,20 +536,13 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
       unpack2(add2(acc[2], acc[3]), b0, b1);
       lsum = (a0 + a1) + (b0 + b1);
     }
-#ifdef ISD_DEBUG_TIMING
-    const long long _t1 = clock64();
-#endif
     TMEM_ST32(ts, pk, 0);
     TMEM_ST32(ts + 32, pk, 32);
     tmem_wait_st();
-#ifdef ISD_DEBUG_TIMING
-    dbg_acc[11] += clock64() - _t1;
-#endif
     l += lsum;
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(bar(BAR_PFULL + (nn & 1u)));
-    DBG_ADD(6);
   }
   if (!ok) return false;
   if (sg_next != nullptr) stage_q(P, *sg_next, sc, sc.seg + 1);
@@ -684,11 +653,8 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   const int cta = blockIdx.x;
   auto bar = [&](int i) { return bar_base + 8u * (uint32_t)i; };
 
-  if (sm_base & 1023u) {  // the swizzled layouts below assume a 1 KiB aligned window
-    if (threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
-    return;
-  }
-  // ---- setup: barriers, TMEM, zero the ring (stale V rows of a ragged tile must be finite)
+  // ---- setup that touches nothing an earlier kernel wrote (it runs while the K/V append drains): barriers,
+  // TMEM, zero the ring (stale V rows of a ragged tile must be finite)
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_SFULL + i), 1); mbar_init(bar(BAR_PFULL + i), 4); }
@@ -696,7 +662,8 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
     mbar_init(bar(BAR_ODONE + 1), 1);
     mbar_init(bar(BAR_OFREE), 4);
     mbar_init(bar(BAR_QFULL), 4);
-    *abort_flag = 0;
+    *abort_flag = (sm_base & 1023u) ? 1 : 0;  // the swizzled layouts below assume a 1 KiB aligned window
+    *reinterpret_cast<volatile unsigned long long*>(abort_flag + 2) = P.wait_ns;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   {
@@ -709,6 +676,8 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   }
   fence_async_smem();
   tc_fence_before();
+  pdl_wait();               // the block's K/V rows are in the pages from here on
+  pdl_launch_dependents();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
@@ -721,12 +690,6 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
     prefix = sm_prefix;
     slot_info = sm_slot;
   }
-#ifdef ISD_DEBUG_TIMING
-  long long dbg_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-  const long long dbg_start = clock64();
-  unsigned long long dbg_gt0;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(dbg_gt0));
-#endif
   const uint32_t tmem_s0 = tmem + kTmS, tmem_o = tmem + kTmO, tmem_q = tmem + kTmQ;
 
   if (warp >= 4 && warp < 4 + kProducerWarps) {
@@ -759,11 +722,8 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
         const uint32_t s = fill % kStages, ph = (fill / kStages) & 1u;
         if (fill % kProducerWarps == pw) {
           {
-            DBG_T0();
             if (!mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag)) return false;
-            DBG_ADD(0);
           }
-          DBG_T0();
           if (lane == 0) mbar_arrive_expect_tx(bar(BAR_FULL + s), (uint32_t)valid * 4096u);
           __syncwarp();
           const int pg = lane >> 1, half = lane & 1;
@@ -773,7 +733,6 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
             tma_load_3d(dst, is_v ? &tmap_v : &tmap_k, half * 64, 0, pid * P.Hkv + sg.g, bar(BAR_FULL + s));
           }
           __syncwarp();
-          DBG_ADD(3);
         }
         ++fill;
         if (is_v && (i & 3) == 3) {  // V(i) is the last user of chunk i / 4
@@ -813,14 +772,11 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
       auto qk = [&](uint32_t nn) -> bool {
         const uint32_t s = cons % kStages, ph = (cons / kStages) & 1u;
         {
-          DBG_T0();
           if (!mbar_wait(bar(BAR_FULL + s), ph, abort_flag)) return false;
-          DBG_ADD(1);
         }
         // S[nn & 1] is free: QK(nn) follows PV(nn-2) in issue order, and PV(nn-2) was issued only after
         // the softmax warps had read S(nn-2) and stored P(nn-2) over it
         tc_fence_after();
-        DBG_T0();
         if (elect_one()) {
           const uint32_t kb = sm_base + kSmRing + s * kStageBytes;
 #pragma unroll
@@ -831,7 +787,6 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
           tc_commit(bar(BAR_EMPTY + s));
           tc_commit(bar(BAR_SFULL + (nn & 1u)));
         }
-        DBG_ADD(8);
         __syncwarp();
         ++cons;
         return true;
@@ -839,18 +794,13 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
       auto pv = [&](uint32_t nn, bool first) -> bool {
         const uint32_t s = cons % kStages, ph = (cons / kStages) & 1u;
         {
-          DBG_T0();
           if (!mbar_wait(bar(BAR_FULL + s), ph, abort_flag)) return false;
-          DBG_ADD(2);
         }
         {
-          DBG_T0();
           if (!mbar_wait(bar(BAR_PFULL + (nn & 1u)), (nn >> 1) & 1u, abort_flag)) return false;
-          DBG_ADD(4);
         }
         if (first && seg > 0 && !mbar_wait(bar(BAR_OFREE), (seg - 1u) & 1u, abort_flag)) return false;
         tc_fence_after();
-        DBG_T0();
         if (elect_one()) {
           const uint32_t vb = sm_base + kSmRing + s * kStageBytes;
           const uint32_t pt_ = tmem_s0 + (nn & 1u) * 128u;
@@ -861,7 +811,6 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
           tc_commit(bar(BAR_EMPTY + s));
           tc_commit(bar(BAR_ODONE + (nn & 1u)));
         }
-        DBG_ADD(9);
         __syncwarp();
         ++cons;
         return true;
@@ -883,9 +832,6 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
     sc.smem = smem; sc.bar_base = bar_base; sc.abort_flag = abort_flag;
     sc.tmem_s0 = tmem_s0; sc.tmem_o = tmem_o; sc.tmem_q = tmem_q;
     sc.n = 0; sc.seg = 0;
-#ifdef ISD_DEBUG_TIMING
-    sc.dbg = dbg_acc;
-#endif
     bool ok = true;
     Segment sg_next;
     bool have = it.next(P, cta, sg);
@@ -903,18 +849,6 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
   }
 
   // ---- teardown
-#ifdef ISD_DEBUG_TIMING
-  if (lane == 0 && (warp == 0 || warp >= 4)) {
-    dbg_acc[7] = clock64() - dbg_start;
-    if (warp == 0) {
-      unsigned long long gt1;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1));
-      dbg_acc[2] = (long long)(gt1 - dbg_gt0);  // nanoseconds (slot 2 of warp 0 is otherwise unused)
-    }
-    for (int i = 0; i < 12; ++i)
-      if (dbg_acc[i]) g_isd_dbg[cta * 12 + i] = dbg_acc[i];
-  }
-#endif
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
@@ -935,6 +869,8 @@ attn_tc_kernel(const TcParams P, const __grid_constant__ CUtensorMap tmap_k, con
 constexpr int kCombineThreads = 1024;
 __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const TcParams P) {
   const int c0 = blockIdx.x;
+  pdl_wait();
+  pdl_launch_dependents();
   const long long total = (long long)P.tile_prefix[P.B] * P.Hkv;
   if (total == 0) return;
   const long long per = (total + P.num_ctas - 1) / P.num_ctas;
@@ -1067,11 +1003,6 @@ struct TcHost {
 
 }  // namespace
 
-#ifdef ISD_DEBUG_TIMING
-extern "C" int isd_debug_timing(unsigned long long* host_out, int n) {
-  return cudaMemcpyFromSymbol(host_out, g_isd_dbg, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 int isd_attn_tc_create(isd_ctx* ctx) {
   TcHost* h = new (std::nothrow) TcHost();
@@ -1132,11 +1063,14 @@ int isd_launch_attn_tc(isd_ctx* ctx, const isd_batch_state* st, const void* q, c
   P.q = (const __nv_bfloat16*)q; P.out = (__nv_bfloat16*)out; P.lse = lse;
   P.tile_prefix = h->tile_prefix; P.part_o = ctx->attn_part_o; P.part_ml = ctx->attn_part_ml;
   P.num_ctas = ctx->attn_ctas;
-  if (c.batch > kMaxSmemPrefixSlots) attn_plan_kernel<<<1, 1024, 0, stream>>>(P);
+  P.wait_ns = ctx->wait_ns;
+  cudaError_t e = cudaSuccess;
+  if (c.batch > kMaxSmemPrefixSlots) e = isd_launch_pdl(attn_plan_kernel, dim3(1), dim3(1024), 0, stream, P);
   if (ctx->ev_attn0) cudaEventRecord(ctx->ev_attn0, stream);
-  attn_tc_kernel<<<ctx->attn_ctas, kThreads, kSmemBytes, stream>>>(P, pm->map_k, pm->map_v);
+  if (e == cudaSuccess)
+    e = isd_launch_pdl(attn_tc_kernel, dim3(ctx->attn_ctas), dim3(kThreads), kSmemBytes, stream, P, pm->map_k, pm->map_v);
   if (ctx->ev_attn1) cudaEventRecord(ctx->ev_attn1, stream);
-  attn_combine_kernel<<<ctx->attn_ctas, kCombineThreads, 0, stream>>>(P);
+  if (e == cudaSuccess) e = isd_launch_pdl(attn_combine_kernel, dim3(ctx->attn_ctas), dim3(kCombineThreads), 0, stream, P);
   ctx->launches += 2 + (c.batch > kMaxSmemPrefixSlots ? 1 : 0);
-  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+  return e == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }

@@ -17,10 +17,8 @@
 #define ISD_TAG_FINAL 1u
 #define ISD_TAG_PROPOSE 2u
 
-// internal status bit (not part of the public set): a bounded wait inside a kernel ran out
-#ifndef ISD_ST_KERNEL_TIMEOUT
-#define ISD_ST_KERNEL_TIMEOUT 0x80000000u
-#endif
+// default time limit of a device-side wait (isd_set_wait_limit changes it per context)
+#define ISD_DEFAULT_WAIT_NS 250000000ull
 
 // score gap below which two Gumbel-max candidates are re-judged in fp64
 #define ISD_TIE_EPS 1e-3f
@@ -79,6 +77,10 @@ struct isd_ctx {
   uint32_t* lora_flags;
   // ---- optional device-resident step counter (CUDA-graph replay), owned by the caller
   uint32_t* step_counter;
+  // ---- isd_step: arrivals of the last verification kernel's CTAs (the last one commits), zero between calls
+  int* step_ticket;
+  // ---- time limit of every device-side wait, nanoseconds
+  unsigned long long wait_ns;
   // ---- status
   uint32_t* global_status;  // [1]
   int64_t launches;
@@ -87,6 +89,13 @@ struct isd_ctx {
 // -------------------------------------------------------------------------------------------------
 // Device helpers
 // -------------------------------------------------------------------------------------------------
+// 32 x 32 -> 64 bit product as one instruction (both halves are needed by every Philox round)
+__device__ __forceinline__ void mul_wide_u32(uint32_t a, uint32_t b, uint32_t& hi, uint32_t& lo) {
+  uint64_t p;
+  asm("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"(a), "r"(b));
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(p));
+}
+
 __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
                                                uint32_t k0, uint32_t k1) {
 #pragma unroll
@@ -95,10 +104,39 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
       k0 += 0x9E3779B9u;
       k1 += 0xBB67AE85u;
     }
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    uint32_t hi0, lo0, hi1, lo1;
+    mul_wide_u32(0xD2511F53u, c0, hi0, lo0);
+    mul_wide_u32(0xCD9E8D57u, c2, hi1, lo1);
     const uint32_t n0 = hi1 ^ c1 ^ k0;
     const uint32_t n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+// The ten round keys of a Philox key (k0 + r * 0x9E3779B9, k1 + r * 0xBB67AE85), computed once on the host and
+// passed as kernel parameters: inside the sampling loops a round is then two wide multiplies and two three-input
+// XORs whose third operand comes straight from the constant bank.
+struct PhiloxKeys {
+  uint32_t k[20];
+};
+inline void philox_round_keys(uint64_t seed, PhiloxKeys& rk) {
+  uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    rk.k[2 * r] = k0;
+    rk.k[2 * r + 1] = k1;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+}
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKeys& rk) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0, lo0, hi1, lo1;
+    mul_wide_u32(0xD2511F53u, c0, hi0, lo0);
+    mul_wide_u32(0xCD9E8D57u, c2, hi1, lo1);
+    const uint32_t n0 = hi1 ^ c1 ^ rk.k[2 * r];
+    const uint32_t n2 = hi0 ^ c3 ^ rk.k[2 * r + 1];
     c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
   }
   return make_uint4(c0, c1, c2, c3);
@@ -174,6 +212,44 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 
 // -------------------------------------------------------------------------------------------------
+// Bounded waits.  Every device-side wait of the library (an mbarrier phase, a readiness counter written by
+// another CTA) polls through this routine: after the first 64 failed probes it reads the nanosecond clock
+// every 64 probes and gives up once `budget_ns` has passed since then.  The caller then raises
+// ISD_ST_KERNEL_TIMEOUT, stops issuing work, waits (bounded again) for its copies in flight, frees what it
+// holds and returns, so the context stays usable.  `abort_flag` (may be null) is the CTA's shared flag: a wait
+// also ends when another thread of the CTA has given up, and raises it when its own limit runs out.
+// -------------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long isd_now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+template <class Probe>
+__device__ __forceinline__ bool isd_bounded_wait(unsigned long long budget_ns, volatile int* abort_flag, Probe probe) {
+  unsigned long long t0 = 0;
+  for (uint32_t i = 1;; ++i) {
+    if (probe()) return true;
+    if ((i & 63u) == 0u) {
+      if (abort_flag && *abort_flag) return false;
+      const unsigned long long now = isd_now_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > budget_ns) {
+        if (abort_flag) *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+
+// Programmatic dependent launch: the kernels of a step are launched with the programmatic-serialisation
+// attribute, so a kernel's CTAs may become resident while the kernel before it in the stream is still draining.
+// pdl_wait() returns once that kernel has completed and its writes are visible; every kernel executes it before
+// it reads anything an earlier kernel wrote and before any return, so completion stays transitive along the chain.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// -------------------------------------------------------------------------------------------------
 // mbarrier / bulk-copy helpers for shared-memory rings (one producer thread, many consumers)
 // -------------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t ring_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -186,29 +262,23 @@ __device__ __forceinline__ void ring_mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void ring_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait on a phase parity; false when the limit expires (the caller raises a status bit and leaves).
-__device__ __forceinline__ bool ring_mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < (1u << 24); ++i) {
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    if (ok) return true;
-  }
-  return false;
-}
-// The same wait where the phase has normally completed already: one probe, then the bounded loop.
-__device__ __forceinline__ bool mbar_wait_likely(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool ring_mbar_probe(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n.reg .pred p;\n"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
       "selp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  if (__builtin_expect(ok != 0, 1)) return true;
-  return ring_mbar_wait(bar, parity);
+  return ok != 0;
+}
+// Bounded wait on a phase parity; false when the time limit expires (the caller raises a status bit and leaves).
+__device__ __forceinline__ bool ring_mbar_wait(uint32_t bar, uint32_t parity, unsigned long long budget_ns) {
+  return isd_bounded_wait(budget_ns, nullptr, [&]() { return ring_mbar_probe(bar, parity); });
+}
+// The same wait where the phase has normally completed already: one probe, then the bounded loop.
+__device__ __forceinline__ bool mbar_wait_likely(uint32_t bar, uint32_t parity, unsigned long long budget_ns) {
+  if (__builtin_expect(ring_mbar_probe(bar, parity), 1)) return true;
+  return ring_mbar_wait(bar, parity, budget_ns);
 }
 // Contiguous global -> shared copy (16-byte aligned addresses, size a multiple of 16) that signals `bar`.
 __device__ __forceinline__ void ring_bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -268,11 +338,31 @@ __device__ __forceinline__ void lse_merge(float& m, float& s, float om, float os
 }
 
 // -------------------------------------------------------------------------------------------------
+// Host side: launch with the programmatic-serialisation attribute (see pdl_wait above)
+// -------------------------------------------------------------------------------------------------
+template <typename... KArgs, typename... Args>
+inline cudaError_t isd_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                  Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// -------------------------------------------------------------------------------------------------
 // Host-side launchers implemented in the .cu files
 // -------------------------------------------------------------------------------------------------
+// commit_st != nullptr: the last CTA of the last verification kernel also commits (isd_step)
 int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
                       const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
-                      cudaStream_t stream);
+                      cudaStream_t stream, isd_batch_state* commit_st = nullptr);
 int isd_verify_topk_create(isd_ctx* ctx);
 void isd_verify_topk_destroy(isd_ctx* ctx);
 int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
@@ -284,9 +374,8 @@ void isd_lora_destroy(isd_ctx* ctx);
 int isd_launch_commit(isd_ctx* ctx, isd_batch_state* st, const isd_verify_out* out, cudaStream_t stream);
 int isd_launch_release(isd_ctx* ctx, isd_batch_state* st, const int32_t* slots, int32_t n,
                        cudaStream_t stream);
-int isd_launch_attn_plain(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void* k_new,
-                          const void* v_new, void* k_pool, void* v_pool, void* out, float* lse,
-                          cudaStream_t stream);
+int isd_launch_kv_append(isd_ctx* ctx, const isd_batch_state* st, const void* k_new, const void* v_new,
+                         void* k_pool, void* v_pool, cudaStream_t stream);
 int isd_launch_attn_tc(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void* k_new,
                        const void* v_new, void* k_pool, void* v_pool, void* out, float* lse,
                        cudaStream_t stream);

@@ -1,7 +1,6 @@
-// K/V append (batched scatter of the block rows into the slot's pages, Sec. 3.3 (2)) and a plain
-// CUDA-core attention kernel.  The plain kernel is the slow, obviously-correct device path
-// (attn_impl = 1): one CTA per (slot, block row, query head), fp32 FMA, online softmax per warp.
-// The tensor-core kernel in isd_attn_tc.cu is the product path.
+// K/V append: batched scatter of the block rows into the slot's pages (Sec. 3.3 (2): "KV slots are allocated
+// via a single batched scatter"; Sec. 3.3 (1): the paged-only attention kernel finds the block's own keys in the
+// pages).  Runs right before the attention kernel of isd_attn_tc.cu, which starts its set-up under it.
 #include "isd_internal.cuh"
 
 namespace {
@@ -34,6 +33,8 @@ __device__ __forceinline__ int slot_q_len(const AttnParams& P, int b) {
 // one CTA per (slot, kv head): validate the slot's page-table prefix, then scatter the block rows
 __global__ void __launch_bounds__(128) kv_append_kernel(const AttnParams P) {
   const int b = blockIdx.x, g = blockIdx.y;
+  pdl_wait();
+  pdl_launch_dependents();
   const int ql = slot_q_len(P, b);
   if (ql == 0) return;
   const int ctx = P.ctx_len[b];
@@ -89,64 +90,6 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const AttnParams P) {
   }
 }
 
-__global__ void __launch_bounds__(128) attn_plain_kernel(const AttnParams P) {
-  const int h = blockIdx.x, r = blockIdx.y, b = blockIdx.z;
-  const int ql = slot_q_len(P, b);
-  if (r >= ql) return;
-  if (P.slot_status[b] & (ISD_ST_BAD_PAGE_ID | ISD_ST_SLOT_CAPACITY)) return;
-  const int ctx = P.ctx_len[b];
-  const int g = h / P.G;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nkeys = ctx + r + 1;
-
-  const __nv_bfloat16* qp = P.q + (((size_t)b * P.Q + r) * P.Hq + h) * ISD_HEAD_DIM + lane * 4;
-  float qv[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) qv[i] = __bfloat162float(qp[i]) * P.sm_scale;
-
-  float m = -INFINITY, l = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
-  for (int j = warp; j < nkeys; j += 4) {
-    int page = P.page_table[(size_t)b * P.max_pages + j / ISD_PAGE];
-    page = min(max(page, 0), P.num_pages - 1);
-    const size_t off = (((size_t)page * P.Hkv + g) * ISD_PAGE + (j % ISD_PAGE)) * ISD_HEAD_DIM + lane * 4;
-    const uint2 kb = *reinterpret_cast<const uint2*>(P.k_pool + off);
-    float s = qv[0] * __uint_as_float(kb.x << 16) + qv[1] * __uint_as_float(kb.x & 0xFFFF0000u) +
-              qv[2] * __uint_as_float(kb.y << 16) + qv[3] * __uint_as_float(kb.y & 0xFFFF0000u);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    const float mn = fmaxf(m, s);
-    const float corr = __expf(m - mn);
-    const float p = __expf(s - mn);
-    const uint2 vb = *reinterpret_cast<const uint2*>(P.v_pool + off);
-    l = l * corr + p;
-    acc[0] = acc[0] * corr + p * __uint_as_float(vb.x << 16);
-    acc[1] = acc[1] * corr + p * __uint_as_float(vb.x & 0xFFFF0000u);
-    acc[2] = acc[2] * corr + p * __uint_as_float(vb.y << 16);
-    acc[3] = acc[3] * corr + p * __uint_as_float(vb.y & 0xFFFF0000u);
-    m = mn;
-  }
-  __shared__ float sm_m[4], sm_l[4], sm_acc[4][ISD_HEAD_DIM];
-  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
-#pragma unroll
-  for (int i = 0; i < 4; ++i) sm_acc[warp][lane * 4 + i] = acc[i];
-  __syncthreads();
-  if (warp == 0) {
-    float M = fmaxf(fmaxf(sm_m[0], sm_m[1]), fmaxf(sm_m[2], sm_m[3]));
-    float L = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const float c = (sm_m[w] == -INFINITY) ? 0.f : __expf(sm_m[w] - M);
-      L += sm_l[w] * c;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) o[i] += sm_acc[w][lane * 4 + i] * c;
-    }
-    __nv_bfloat16* op = P.out + (((size_t)b * P.Q + r) * P.Hq + h) * ISD_HEAD_DIM + lane * 4;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) op[i] = __float2bfloat16_rn(o[i] / L);
-    if (P.lse && lane == 0) P.lse[((size_t)b * P.Q + r) * P.Hq + h] = M + logf(L);
-  }
-}
-
 AttnParams make_params(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void* k_new,
                        const void* v_new, void* k_pool, void* v_pool, void* out, float* lse) {
   const isd_config& c = ctx->cfg;
@@ -164,20 +107,9 @@ AttnParams make_params(isd_ctx* ctx, const isd_batch_state* st, const void* q, c
 
 int isd_launch_kv_append(isd_ctx* ctx, const isd_batch_state* st, const void* k_new, const void* v_new,
                          void* k_pool, void* v_pool, cudaStream_t stream) {
-  AttnParams P = make_params(ctx, st, nullptr, k_new, v_new, k_pool, v_pool, nullptr, nullptr);
-  kv_append_kernel<<<dim3(ctx->cfg.batch, ctx->cfg.n_kv_heads), 128, 0, stream>>>(P);
+  const AttnParams P = make_params(ctx, st, nullptr, k_new, v_new, k_pool, v_pool, nullptr, nullptr);
+  const cudaError_t e = isd_launch_pdl(kv_append_kernel, dim3(ctx->cfg.batch, ctx->cfg.n_kv_heads), dim3(128), 0, stream, P);
   ctx->launches++;
-  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+  return e == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
 }
 
-int isd_launch_attn_plain(isd_ctx* ctx, const isd_batch_state* st, const void* q, const void* k_new,
-                          const void* v_new, void* k_pool, void* v_pool, void* out, float* lse,
-                          cudaStream_t stream) {
-  int rc = isd_launch_kv_append(ctx, st, k_new, v_new, k_pool, v_pool, stream);
-  if (rc != ISD_OK) return rc;
-  AttnParams P = make_params(ctx, st, q, k_new, v_new, k_pool, v_pool, out, lse);
-  const dim3 grid(ctx->cfg.n_q_heads, ctx->Q, ctx->cfg.batch);
-  attn_plain_kernel<<<grid, 128, 0, stream>>>(P);
-  ctx->launches++;
-  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
-}

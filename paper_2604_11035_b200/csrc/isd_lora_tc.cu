@@ -14,7 +14,7 @@
 //
 // Two forms of the kernel.  gemm_tc2_kernel (further down, the one normally used) works on CTA pairs; the one-CTA
 // form below serves shapes the pairs cannot take (ranks above 256 that are not multiples of 256, more blocks of t
-// than CTA pairs) and comparison runs.
+// than CTA pairs).
 //
 // One-CTA kernel: persistent CTAs, one 128 x BN output tile at a time.  Warp 4 streams the operands with TMA
 // (2-D maps, 64-element K slices = 128-byte rows, SWIZZLE_128B, every CTA loads for itself) into a 4-stage ring; warp 5
@@ -25,8 +25,6 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
-#include <cstdlib>
-
 #include "isd_internal.cuh"
 
 namespace {
@@ -34,11 +32,7 @@ namespace {
 constexpr int kThreads = 192;
 constexpr int kBM = 128;
 constexpr int kBK = 64;                       // bf16 elements per K slice = one 128-byte swizzled row
-#ifndef ISD_LORA_STAGES
-#define ISD_LORA_STAGES 4
-#endif
-constexpr int kStages = ISD_LORA_STAGES;
-constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr int kStages = 4;                    // 4 x 48 KiB ring of the one-CTA kernel
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -59,14 +53,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: false (and the abort flag raised) when the limit is reached or somebody else gave up.
+// Bounded wait: false (and the abort flag raised) when the time limit is reached or somebody else gave up.
+// The limit (nanoseconds) sits in shared memory two words behind the abort flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long budget = *reinterpret_cast<const volatile unsigned long long*>(abort_flag + 2);
+  return isd_bounded_wait(budget, abort_flag, [&]() { return mbar_try_wait(bar, parity); });
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
   asm volatile(
@@ -133,6 +125,7 @@ struct GemmParams {
   float t_scale;
   uint32_t* flags;            // [tiles_m] blocks of t written for that row block (all zero between launches)
   uint32_t* done;             // [1] CTAs that have finished (zero between launches)
+  unsigned long long wait_ns; // time limit of a device-side wait
 };
 
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
@@ -168,6 +161,7 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
     for (int i = 0; i < kStages; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_ACC_FULL + i), 1); mbar_init(bar(BAR_ACC_FREE + i), 4); }
     *abort_flag = 0;
+    *reinterpret_cast<volatile unsigned long long*>(abort_flag + 2) = P.wait_ns;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 4) {
@@ -182,9 +176,14 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
   const int tiles_m = (P.M + kBM - 1) / kBM, tiles_n = (P.N + BN - 1) / BN;
   const int n_tiles = tiles_m * tiles_n;
   const int ks1 = P.K1 / kBK, ks2 = P.K2 / kBK, ks = ks1 + ks2;  // K slices per tile
-  // Work items of this CTA: with the fused down-projection, the last tiles_m * t_chunks CTAs (the ones with the
-  // fewest output tiles) start with one block of t; then the output tiles blockIdx.x, blockIdx.x + grid, ...
-  const int t_item = P.fuse ? (int)blockIdx.x - ((int)gridDim.x - tiles_m * P.t_chunks) : -1;  // >= 0: this CTA computes a block of t
+  // Work items of this CTA.  Work is assigned by the mirrored index v = grid - 1 - blockIdx.x.  With the fused
+  // down-projection the CTAs v >= grid - tiles_m * t_chunks (the ones with the fewest output tiles) start with one
+  // block of t; then come the output tiles v, v + grid, ...  The mirror puts the blocks of t on the LOWEST block
+  // indices: the hardware hands out CTAs in index order, so the producers of t are resident before any consumer of
+  // it, and they never wait before they publish.  A grid that is only partly resident (another kernel holds SMs)
+  // therefore still makes progress; the consumers' bounded spin below needs no co-residency of the whole grid.
+  const int v_cta = (int)gridDim.x - 1 - (int)blockIdx.x;
+  const int t_item = P.fuse ? v_cta - ((int)gridDim.x - tiles_m * P.t_chunks) : -1;  // >= 0: this CTA computes a block of t
   const int t_block = t_item >= 0 ? t_item % tiles_m : 0, t_chunk = t_item >= 0 ? t_item / tiles_m : 0;
   const int n_pre = t_item >= 0 ? 1 : 0;
   // The output tiles: whole rounds of the grid as 128 x BN tiles; the tiles of the last, partial round are cut
@@ -192,7 +191,7 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
   // tail0 + u / tail_split, columns (u % tail_split) * BN / tail_split ...).  No CTA gets a strip and a block of t.
   const int rounds = n_tiles / (int)gridDim.x, tail0 = rounds * (int)gridDim.x;
   const int n_strips = (n_tiles - tail0) * P.tail_split, strip_cols = BN / P.tail_split;
-  const int n_items = n_pre + rounds + ((int)blockIdx.x < n_strips ? 1 : 0);
+  const int n_items = n_pre + rounds + (v_cta < n_strips ? 1 : 0);
   struct Item { bool pre; int m0, n0, cols; };
   auto item = [&](int it) {
     Item w;
@@ -200,11 +199,11 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
     if (w.pre) {
       w.m0 = t_block * kBM; w.n0 = t_chunk * P.Rc; w.cols = P.Rc;
     } else if (it - n_pre < rounds) {
-      const int tile = (int)blockIdx.x + (it - n_pre) * (int)gridDim.x;
+      const int tile = v_cta + (it - n_pre) * (int)gridDim.x;
       w.m0 = (tile % tiles_m) * kBM; w.n0 = (tile / tiles_m) * BN; w.cols = BN;  // neighbouring CTAs share a B panel
     } else {
-      const int tile = tail0 + (int)blockIdx.x / P.tail_split;
-      w.m0 = (tile % tiles_m) * kBM; w.n0 = (tile / tiles_m) * BN + ((int)blockIdx.x % P.tail_split) * strip_cols; w.cols = strip_cols;
+      const int tile = tail0 + v_cta / P.tail_split;
+      w.m0 = (tile % tiles_m) * kBM; w.n0 = (tile / tiles_m) * BN + (v_cta % P.tail_split) * strip_cols; w.cols = strip_cols;
     }
     return w;
   };
@@ -225,11 +224,9 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
         if (!ok) break;
         const bool seg2 = !pre && i >= ks1;
         if (P.fuse && seg2 && i == ks1) {
-          // the second segment reads t: wait until this row block of it has been published
-          uint32_t spins = 0;
-          while (ld_acquire(P.flags + m0 / kBM) != (uint32_t)P.t_chunks) {
-            if (++spins >= kSpinLimit || ((spins & 1023u) == 0u && *abort_flag)) { *abort_flag = 1; ok = false; break; }
-          }
+          // the second segment reads t: wait (bounded in time) until this row block of it has been published.
+          // Its producers are the CTAs with the lowest block indices, which never wait before they publish.
+          ok = isd_bounded_wait(P.wait_ns, abort_flag, [&]() { return ld_acquire(P.flags + m0 / kBM) == (uint32_t)P.t_chunks; });
           if (!ok) break;
           fence_proxy_async();
         }
@@ -409,6 +406,7 @@ gemm_tc2_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, 
     for (int i = 0; i < kStages2; ++i) { mbar_init(bar(B2_FULL + i), 1); mbar_init(bar(B2_EMPTY + i), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar(B2_ACC_FULL + i), 1); mbar_init(bar(B2_ACC_FREE + i), 8); }
     *abort_flag = (sm_base & 1023u) ? 1 : 0;  // the swizzled layout assumes a 1 KiB aligned window
+    *reinterpret_cast<volatile unsigned long long*>(abort_flag + 2) = P.wait_ns;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 4) {  // the same warp in both CTAs
@@ -424,8 +422,10 @@ gemm_tc2_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, 
   const int tiles_m = (P.M + 2 * kBM - 1) / (2 * kBM), tiles_n = (P.N + kBN2 - 1) / kBN2;
   const int n_tiles = tiles_m * tiles_n;
   const int ks1 = P.K1 / kBK, ks2 = P.K2 / kBK, ks = ks1 + ks2;
-  const int pr = (int)blockIdx.x >> 1, n_pairs = (int)gridDim.x >> 1;
-  // work items of the pair, as in the one-CTA kernel: a block of t first (last pairs), whole tiles, one column strip
+  // work items of the pair, as in the one-CTA kernel and by the same mirrored index (the pairs with the lowest
+  // block indices compute the blocks of t, so the producers of t are resident before any of its consumers):
+  // a block of t first, whole tiles, one column strip
+  const int n_pairs = (int)gridDim.x >> 1, pr = n_pairs - 1 - ((int)blockIdx.x >> 1);
   const int t_item = P.fuse ? pr - (n_pairs - tiles_m * P.t_chunks) : -1;
   const int t_block = t_item >= 0 ? t_item % tiles_m : 0, t_chunk = t_item >= 0 ? t_item / tiles_m : 0;
   const int n_pre = t_item >= 0 ? 1 : 0;
@@ -465,10 +465,9 @@ gemm_tc2_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, 
         if (!ok) break;
         const bool seg2 = !pre && i >= ks1;
         if (P.fuse && seg2 && i == ks1) {
-          uint32_t spins = 0;
-          while (ld_acquire(P.flags + w.m0 / (2 * kBM)) != 2u * (uint32_t)P.t_chunks) {
-            if (++spins >= kSpinLimit || ((spins & 1023u) == 0u && *abort_flag)) { *abort_flag = 1; ok = false; break; }
-          }
+          // bounded in time; the producers of t are the pairs with the lowest block indices (see above)
+          ok = isd_bounded_wait(P.wait_ns, abort_flag,
+                                [&]() { return ld_acquire(P.flags + w.m0 / (2 * kBM)) == 2u * (uint32_t)P.t_chunks; });
           if (!ok) break;
           fence_proxy_async();
         }
@@ -696,9 +695,8 @@ void isd_lora_destroy(isd_ctx* ctx) {
   ctx->lora_flags = nullptr;
 }
 
-#ifndef ISD_LORA_BN
-#define ISD_LORA_BN 256
-#endif
+// Width of an output tile of the one-CTA kernel = widest MMA (N = 256): the fewest B-panel re-reads per flop.
+constexpr int kLoraBN = 256;
 
 int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t stream) {
   const int tiles_m = (a->m + kBM - 1) / kBM;
@@ -708,15 +706,15 @@ int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t st
   P2.global_status = ctx->global_status;
   P2.fuse = 0; P2.R = a->rank; P2.Rc = a->rank; P2.t_chunks = 1; P2.t = reinterpret_cast<__nv_bfloat16*>(a->t); P2.t_gate = a->gate; P2.t_scale = a->scale;
   P2.flags = ctx->lora_flags; P2.done = ctx->lora_flags + kMaxFlags;
+  P2.wait_ns = ctx->wait_ns;
   // One launch when t divides into blocks of one MMA's width (rank <= the tile width, or a multiple of it) and
   // every block gets its own CTA: the last CTAs compute t = gate * scale * (x A^T) block by block before their
   // output tiles, and the second K segment of y = x W^T + t B^T waits for the blocks of the rows it reads.
-  const int chunks = a->rank <= ISD_LORA_BN ? 1 : (a->rank % ISD_LORA_BN == 0 ? a->rank / ISD_LORA_BN : 0);
-  // ISD_LORA_PAIR=0 in the environment keeps the CTA-pair kernel out (comparison runs, tests of the one-CTA form)
-  const char* env_pair = getenv("ISD_LORA_PAIR");
-  const bool use_pairs = !(env_pair && env_pair[0] == '0');
+  const int chunks = a->rank <= kLoraBN ? 1 : (a->rank % kLoraBN == 0 ? a->rank / kLoraBN : 0);
+  // The form is chosen by shape alone: CTA pairs when every block of t gets a pair of its own, else the one-CTA
+  // kernel with the fused down-projection when every block gets a CTA, else two launches.
   const int blocks2 = (a->m + 2 * kBM - 1) / (2 * kBM);  // 256-row blocks
-  if (use_pairs && chunks > 0 && blocks2 * chunks <= ctx->num_sms / 2 && blocks2 <= kMaxFlags) {
+  if (chunks > 0 && blocks2 * chunks <= ctx->num_sms / 2 && blocks2 <= kMaxFlags) {
     // CTA pairs: 256 x 256 tiles, blocks of t of 256 rows
     P2.fuse = 1;
     P2.t_chunks = chunks;
@@ -727,7 +725,7 @@ int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t st
     P2.fuse = 1;
     P2.t_chunks = chunks;
     P2.Rc = a->rank / chunks;
-    return launch_gemm<ISD_LORA_BN>(ctx, P2, a->x, a->w, a->t, a->b, a->a, stream);
+    return launch_gemm<kLoraBN>(ctx, P2, a->x, a->w, a->t, a->b, a->a, stream);
   }
   // Otherwise two launches.  1. t = gate * scale * (x A^T): N = rank, one K segment
   GemmParams P1 = P2;
@@ -735,5 +733,5 @@ int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t st
   int rc = launch_gemm<128>(ctx, P1, a->x, a->a, nullptr, nullptr, nullptr, stream);
   if (rc != ISD_OK) return rc;
   // 2. y = x W^T + t B^T: two K segments, no gate (it is already in t)
-  return launch_gemm<ISD_LORA_BN>(ctx, P2, a->x, a->w, a->t, a->b, nullptr, stream);
+  return launch_gemm<kLoraBN>(ctx, P2, a->x, a->w, a->t, a->b, nullptr, stream);
 }

@@ -1,6 +1,6 @@
 // Streaming of logits rows through shared memory, shared by the verification kernels: a ring of
 // kRowStages x kRowStageBytes that one thread of a producer warp fills with bulk copies (mbarrier
-// full / empty pairs, bounded waits) and 256 worker threads read back as 16-byte vectors.
+// full / empty pairs, waits bounded in time) and 256 worker threads read back as 16-byte vectors.
 #pragma once
 #include "isd_internal.cuh"
 
@@ -65,12 +65,13 @@ struct RowRing {
 // Producer (one thread): streams bytes [byte_lo, byte_hi) of a row into the ring, one contiguous bulk copy
 // per stage.  c is the ring's running stage counter: it carries on over consecutive ranges, so that several
 // ranges can go through one ring without re-initialising its barriers.  Returns false when a wait ran out.
-__device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t byte_lo, size_t byte_hi, int& c) {
+__device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t byte_lo, size_t byte_hi, int& c,
+                                             unsigned long long wait_ns) {
   const uint32_t full0 = ring_smem_u32(R.full), empty0 = ring_smem_u32(R.empty), st0 = ring_smem_u32(R.stage);
   for (size_t off = byte_lo; off < byte_hi; off += kRowStageBytes, ++c) {
     const int s = c & (kRowStages - 1);
     const uint32_t ph = (c / kRowStages) & 1;
-    if (!ring_mbar_wait(empty0 + 8 * s, ph ^ 1)) return false;
+    if (!ring_mbar_wait(empty0 + 8 * s, ph ^ 1, wait_ns)) return false;
     const size_t left = byte_hi - off;
     const uint32_t bytes = left < (size_t)kRowStageBytes ? (uint32_t)left : (uint32_t)kRowStageBytes;
     ring_mbar_expect_tx(full0 + 8 * s, bytes);
@@ -79,9 +80,10 @@ __device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t
   return true;
 }
 
-__device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t byte_lo, size_t byte_hi) {
+__device__ __forceinline__ bool row_producer(RowRing& R, const char* row, size_t byte_lo, size_t byte_hi,
+                                             unsigned long long wait_ns) {
   int c = 0;
-  return row_producer(R, row, byte_lo, byte_hi, c);
+  return row_producer(R, row, byte_lo, byte_hi, c, wait_ns);
 }
 
 

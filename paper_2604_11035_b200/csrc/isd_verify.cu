@@ -27,6 +27,7 @@
 // ISD_TIE_EPS.
 #include "isd_internal.cuh"
 #include "isd_stream.cuh"
+#include "isd_commit.cuh"
 
 namespace {
 
@@ -37,6 +38,8 @@ struct VerifyParams {
   int B, N, Q, V;
   int logits_dtype, q_mode, propose_mode;
   float inv_t, tau;
+  unsigned long long wait_ns;  // time limit of a device-side wait
+  PhiloxKeys rk;               // round keys of the seed
   uint32_t seed_lo, seed_hi, step;
   const uint32_t* step_dev;  // when set, the step number is read from here (CUDA-graph replay) instead of `step`
   int row_splits, sample_splits;
@@ -57,6 +60,10 @@ struct VerifyParams {
   int* reject_pos;
   int* row_arg;
   float* lse_p_rej;
+  // isd_step: the CTA of the sampling pass that finishes last commits the batch (fuse_commit != 0)
+  int fuse_commit;
+  int* step_ticket;
+  CommitParams commit;
 };
 
 // rows nv .. nv + rows_sampled - 1 of a slot are drawn by the sampling pass
@@ -265,7 +272,7 @@ __device__ __forceinline__ bool row_pass(const VerifyParams& P, RowRing& R, cons
   };
   // s = stage (a compile-time constant in the unrolled main loop), ph = parity of its current fill
   auto read_stage = [&](int s, uint32_t ph, float (&l)[U][8]) {
-    ok = ok && mbar_wait_likely(full0 + 8 * s, ph);
+    ok = ok && mbar_wait_likely(full0 + 8 * s, ph, P.wait_ns);
     const uint32_t base = mine + s * kRowStageBytes;
 #pragma unroll
     for (int g = 0; g < U; ++g) {
@@ -331,6 +338,13 @@ __device__ __forceinline__ bool row_pass(const VerifyParams& P, RowRing& R, cons
   return ok;
 }
 
+// A wait of the row pass ran out: the slot's statistics are incomplete, so the slot is marked (the decision
+// phase and the commit then leave it alone) and the global word tells the host.
+__device__ __forceinline__ void row_timeout(const VerifyParams& P, int b) {
+  atomicOr(&P.slot_status[b], ISD_ST_KERNEL_TIMEOUT);
+  atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Pass 1: row statistics + decision
 // ------------------------------------------------------------------------------------------------
@@ -339,6 +353,19 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
   // Launch order = (split, slot, k): the rows that the sampling pass reads again come last, so that
   // they are the most recent lines in L2 when it starts.
   const int split = blockIdx.x, b = blockIdx.y, k = blockIdx.z;
+  __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
+  __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
+  __shared__ int sm_last;
+  __shared__ RowRing sm_ring;
+  if (threadIdx.x == 0) {  // needs nothing from memory: runs while the kernel before this one drains
+    for (int i = 0; i < kRowStages; ++i) {
+      ring_mbar_init(ring_smem_u32(&sm_ring.full[i]), 1);
+      ring_mbar_init(ring_smem_u32(&sm_ring.empty[i]), kThreads / 32);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  pdl_wait();
+  pdl_launch_dependents();
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
   if (nv < 0 || nv > P.N - 1) {
@@ -353,37 +380,23 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
   if (r >= P.Q) r -= P.Q;
   if (r >= q_len) return;
 
-  __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
-  __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
-  __shared__ int sm_last;
-  __shared__ RowRing sm_ring;
-
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
   int lo, hi;
   chunk_range(P.V, P.row_splits, split, lo, hi);
-
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < kRowStages; ++i) {
-      ring_mbar_init(ring_smem_u32(&sm_ring.full[i]), 1);
-      ring_mbar_init(ring_smem_u32(&sm_ring.empty[i]), kThreads / 32);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
   __syncthreads();
   if (threadIdx.x >= kThreads) {
     // producer warp: one thread feeds the ring, then the warp is done (every copy it issued is consumed
     // by the workers before they leave; a wait that runs out raises the status bit and stops feeding)
     if (threadIdx.x == kThreads && hi > lo) {
-      if (!row_producer(sm_ring, row, (size_t)lo * elt, (size_t)hi * elt)) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+      if (!row_producer(sm_ring, row, (size_t)lo * elt, (size_t)hi * elt, P.wait_ns)) row_timeout(P, b);
     }
     return;
   }
 
   float m_nat, S, raw_max;
   int raw_idx;
-  if (!row_pass<DT>(P, sm_ring, row, lo, hi, m_nat, S, raw_max, raw_idx) && threadIdx.x == 0)
-    atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  if (!row_pass<DT>(P, sm_ring, row, lo, hi, m_nat, S, raw_max, raw_idx) && threadIdx.x == 0) row_timeout(P, b);
 
   // ---- block reduction -> partial
   block_merge_lse(m_nat, S, sm_f0, sm_f1);
@@ -488,6 +501,8 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
     }
   }
   if (a >= 0 && rej == 0 && d_bad[nv]) status |= ISD_ST_NONFINITE_LOGIT;
+  // a CTA of this slot gave up on a wait: its partial is incomplete, nothing of the slot may be committed
+  status |= *reinterpret_cast<volatile uint32_t*>(&P.slot_status[b]) & ISD_ST_KERNEL_TIMEOUT;
   for (int j = 0; j < P.N; ++j) P.out.out_tok[(size_t)b * P.N + j] = -1;
   P.out.repl_tok[b] = -1;  // the sampling pass fills the drawn token
   if (a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL)) {
@@ -545,9 +560,7 @@ __device__ __forceinline__ float job_score(const VerifyParams& P, const SampleJo
 
 // resident CTAs per SM the sampling kernel is compiled for: three keep it at 80 registers (without the bound
 // the compiler takes 89 and only two CTAs fit)
-#ifndef ISD_SAMPLE_MINB
-#define ISD_SAMPLE_MINB 3
-#endif
+constexpr int kSampleMinBlocks = 4;
 // Per-warp queue of groups of four logits that survived the first skip test.
 constexpr int kQueueCap = 128;  // < 32 left over + at most 64 new per iteration
 struct SampleQueue {
@@ -560,9 +573,8 @@ struct SampleQueue {
 // shared by the CTA through sm_best, and a stale value only makes the skip tests weaker.
 template <int DT>
 __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJob& J, int lo, int hi, int b,
-                                            float best, Top2& top, SampleQueue& Q, unsigned* sm_best, uint4* ring) {
-  RowStream<DT, 1, kSampleRingBytes> in;
-  in.start(ring, J.prow, lo, hi);
+                                            float best, Top2& top, SampleQueue& Q, unsigned* sm_best,
+                                            RowStream<DT, 1, kSampleRingBytes>& in) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const unsigned below = (1u << lane) - 1u;
   float4* ql = Q.l[warp];
@@ -575,16 +587,23 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
   top.init();
   int head = 0, tail = 0;  // warp-uniform queue positions
 
-  // Draw the noise of one queued group and keep its candidates.
-  auto drain = [&](int pos) {
-    const int idx = qi[pos & (kQueueCap - 1)];
-    const float4 v = ql[pos & (kQueueCap - 1)];
-    const float l4[4] = {v.x, v.y, v.z, v.w};
-    const uint4 rnd = philox4x32_10((uint32_t)idx >> 2, J.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
-    const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-    // -ln u' >= 1 - u' >= nf 2^-24 with nf = floor(2^24 (1 - u')), so g_i <= -ln(nf 2^-24): the element
-    // cannot come within 2e-3 of the running best when nf >= 1.002 * 2^24 * exp(l_i invT - shift - best)
+  // Judge one queued group whose noise `rnd` has been drawn, and keep its candidates.
+  auto judge = [&](int idx, const float4& v, const uint4& rnd) {
+    // -ln u' >= 1 - u' >= nf 2^-24 with nf = floor(2^24 (1 - u')) = (~word) >> 8, so g_i <= -ln(nf 2^-24): element i
+    // cannot come within 2e-3 of the running best when nf >= 1.002 * 2^24 * exp(l_i invT - shift - best).
+    // First for the whole group, with the group's largest logit and in integers: nf >= kb for the integer
+    // kb >= that bound is the same as word <= ~(kb << 8), one compare per element and no conversion.  Nearly
+    // every group ends here.
     float K2 = 24.0028853901f - (shift + best) * kLog2e;  // log2 of the factor; +inf while there is no best
+    const float xg = fmaf(fmaxf(max3(v.x, v.y, v.z), v.w), scale2, K2);
+    if (xg < 23.9f) {  // false for NaN (no best yet) and for groups that reach the running best
+      uint32_t kb;
+      asm("cvt.rpi.u32.f32 %0, %1;" : "=r"(kb) : "f"(ex2f(xg)));
+      const uint32_t wt = ~(kb << 8);
+      if (rnd.x <= wt && rnd.y <= wt && rnd.z <= wt && rnd.w <= wt) return;
+    }
+    const float l4[4] = {v.x, v.y, v.z, v.w};
+    const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
     bool improved = false;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -603,6 +622,12 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
       }
     }
     if (improved) atomicMax(sm_best, enc_ordered(best));
+  };
+  auto drain = [&](int pos) {
+    const int idx = qi[pos & (kQueueCap - 1)];
+    const float4 v = ql[pos & (kQueueCap - 1)];
+    const uint4 rnd = philox4x32_10((uint32_t)idx >> 2, J.step, (uint32_t)b, J.tagpos, P.rk);
+    judge(idx, v, rnd);
   };
 
   // uniform trip count per block (the warp votes inside the loop)
@@ -646,7 +671,7 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads, ISD_SAMPLE_MINB) verify_sample_kernel(const VerifyParams P) {
+__device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
   const int split = blockIdx.x, k = blockIdx.y, b = blockIdx.z;
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
@@ -690,6 +715,12 @@ __global__ void __launch_bounds__(kThreads, ISD_SAMPLE_MINB) verify_sample_kerne
   }
   J.prow = cur + (size_t)r * row_bytes;
 
+  // the first stages of this CTA's piece of the row are on their way while thread 0 works out the seed
+  int lo, hi;
+  chunk_range(P.V, P.sample_splits, split, lo, hi);
+  RowStream<DT, 1, kSampleRingBytes> in;
+  in.start(sm_ring, J.prow, lo, hi);
+
   // ---- seed: the true noisy score of the row's argmax (for the residual: if it has residual mass)
   if (threadIdx.x == 0) {
     float seed = -INFINITY;
@@ -703,10 +734,8 @@ __global__ void __launch_bounds__(kThreads, ISD_SAMPLE_MINB) verify_sample_kerne
   __syncthreads();
   const float best0 = dec_ordered(sm_best);  // NaN when there is no seed
 
-  int lo, hi;
-  chunk_range(P.V, P.sample_splits, split, lo, hi);
   Top2 top;
-  sample_pass<DT>(P, J, lo, hi, b, fmaxf(-INFINITY, best0), top, sm_queue, &sm_best, sm_ring);
+  sample_pass<DT>(P, J, lo, hi, b, fmaxf(-INFINITY, best0), top, sm_queue, &sm_best, in);
 
   block_merge_top2(top, sm_f0, sm_i0, sm_f1, sm_i1);
   int* ticket = P.samp_ticket + (size_t)b * P.N + k;
@@ -755,7 +784,8 @@ __global__ void __launch_bounds__(kThreads, ISD_SAMPLE_MINB) verify_sample_kerne
     if (threadIdx.x == 0) sm_best = 0u;
     __syncthreads();
     Top2 t;
-    sample_pass<DT>(P, J, 0, P.V, b, -INFINITY, t, sm_queue, &sm_best, sm_ring);
+    in.start(sm_ring, J.prow, 0, P.V);
+    sample_pass<DT>(P, J, 0, P.V, b, -INFINITY, t, sm_queue, &sm_best, in);
     block_merge_top2(t, sm_f0, sm_i0, sm_f1, sm_i1);
     if (threadIdx.x == 0) {
       y = t.i1;
@@ -780,16 +810,39 @@ __global__ void __launch_bounds__(kThreads, ISD_SAMPLE_MINB) verify_sample_kerne
   }
 }
 
+template <int DT>
+__global__ void __launch_bounds__(kThreads, kSampleMinBlocks) verify_sample_kernel(const VerifyParams P) {
+  pdl_wait();
+  pdl_launch_dependents();
+  verify_sample_body<DT>(P);
+  if (!P.fuse_commit) return;
+  // ---- isd_step: the CTA that finishes last (a ticket over the whole grid; nobody waits) has every slot's
+  // decision and tokens in front of it and commits the batch, which saves the launch of a kernel for it
+  __shared__ int sm_commit[36];
+  if (threadIdx.x == 0) {
+    __threadfence();  // thread 0 wrote everything this CTA contributes (tokens, status bits)
+    const int arrived = atomicAdd(P.step_ticket, 1);
+    sm_commit[35] = (arrived == (int)(gridDim.x * gridDim.y * gridDim.z) - 1);
+  }
+  __syncthreads();
+  if (!sm_commit[35]) return;
+  if (threadIdx.x == 0) *P.step_ticket = 0;  // ready for the next call
+  __threadfence();
+  commit_block(P.commit, sm_commit, sm_commit + 33);
+}
+
 }  // namespace
 
 int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
                       const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
-                      cudaStream_t stream) {
+                      cudaStream_t stream, isd_batch_state* commit_st) {
   const isd_config& c = ctx->cfg;
   VerifyParams P;
   P.B = c.batch; P.N = c.stride; P.Q = ctx->Q; P.V = c.vocab;
   P.logits_dtype = c.logits_dtype; P.q_mode = c.q_mode; P.propose_mode = c.propose_mode;
   P.inv_t = c.inv_temperature; P.tau = c.tau;
+  P.wait_ns = ctx->wait_ns;
+  philox_round_keys(c.seed, P.rk);
   P.seed_lo = (uint32_t)c.seed; P.seed_hi = (uint32_t)(c.seed >> 32); P.step = step;
   P.step_dev = ctx->step_counter;
   P.row_splits = ctx->row_splits; P.sample_splits = ctx->sample_splits;
@@ -799,20 +852,26 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   P.row_part = ctx->row_part; P.samp_part = ctx->samp_part; P.row_ticket = ctx->row_ticket;
   P.samp_ticket = ctx->samp_ticket; P.reject_pos = ctx->reject_pos; P.row_arg = ctx->row_arg;
   P.lse_p_rej = ctx->lse_p_rej;
+  P.fuse_commit = commit_st != nullptr && ctx->step_ticket != nullptr;
+  P.step_ticket = ctx->step_ticket;
+  P.commit = make_commit_params(ctx, P.fuse_commit ? commit_st : st, out);
 
   const dim3 grid1(ctx->row_splits, c.batch, ctx->Q);
   const dim3 grid2(ctx->sample_splits, c.propose_mode == 0 ? c.stride : 1, c.batch);
   if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
+  cudaError_t e1, e2;
   if (c.logits_dtype == ISD_LOGITS_BF16) {
-    verify_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads + 32, 0, stream>>>(P);
-    verify_sample_kernel<ISD_LOGITS_BF16><<<grid2, kThreads, 0, stream>>>(P);
+    e1 = isd_launch_pdl(verify_rows_kernel<ISD_LOGITS_BF16>, grid1, dim3(kThreads + 32), 0, stream, P);
+    e2 = isd_launch_pdl(verify_sample_kernel<ISD_LOGITS_BF16>, grid2, dim3(kThreads), 0, stream, P);
   } else {
-    verify_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads + 32, 0, stream>>>(P);
-    verify_sample_kernel<ISD_LOGITS_F32><<<grid2, kThreads, 0, stream>>>(P);
+    e1 = isd_launch_pdl(verify_rows_kernel<ISD_LOGITS_F32>, grid1, dim3(kThreads + 32), 0, stream, P);
+    e2 = isd_launch_pdl(verify_sample_kernel<ISD_LOGITS_F32>, grid2, dim3(kThreads), 0, stream, P);
   }
   if (ctx->ev_verify1) cudaEventRecord(ctx->ev_verify1, stream);
   ctx->launches += 2;
-  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+  if (e1 != cudaSuccess || e2 != cudaSuccess) return ISD_ERR_CUDA;
+  // without the fused commit the caller launches the commit kernel itself
+  return ISD_OK;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -917,6 +976,7 @@ extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* s
   tmp.lse_p_rej = reinterpret_cast<float*>(base + kOffLse);
   tmp.samp_part = reinterpret_cast<SamplePartial*>(base + kOffSampPart);
   tmp.row_part = reinterpret_cast<RowPartial*>(base + kOffRowPart);
+  tmp.wait_ns = ISD_DEFAULT_WAIT_NS;
 
   // the array keeps the previous call's contents: counters and flags must start at zero
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);

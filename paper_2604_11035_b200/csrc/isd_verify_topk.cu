@@ -33,6 +33,7 @@ struct TopkParams {
   int B, N, Q, V;
   int logits_dtype, q_mode, propose_mode, top_k;
   float inv_t, tau, top_p;
+  unsigned long long wait_ns;  // time limit of a device-side wait
   uint32_t seed_lo, seed_hi, step;
   const uint32_t* step_dev;
   const int32_t* n_ver;
@@ -198,7 +199,7 @@ __device__ unsigned bound_from_maxima(unsigned vkey, int k, unsigned* sm_offer) 
 // buffer (many equal values), the k-th best of what was collected is a strictly better bound and the second
 // stream is repeated.
 template <int DT>
-__device__ bool block_topk_two_stream(TopkShared& sh, const char* row, int e_lo, int e_hi, int k) {
+__device__ bool block_topk_two_stream(TopkShared& sh, const char* row, int e_lo, int e_hi, int k, unsigned long long wait_ns) {
   constexpr int kElt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   constexpr int U = DT == ISD_LOGITS_BF16 ? 2 : 1;
   constexpr int kStageElems = kRowStageBytes / kElt;
@@ -223,13 +224,13 @@ __device__ bool block_topk_two_stream(TopkShared& sh, const char* row, int e_lo,
     }
     __syncthreads();
     if (!worker) {
-      if (threadIdx.x == kThreads) ok = row_producer(sh.ring, row, (size_t)e_lo * kElt, (size_t)e_hi * kElt) && ok;
+      if (threadIdx.x == kThreads) ok = row_producer(sh.ring, row, (size_t)e_lo * kElt, (size_t)e_hi * kElt, wait_ns) && ok;
     } else {
       float tmax = -INFINITY;  // first stream: the best value this thread has seen
       int e = e_lo + threadIdx.x * 8;
       for (int c = 0; c < stages; ++c, e += kStageElems) {
         const int s = c & (kRowStages - 1);
-        ok = mbar_wait_likely(full0 + 8 * s, (uint32_t)(c / kRowStages) & 1u) && ok;
+        ok = mbar_wait_likely(full0 + 8 * s, (uint32_t)(c / kRowStages) & 1u, wait_ns) && ok;
         float l[U][8];
 #pragma unroll
         for (int g = 0; g < U; ++g) {
@@ -304,9 +305,10 @@ constexpr int kCompactAt = 96;  // candidates from which they are cut back to th
 
 // One stage of the ring: waits for it, takes this thread's groups of eight as packed words, releases the stage.
 template <int DT, int U>
-__device__ __forceinline__ bool take_stage(uint32_t full0, uint32_t empty0, uint32_t mine, int cc, uint4 (&a)[U], uint4 (&b)[U]) {
+__device__ __forceinline__ bool take_stage(uint32_t full0, uint32_t empty0, uint32_t mine, int cc, uint4 (&a)[U], uint4 (&b)[U],
+                                           unsigned long long wait_ns) {
   const int s = cc & (kRowStages - 1);
-  const bool ok = mbar_wait_likely(full0 + 8 * s, (uint32_t)(cc / kRowStages) & 1u);
+  const bool ok = mbar_wait_likely(full0 + 8 * s, (uint32_t)(cc / kRowStages) & 1u, wait_ns);
 #pragma unroll
   for (int g = 0; g < U; ++g) {
     b[g] = make_uint4(0u, 0u, 0u, 0u);
@@ -335,7 +337,7 @@ __device__ __forceinline__ bool take_stage(uint32_t full0, uint32_t empty0, uint
 // between two looks than the buffers hold (a row sorted upwards, long runs of equal values), nothing more is
 // noted, the stream is drained and the two-stream routine, which handles any input, starts over.
 template <int DT>
-__device__ bool block_topk(TopkShared& sh, const char* row, int e_lo, int e_hi, int k) {
+__device__ bool block_topk(TopkShared& sh, const char* row, int e_lo, int e_hi, int k, unsigned long long wait_ns) {
   constexpr int kElt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   constexpr int U = DT == ISD_LOGITS_BF16 ? 2 : 1;
   constexpr int kStageElems = kRowStageBytes / kElt;
@@ -362,8 +364,8 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int e_lo, int e_hi, 
     if (threadIdx.x == kThreads) {
       const size_t lo = (size_t)e_lo * kElt, hi = (size_t)e_hi * kElt, head_hi = lo + (size_t)head * kRowStageBytes;
       int c = 0;
-      ok = row_producer(sh.ring, row, lo, head_hi < hi ? head_hi : hi, c);
-      ok = ok && row_producer(sh.ring, row, lo, hi, c);
+      ok = row_producer(sh.ring, row, lo, head_hi < hi ? head_hi : hi, c, wait_ns);
+      ok = ok && row_producer(sh.ring, row, lo, hi, c, wait_ns);
     }
   } else {
     const uint32_t full0 = ring_smem_u32(sh.ring.full), empty0 = ring_smem_u32(sh.ring.empty);
@@ -372,7 +374,7 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int e_lo, int e_hi, 
     // ---- the head: the best value this thread sees
     float tmax = -INFINITY;
     for (int c = 0; c < head; ++c) {
-      ok = take_stage<DT, U>(full0, empty0, mine, c, a, b) && ok;
+      ok = take_stage<DT, U>(full0, empty0, mine, c, a, b, wait_ns) && ok;
       const int e = e_lo + c * kStageElems + threadIdx.x * 8;
 #pragma unroll
       for (int g = 0; g < U; ++g) {
@@ -387,7 +389,7 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int e_lo, int e_hi, 
     bool over = false;
     // ---- the range
     for (int c = 0; c < stages; ++c) {
-      ok = take_stage<DT, U>(full0, empty0, mine, head + c, a, b) && ok;
+      ok = take_stage<DT, U>(full0, empty0, mine, head + c, a, b, wait_ns) && ok;
       const int e = e_lo + c * kStageElems + threadIdx.x * 8;
       const bool last = c == stages - 1;
 #pragma unroll
@@ -471,7 +473,7 @@ __device__ bool block_topk(TopkShared& sh, const char* row, int e_lo, int e_hi, 
     if (over && threadIdx.x == 0) sh.over = 1;
   }
   __syncthreads();  // producer warp and workers meet
-  if (sh.over) return block_topk_two_stream<DT>(sh, row, e_lo, e_hi, k) && ok;
+  if (sh.over) return block_topk_two_stream<DT>(sh, row, e_lo, e_hi, k, wait_ns) && ok;
   return ok;
 }
 
@@ -769,7 +771,10 @@ __global__ void __launch_bounds__(kThreads + 32, 5) topk_rows_kernel(const TopkP
   if (r >= nv + P.N) return;
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
-  if (!block_topk<DT>(sh, row, 0, P.V, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  if (!block_topk<DT>(sh, row, 0, P.V, P.top_k, P.wait_ns) && threadIdx.x == 0) {
+    atomicOr(&P.slot_status[b], ISD_ST_KERNEL_TIMEOUT);
+    atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  }
   const size_t base = ((size_t)b * P.Q + r) * kMaxTopK;
   if (threadIdx.x < sh.list_n) {
     P.list_val[base + threadIdx.x] = sh.list_val[threadIdx.x];
@@ -853,7 +858,10 @@ __global__ void __cluster_dims__(kQSplit, 1, 1) __launch_bounds__(kThreads + 32)
   const int per = ((P.V + stage_elems - 1) / stage_elems + kQSplit - 1) / kQSplit * stage_elems;
   const int e_lo = piece * per < P.V ? piece * per : P.V;
   const int e_hi = e_lo + per < P.V ? e_lo + per : P.V;
-  if (!block_topk<DT>(sh, qrow, e_lo, e_hi, P.top_k) && threadIdx.x == 0) atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  if (!block_topk<DT>(sh, qrow, e_lo, e_hi, P.top_k, P.wait_ns) && threadIdx.x == 0) {
+    atomicOr(&P.slot_status[b], ISD_ST_KERNEL_TIMEOUT);
+    atomicOr(P.global_status, ISD_ST_KERNEL_TIMEOUT);
+  }
   if (threadIdx.x < sh.list_n)
     P.q_key[((size_t)b * kQSplit + piece) * kMaxTopK + threadIdx.x] = cand_key(sh.list_val[threadIdx.x], sh.list_idx[threadIdx.x]);
   if (threadIdx.x == 0) P.q_n[(size_t)b * kQSplit + piece] = sh.list_n;
@@ -936,6 +944,7 @@ int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* 
   P.B = c.batch; P.N = c.stride; P.Q = ctx->Q; P.V = c.vocab;
   P.logits_dtype = c.logits_dtype; P.q_mode = c.q_mode; P.propose_mode = c.propose_mode; P.top_k = c.top_k;
   P.inv_t = c.inv_temperature; P.tau = c.tau; P.top_p = c.top_p;
+  P.wait_ns = ctx->wait_ns;
   P.seed_lo = (uint32_t)c.seed; P.seed_hi = (uint32_t)(c.seed >> 32); P.step = step;
   P.step_dev = ctx->step_counter;
   P.n_ver = st->n_ver; P.active = st->active; P.block_tok = st->block_tok; P.q_row0 = st->q_row0;

@@ -14,7 +14,6 @@ overwritten with the oracle's so that the chain stays comparable.
 """
 from __future__ import annotations
 
-import os
 import time
 
 import numpy as np
@@ -33,16 +32,14 @@ def _bf16_to_f64(bits):
     return torch.from_numpy(bits.astype(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
 
 
-def run_chain_parity(w: wl.Workload, steps: int, device="cuda:0", attn_slots=None, attn_impl=None,
+def run_chain_parity(w: wl.Workload, steps: int, device="cuda:0", attn_slots=None,
                      oracle_threads=None, check_pools=True, verbose=False, **isd_kw):
     dev = torch.device(device)
     N, B, Q, NP = w.stride, w.batch, w.Q, w.stride - 1
-    if attn_impl is None:
-        attn_impl = int(os.environ.get("ISD_TEST_ATTN_IMPL", "0"))
     oracle.set_threads(oracle_threads or oracle.max_threads())
     st = wl.make_state(w, dev)
     s = state_to_np(st)                      # oracle state (inputs come from the generator)
-    eng = isd_pkg.isd_for_workload(w, st, attn_impl=attn_impl, **isd_kw)
+    eng = isd_pkg.isd_for_workload(w, st, **isd_kw)
     out = isd_pkg.alloc_verify_out(B, N, dev)
     attn_out = torch.zeros(B, Q, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
     attn_lse = torch.zeros(B, Q, w.n_q_heads, dtype=torch.float32, device=dev)

@@ -80,7 +80,7 @@ def test_multi_layer_step_matches_oracle_layer_by_layer():
         prev, prev_np = lg, lg_np
     assert rejections > 0
     assert eng.isd_read_status() == 0
-    assert eng.isd_launch_count() == steps * (3 * L + 3)   # per layer: append, attention, combine; then 2 + 1
+    assert eng.isd_launch_count() == steps * (3 * L + 2)   # per layer: append, attention, combine; then rows, sampling (+ commit)
     eng.close()
 
 

@@ -101,15 +101,18 @@ def test_repeated_calls_reuse_the_scratch_and_big_ranks_take_two_launches():
     eng.close()
 
 
-@pytest.mark.parametrize("M,N,K,R", [(517, 544, 448, 192), (300, 544, 192, 512), (700, 1120, 128, 64)])
-def test_one_cta_form_of_the_kernel(M, N, K, R, monkeypatch):
-    # ISD_LORA_PAIR=0 keeps the CTA-pair kernel out: the one-CTA kernel with the fused down-projection and the
-    # column strips of the last round takes the same shapes (the library reads the variable at every call)
-    monkeypatch.setenv("ISD_LORA_PAIR", "0")
+@pytest.mark.parametrize("M,N,K,R,launches", [(6200, 288, 128, 768, 1), (6200, 544, 192, 320, 2)])
+def test_one_cta_form_of_the_kernel(M, N, K, R, launches):
+    # The library picks the kernel by shape alone.  Rank 768 at 6200 rows has 25 x 3 blocks of t (256 rows each):
+    # more than the 74 CTA pairs, but its 49 x 3 blocks of 128 rows fit the 148 CTAs, so the one-CTA kernel runs
+    # with the fused down-projection and the column strips of its last round.  Rank 320 is neither below 256 nor a
+    # multiple of it: two launches of the one-CTA kernel, t first.
     eng = _engine()
     x, w, a, b, gate = _inputs(M, N, K, R, seed=7 * M + R)
+    n0 = eng.isd_launch_count()
     y = eng.isd_lora_linear(x, w, a, b, gate, 0.6)
     torch.cuda.synchronize()
+    assert eng.isd_launch_count() - n0 == launches
     ref = oracle.lora_linear(_f64(x), _f64(w), _f64(a), _f64(b), gate.cpu().numpy(), 0.6)
     tol = _tolerance(ref, _f64(x), _f64(a), _f64(b), gate.cpu().numpy(), 0.6)
     err = np.abs(_f64(y) - ref)
