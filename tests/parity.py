@@ -43,9 +43,6 @@ def run_chain_parity(w: wl.Workload, steps: int, device="cuda:0", attn_slots=Non
     out = isd_pkg.alloc_verify_out(B, N, dev)
     attn_out = torch.zeros(B, Q, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
     attn_lse = torch.zeros(B, Q, w.n_q_heads, dtype=torch.float32, device=dev)
-    attn_sel = np.arange(B) if attn_slots is None else np.asarray(attn_slots)
-    attn_active = np.zeros(B, np.uint8)
-    attn_active[attn_sel] = 1
 
     rep = dict(workload=w.name, steps=steps, mismatches=0, exempt_flips=0, near_threshold=0,
                fragile_samples=0, attn_max_abs_err=0.0, lse_max_abs_err=0.0, alpha_max_abs_err=0.0,
@@ -73,8 +70,21 @@ def run_chain_parity(w: wl.Workload, steps: int, device="cuda:0", attn_slots=Non
         eng.isd_step(st, args, t)
         torch.cuda.synchronize()
 
-        # ---- oracle: attention on the selected slots, verify + commit on all slots
+        # ---- oracle: attention on the selected slots (a list, or a function of the step for a rotating sample),
+        # verify + commit on all slots
         t0 = time.time()
+        sel_t = attn_slots(t) if callable(attn_slots) else attn_slots
+        attn_sel = np.arange(B) if sel_t is None else np.asarray(sel_t, dtype=np.int64)
+        attn_active = np.zeros(B, np.uint8)
+        attn_active[attn_sel] = 1
+        # slots outside the sample: only the batched scatter of the block's K/V rows (input plumbing, so that the
+        # oracle's pools stay complete when the sample moves on)
+        for b in np.nonzero((s["active"] != 0) & (attn_active == 0))[0]:
+            ql_b, ctx_b = int(s["n_ver"][b]) + N, int(s["ctx_len"][b])
+            pos = ctx_b + np.arange(ql_b)
+            pages = s["page_table"][b, pos // wl.PAGE]
+            s["k_pool"][pages, :, pos % wl.PAGE, :] = k_np[b, :ql_b]
+            s["v_pool"][pages, :, pos % wl.PAGE, :] = v_np[b, :ql_b]
         save_active = s["active"]
         s["active"] = (save_active & attn_active).astype(np.uint8)
         q_len = np.where(s["active"] != 0, s["n_ver"] + N, 0).astype(np.int32)
@@ -107,16 +117,17 @@ def run_chain_parity(w: wl.Workload, steps: int, device="cuda:0", attn_slots=Non
                 bad(f"step {t} slot {b}: attention err {e:.3e} above the derived bound {tight:.3e}")
         # ---- compare KV rows: every logical position below the new committed length
         if check_pools:
-            gk, gv = bits16(st["k_pool"]), bits16(st["v_pool"])
             for b in attn_sel:
                 n = int(ctx_before[b] + q_len[b])       # rows beyond n are "don't care"
                 pages = s["page_table"][b, :(n + 15) // 16]
+                pg_dev = torch.from_numpy(pages.astype(np.int64)).to(dev)
+                gk, gv = bits16(st["k_pool"][pg_dev]), bits16(st["v_pool"][pg_dev])   # only this slot's pages travel
+                ok_, ov_ = s["k_pool"][pages], s["v_pool"][pages]
                 full, rem = n // 16, n % 16
-                same = (np.array_equal(gk[pages[:full]], s["k_pool"][pages[:full]]) and
-                        np.array_equal(gv[pages[:full]], s["v_pool"][pages[:full]]))
+                same = np.array_equal(gk[:full], ok_[:full]) and np.array_equal(gv[:full], ov_[:full])
                 if rem:
-                    same = same and np.array_equal(gk[pages[full], :, :rem], s["k_pool"][pages[full], :, :rem]) \
-                        and np.array_equal(gv[pages[full], :, :rem], s["v_pool"][pages[full], :, :rem])
+                    same = same and np.array_equal(gk[full, :, :rem], ok_[full, :, :rem]) \
+                        and np.array_equal(gv[full, :, :rem], ov_[full, :, :rem])
                 if not same:
                     bad(f"step {t} slot {b}: KV rows differ after append")
 

@@ -151,7 +151,7 @@ def test_temperature_and_relaxed_acceptance():
 
 
 def test_config1_moderate_full():
-    rep = run_chain_parity(wl.config(1), steps=2, device=DEV, attn_slots=[0, 7, 31])
+    rep = run_chain_parity(wl.config(1), steps=2, device=DEV, attn_slots=lambda t: [t, 7 + 3 * t, 31 - t])
     assert_clean(rep)
     assert rep["rejections"] > 0
 
@@ -160,14 +160,41 @@ def test_config2_stationary_batch_full_size_sampled_attention():
     # full launch configuration of the benchmark; verify/commit compared on all 256 slots,
     # attention on sampled slots (the oracle needs ~1 s per slot)
     w = wl.config(2, steps=4)
-    rep = run_chain_parity(w, steps=3, device=DEV, attn_slots=[0, 100, 255], check_pools=True)
+    rep = run_chain_parity(w, steps=3, device=DEV, attn_slots=lambda t: [(37 * t) % 256, (100 + 41 * t) % 256, 255 - t],
+                           check_pools=True)
     assert_clean(rep)
     assert rep["positions"] >= 256 * 8
 
 
 def test_config3_long_context_sampled():
-    rep = run_chain_parity(wl.config(3), steps=2, device=DEV, attn_slots=[3])
+    rep = run_chain_parity(wl.config(3), steps=2, device=DEV, attn_slots=lambda t: [(5 * t + 3) % 16])
     assert_clean(rep)
+
+
+def test_config2_hundred_chained_steps_at_full_batch():
+    # the stationary batch as the benchmark definition states it: 100 chained isd_step calls at batch 256 with the
+    # accept lengths fed back; verification, commit, page tables and the free stack are compared on every slot at
+    # every step (about fifty fresh pages per slot come off the stack over the run), attention and the appended
+    # K/V rows on a rotating pair of slots every tenth step
+    w = wl.config(2)
+    assert w.steps == 100 and w.batch == 256
+    pick = lambda t: [(7 * t) % w.batch, (7 * t + 131) % w.batch] if t % 10 == 0 else []
+    rep = run_chain_parity(w, steps=100, device=DEV, attn_slots=pick)
+    assert_clean(rep)
+    assert rep["positions"] > 100 * 256 * 8 and rep["rejections"] > 1000
+    assert 3.5 < rep["tpf"] < 4.6            # the workload is tuned to the paper's stride-8 operating point (TPF 4.01)
+
+
+@pytest.mark.parametrize("stride,batch", [(2, 1), (2, 512), (16, 1), (16, 512), (8, 64), (4, 256)])
+def test_config4_sweep_points(stride, batch):
+    # corners and centre of the sweep (stride in 2..16 x batch in 1..512 at context 4,096, seeds fixed per point):
+    # two chained steps (an NP step, then a P step) with verification and commit compared on every slot and
+    # attention on a sample of at most three slots that moves with the step
+    w = wl.sweep_point(stride, batch)
+    pick = lambda t: sorted({(11 * t + 1) % batch, (batch // 2 + 5 * t) % batch, (batch - 1 - t) % batch})
+    rep = run_chain_parity(w, steps=2, device=DEV, attn_slots=pick)
+    assert_clean(rep)
+    assert rep["positions"] == batch * stride + batch * (2 * stride - 1)
 
 
 def _fresh(w, **kw):
