@@ -66,8 +66,9 @@ def config(i: int, **kw) -> Workload:
         w = Workload("moderate_b32_n4_ctx512-4096", batch=32, stride=4, ctx_min=512, ctx_max=4096,
                      logit_sigma=3.0, peaked_frac=0.2, propose_mode=0, seed=1)
     elif i == 2:
+        # argmax proposals judged against a point mass: the paper's serving setting in its distribution-preserving form
         w = Workload("stationary_b256_n8_ctx1k-8k", batch=256, stride=8, ctx_min=1024, ctx_max=8192,
-                     logit_sigma=3.0, peaked_frac=0.9, steps=100, seed=2)
+                     logit_sigma=3.0, peaked_frac=0.9, steps=100, q_mode=1, seed=2)
     elif i == 3:
         w = Workload("longctx_b16_n4_ctx32k", batch=16, stride=4, ctx_min=32768, ctx_max=32768,
                      logit_sigma=2.0, propose_mode=0, seed=3)
@@ -82,7 +83,7 @@ def sweep_point(stride: int, batch: int) -> Workload:
     strides, batches = [2, 4, 8, 16], [1, 8, 64, 256, 512]
     seed = 5000 + 100 * strides.index(stride) + batches.index(batch)
     return Workload(f"sweep_n{stride}_b{batch}_ctx4096", batch=batch, stride=stride, ctx_min=4096,
-                    ctx_max=4096, peaked_frac=0.9, seed=seed)
+                    ctx_max=4096, peaked_frac=0.9, q_mode=1, seed=seed)
 
 
 def _gen(device, *keys) -> torch.Generator:

@@ -159,7 +159,9 @@ def test_config1_moderate_full():
 def test_config2_stationary_batch_full_size_sampled_attention():
     # full launch configuration of the benchmark; verify/commit compared on all 256 slots,
     # attention on sampled slots (the oracle needs ~1 s per slot)
-    w = wl.config(2, steps=4)
+    # (here with sampled proposals judged against their softmax law, Algorithm 1 to the letter; the 100-step chain
+    # below runs the workload's own pairing, argmax proposals against a point mass)
+    w = wl.config(2, steps=4, propose_mode=0, q_mode=0)
     rep = run_chain_parity(w, steps=3, device=DEV, attn_slots=lambda t: [(37 * t) % 256, (100 + 41 * t) % 256, 255 - t],
                            check_pools=True)
     assert_clean(rep)
@@ -185,12 +187,14 @@ def test_config2_hundred_chained_steps_at_full_batch():
     assert 3.5 < rep["tpf"] < 4.6            # the workload is tuned to the paper's stride-8 operating point (TPF 4.01)
 
 
-@pytest.mark.parametrize("stride,batch", [(2, 1), (2, 512), (16, 1), (16, 512), (8, 64), (4, 256)])
-def test_config4_sweep_points(stride, batch):
+@pytest.mark.parametrize("stride,batch,pairing", [(2, 1, (1, 1)), (2, 512, (1, 1)), (16, 1, (0, 0)), (16, 512, (1, 1)),
+                                                  (8, 64, (1, 0)), (4, 256, (0, 0))])
+def test_config4_sweep_points(stride, batch, pairing):
     # corners and centre of the sweep (stride in 2..16 x batch in 1..512 at context 4,096, seeds fixed per point):
     # two chained steps (an NP step, then a P step) with verification and commit compared on every slot and
     # attention on a sample of at most three slots that moves with the step
-    w = wl.sweep_point(stride, batch)
+    from dataclasses import replace
+    w = replace(wl.sweep_point(stride, batch), propose_mode=pairing[0], q_mode=pairing[1])
     pick = lambda t: sorted({(11 * t + 1) % batch, (batch // 2 + 5 * t) % batch, (batch - 1 - t) % batch})
     rep = run_chain_parity(w, steps=2, device=DEV, attn_slots=pick)
     assert_clean(rep)
