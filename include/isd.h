@@ -303,6 +303,18 @@ int isd_read_status(isd_ctx* ctx, uint32_t* host_status, void* cuda_stream);
  */
 int isd_set_wait_limit(isd_ctx* ctx, uint32_t milliseconds);
 
+/*
+ * Test hook for the wait limit (the paper has no counterpart; not for production use).  The fused LoRA layer
+ * hands blocks of its intermediate t from the CTAs that compute them to the CTAs that read them through one
+ * readiness counter per row block, which a reader waits on until it EQUALS the number of blocks.  This call
+ * writes `value` into the counter of `row_block` (asynchronously on `cuda_stream`), so that with a value the
+ * count can never reach, the readers of that row block wait until their time limit runs out: the next
+ * isd_lora_linear on this context then returns normally, the rows of that block in y are incomplete, and
+ * isd_read_status carries ISD_ST_KERNEL_TIMEOUT.  The kernel clears all counters when it ends, so the call
+ * after that is an ordinary one again.  Nothing faults or hangs; set a short limit first (isd_set_wait_limit).
+ */
+int isd_test_preset_lora_counter(isd_ctx* ctx, int32_t row_block, uint32_t value, void* cuda_stream);
+
 /* Optional instrumentation (the paper has no counterpart): cudaEvent_t handles, passed as void*,
  * that later calls record on their stream immediately before / after the attention main kernel
  * (attn_*) and the kernels of isd_verify together (verify_*).  NULL switches a pair off.

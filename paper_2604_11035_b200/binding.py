@@ -20,7 +20,8 @@ ST_KERNEL_TIMEOUT = 0x80000000
 
 EXPORTS = ["isd_create", "isd_destroy", "isd_attn", "isd_verify", "isd_commit", "isd_step",
            "isd_release", "isd_read_status", "isd_set_profile_events", "isd_launch_count", "isd_strerror",
-           "isd_verify_static", "isd_step_layers", "isd_set_step_counter", "isd_lora_linear", "isd_set_wait_limit"]
+           "isd_verify_static", "isd_step_layers", "isd_set_step_counter", "isd_lora_linear", "isd_set_wait_limit",
+           "isd_test_preset_lora_counter"]
 
 
 class IsdConfig(C.Structure):
@@ -90,6 +91,8 @@ def load():
         lib.isd_lora_linear.restype = C.c_int
         lib.isd_set_wait_limit.argtypes = [vp, C.c_uint32]
         lib.isd_set_wait_limit.restype = C.c_int
+        lib.isd_test_preset_lora_counter.argtypes = [vp, C.c_int32, C.c_uint32, vp]
+        lib.isd_test_preset_lora_counter.restype = C.c_int
         lib.isd_launch_count.argtypes = [vp]
         lib.isd_launch_count.restype = C.c_int64
         lib.isd_strerror.argtypes = [C.c_int]
@@ -233,6 +236,10 @@ class Isd:
     def isd_set_wait_limit(self, milliseconds: int):
         """Time limit of every wait inside the kernels (default 250 ms); see include/isd.h."""
         _check(self.lib.isd_set_wait_limit(self.ctx, int(milliseconds)), "isd_set_wait_limit")
+
+    def isd_test_preset_lora_counter(self, row_block: int, value: int):
+        """Test hook: see include/isd.h (makes the readers of one row block of t run into their wait limit)."""
+        _check(self.lib.isd_test_preset_lora_counter(self.ctx, row_block, value, _stream()), "isd_test_preset_lora_counter")
 
     def isd_release(self, st, slots):
         s = self.state_struct(st)

@@ -230,6 +230,13 @@ int isd_set_wait_limit(isd_ctx* ctx, uint32_t milliseconds) {
   return ISD_OK;
 }
 
+int isd_test_preset_lora_counter(isd_ctx* ctx, int32_t row_block, uint32_t value, void* cuda_stream) {
+  if (!ctx || !ctx->lora_flags || row_block < 0 || row_block >= 4096) return ISD_ERR_INVALID_ARG;
+  // (pageable host source: the runtime stages the four bytes before it returns)
+  return cudaMemcpyAsync(ctx->lora_flags + row_block, &value, sizeof(uint32_t), cudaMemcpyHostToDevice,
+                         reinterpret_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+}
+
 int isd_set_step_counter(isd_ctx* ctx, uint32_t* device_counter) {
   if (!ctx) return ISD_ERR_INVALID_ARG;
   ctx->step_counter = device_counter;
