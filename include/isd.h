@@ -315,6 +315,19 @@ int isd_set_wait_limit(isd_ctx* ctx, uint32_t milliseconds);
  */
 int isd_test_preset_lora_counter(isd_ctx* ctx, int32_t row_block, uint32_t value, void* cuda_stream);
 
+/*
+ * Test hook, host only (the paper has no counterpart; needs no GPU): how isd_lora_linear assigns its work for a
+ * shape on a GPU of num_sms SMs.  For unit `unit_index` (a CTA, or a pair of CTAs, in block-index order) of the
+ * launch that writes y and its work item `item`: out[0] = kernel form (2 CTA pairs with the down-projection fused,
+ * 1 one-CTA kernel fused, 0 two launches), out[1] = units of the launch, out[2] = items of this unit, out[3] = 1 for
+ * a block of the intermediate t / 0 for an output tile or strip, out[4..6] = first row, first column, columns,
+ * out[7..8] = rows and columns of a full tile (out[3..6] = -1 past the unit's last item).  The CPU tests use it to
+ * check that every output element is computed exactly once and that the blocks of t fall to the lowest block
+ * indices, whose CTAs the hardware makes resident first.
+ */
+int isd_test_lora_work_item(int32_t m, int32_t n, int32_t rank, int32_t num_sms, int32_t unit_index, int32_t item,
+                            int32_t* out);
+
 /* Optional instrumentation (the paper has no counterpart): cudaEvent_t handles, passed as void*,
  * that later calls record on their stream immediately before / after the attention main kernel
  * (attn_*) and the kernels of isd_verify together (verify_*).  NULL switches a pair off.

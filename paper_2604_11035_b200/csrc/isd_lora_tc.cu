@@ -26,6 +26,7 @@
 #include <cuda_bf16.h>
 
 #include "isd_internal.cuh"
+#include "isd_lora_work.cuh"
 
 namespace {
 
@@ -173,40 +174,14 @@ gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, c
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  const int tiles_m = (P.M + kBM - 1) / kBM, tiles_n = (P.N + BN - 1) / BN;
-  const int n_tiles = tiles_m * tiles_n;
   const int ks1 = P.K1 / kBK, ks2 = P.K2 / kBK, ks = ks1 + ks2;  // K slices per tile
-  // Work items of this CTA.  Work is assigned by the mirrored index v = grid - 1 - blockIdx.x.  With the fused
-  // down-projection the CTAs v >= grid - tiles_m * t_chunks (the ones with the fewest output tiles) start with one
-  // block of t; then come the output tiles v, v + grid, ...  The mirror puts the blocks of t on the LOWEST block
-  // indices: the hardware hands out CTAs in index order, so the producers of t are resident before any consumer of
-  // it, and they never wait before they publish.  A grid that is only partly resident (another kernel holds SMs)
-  // therefore still makes progress; the consumers' bounded spin below needs no co-residency of the whole grid.
-  const int v_cta = (int)gridDim.x - 1 - (int)blockIdx.x;
-  const int t_item = P.fuse ? v_cta - ((int)gridDim.x - tiles_m * P.t_chunks) : -1;  // >= 0: this CTA computes a block of t
-  const int t_block = t_item >= 0 ? t_item % tiles_m : 0, t_chunk = t_item >= 0 ? t_item / tiles_m : 0;
-  const int n_pre = t_item >= 0 ? 1 : 0;
-  // The output tiles: whole rounds of the grid as 128 x BN tiles; the tiles of the last, partial round are cut
-  // into tail_split column strips each, one strip per CTA, so that more CTAs share that round (strip u: tile
-  // tail0 + u / tail_split, columns (u % tail_split) * BN / tail_split ...).  No CTA gets a strip and a block of t.
-  const int rounds = n_tiles / (int)gridDim.x, tail0 = rounds * (int)gridDim.x;
-  const int n_strips = (n_tiles - tail0) * P.tail_split, strip_cols = BN / P.tail_split;
-  const int n_items = n_pre + rounds + (v_cta < n_strips ? 1 : 0);
-  struct Item { bool pre; int m0, n0, cols; };
-  auto item = [&](int it) {
-    Item w;
-    w.pre = it < n_pre;
-    if (w.pre) {
-      w.m0 = t_block * kBM; w.n0 = t_chunk * P.Rc; w.cols = P.Rc;
-    } else if (it - n_pre < rounds) {
-      const int tile = v_cta + (it - n_pre) * (int)gridDim.x;
-      w.m0 = (tile % tiles_m) * kBM; w.n0 = (tile / tiles_m) * BN; w.cols = BN;  // neighbouring CTAs share a B panel
-    } else {
-      const int tile = tail0 + v_cta / P.tail_split;
-      w.m0 = (tile % tiles_m) * kBM; w.n0 = (tile / tiles_m) * BN + (v_cta % P.tail_split) * strip_cols; w.cols = strip_cols;
-    }
-    return w;
-  };
+  // Work items of this CTA (isd_lora_work.cuh): assigned by the mirrored block index, so that the blocks of t fall
+  // to the lowest block indices; the readers' bounded wait below needs no co-residency of the whole grid.
+  LoraWork work;
+  work.init((int)blockIdx.x, (int)gridDim.x, P.M, P.N, kBM, BN, P.fuse, P.t_chunks, P.Rc, P.tail_split);
+  const int tiles_m = work.tiles_m, n_items = work.n_items, t_block = work.t_block;
+  using Item = LoraWorkItem;
+  auto item = [&](int it) { return work.item(it); };
 
   if (warp == 4) {
     // ============================================================================ TMA producer
@@ -419,34 +394,14 @@ gemm_tc2_kernel(const GemmParams P, const __grid_constant__ CUtensorMap map_a1, 
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  const int tiles_m = (P.M + 2 * kBM - 1) / (2 * kBM), tiles_n = (P.N + kBN2 - 1) / kBN2;
-  const int n_tiles = tiles_m * tiles_n;
   const int ks1 = P.K1 / kBK, ks2 = P.K2 / kBK, ks = ks1 + ks2;
-  // work items of the pair, as in the one-CTA kernel and by the same mirrored index (the pairs with the lowest
-  // block indices compute the blocks of t, so the producers of t are resident before any of its consumers):
-  // a block of t first, whole tiles, one column strip
-  const int n_pairs = (int)gridDim.x >> 1, pr = n_pairs - 1 - ((int)blockIdx.x >> 1);
-  const int t_item = P.fuse ? pr - (n_pairs - tiles_m * P.t_chunks) : -1;
-  const int t_block = t_item >= 0 ? t_item % tiles_m : 0, t_chunk = t_item >= 0 ? t_item / tiles_m : 0;
-  const int n_pre = t_item >= 0 ? 1 : 0;
-  const int rounds = n_tiles / n_pairs, tail0 = rounds * n_pairs;
-  const int n_strips = (n_tiles - tail0) * P.tail_split, strip_cols = kBN2 / P.tail_split;
-  const int n_items = n_pre + rounds + (pr < n_strips ? 1 : 0);
-  struct Item { bool pre; int m0, n0, cols; };
-  auto item = [&](int it) {
-    Item w;
-    w.pre = it < n_pre;
-    if (w.pre) {
-      w.m0 = t_block * 2 * kBM; w.n0 = t_chunk * P.Rc; w.cols = P.Rc;
-    } else if (it - n_pre < rounds) {
-      const int tile = pr + (it - n_pre) * n_pairs;
-      w.m0 = (tile % tiles_m) * 2 * kBM; w.n0 = (tile / tiles_m) * kBN2; w.cols = kBN2;
-    } else {
-      const int tile = tail0 + pr / P.tail_split;
-      w.m0 = (tile % tiles_m) * 2 * kBM; w.n0 = (tile / tiles_m) * kBN2 + (pr % P.tail_split) * strip_cols; w.cols = strip_cols;
-    }
-    return w;
-  };
+  // work items of the pair (isd_lora_work.cuh), by the mirrored pair index: a block of t first, whole tiles, one
+  // column strip
+  LoraWork work;
+  work.init((int)blockIdx.x >> 1, (int)gridDim.x >> 1, P.M, P.N, 2 * kBM, kBN2, P.fuse, P.t_chunks, P.Rc, P.tail_split);
+  const int tiles_m = work.tiles_m, n_items = work.n_items, t_block = work.t_block;
+  using Item = LoraWorkItem;
+  auto item = [&](int it) { return work.item(it); };
 
   if (warp == 4) {
     // ============================================================================ TMA producer (both CTAs)
@@ -632,16 +587,9 @@ int launch_gemm(isd_ctx* ctx, GemmParams P, const void* a1, const void* b1, cons
   if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&mb2, b2, P.N, P.K2, BN) : encode_matrix(&mb2, b1, P.N, P.K1, BN);
   if (rc == ISD_OK) rc = P.fuse ? encode_matrix(&mbt, bt, P.R, P.K1, P.Rc) : encode_matrix(&mbt, b1, P.N, P.K1, BN);
   if (rc != ISD_OK) return rc;
-  const int tiles_m = (P.M + kBM - 1) / kBM;
-  const int n_tiles = tiles_m * ((P.N + BN - 1) / BN), n_t = P.fuse ? tiles_m * P.t_chunks : 0;
-  int tiles = n_tiles;
-  if (tiles < n_t) tiles = n_t;  // every block of t needs a CTA
-  const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
-  // column strips for the last, partial round of tiles: as many as the CTAs without a block of t can take
-  const int tail = n_tiles % grid;
-  P.tail_split = 1;
-  for (int sp = 4; sp > 1; sp >>= 1)
-    if (tail > 0 && tail * sp <= grid - n_t && (BN / sp) % 32 == 0) { P.tail_split = sp; break; }
+  // grid and column strips of the last, partial round (isd_lora_work.cuh)
+  int grid;
+  lora_grid(P.M, P.N, kBM, BN, P.fuse, P.t_chunks, ctx->num_sms, true, grid, P.tail_split);
   rc = encode_matrix(&mb1n, b1, P.N, P.K1, BN / P.tail_split);
   if (rc == ISD_OK) rc = P.K2 ? encode_matrix(&mb2n, b2, P.N, P.K2, BN / P.tail_split) : encode_matrix(&mb2n, b1, P.N, P.K1, BN / P.tail_split);
   if (rc != ISD_OK) return rc;
@@ -660,14 +608,8 @@ int launch_gemm_pair(isd_ctx* ctx, GemmParams P, const void* a1, const void* b1,
       return ISD_ERR_CUDA;
     attr_set = true;
   }
-  const int tiles_m = (P.M + 2 * kBM - 1) / (2 * kBM);
-  const int n_tiles = tiles_m * ((P.N + kBN2 - 1) / kBN2), n_t = P.fuse ? tiles_m * P.t_chunks : 0;
-  int pairs = n_tiles < n_t ? n_t : n_tiles;
-  if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;
-  const int tail = n_tiles % pairs;
-  P.tail_split = 1;
-  for (int sp = 4; sp > 1; sp >>= 1)
-    if (tail > 0 && tail * sp <= pairs - n_t) { P.tail_split = sp; break; }
+  int pairs;
+  lora_grid(P.M, P.N, 2 * kBM, kBN2, P.fuse, P.t_chunks, ctx->num_sms / 2, false, pairs, P.tail_split);
   const int strip_half = kBN2 / P.tail_split / 2;
   CUtensorMap ma1, mb1, ma2, mb2, mbt, mb1n, mb2n;
   int rc = encode_matrix(&ma1, a1, P.M, P.K1, kBM);
@@ -699,7 +641,6 @@ void isd_lora_destroy(isd_ctx* ctx) {
 constexpr int kLoraBN = 256;
 
 int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t stream) {
-  const int tiles_m = (a->m + kBM - 1) / kBM;
   GemmParams P2;
   P2.M = a->m; P2.N = a->n; P2.K1 = a->k; P2.K2 = a->rank;
   P2.c = reinterpret_cast<__nv_bfloat16*>(a->y); P2.gate = nullptr; P2.scale = 1.f;
@@ -710,21 +651,18 @@ int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t st
   // One launch when t divides into blocks of one MMA's width (rank <= the tile width, or a multiple of it) and
   // every block gets its own CTA: the last CTAs compute t = gate * scale * (x A^T) block by block before their
   // output tiles, and the second K segment of y = x W^T + t B^T waits for the blocks of the rows it reads.
-  const int chunks = a->rank <= kLoraBN ? 1 : (a->rank % kLoraBN == 0 ? a->rank / kLoraBN : 0);
-  // The form is chosen by shape alone: CTA pairs when every block of t gets a pair of its own, else the one-CTA
-  // kernel with the fused down-projection when every block gets a CTA, else two launches.
-  const int blocks2 = (a->m + 2 * kBM - 1) / (2 * kBM);  // 256-row blocks
-  if (chunks > 0 && blocks2 * chunks <= ctx->num_sms / 2 && blocks2 <= kMaxFlags) {
+  const LoraPlan plan = lora_plan(a->m, a->n, a->rank, ctx->num_sms, kMaxFlags);
+  if (plan.form == 2) {
     // CTA pairs: 256 x 256 tiles, blocks of t of 256 rows
     P2.fuse = 1;
-    P2.t_chunks = chunks;
-    P2.Rc = a->rank / chunks;
+    P2.t_chunks = plan.t_chunks;
+    P2.Rc = plan.Rc;
     return launch_gemm_pair(ctx, P2, a->x, a->w, a->t, a->b, a->a, stream);
   }
-  if (chunks > 0 && tiles_m * chunks <= ctx->num_sms && tiles_m <= kMaxFlags) {
+  if (plan.form == 1) {
     P2.fuse = 1;
-    P2.t_chunks = chunks;
-    P2.Rc = a->rank / chunks;
+    P2.t_chunks = plan.t_chunks;
+    P2.Rc = plan.Rc;
     return launch_gemm<kLoraBN>(ctx, P2, a->x, a->w, a->t, a->b, a->a, stream);
   }
   // Otherwise two launches.  1. t = gate * scale * (x A^T): N = rank, one K segment
@@ -734,4 +672,22 @@ int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t st
   if (rc != ISD_OK) return rc;
   // 2. y = x W^T + t B^T: two K segments, no gate (it is already in t)
   return launch_gemm<kLoraBN>(ctx, P2, a->x, a->w, a->t, a->b, nullptr, stream);
+}
+
+// Host-only view of the work assignment (no GPU needed): what unit `unit_index` of the launch that writes y does as
+// its item `item`.  out = {form, units, items of this unit, pre, m0, n0, cols, tile rows, tile columns}.
+extern "C" int isd_test_lora_work_item(int32_t m, int32_t n, int32_t rank, int32_t num_sms, int32_t unit_index, int32_t item,
+                                       int32_t* out) {
+  if (!out || m < 1 || n < 1 || rank < 1 || num_sms < 2) return ISD_ERR_INVALID_ARG;
+  const LoraPlan p = lora_plan(m, n, rank, num_sms, kMaxFlags);
+  if (unit_index < 0 || unit_index >= p.units) return ISD_ERR_INVALID_ARG;
+  LoraWork w;
+  w.init(unit_index, p.units, m, n, p.bm, p.bn, p.fuse, p.t_chunks, p.Rc, p.tail_split);
+  out[0] = p.form; out[1] = p.units; out[2] = w.n_items; out[7] = p.bm; out[8] = p.bn;
+  out[3] = out[4] = out[5] = out[6] = -1;
+  if (item >= 0 && item < w.n_items) {
+    const LoraWorkItem it = w.item(item);
+    out[3] = it.pre; out[4] = it.m0; out[5] = it.n0; out[6] = it.cols;
+  }
+  return ISD_OK;
 }
