@@ -171,11 +171,14 @@ def run_model_step(args):
         eng.isd_step_layers(st, layers, cur, prev, out, 0, st_struct)
 
     graph = None
+    launches_in_graph = 0
     if args.graph:
         torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()
+        n0 = eng.isd_launch_count()
         with torch.cuda.graph(graph):
             launch()
+        launches_in_graph = eng.isd_launch_count() - n0      # kernels recorded by the capture = launched per replay
     ev = lambda: torch.cuda.Event(enable_timing=True)
     e_step = [(ev(), ev()) for _ in range(W + K)]
     pos_acc = torch.zeros(W + K, dtype=torch.int64, device=dev)
@@ -225,7 +228,7 @@ def run_model_step(args):
                    "ctx": [w.ctx_min, w.ctx_max], "l2": "flushed before every step (512 MB written, then read back)"},
         "emitted_tokens_per_s": int(emit_acc[W:].sum().item()) / t_total,
         "step_algorithmic_gbs": gbs, "step_frac_of_8TBs": gbs / HBM_NOMINAL_GBS, "step_frac_of_measured_copy": gbs / peak,
-        "gpu_launches": launches if graph is None else K * (3 * L + (3 if w.top_k else 2)), "launches_issued_by_host": launches,
+        "gpu_launches": launches if graph is None else K * launches_in_graph, "launches_issued_by_host": launches,
         "status_word": status, "clocks": clocks,
     }
     print(json.dumps(line))

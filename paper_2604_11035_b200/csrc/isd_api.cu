@@ -175,15 +175,10 @@ int isd_commit(isd_ctx* ctx, isd_batch_state* st, const isd_verify_out* out, voi
   return isd_launch_commit(ctx, st, out, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
-// Verification followed by the commit.  With plain softmax laws the last CTA of the sampling kernel commits
-// (no kernel of its own for it); the filtered path keeps the commit kernel.
+// Verification followed by the commit: the last CTA of the last verification kernel commits (no kernel of its
+// own for it), except on the filtered path when the proposal-law rows have to be streamed by a second kernel.
 static int verify_then_commit(isd_ctx* ctx, isd_batch_state* st, const void* logits_cur, const void* q_prev_logits,
                               uint64_t step, const isd_verify_out* out, void* cuda_stream) {
-  if (ctx->cfg.top_k > 0) {
-    const int rc = isd_verify(ctx, st, logits_cur, q_prev_logits, step, out, cuda_stream);
-    if (rc != ISD_OK) return rc;
-    return isd_commit(ctx, st, out, cuda_stream);
-  }
   int rc = check_state(st);
   if (rc != ISD_OK) return rc;
   rc = check_out(ctx, out);
@@ -191,8 +186,14 @@ static int verify_then_commit(isd_ctx* ctx, isd_batch_state* st, const void* log
   if (!logits_cur || step > 0xFFFFFFFFull) return ISD_ERR_INVALID_ARG;
   if (ctx->cfg.stride > 1 && !st->q_stats) return ISD_ERR_INVALID_ARG;
   if (!aligned16(logits_cur) || (q_prev_logits && !aligned16(q_prev_logits))) return ISD_ERR_ALIGNMENT;
-  return isd_launch_verify(ctx, st, logits_cur, q_prev_logits, (uint32_t)step, out,
-                           reinterpret_cast<cudaStream_t>(cuda_stream), st);
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (ctx->cfg.top_k > 0) {
+    bool committed = false;
+    rc = isd_launch_verify_topk(ctx, st, logits_cur, q_prev_logits, (uint32_t)step, out, s, st, &committed);
+    if (rc != ISD_OK || committed) return rc;
+    return isd_launch_commit(ctx, st, out, s);
+  }
+  return isd_launch_verify(ctx, st, logits_cur, q_prev_logits, (uint32_t)step, out, s, st);
 }
 
 int isd_step(isd_ctx* ctx, isd_batch_state* st, const isd_step_args* a, uint64_t step, void* cuda_stream) {

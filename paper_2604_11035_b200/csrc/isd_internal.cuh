@@ -365,9 +365,10 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
                       cudaStream_t stream, isd_batch_state* commit_st = nullptr);
 int isd_verify_topk_create(isd_ctx* ctx);
 void isd_verify_topk_destroy(isd_ctx* ctx);
+// commit_st != nullptr: the row kernel's last CTA commits when no decide kernel follows it; *committed says whether
 int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
                            const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
-                           cudaStream_t stream);
+                           cudaStream_t stream, isd_batch_state* commit_st = nullptr, bool* committed = nullptr);
 int isd_launch_lora_linear(isd_ctx* ctx, const isd_lora_args* a, cudaStream_t stream);
 int isd_lora_create(isd_ctx* ctx);
 void isd_lora_destroy(isd_ctx* ctx);

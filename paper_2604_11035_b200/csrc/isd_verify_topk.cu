@@ -19,6 +19,7 @@
 //      pieces and draws the replacement.
 #include "isd_internal.cuh"
 #include "isd_stream.cuh"
+#include "isd_commit.cuh"
 
 #include <cooperative_groups.h>
 
@@ -61,6 +62,10 @@ struct TopkParams {
   int* nuc_bad;               // [B, Q] 1 = the row holds a NaN or +inf
   double* nuc_lse;            // [B, Q] log-normaliser of the support
   int* row_ticket;            // [B] rows of the slot that are done (zero between launches)
+  // isd_step: the CTA of the row kernel that finishes last commits the batch (fuse_commit != 0)
+  int fuse_commit;
+  int* step_ticket;
+  CommitParams commit;
 };
 
 struct TopkShared {
@@ -755,9 +760,7 @@ __device__ void draw_residual(const TopkParams& P, const TopkShared& sh, const i
 // Pass 1: the top-k list of every valid row
 // ------------------------------------------------------------------------------------------------
 template <int DT>
-__global__ void __launch_bounds__(kThreads + 32, 5) topk_rows_kernel(const TopkParams P) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
+__device__ __forceinline__ void topk_rows_body(const TopkParams& P, TopkShared& sh) {
   const int b = blockIdx.x, r = blockIdx.y;
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
@@ -822,6 +825,30 @@ __global__ void __launch_bounds__(kThreads + 32, 5) topk_rows_kernel(const TopkP
   }
 }
 
+template <int DT>
+__global__ void __launch_bounds__(kThreads + 32, 5) topk_rows_kernel(const TopkParams P) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
+  pdl_wait();
+  pdl_launch_dependents();
+  topk_rows_body<DT>(P, sh);
+  if (!P.fuse_commit) return;
+  // ---- isd_step, when this kernel is the whole verification: the CTA that finishes last (a ticket over the grid;
+  // nobody waits) commits the batch
+  __shared__ int sm_commit[36];
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int arrived = atomicAdd(P.step_ticket, 1);
+    sm_commit[35] = (arrived == (int)(gridDim.x * gridDim.y) - 1);
+  }
+  __syncthreads();
+  if (!sm_commit[35]) return;
+  if (threadIdx.x == 0) *P.step_ticket = 0;  // ready for the next call
+  __threadfence();
+  commit_block(P.commit, sm_commit, sm_commit + 33);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Pass 2: everything else, one CTA per slot
 // ------------------------------------------------------------------------------------------------
@@ -838,6 +865,8 @@ __global__ void __cluster_dims__(kQSplit, 1, 1) __launch_bounds__(kThreads + 32)
   // the same decision, so they leave before the cluster barrier together or not at all.
   const int b = blockIdx.x / kQSplit, piece = blockIdx.x % kQSplit;
   const bool lead = piece == 0;
+  pdl_wait();
+  pdl_launch_dependents();
   if (!P.active[b]) return;
   const int nv = P.n_ver[b];
   if (nv < 0 || nv > P.N - 1) return;
@@ -938,7 +967,7 @@ void isd_verify_topk_destroy(isd_ctx* ctx) {
 
 int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* logits_cur,
                            const void* q_prev_logits, uint32_t step, const isd_verify_out* out,
-                           cudaStream_t stream) {
+                           cudaStream_t stream, isd_batch_state* commit_st, bool* committed) {
   const isd_config& c = ctx->cfg;
   TopkParams P;
   P.B = c.batch; P.N = c.stride; P.Q = ctx->Q; P.V = c.vocab;
@@ -970,15 +999,21 @@ int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* 
   const dim3 grid1(c.batch, ctx->Q);
   // a second kernel only when rejections need proposal-law rows that have to be streamed
   const bool stream_q = c.q_mode == 0 && q_prev_logits != nullptr && !P.prev_valid;
+  // the row kernel commits by itself when it is the whole verification (no decide kernel after it)
+  P.fuse_commit = (commit_st != nullptr && !stream_q && ctx->step_ticket != nullptr) ? 1 : 0;
+  P.step_ticket = ctx->step_ticket;
+  P.commit = make_commit_params(ctx, P.fuse_commit ? commit_st : st, out);
+  if (committed) *committed = P.fuse_commit != 0;
   if (ctx->ev_verify0) cudaEventRecord(ctx->ev_verify0, stream);
+  cudaError_t e;
   if (c.logits_dtype == ISD_LOGITS_BF16) {
-    topk_rows_kernel<ISD_LOGITS_BF16><<<grid1, kThreads + 32, kTopkSmem, stream>>>(P);
+    e = isd_launch_pdl(topk_rows_kernel<ISD_LOGITS_BF16>, grid1, dim3(kThreads + 32), kTopkSmem, stream, P);
     if (stream_q) topk_decide_kernel<ISD_LOGITS_BF16><<<c.batch * kQSplit, kThreads + 32, kTopkSmem, stream>>>(P);
   } else {
-    topk_rows_kernel<ISD_LOGITS_F32><<<grid1, kThreads + 32, kTopkSmem, stream>>>(P);
+    e = isd_launch_pdl(topk_rows_kernel<ISD_LOGITS_F32>, grid1, dim3(kThreads + 32), kTopkSmem, stream, P);
     if (stream_q) topk_decide_kernel<ISD_LOGITS_F32><<<c.batch * kQSplit, kThreads + 32, kTopkSmem, stream>>>(P);
   }
   if (ctx->ev_verify1) cudaEventRecord(ctx->ev_verify1, stream);
   ctx->launches += stream_q ? 2 : 1;
-  return cudaGetLastError() == cudaSuccess ? ISD_OK : ISD_ERR_CUDA;
+  return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ISD_OK : ISD_ERR_CUDA;
 }
