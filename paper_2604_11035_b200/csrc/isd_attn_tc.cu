@@ -203,6 +203,15 @@ __device__ __forceinline__ uint32_t pack_bf16_alu(float a, float b) {
   return d;
 }
 
+// bf16 pair (a in the low half, b in the high half) with the conversion instruction: one instruction instead of
+// three, which matters more than the pipe it runs on -- the softmax warps are bound by instruction issue (one warp
+// per scheduler), not by the transcendental unit
+__device__ __forceinline__ uint32_t pack_bf16_cvt(float a, float b) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(b), "f"(a));
+  return d;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Work split: identical, independent enumeration in every warp role
 // ------------------------------------------------------------------------------------------------
@@ -514,20 +523,28 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
     const float mref = (m2 == -INFINITY) ? 0.f : m2;
     const uint64_t sc2 = pack2(P.scale2, P.scale2), nm2 = pack2(-mref, -mref);
     uint64_t acc[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
-    uint32_t pk[64];
+    // F = 2: the thread's 32 packed columns go straight to its half of the P tile and zeros to the other half (two
+    // stores at run-time column offsets); F = 4 places its 16 columns among zeros with compile-time selects
+    uint32_t pk[F == 2 ? 32 : 64];
+    if (F == 4) {
 #pragma unroll
-    for (int c = 0; c < 64; ++c) pk[c] = 0u;
+      for (int c = 0; c < 64; ++c) pk[c] = 0u;
+    }
 #pragma unroll
     for (int c = 0; c < C / 2; ++c) {
       float x0, x1;
       unpack2(fma2(pack2(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1])), sc2, nm2), x0, x1);
       const float p0 = ex2f(x0), p1 = ex2f(x1);
       acc[c & 3] = add2(acc[c & 3], pack2(p0, p1));
-      const uint32_t w = pack_bf16_alu(p0, p1);
-      // static placement: replica `part` owns packed columns [part * C / 2, (part + 1) * C / 2)
+      const uint32_t w = pack_bf16_cvt(p0, p1);
+      if (F == 4) {
+        // static placement: replica `part` owns packed columns [part * C / 2, (part + 1) * C / 2)
 #pragma unroll
-      for (int pp = 0; pp < F; ++pp)
-        if (pp == part) pk[pp * (C / 2) + c] = w;
+        for (int pp = 0; pp < F; ++pp)
+          if (pp == part) pk[pp * (C / 2) + c] = w;
+      } else {
+        pk[c] = w;
+      }
     }
     float lsum;
     {
@@ -536,8 +553,16 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
       unpack2(add2(acc[2], acc[3]), b0, b1);
       lsum = (a0 + a1) + (b0 + b1);
     }
-    TMEM_ST32(ts, pk, 0);
-    TMEM_ST32(ts + 32, pk, 32);
+    if (F == 2) {
+      uint32_t zero[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) zero[c] = 0u;
+      TMEM_ST32(ts + (uint32_t)part * 32u, pk, 0);
+      TMEM_ST32(ts + (uint32_t)(1 - part) * 32u, zero, 0);
+    } else {
+      TMEM_ST32(ts, pk, 0);
+      TMEM_ST32(ts + 32, pk, F == 2 ? 0 : 32);
+    }
     tmem_wait_st();
     l += lsum;
     tc_fence_before();
