@@ -181,6 +181,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
         "r"(v[o + 29]), "r"(v[o + 30]), "r"(v[o + 31])                                                  \
       : "memory")
 
+#define TMEM_ST16(taddr, v, o)                                                                          \
+  asm volatile(                                                                                         \
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "                                                   \
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"                                       \
+      ::"r"(taddr), "r"(v[o + 0]), "r"(v[o + 1]), "r"(v[o + 2]), "r"(v[o + 3]), "r"(v[o + 4]),          \
+        "r"(v[o + 5]), "r"(v[o + 6]), "r"(v[o + 7]), "r"(v[o + 8]), "r"(v[o + 9]), "r"(v[o + 10]),      \
+        "r"(v[o + 11]), "r"(v[o + 12]), "r"(v[o + 13]), "r"(v[o + 14]), "r"(v[o + 15])                  \
+      : "memory")
+
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -523,28 +532,16 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
     const float mref = (m2 == -INFINITY) ? 0.f : m2;
     const uint64_t sc2 = pack2(P.scale2, P.scale2), nm2 = pack2(-mref, -mref);
     uint64_t acc[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
-    // F = 2: the thread's 32 packed columns go straight to its half of the P tile and zeros to the other half (two
-    // stores at run-time column offsets); F = 4 places its 16 columns among zeros with compile-time selects
-    uint32_t pk[F == 2 ? 32 : 64];
-    if (F == 4) {
-#pragma unroll
-      for (int c = 0; c < 64; ++c) pk[c] = 0u;
-    }
+    // F > 1: the thread's C / 2 packed columns go straight to its replica's part of the P tile and zeros to the
+    // rest (stores at run-time column offsets, no per-element selects)
+    uint32_t pk[C / 2];
 #pragma unroll
     for (int c = 0; c < C / 2; ++c) {
       float x0, x1;
       unpack2(fma2(pack2(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1])), sc2, nm2), x0, x1);
       const float p0 = ex2f(x0), p1 = ex2f(x1);
       acc[c & 3] = add2(acc[c & 3], pack2(p0, p1));
-      const uint32_t w = pack_bf16_cvt(p0, p1);
-      if (F == 4) {
-        // static placement: replica `part` owns packed columns [part * C / 2, (part + 1) * C / 2)
-#pragma unroll
-        for (int pp = 0; pp < F; ++pp)
-          if (pp == part) pk[pp * (C / 2) + c] = w;
-      } else {
-        pk[c] = w;
-      }
+      pk[c] = pack_bf16_cvt(p0, p1);
     }
     float lsum;
     {
@@ -553,15 +550,21 @@ __device__ __forceinline__ bool softmax_segment(const TcParams& P, const Segment
       unpack2(add2(acc[2], acc[3]), b0, b1);
       lsum = (a0 + a1) + (b0 + b1);
     }
-    if (F == 2) {
+    if (F == 1) {
+      TMEM_ST32(ts, pk, 0);
+      TMEM_ST32(ts + 32, pk, 32);
+    } else {
       uint32_t zero[32];
 #pragma unroll
       for (int c = 0; c < 32; ++c) zero[c] = 0u;
-      TMEM_ST32(ts + (uint32_t)part * 32u, pk, 0);
-      TMEM_ST32(ts + (uint32_t)(1 - part) * 32u, zero, 0);
-    } else {
-      TMEM_ST32(ts, pk, 0);
-      TMEM_ST32(ts + 32, pk, F == 2 ? 0 : 32);
+      if (F == 2) {
+        TMEM_ST32(ts + (uint32_t)part * 32u, pk, 0);
+        TMEM_ST32(ts + (uint32_t)(1 - part) * 32u, zero, 0);
+      } else {  // F = 4: own quarter, then zeros over the other quarter of the same half and over the other half
+        TMEM_ST16(ts + (uint32_t)part * 16u, pk, 0);
+        TMEM_ST16(ts + (uint32_t)(part ^ 1) * 16u, zero, 0);
+        TMEM_ST32(ts + (uint32_t)((part >> 1) ^ 1) * 32u, zero, 0);
+      }
     }
     tmem_wait_st();
     l += lsum;
