@@ -86,7 +86,7 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   ctx->sample_splits = ps;
 
   int rc = ISD_OK;
-  if (rc == ISD_OK) rc = dev_alloc(&ctx->row_part, (size_t)rows * rs);
+  if (rc == ISD_OK) rc = dev_alloc(&ctx->row_part, (size_t)rows * rs * 8);  // one partial per worker warp of a row piece
   if (rc == ISD_OK) rc = dev_alloc(&ctx->samp_part, (size_t)c.batch * c.stride * ps);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->row_ticket, c.batch);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->samp_ticket, (size_t)c.batch * c.stride);

@@ -239,7 +239,7 @@ struct OnlineSoftmax {
 // groups of eight logits per stage; fp32: one group from two adjacent vectors).
 template <int DT>
 __device__ __forceinline__ bool row_pass(const VerifyParams& P, RowRing& R, const char* row, int lo, int hi,
-                                         float& m_nat, float& S_out, float& raw_max, int& raw_idx) {
+                                         float& warp_max, float& S_out, float& raw_max, int& raw_idx) {
   constexpr int kElt = DT == ISD_LOGITS_BF16 ? 2 : 4;
   constexpr int U = DT == ISD_LOGITS_BF16 ? 2 : 1;      // groups of eight logits per thread and stage
   constexpr int kStageElems = kRowStageBytes / kElt;
@@ -334,7 +334,7 @@ __device__ __forceinline__ bool row_pass(const VerifyParams& P, RowRing& R, cons
     }
   }
   S_out = os.sum();
-  m_nat = os.M * P.inv_t;
+  warp_max = os.M;  // the same in every lane
   return ok;
 }
 
@@ -353,21 +353,20 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
   // Launch order = (split, slot, k): the rows that the sampling pass reads again come last, so that
   // they are the most recent lines in L2 when it starts.
   const int split = blockIdx.x, b = blockIdx.y, k = blockIdx.z;
-  __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
-  __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
-  __shared__ int sm_last;
   __shared__ RowRing sm_ring;
-  if (threadIdx.x == 0) {  // needs nothing from memory: runs while the kernel before this one drains
+  if (threadIdx.x == kThreads) {  // needs nothing from memory: runs while the kernel before this one drains
     for (int i = 0; i < kRowStages; ++i) {
       ring_mbar_init(ring_smem_u32(&sm_ring.full[i]), 1);
       ring_mbar_init(ring_smem_u32(&sm_ring.empty[i]), kThreads / 32);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  __syncthreads();  // the only CTA-wide barrier of the kernel, still ahead of the wait
   pdl_wait();
   pdl_launch_dependents();
-  if (!P.active[b]) return;
-  const int nv = P.n_ver[b];
+  const int act = P.active[b];
+  const int nv = P.n_ver[b];  // both loads in flight together
+  if (!act) return;
   if (nv < 0 || nv > P.N - 1) {
     if (split == 0 && k == 0 && threadIdx.x == 0) {
       atomicOr(&P.slot_status[b], ISD_ST_SLOT_CAPACITY);
@@ -384,7 +383,6 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
   const char* row = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + r) * (size_t)P.V * elt;
   int lo, hi;
   chunk_range(P.V, P.row_splits, split, lo, hi);
-  __syncthreads();
   if (threadIdx.x >= kThreads) {
     // producer warp: one thread feeds the ring, then the warp is done (every copy it issued is consumed
     // by the workers before they leave; a wait that runs out raises the status bit and stops feeding)
@@ -394,53 +392,63 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
     return;
   }
 
-  float m_nat, S, raw_max;
+  float wmax, S, raw_max;
   int raw_idx;
-  if (!row_pass<DT>(P, sm_ring, row, lo, hi, m_nat, S, raw_max, raw_idx) && threadIdx.x == 0) row_timeout(P, b);
+  const bool ok = row_pass<DT>(P, sm_ring, row, lo, hi, wmax, S, raw_max, raw_idx);
 
-  // ---- block reduction -> partial
-  block_merge_lse(m_nat, S, sm_f0, sm_f1);
-  Top2 top;
-  top.init();
-  top.push(raw_max, raw_idx);
-  block_merge_top2(top, sm_f0, sm_i0, sm_f1, sm_i1);
-  if (threadIdx.x == 0) {
+  // ---- warp reduction -> partial.  From here on the warps of a CTA go their own ways: a CTA-wide merge would
+  // cost three more barriers and leave the CTA's share of the SM without a copy in flight for as long, which
+  // at five CTAs per SM showed as a tenth of the kernel's time.  Every lane of a warp holds the same maximum
+  // (the warp agreed on it in every iteration), so its sums add up as they are, and the lowest index among the
+  // lanes that recorded this maximum is the first occurrence in the warp's share.
+  constexpr int kWarps = kThreads / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) S += __shfl_xor_sync(0xffffffffu, S, off);
+  const int widx = __reduce_min_sync(0xffffffffu, (raw_idx >= 0 && raw_max == wmax) ? raw_idx : 0x7FFFFFFF);
+  int last = 0;
+  if (lane == 0) {
+    if (!ok) row_timeout(P, b);
     RowPartial rp;
-    rp.m = m_nat; rp.s = S; rp.raw_max = top.s1; rp.idx = top.i1;
-    P.row_part[((size_t)b * P.Q + r) * P.row_splits + split] = rp;
+    rp.m = wmax * P.inv_t; rp.s = S; rp.raw_max = wmax; rp.idx = widx == 0x7FFFFFFF ? -1 : widx;
+    P.row_part[(((size_t)b * P.Q + r) * P.row_splits + split) * kWarps + warp] = rp;
     __threadfence();
     const int arrived = atomicAdd(&P.row_ticket[b], 1);
-    sm_last = (arrived == q_len * P.row_splits - 1);
+    last = (arrived == q_len * P.row_splits * kWarps - 1);
   }
-  worker_sync();
-  if (!sm_last) return;
+  if (!__shfl_sync(0xffffffffu, last, 0)) return;
 
-  // ---- decision phase: last CTA of the slot, warp 0 -------------------------------------------
-  if (threadIdx.x >= 32) return;
+  // ---- decision phase: the warp of the slot that arrives last ----------------------------------
   __threadfence();
-  const int lane = threadIdx.x;
   __shared__ float d_lse[32];
   __shared__ int d_tok[32];
   __shared__ int d_bad[32];
   if (lane == 0) P.row_ticket[b] = 0;  // ready for the next call
   {
-    // lane = block row: merge its splits
-    float m = -INFINITY, s = 0.f;
-    Top2 t;
-    t.init();
-    int bad = 0;
+    // lane = block row: merge the partials of its warps (empty pieces wrote neutral values)
+    float m = -INFINITY, s = 0.f, best = -INFINITY;
+    int tok = -1, bad = 0;
     if (lane < q_len) {
-      const volatile RowPartial* rp = P.row_part + ((size_t)b * P.Q + lane) * P.row_splits;
-      for (int i = 0; i < P.row_splits; ++i) {  // empty splits wrote neutral values
-        lse_merge(m, s, rp[i].m, rp[i].s);
-        t.push(rp[i].raw_max, rp[i].idx);
+      const volatile RowPartial* rp = P.row_part + ((size_t)b * P.Q + lane) * P.row_splits * kWarps;
+      const int n = P.row_splits * kWarps;
+      for (int i = 0; i < n; ++i) {
+        m = fmaxf(m, rp[i].m);
+        const float rm = rp[i].raw_max;
+        const int id = rp[i].idx;
+        if (id >= 0 && (rm > best || (rm == best && id < tok) || tok < 0)) { best = rm; tok = id; }
+      }
+      if (m > -INFINITY) {
+        for (int i = 0; i < n; ++i) {
+          const float mi = rp[i].m;
+          if (mi > -INFINITY) s += rp[i].s * __expf(mi - m);  // NaN sums and m = +inf poison s
+        }
       }
       // NaN anywhere poisons s; +inf logits give m = +inf
       bad = (s != s) || (m == INFINITY) || (m != m);
-      P.row_arg[(size_t)b * P.Q + lane] = t.i1;
+      P.row_arg[(size_t)b * P.Q + lane] = tok;
     }
     d_lse[lane] = m + logf(s);
-    d_tok[lane] = t.i1;
+    d_tok[lane] = tok;
     d_bad[lane] = bad;
   }
   __syncwarp();
@@ -907,7 +915,10 @@ constexpr size_t kOffLse = kOffRowArg + align256(sizeof(int) * kStaticMaxBatch *
 constexpr size_t kOffSampPart = kOffLse + align256(sizeof(float) * kStaticMaxBatch);
 constexpr size_t kOffRowPart =
     kOffSampPart + align256(sizeof(SamplePartial) * kStaticMaxBatch * kStaticMaxStride * kStaticMaxSplits);
-constexpr size_t kStaticBytes = kOffRowPart + align256(sizeof(RowPartial) * kStaticMaxBatch * ISD_MAX_Q * kStaticMaxSplits);
+// row pieces of one call: rows * row_splits <= rows + 4 * SMs by the rule that picks row_splits; the entry point
+// lowers row_splits where a device with more SMs would exceed this.  One partial per worker warp of a piece.
+constexpr int kStaticMaxRowPieces = kStaticMaxBatch * ISD_MAX_Q + 1024;
+constexpr size_t kStaticBytes = kOffRowPart + align256(sizeof(RowPartial) * kStaticMaxRowPieces * (kThreads / 32));
 
 constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
@@ -964,6 +975,7 @@ extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* s
   int rs = (target + rows - 1) / rows;
   rs = rs < 1 ? 1 : (rs > kStaticMaxSplits ? kStaticMaxSplits : rs);
   rs = rs > max_by_len ? max_by_len : rs;
+  if (rows * rs > kStaticMaxRowPieces) rs = kStaticMaxRowPieces / rows;  // >= 1: rows <= 64 * ISD_MAX_Q
   int ps = 4;  // same cut as isd_create uses
   ps = ps > max_by_len ? max_by_len : ps;
   tmp.row_splits = rs;
