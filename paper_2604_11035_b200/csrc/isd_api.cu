@@ -88,19 +88,12 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   int rc = ISD_OK;
   if (rc == ISD_OK) rc = dev_alloc(&ctx->row_part, (size_t)rows * rs * 8);  // one partial per worker warp of a row piece
   if (rc == ISD_OK) rc = dev_alloc(&ctx->samp_part, (size_t)c.batch * c.stride * ps);
-  if (rc == ISD_OK) rc = dev_alloc(&ctx->row_ticket, c.batch);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->samp_ticket, (size_t)c.batch * c.stride);
-  if (rc == ISD_OK) rc = dev_alloc(&ctx->reject_pos, c.batch);
-  if (rc == ISD_OK) rc = dev_alloc(&ctx->row_arg, (size_t)rows);
-  if (rc == ISD_OK) rc = dev_alloc(&ctx->lse_p_rej, c.batch);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->global_status, 1);
   if (rc == ISD_OK) rc = dev_alloc(&ctx->step_ticket, 1);
   if (rc == ISD_OK) {
     cudaMemset(ctx->step_ticket, 0, sizeof(int));
-    cudaMemset(ctx->row_ticket, 0, sizeof(int) * c.batch);
     cudaMemset(ctx->samp_ticket, 0, sizeof(int) * c.batch * c.stride);
-    cudaMemset(ctx->reject_pos, 0xFF, sizeof(int) * c.batch);
-    cudaMemset(ctx->row_arg, 0xFF, sizeof(int) * rows);
     cudaMemset(ctx->global_status, 0, sizeof(uint32_t));
   }
   if (rc == ISD_OK && c.top_k > 0) rc = isd_verify_topk_create(ctx);
@@ -123,11 +116,7 @@ int isd_destroy(isd_ctx* ctx) {
   isd_lora_destroy(ctx);
   cudaFree(ctx->row_part);
   cudaFree(ctx->samp_part);
-  cudaFree(ctx->row_ticket);
   cudaFree(ctx->samp_ticket);
-  cudaFree(ctx->reject_pos);
-  cudaFree(ctx->row_arg);
-  cudaFree(ctx->lse_p_rej);
   cudaFree(ctx->global_status);
   cudaFree(ctx->step_ticket);
   delete ctx;

@@ -49,13 +49,9 @@ struct isd_ctx {
   // ---- verify scratch
   int row_splits;        // CTAs per logits row in the row pass
   int sample_splits;     // CTAs per sampled row in the sampling pass
-  RowPartial* row_part;  // [B, Q, row_splits]
+  RowPartial* row_part;  // [B, Q, row_splits, worker warps of a CTA]
   SamplePartial* samp_part;  // [B, N, sample_splits]
-  int* row_ticket;       // [B] arrivals of the row pass
   int* samp_ticket;      // [B, N] arrivals of the sampling pass
-  int* reject_pos;       // [B] -1 = slot frozen (nothing to sample), 0 = nothing rejected, j = first rejected proposal
-  int* row_arg;          // [B, Q] argmax of every valid row (seeds the sampling pass)
-  float* lse_p_rej;      // [B] LSE of the anchor row that rejected
   // ---- attention scratch
   int attn_ctas;         // persistent CTAs of the tensor-core kernel
   float* attn_part_o;    // [attn_ctas * 2, 128, 128] un-normalised partial outputs

@@ -55,11 +55,7 @@ struct VerifyParams {
   isd_verify_out out;
   RowPartial* row_part;
   SamplePartial* samp_part;
-  int* row_ticket;
   int* samp_ticket;
-  int* reject_pos;
-  int* row_arg;
-  float* lse_p_rej;
   // isd_step: the CTA of the sampling pass that finishes last commits the batch (fuse_commit != 0)
   int fuse_commit;
   int* step_ticket;
@@ -346,7 +342,7 @@ __device__ __forceinline__ void row_timeout(const VerifyParams& P, int b) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Pass 1: row statistics + decision
+// Pass 1: row statistics
 // ------------------------------------------------------------------------------------------------
 template <int DT>
 __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const VerifyParams P) {
@@ -396,9 +392,11 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
   int raw_idx;
   const bool ok = row_pass<DT>(P, sm_ring, row, lo, hi, wmax, S, raw_max, raw_idx);
 
-  // ---- warp reduction -> partial.  From here on the warps of a CTA go their own ways: a CTA-wide merge would
-  // cost three more barriers and leave the CTA's share of the SM without a copy in flight for as long, which
-  // at five CTAs per SM showed as a tenth of the kernel's time.  Every lane of a warp holds the same maximum
+  // ---- warp reduction -> partial, and the warp is done: one 16-byte store that nobody in this kernel reads.
+  // Anything more at the end of a CTA (a CTA-wide merge, a fence and a ticket for a last-arriver decision)
+  // keeps its share of the SM without a copy in flight for two or three round trips through a saturated memory
+  // system, which at five CTAs per SM was an eighth of the kernel's time; the decision that needs all rows of
+  // a slot is taken at the head of the sampling kernel instead.  Every lane of a warp holds the same maximum
   // (the warp agreed on it in every iteration), so its sums add up as they are, and the lowest index among the
   // lanes that recorded this maximum is the first occurrence in the warp's share.
   constexpr int kWarps = kThreads / 32;
@@ -406,46 +404,75 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) S += __shfl_xor_sync(0xffffffffu, S, off);
   const int widx = __reduce_min_sync(0xffffffffu, (raw_idx >= 0 && raw_max == wmax) ? raw_idx : 0x7FFFFFFF);
-  int last = 0;
   if (lane == 0) {
     if (!ok) row_timeout(P, b);
     RowPartial rp;
     rp.m = wmax * P.inv_t; rp.s = S; rp.raw_max = wmax; rp.idx = widx == 0x7FFFFFFF ? -1 : widx;
     P.row_part[(((size_t)b * P.Q + r) * P.row_splits + split) * kWarps + warp] = rp;
-    __threadfence();
-    const int arrived = atomicAdd(&P.row_ticket[b], 1);
-    last = (arrived == q_len * P.row_splits * kWarps - 1);
   }
-  if (!__shfl_sync(0xffffffffu, last, 0)) return;
+}
 
-  // ---- decision phase: the warp of the slot that arrives last ----------------------------------
-  __threadfence();
-  __shared__ float d_lse[32];
-  __shared__ int d_tok[32];
-  __shared__ int d_bad[32];
-  if (lane == 0) P.row_ticket[b] = 0;  // ready for the next call
-  {
-    // lane = block row: merge the partials of its warps (empty pieces wrote neutral values)
-    float m = -INFINITY, s = 0.f, best = -INFINITY;
+// ------------------------------------------------------------------------------------------------
+// The decision of a slot (Algorithm 1, introspection loop), taken by one warp at the head of the sampling
+// kernel from the row pass's partials.  Every sampling CTA that draws the slot's emission (k = 0) takes it
+// for itself; the one with split 0 records the slot's outputs that need no random sample (write).
+// ------------------------------------------------------------------------------------------------
+// One lane's merge of the partials of a block row: max and sum of the online softmax, first argmax.
+__device__ __forceinline__ void merge_row(const VerifyParams& P, int b, int row, float& m, float& s, int& tok) {
+  const int n = P.row_splits * (kThreads / 32);
+  const RowPartial* rp = P.row_part + ((size_t)b * P.Q + row) * n;
+  float best = -INFINITY;
+  m = -INFINITY; s = 0.f; tok = -1;
+  for (int i = 0; i < n; ++i) {  // empty pieces wrote neutral values
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(rp + i));
+    const int id = __float_as_int(v.w);
+    m = fmaxf(m, v.x);
+    if (id >= 0 && (v.z > best || (v.z == best && id < tok) || tok < 0)) { best = v.z; tok = id; }
+  }
+  if (m > -INFINITY) {
+    for (int i = 0; i < n; ++i) {
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(rp + i));
+      if (v.x > -INFINITY) s += v.y * __expf(v.x - m);  // NaN sums and m = +inf poison s
+    }
+  }
+}
+
+struct SlotDecision {
+  int rej;      // -1: frozen, nothing is drawn for the emission; 0: nothing rejected; j: first rejected proposal
+  int i0;       // argmax of the row the emission is drawn from
+  float lse_p;  // LSE of the row that rejected
+};
+
+// Called by all 32 lanes of warp 0.  d_lse / d_tok / d_bad: 32 entries of shared memory each.
+template <int DT>
+__device__ __forceinline__ void decide_slot(const VerifyParams& P, int b, int nv, bool write, float* d_lse, int* d_tok,
+                                            int* d_bad, SlotDecision* out) {
+  const unsigned full = 0xffffffffu;
+  const int lane = threadIdx.x & 31;
+  const int NP = P.N - 1, q_len = nv + P.N;
+  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  const char* cur = reinterpret_cast<const char*>(P.logits_cur) + (size_t)b * P.Q * (size_t)P.V * elt;
+
+  // lane = proposal position j: what its accept test needs besides the row statistics is fetched first
+  const bool pos = lane >= 1 && lane <= nv;
+  const int x = pos ? P.block_tok[(size_t)b * P.Q + lane] : 0;
+  float logq = 0.f;
+  if (pos && P.q_mode == 0) {
+    const float* qs = P.q_stats + ((size_t)b * NP + lane - 1) * 2;
+    logq = qs[1] - qs[0];
+  }
+  // a warp of the row pass gave up on a wait: a partial is incomplete, nothing of the slot may be committed
+  const uint32_t timeout = *reinterpret_cast<volatile uint32_t*>(&P.slot_status[b]) & ISD_ST_KERNEL_TIMEOUT;
+  const bool badtok = pos && (x < 0 || x >= P.V);
+  float lx = 0.f;  // the raw logit of the proposal in the row that judges it
+  if (pos && !badtok) lx = load_logit(cur + (size_t)(lane - 1) * P.V * elt, P.logits_dtype, (size_t)x);
+
+  {  // lane = block row: merge its partials
+    float m = -INFINITY, s = 0.f;
     int tok = -1, bad = 0;
     if (lane < q_len) {
-      const volatile RowPartial* rp = P.row_part + ((size_t)b * P.Q + lane) * P.row_splits * kWarps;
-      const int n = P.row_splits * kWarps;
-      for (int i = 0; i < n; ++i) {
-        m = fmaxf(m, rp[i].m);
-        const float rm = rp[i].raw_max;
-        const int id = rp[i].idx;
-        if (id >= 0 && (rm > best || (rm == best && id < tok) || tok < 0)) { best = rm; tok = id; }
-      }
-      if (m > -INFINITY) {
-        for (int i = 0; i < n; ++i) {
-          const float mi = rp[i].m;
-          if (mi > -INFINITY) s += rp[i].s * __expf(mi - m);  // NaN sums and m = +inf poison s
-        }
-      }
-      // NaN anywhere poisons s; +inf logits give m = +inf
-      bad = (s != s) || (m == INFINITY) || (m != m);
-      P.row_arg[(size_t)b * P.Q + lane] = tok;
+      merge_row(P, b, lane, m, s, tok);
+      bad = (s != s) || (m == INFINITY) || (m != m);  // NaN anywhere poisons s; +inf logits give m = +inf
     }
     d_lse[lane] = m + logf(s);
     d_tok[lane] = tok;
@@ -453,78 +480,71 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
   }
   __syncwarp();
 
-  const int NP = P.N - 1;
   // proposal-law statistics (lanes 1..N-1 = MASK row m); argmax proposals are final here, sampled ones
-  // and their logit are written by the sampling pass
-  if (lane >= 1 && lane <= NP) {
+  // and their logit are written by the CTAs that draw them
+  if (write && lane >= 1 && lane <= NP) {
     const int rr = nv + lane;
     P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 0] = d_lse[rr];
     if (P.propose_mode == 1) {
       const int xh = d_tok[rr];
-      const char* rw = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + rr) * (size_t)P.V * elt;
       P.out.new_prop_tok[(size_t)b * NP + lane - 1] = xh;
       P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 1] =
-          xh >= 0 ? load_logit(rw, P.logits_dtype, (size_t)xh) * P.inv_t : NAN;
+          xh >= 0 ? load_logit(cur + (size_t)rr * P.V * elt, P.logits_dtype, (size_t)xh) * P.inv_t : NAN;
     }
   }
-  if (lane != 0) return;
 
-  // sequential accept test (Algorithm 1, introspection loop)
-  uint32_t status = 0;
-  int a = nv, rej = 0;
-  for (int m = 1; m <= NP; ++m) status |= d_bad[nv + m] ? ISD_ST_NONFINITE_LOGIT : 0u;
-  for (int j = 1; j <= NP; ++j) {
-    P.out.accept[(size_t)b * NP + j - 1] = -1;
-    P.out.alpha[(size_t)b * NP + j - 1] = NAN;
-  }
-  for (int j = 1; j <= nv; ++j) {
-    const int x = P.block_tok[(size_t)b * P.Q + j];
-    if (x < 0 || x >= P.V) {
-      status |= ISD_ST_BAD_TOKEN_ID;
-      a = -1;
-      break;
-    }
-    if (d_bad[j - 1]) status |= ISD_ST_NONFINITE_LOGIT;
-    const char* rw = reinterpret_cast<const char*>(P.logits_cur) + ((size_t)b * P.Q + (j - 1)) * (size_t)P.V * elt;
-    const float logp = load_logit(rw, P.logits_dtype, (size_t)x) * P.inv_t - d_lse[j - 1];
-    float logq = 0.f;
-    if (P.q_mode == 0) {
-      const float* qs = P.q_stats + ((size_t)b * NP + j - 1) * 2;
-      logq = qs[1] - qs[0];
-    }
-    float al = (1.f + P.tau) * expf(logp - logq);
+  // The accept tests of all positions at once (a test depends on nothing an earlier one decides); the first
+  // position that rejects, or whose token id is out of range, ends the sequence.
+  float al = NAN;
+  bool acc = true;
+  if (pos && !badtok) {
+    const float logp = lx * P.inv_t - d_lse[lane - 1];
+    al = (1.f + P.tau) * expf(logp - logq);
     al = fminf(al, 1.f);
     if (al != al) al = 0.f;
-    const uint4 rnd = philox4x32_10(0u, step_of(P), (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)j, P.seed_lo, P.seed_hi);
+    const uint4 rnd = philox4x32_10(0u, step_of(P), (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)lane, P.seed_lo, P.seed_hi);
     const float u = (float)(rnd.x >> 8) * 0x1p-24f;
-    P.out.alpha[(size_t)b * NP + j - 1] = al;
-    if (u < al) {
-      P.out.accept[(size_t)b * NP + j - 1] = 1;
-    } else {
-      P.out.accept[(size_t)b * NP + j - 1] = 0;
-      a = j - 1;
-      rej = j;
-      P.lse_p_rej[b] = d_lse[j - 1];
-      break;
+    acc = u < al;
+  }
+  const unsigned m_badtok = __ballot_sync(full, badtok);
+  const unsigned m_stop = m_badtok | __ballot_sync(full, pos && !badtok && !acc);
+  const int first = m_stop ? __ffs(m_stop) - 1 : nv + 1;
+  const bool bad_first = m_stop && ((m_badtok >> first) & 1u);
+  const int rej = (m_stop && !bad_first) ? first : 0;
+  const int a = bad_first ? -1 : (rej ? rej - 1 : nv);
+  const bool evald = pos && lane <= first && !badtok;  // positions whose test was run
+  const bool nonfinite = (evald && d_bad[lane - 1]) || (lane >= 1 && lane <= NP && d_bad[nv + lane]) ||
+                         (lane == 0 && a >= 0 && rej == 0 && d_bad[nv]);
+  uint32_t status = timeout;
+  if (__ballot_sync(full, nonfinite)) status |= ISD_ST_NONFINITE_LOGIT;
+  if (bad_first) status |= ISD_ST_BAD_TOKEN_ID;
+  const bool frozen = a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL);
+  const int x_next = __shfl_down_sync(full, x, 1);  // lane j - 1 gets proposal j
+
+  if (lane == 0) {
+    out->rej = frozen ? -1 : rej;
+    out->i0 = d_tok[rej > 0 ? rej - 1 : nv];
+    out->lse_p = rej > 0 ? d_lse[rej - 1] : 0.f;
+  }
+  if (!write) return;
+  if (lane >= 1 && lane <= NP) {
+    P.out.accept[(size_t)b * NP + lane - 1] = evald ? (lane == rej ? 0 : 1) : -1;
+    P.out.alpha[(size_t)b * NP + lane - 1] = evald ? al : NAN;
+  }
+  // the emission: accepted proposals now; the drawn token and the copy of it in repl_tok come from the CTA
+  // of the sampling pass that finishes the draw, unless nothing is drawn
+  const bool draws = !frozen && !(rej > 0 && P.q_mode == 0 && P.q_prev == nullptr);
+  if (lane < P.N && !(draws && lane == a))
+    P.out.out_tok[(size_t)b * P.N + lane] = (!frozen && lane < a) ? x_next : -1;
+  if (lane == 0) {
+    if (!draws) P.out.repl_tok[b] = -1;
+    P.out.accept_len[b] = frozen ? 0 : a;
+    P.out.n_emit[b] = frozen ? 0 : a + 1;
+    if (frozen) {
+      atomicOr(&P.slot_status[b], status);
+      atomicOr(P.global_status, status);
     }
   }
-  if (a >= 0 && rej == 0 && d_bad[nv]) status |= ISD_ST_NONFINITE_LOGIT;
-  // a CTA of this slot gave up on a wait: its partial is incomplete, nothing of the slot may be committed
-  status |= *reinterpret_cast<volatile uint32_t*>(&P.slot_status[b]) & ISD_ST_KERNEL_TIMEOUT;
-  for (int j = 0; j < P.N; ++j) P.out.out_tok[(size_t)b * P.N + j] = -1;
-  P.out.repl_tok[b] = -1;  // the sampling pass fills the drawn token
-  if (a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL)) {
-    P.out.accept_len[b] = 0;
-    P.out.n_emit[b] = 0;
-    P.reject_pos[b] = -1;  // frozen: nothing is drawn for the emission
-    atomicOr(&P.slot_status[b], status);
-    atomicOr(P.global_status, status);
-    return;
-  }
-  P.out.accept_len[b] = a;
-  P.out.n_emit[b] = a + 1;
-  for (int j = 1; j <= a; ++j) P.out.out_tok[(size_t)b * P.N + j - 1] = P.block_tok[(size_t)b * P.Q + j];
-  P.reject_pos[b] = rej;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -681,11 +701,10 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
 template <int DT>
 __device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
   const int split = blockIdx.x, k = blockIdx.y, b = blockIdx.z;
-  if (!P.active[b]) return;
-  const int nv = P.n_ver[b];
-  if (nv < 0 || nv > P.N - 1) return;  // flagged by the row pass; its scratch entries are stale
-  const int rej = P.reject_pos[b];
-  if (k == 0 && rej < 0) return;       // frozen slot: no emission
+  const int act = P.active[b];
+  const int nv = P.n_ver[b];  // both loads in flight together
+  if (!act) return;
+  if (nv < 0 || nv > P.N - 1) return;  // flagged by the row pass
 
   __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
   __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
@@ -693,6 +712,24 @@ __device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
   __shared__ unsigned sm_best;
   __shared__ SampleQueue sm_queue;
   __shared__ __align__(16) uint4 sm_ring[kSampleRingBytes / 16];
+  __shared__ float d_lse[32];
+  __shared__ int d_tok[32], d_bad[32];
+  __shared__ SlotDecision sm_dec;
+
+  // ---- what the row pass found: the slot's decision (k = 0), or just the argmax of the MASK row (k >= 1)
+  if (threadIdx.x < 32) {
+    if (k == 0) {
+      decide_slot<DT>(P, b, nv, split == 0, d_lse, d_tok, d_bad, &sm_dec);
+    } else if (threadIdx.x == 0) {
+      float m, s;
+      int tok;
+      merge_row(P, b, nv + k, m, s, tok);
+      sm_dec.rej = 0; sm_dec.i0 = tok; sm_dec.lse_p = 0.f;
+    }
+  }
+  __syncthreads();
+  const int rej = sm_dec.rej;
+  if (k == 0 && rej < 0) return;       // frozen slot: no emission
 
   const int NP = P.N - 1;
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
@@ -710,7 +747,7 @@ __device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
     r = rej - 1;
     J.resid = true;
     J.x = P.block_tok[(size_t)b * P.Q + rej];
-    J.lse_p = P.lse_p_rej[b];
+    J.lse_p = sm_dec.lse_p;
     if (P.q_mode == 0) {
       J.qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + (P.q_row0[b] + rej - 1)) * row_bytes;
       J.lse_q = P.q_stats[((size_t)b * NP + rej - 1) * 2 + 0];
@@ -732,7 +769,7 @@ __device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
   // ---- seed: the true noisy score of the row's argmax (for the residual: if it has residual mass)
   if (threadIdx.x == 0) {
     float seed = -INFINITY;
-    const int i0 = P.row_arg[(size_t)b * P.Q + r];
+    const int i0 = sm_dec.i0;
     if (i0 >= 0 && i0 < P.V) {
       const uint4 rnd = philox4x32_10((uint32_t)i0 >> 2, J.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
       seed = job_score(P, J, load_logit(J.prow, P.logits_dtype, (size_t)i0), i0, philox_word(rnd, i0 & 3));
@@ -857,9 +894,7 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   P.n_ver = st->n_ver; P.active = st->active; P.block_tok = st->block_tok; P.q_row0 = st->q_row0;
   P.q_stats = st->q_stats; P.slot_status = st->slot_status; P.global_status = ctx->global_status;
   P.logits_cur = logits_cur; P.q_prev = q_prev_logits; P.out = *out;
-  P.row_part = ctx->row_part; P.samp_part = ctx->samp_part; P.row_ticket = ctx->row_ticket;
-  P.samp_ticket = ctx->samp_ticket; P.reject_pos = ctx->reject_pos; P.row_arg = ctx->row_arg;
-  P.lse_p_rej = ctx->lse_p_rej;
+  P.row_part = ctx->row_part; P.samp_part = ctx->samp_part; P.samp_ticket = ctx->samp_ticket;
   P.fuse_commit = commit_st != nullptr && ctx->step_ticket != nullptr;
   P.step_ticket = ctx->step_ticket;
   P.commit = make_commit_params(ctx, P.fuse_commit ? commit_st : st, out);
@@ -903,16 +938,12 @@ namespace {
 constexpr int kStaticMaxBatch = ISD_STATIC_MAX_BATCH;
 constexpr int kStaticMaxSplits = 16;
 constexpr size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
-// layout of the array: [zeroed every call: tickets, reject positions, status word][partials]
+// layout of the array: [zeroed every call: tickets of the sampling pass, status word][partials of both passes]
 constexpr int kStaticMaxStride = (ISD_MAX_Q + 1) / 2;
-constexpr size_t kOffRowTicket = 0;
-constexpr size_t kOffSampTicket = kOffRowTicket + align256(sizeof(int) * kStaticMaxBatch);
+constexpr size_t kOffSampTicket = 0;
 constexpr size_t kOffStatus = kOffSampTicket + align256(sizeof(int) * kStaticMaxBatch * kStaticMaxStride);
 constexpr size_t kZeroedBytes = kOffStatus + align256(sizeof(uint32_t));
-constexpr size_t kOffRejectPos = kZeroedBytes;  // written by the row pass for every slot the sampling pass reads
-constexpr size_t kOffRowArg = kOffRejectPos + align256(sizeof(int) * kStaticMaxBatch);
-constexpr size_t kOffLse = kOffRowArg + align256(sizeof(int) * kStaticMaxBatch * ISD_MAX_Q);
-constexpr size_t kOffSampPart = kOffLse + align256(sizeof(float) * kStaticMaxBatch);
+constexpr size_t kOffSampPart = kZeroedBytes;
 constexpr size_t kOffRowPart =
     kOffSampPart + align256(sizeof(SamplePartial) * kStaticMaxBatch * kStaticMaxStride * kStaticMaxSplits);
 // row pieces of one call: rows * row_splits <= rows + 4 * SMs by the rule that picks row_splits; the entry point
@@ -980,12 +1011,8 @@ extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* s
   ps = ps > max_by_len ? max_by_len : ps;
   tmp.row_splits = rs;
   tmp.sample_splits = ps;
-  tmp.row_ticket = reinterpret_cast<int*>(base + kOffRowTicket);
   tmp.samp_ticket = reinterpret_cast<int*>(base + kOffSampTicket);
-  tmp.row_arg = reinterpret_cast<int*>(base + kOffRowArg);
-  tmp.reject_pos = reinterpret_cast<int*>(base + kOffRejectPos);
   tmp.global_status = reinterpret_cast<uint32_t*>(base + kOffStatus);
-  tmp.lse_p_rej = reinterpret_cast<float*>(base + kOffLse);
   tmp.samp_part = reinterpret_cast<SamplePartial*>(base + kOffSampPart);
   tmp.row_part = reinterpret_cast<RowPartial*>(base + kOffRowPart);
   tmp.wait_ns = ISD_DEFAULT_WAIT_NS;
