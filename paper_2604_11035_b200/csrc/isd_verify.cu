@@ -156,22 +156,6 @@ __device__ __forceinline__ void chunk_range(int V, int splits, int split, int& l
 }
 
 // Block-wide merge helpers (8 worker warps) -------------------------------------------------------
-__device__ __forceinline__ void block_merge_lse(float& m, float& s, float* sm_m, float* sm_s) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    const float om = __shfl_xor_sync(0xffffffffu, m, off);
-    const float os = __shfl_xor_sync(0xffffffffu, s, off);
-    lse_merge(m, s, om, os);
-  }
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (lane == 0) { sm_m[warp] = m; sm_s[warp] = s; }
-  worker_sync();
-  if (threadIdx.x == 0) {
-    for (int w = 1; w < kThreads / 32; ++w) lse_merge(m, s, sm_m[w], sm_s[w]);
-  }
-  worker_sync();
-}
-
 __device__ __forceinline__ void block_merge_top2(Top2& t, float* sm_s1, int* sm_i1, float* sm_s2, int* sm_i2) {
   warp_merge_top2(t);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -413,141 +397,6 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
 }
 
 // ------------------------------------------------------------------------------------------------
-// The decision of a slot (Algorithm 1, introspection loop), taken by one warp at the head of the sampling
-// kernel from the row pass's partials.  Every sampling CTA that draws the slot's emission (k = 0) takes it
-// for itself; the one with split 0 records the slot's outputs that need no random sample (write).
-// ------------------------------------------------------------------------------------------------
-// One lane's merge of the partials of a block row: max and sum of the online softmax, first argmax.
-__device__ __forceinline__ void merge_row(const VerifyParams& P, int b, int row, float& m, float& s, int& tok) {
-  const int n = P.row_splits * (kThreads / 32);
-  const RowPartial* rp = P.row_part + ((size_t)b * P.Q + row) * n;
-  float best = -INFINITY;
-  m = -INFINITY; s = 0.f; tok = -1;
-  for (int i = 0; i < n; ++i) {  // empty pieces wrote neutral values
-    const float4 v = __ldcg(reinterpret_cast<const float4*>(rp + i));
-    const int id = __float_as_int(v.w);
-    m = fmaxf(m, v.x);
-    if (id >= 0 && (v.z > best || (v.z == best && id < tok) || tok < 0)) { best = v.z; tok = id; }
-  }
-  if (m > -INFINITY) {
-    for (int i = 0; i < n; ++i) {
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(rp + i));
-      if (v.x > -INFINITY) s += v.y * __expf(v.x - m);  // NaN sums and m = +inf poison s
-    }
-  }
-}
-
-struct SlotDecision {
-  int rej;      // -1: frozen, nothing is drawn for the emission; 0: nothing rejected; j: first rejected proposal
-  int i0;       // argmax of the row the emission is drawn from
-  float lse_p;  // LSE of the row that rejected
-};
-
-// Called by all 32 lanes of warp 0.  d_lse / d_tok / d_bad: 32 entries of shared memory each.
-template <int DT>
-__device__ __forceinline__ void decide_slot(const VerifyParams& P, int b, int nv, bool write, float* d_lse, int* d_tok,
-                                            int* d_bad, SlotDecision* out) {
-  const unsigned full = 0xffffffffu;
-  const int lane = threadIdx.x & 31;
-  const int NP = P.N - 1, q_len = nv + P.N;
-  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
-  const char* cur = reinterpret_cast<const char*>(P.logits_cur) + (size_t)b * P.Q * (size_t)P.V * elt;
-
-  // lane = proposal position j: what its accept test needs besides the row statistics is fetched first
-  const bool pos = lane >= 1 && lane <= nv;
-  const int x = pos ? P.block_tok[(size_t)b * P.Q + lane] : 0;
-  float logq = 0.f;
-  if (pos && P.q_mode == 0) {
-    const float* qs = P.q_stats + ((size_t)b * NP + lane - 1) * 2;
-    logq = qs[1] - qs[0];
-  }
-  // a warp of the row pass gave up on a wait: a partial is incomplete, nothing of the slot may be committed
-  const uint32_t timeout = *reinterpret_cast<volatile uint32_t*>(&P.slot_status[b]) & ISD_ST_KERNEL_TIMEOUT;
-  const bool badtok = pos && (x < 0 || x >= P.V);
-  float lx = 0.f;  // the raw logit of the proposal in the row that judges it
-  if (pos && !badtok) lx = load_logit(cur + (size_t)(lane - 1) * P.V * elt, P.logits_dtype, (size_t)x);
-
-  {  // lane = block row: merge its partials
-    float m = -INFINITY, s = 0.f;
-    int tok = -1, bad = 0;
-    if (lane < q_len) {
-      merge_row(P, b, lane, m, s, tok);
-      bad = (s != s) || (m == INFINITY) || (m != m);  // NaN anywhere poisons s; +inf logits give m = +inf
-    }
-    d_lse[lane] = m + logf(s);
-    d_tok[lane] = tok;
-    d_bad[lane] = bad;
-  }
-  __syncwarp();
-
-  // proposal-law statistics (lanes 1..N-1 = MASK row m); argmax proposals are final here, sampled ones
-  // and their logit are written by the CTAs that draw them
-  if (write && lane >= 1 && lane <= NP) {
-    const int rr = nv + lane;
-    P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 0] = d_lse[rr];
-    if (P.propose_mode == 1) {
-      const int xh = d_tok[rr];
-      P.out.new_prop_tok[(size_t)b * NP + lane - 1] = xh;
-      P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 1] =
-          xh >= 0 ? load_logit(cur + (size_t)rr * P.V * elt, P.logits_dtype, (size_t)xh) * P.inv_t : NAN;
-    }
-  }
-
-  // The accept tests of all positions at once (a test depends on nothing an earlier one decides); the first
-  // position that rejects, or whose token id is out of range, ends the sequence.
-  float al = NAN;
-  bool acc = true;
-  if (pos && !badtok) {
-    const float logp = lx * P.inv_t - d_lse[lane - 1];
-    al = (1.f + P.tau) * expf(logp - logq);
-    al = fminf(al, 1.f);
-    if (al != al) al = 0.f;
-    const uint4 rnd = philox4x32_10(0u, step_of(P), (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)lane, P.seed_lo, P.seed_hi);
-    const float u = (float)(rnd.x >> 8) * 0x1p-24f;
-    acc = u < al;
-  }
-  const unsigned m_badtok = __ballot_sync(full, badtok);
-  const unsigned m_stop = m_badtok | __ballot_sync(full, pos && !badtok && !acc);
-  const int first = m_stop ? __ffs(m_stop) - 1 : nv + 1;
-  const bool bad_first = m_stop && ((m_badtok >> first) & 1u);
-  const int rej = (m_stop && !bad_first) ? first : 0;
-  const int a = bad_first ? -1 : (rej ? rej - 1 : nv);
-  const bool evald = pos && lane <= first && !badtok;  // positions whose test was run
-  const bool nonfinite = (evald && d_bad[lane - 1]) || (lane >= 1 && lane <= NP && d_bad[nv + lane]) ||
-                         (lane == 0 && a >= 0 && rej == 0 && d_bad[nv]);
-  uint32_t status = timeout;
-  if (__ballot_sync(full, nonfinite)) status |= ISD_ST_NONFINITE_LOGIT;
-  if (bad_first) status |= ISD_ST_BAD_TOKEN_ID;
-  const bool frozen = a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL);
-  const int x_next = __shfl_down_sync(full, x, 1);  // lane j - 1 gets proposal j
-
-  if (lane == 0) {
-    out->rej = frozen ? -1 : rej;
-    out->i0 = d_tok[rej > 0 ? rej - 1 : nv];
-    out->lse_p = rej > 0 ? d_lse[rej - 1] : 0.f;
-  }
-  if (!write) return;
-  if (lane >= 1 && lane <= NP) {
-    P.out.accept[(size_t)b * NP + lane - 1] = evald ? (lane == rej ? 0 : 1) : -1;
-    P.out.alpha[(size_t)b * NP + lane - 1] = evald ? al : NAN;
-  }
-  // the emission: accepted proposals now; the drawn token and the copy of it in repl_tok come from the CTA
-  // of the sampling pass that finishes the draw, unless nothing is drawn
-  const bool draws = !frozen && !(rej > 0 && P.q_mode == 0 && P.q_prev == nullptr);
-  if (lane < P.N && !(draws && lane == a))
-    P.out.out_tok[(size_t)b * P.N + lane] = (!frozen && lane < a) ? x_next : -1;
-  if (lane == 0) {
-    if (!draws) P.out.repl_tok[b] = -1;
-    P.out.accept_len[b] = frozen ? 0 : a;
-    P.out.n_emit[b] = frozen ? 0 : a + 1;
-    if (frozen) {
-      atomicOr(&P.slot_status[b], status);
-      atomicOr(P.global_status, status);
-    }
-  }
-}
-
-// ------------------------------------------------------------------------------------------------
 // Pass 2: the random draws
 // ------------------------------------------------------------------------------------------------
 // fp64 score of vocabulary index i of the residual law: ln max(0, p_i - q_i) + g
@@ -584,6 +433,213 @@ __device__ __forceinline__ float job_score(const VerifyParams& P, const SampleJo
                                  : (i == J.x ? 1.f : 0.f);
   const float rr = pi - qi;
   return rr > 0.f ? logf(rr) + gumbel_f32(w) : -INFINITY;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Head of a sampling CTA, run by its warp 0: what the row pass found about the slot, the slot's decision
+// (Algorithm 1, introspection loop) when the CTA draws the slot's emission (k = 0), the job of the CTA and the
+// seed of its draw.  Every CTA takes the decision for itself; the one with split 0 records the slot's outputs
+// that need no random sample (write).  Everything the head reads that does not depend on something else it
+// reads is fetched in one go, so that the head costs two trips to memory (three for a residual against softmax q).
+// ------------------------------------------------------------------------------------------------
+struct SampleHead {
+  int rej;        // -2: slot inactive or invalid; -1: frozen, nothing is drawn for the emission; 0: nothing rejected;
+                  // j: first rejected proposal
+  int nv;
+  int r;          // row of this step's logits that the CTA draws from
+  int x;          // residual: the rejected token
+  int q_row;      // residual against softmax q: the row of q_prev that holds the proposal law
+  float lse_p, lse_q;
+  unsigned best;  // ordered code of the seed score (0: none)
+};
+
+constexpr int kHeadChunk = 8;  // partials of a row merged per pass (one pass when the row pass ran one CTA per row)
+
+// Called by all 32 lanes of warp 0.  d_*: 32 entries of shared memory each.
+template <int DT>
+__device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k, int split, float* d_lse, float* d_raw,
+                                            int* d_tok, int* d_bad, SampleHead* H) {
+  const unsigned full = 0xffffffffu;
+  const int lane = threadIdx.x & 31;
+  const int NP = P.N - 1;
+  const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
+  const size_t row_bytes = (size_t)P.V * elt;
+  const char* cur = reinterpret_cast<const char*>(P.logits_cur) + (size_t)b * P.Q * row_bytes;
+  const bool write = (k == 0 && split == 0);
+
+  // ---- first trip: nothing here depends on anything else that is read
+  const int act = P.active[b];
+  const int nv = P.n_ver[b];
+  const int n_part = P.row_splits * (kThreads / 32);
+  const bool has_row = lane < P.Q;  // lane = block row (rows beyond the slot's block hold stale partials, unused)
+  const float4* rp = reinterpret_cast<const float4*>(P.row_part) + ((size_t)b * P.Q + (has_row ? lane : 0)) * n_part;
+  float4 part[kHeadChunk];
+#pragma unroll
+  for (int i = 0; i < kHeadChunk; ++i) part[i] = __ldcg(rp + i);  // n_part is a multiple of kHeadChunk
+  const bool is_pos = k == 0 && lane >= 1 && lane <= NP;  // lane = proposal position j (valid when j <= nv)
+  int x = 0;
+  float logq = 0.f, lse_q = 0.f;
+  if (is_pos) {
+    x = P.block_tok[(size_t)b * P.Q + lane];
+    if (P.q_mode == 0) {
+      const float* qs = P.q_stats + ((size_t)b * NP + lane - 1) * 2;
+      lse_q = qs[0];
+      logq = qs[1] - lse_q;
+    }
+  }
+  uint32_t timeout = 0;
+  int q_row0 = 0;
+  if (k == 0) {
+    // a warp of the row pass gave up on a wait: a partial is incomplete, nothing of the slot may be committed
+    timeout = *reinterpret_cast<volatile uint32_t*>(&P.slot_status[b]) & ISD_ST_KERNEL_TIMEOUT;
+    if (P.q_mode == 0) q_row0 = P.q_row0[b];
+  }
+
+  if (!act || nv < 0 || nv > NP) {  // an invalid n_ver was flagged by the row pass
+    if (lane == 0) H->rej = -2;
+    return;
+  }
+  const int q_len = nv + P.N;
+  const bool pos = is_pos && lane <= nv;
+  const bool badtok = pos && (x < 0 || x >= P.V);
+  // ---- second trip: the raw logit of the proposal in the row that judges it
+  float lx = 0.f;
+  if (pos && !badtok) lx = load_logit(cur + (size_t)(lane - 1) * row_bytes, P.logits_dtype, (size_t)x);
+
+  {  // lane = block row: merge its partials (max and sum of the online softmax, first argmax)
+    float m = -INFINITY, s = 0.f, best = -INFINITY;
+    int tok = -1;
+    for (int c = 0;; ) {
+      float cm = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < kHeadChunk; ++i) {
+        const int id = __float_as_int(part[i].w);
+        cm = fmaxf(cm, part[i].x);
+        if (id >= 0 && (part[i].z > best || (part[i].z == best && id < tok) || tok < 0)) { best = part[i].z; tok = id; }
+      }
+      const float nm = fmaxf(m, cm);
+      if (nm > -INFINITY) {
+        float acc = (m > -INFINITY) ? s * __expf(m - nm) : 0.f;
+#pragma unroll
+        for (int i = 0; i < kHeadChunk; ++i)
+          if (part[i].x > -INFINITY) acc += part[i].y * __expf(part[i].x - nm);  // NaN sums and m = +inf poison s
+        s = acc;
+      }
+      m = nm;
+      c += kHeadChunk;
+      if (c >= n_part) break;
+#pragma unroll
+      for (int i = 0; i < kHeadChunk; ++i) part[i] = __ldcg(rp + c + i);
+    }
+    const bool valid = lane < q_len;
+    // NaN anywhere poisons s; +inf logits give m = +inf
+    d_bad[lane] = valid && ((s != s) || (m == INFINITY) || (m != m));
+    d_lse[lane] = m + logf(s);
+    d_raw[lane] = best;
+    d_tok[lane] = valid ? tok : -1;
+  }
+  __syncwarp();
+
+  int rej = 0, a = nv;
+  bool frozen = false;
+  if (k == 0) {
+    // proposal-law statistics (lanes 1..N-1 = MASK row m); argmax proposals are final here, sampled ones
+    // and their logit are written by the CTAs that draw them
+    if (write && lane >= 1 && lane <= NP) {
+      const int rr = nv + lane;
+      P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 0] = d_lse[rr];
+      if (P.propose_mode == 1) {
+        const int xh = d_tok[rr];
+        P.out.new_prop_tok[(size_t)b * NP + lane - 1] = xh;
+        // the raw logit at the first argmax is the row's maximum
+        P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 1] = xh >= 0 ? d_raw[rr] * P.inv_t : NAN;
+      }
+    }
+
+    // The accept tests of all positions at once (a test depends on nothing an earlier one decides); the first
+    // position that rejects, or whose token id is out of range, ends the sequence.
+    float al = NAN;
+    bool acc = true;
+    if (pos && !badtok) {
+      const float logp = lx * P.inv_t - d_lse[lane - 1];
+      al = (1.f + P.tau) * expf(logp - logq);
+      al = fminf(al, 1.f);
+      if (al != al) al = 0.f;
+      const uint4 rnd = philox4x32_10(0u, step_of(P), (uint32_t)b, (ISD_TAG_ACCEPT << 16) | (uint32_t)lane, P.seed_lo, P.seed_hi);
+      const float u = (float)(rnd.x >> 8) * 0x1p-24f;
+      acc = u < al;
+    }
+    const unsigned m_badtok = __ballot_sync(full, badtok);
+    const unsigned m_stop = m_badtok | __ballot_sync(full, pos && !badtok && !acc);
+    const int first = m_stop ? __ffs(m_stop) - 1 : nv + 1;
+    const bool bad_first = m_stop && ((m_badtok >> first) & 1u);
+    rej = (m_stop && !bad_first) ? first : 0;
+    a = bad_first ? -1 : (rej ? rej - 1 : nv);
+    const bool evald = pos && lane <= first && !badtok;  // positions whose test was run
+    const bool nonfinite = (evald && d_bad[lane - 1]) || (lane >= 1 && lane <= NP && d_bad[nv + lane]) ||
+                           (lane == 0 && a >= 0 && rej == 0 && d_bad[nv]);
+    uint32_t status = timeout;
+    if (__ballot_sync(full, nonfinite)) status |= ISD_ST_NONFINITE_LOGIT;
+    if (bad_first) status |= ISD_ST_BAD_TOKEN_ID;
+    frozen = a < 0 || (status & ~ISD_ST_EMPTY_RESIDUAL);
+    const int x_next = __shfl_down_sync(full, x, 1);  // lane j - 1 gets proposal j
+    // the rejected token and the LSE of its proposal law, for the residual
+    const int x_rej = __shfl_sync(full, x, rej);
+    const float lse_q_rej = __shfl_sync(full, lse_q, rej);
+    if (lane == 0) {
+      H->x = x_rej;
+      H->lse_q = lse_q_rej;
+    }
+
+    if (write) {
+      if (lane >= 1 && lane <= NP) {
+        P.out.accept[(size_t)b * NP + lane - 1] = evald ? (lane == rej ? 0 : 1) : -1;
+        P.out.alpha[(size_t)b * NP + lane - 1] = evald ? al : NAN;
+      }
+      // the emission: accepted proposals now; the drawn token and the copy of it in repl_tok come from the CTA
+      // of the sampling pass that finishes the draw, unless nothing is drawn
+      const bool draws = !frozen && !(rej > 0 && P.q_mode == 0 && P.q_prev == nullptr);
+      if (lane < P.N && !(draws && lane == a))
+        P.out.out_tok[(size_t)b * P.N + lane] = (!frozen && lane < a) ? x_next : -1;
+      if (lane == 0) {
+        if (!draws) P.out.repl_tok[b] = -1;
+        P.out.accept_len[b] = frozen ? 0 : a;
+        P.out.n_emit[b] = frozen ? 0 : a + 1;
+        if (frozen) {
+          atomicOr(&P.slot_status[b], status);
+          atomicOr(P.global_status, status);
+        }
+      }
+    }
+  }
+  if (lane != 0) return;
+
+  // ---- the CTA's job and the seed of its draw: the true noisy score of the row's argmax, whose raw logit is the
+  // row's maximum (for the residual: if it has residual mass)
+  H->nv = nv;
+  H->rej = frozen ? -1 : rej;
+  const int r = (k == 0 && rej > 0) ? rej - 1 : nv + k;
+  H->r = r;
+  H->q_row = q_row0 + rej - 1;
+  H->lse_p = rej > 0 ? d_lse[rej - 1] : 0.f;
+  H->best = 0u;
+  if (frozen) return;
+  SampleJob J;
+  J.resid = k == 0 && rej > 0;
+  J.x = H->x; J.lse_p = H->lse_p; J.lse_q = H->lse_q;
+  J.qrow = nullptr;
+  if (J.resid && P.q_mode == 0) {
+    if (P.q_prev == nullptr) return;  // nothing to subtract: nothing is drawn
+    J.qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + H->q_row) * row_bytes;
+  }
+  J.step = step_of(P);
+  J.tagpos = k == 0 ? ((ISD_TAG_FINAL << 16) | (uint32_t)(rej > 0 ? rej : nv + 1)) : ((ISD_TAG_PROPOSE << 16) | (uint32_t)k);
+  const int i0 = d_tok[r];
+  if (i0 >= 0 && i0 < P.V) {
+    const uint4 rnd = philox4x32_10((uint32_t)i0 >> 2, J.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
+    const float seed = job_score(P, J, d_raw[r], i0, philox_word(rnd, i0 & 3));
+    if (seed > -INFINITY) H->best = enc_ordered(seed);
+  }
 }
 
 // resident CTAs per SM the sampling kernel is compiled for: three keep it at 80 registers (without the bound
@@ -698,13 +754,11 @@ __device__ __forceinline__ void sample_pass(const VerifyParams& P, const SampleJ
   if (lane < tail - head) drain(head + lane);
 }
 
+// Returns whether this CTA is the one that reports its (slot, k) to the step's ticket: the last of the CTAs that
+// drew for it, or the one with split 0 when none of them has anything to draw.
 template <int DT>
-__device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
+__device__ __forceinline__ bool verify_sample_body(const VerifyParams& P) {
   const int split = blockIdx.x, k = blockIdx.y, b = blockIdx.z;
-  const int act = P.active[b];
-  const int nv = P.n_ver[b];  // both loads in flight together
-  if (!act) return;
-  if (nv < 0 || nv > P.N - 1) return;  // flagged by the row pass
 
   __shared__ float sm_f0[kThreads / 32], sm_f1[kThreads / 32];
   __shared__ int sm_i0[kThreads / 32], sm_i1[kThreads / 32];
@@ -712,24 +766,20 @@ __device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
   __shared__ unsigned sm_best;
   __shared__ SampleQueue sm_queue;
   __shared__ __align__(16) uint4 sm_ring[kSampleRingBytes / 16];
-  __shared__ float d_lse[32];
+  __shared__ float d_lse[32], d_raw[32];
   __shared__ int d_tok[32], d_bad[32];
-  __shared__ SlotDecision sm_dec;
+  __shared__ SampleHead sm_head;
 
-  // ---- what the row pass found: the slot's decision (k = 0), or just the argmax of the MASK row (k >= 1)
+  // ---- what the row pass found, the slot's decision, this CTA's job and its seed (the other warps wait)
   if (threadIdx.x < 32) {
-    if (k == 0) {
-      decide_slot<DT>(P, b, nv, split == 0, d_lse, d_tok, d_bad, &sm_dec);
-    } else if (threadIdx.x == 0) {
-      float m, s;
-      int tok;
-      merge_row(P, b, nv + k, m, s, tok);
-      sm_dec.rej = 0; sm_dec.i0 = tok; sm_dec.lse_p = 0.f;
-    }
+    sample_head<DT>(P, b, k, split, d_lse, d_raw, d_tok, d_bad, &sm_head);
+    if (threadIdx.x == 0) sm_best = sm_head.rej >= 0 ? sm_head.best : 0u;
   }
   __syncthreads();
-  const int rej = sm_dec.rej;
-  if (k == 0 && rej < 0) return;       // frozen slot: no emission
+  const int rej = sm_head.rej;
+  if (rej == -2) return split == 0;             // inactive or invalid slot
+  if (k == 0 && rej < 0) return split == 0;     // frozen slot: no emission
+  const int nv = sm_head.nv;
 
   const int NP = P.N - 1;
   const size_t elt = DT == ISD_LOGITS_BF16 ? 2 : 4;
@@ -740,43 +790,29 @@ __device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
   SampleJob J;
   J.qrow = nullptr; J.x = -1; J.lse_p = 0.f; J.lse_q = 0.f;
   J.step = step_of(P);
-  int r;  // row of this step's logits that is sampled
+  const int r = sm_head.r;  // row of this step's logits that is sampled
   if (k == 0 && rej > 0) {
     // replacement for the first rejected proposal, from normalize(max(0, p - q))
-    if (P.q_mode == 0 && P.q_prev == nullptr) return;  // nothing to subtract: the caller gave no proposal-law rows
-    r = rej - 1;
+    if (P.q_mode == 0 && P.q_prev == nullptr) return split == 0;  // nothing to subtract: the caller gave no proposal-law rows
     J.resid = true;
-    J.x = P.block_tok[(size_t)b * P.Q + rej];
-    J.lse_p = sm_dec.lse_p;
+    J.x = sm_head.x;
+    J.lse_p = sm_head.lse_p;
     if (P.q_mode == 0) {
-      J.qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + (P.q_row0[b] + rej - 1)) * row_bytes;
-      J.lse_q = P.q_stats[((size_t)b * NP + rej - 1) * 2 + 0];
+      J.qrow = reinterpret_cast<const char*>(P.q_prev) + ((size_t)b * P.Q + sm_head.q_row) * row_bytes;
+      J.lse_q = sm_head.lse_q;
     }
     J.tagpos = (ISD_TAG_FINAL << 16) | (uint32_t)rej;
   } else {
-    r = nv + k;  // k = 0: bonus / free token from the row of the last clean token; k >= 1: MASK row k
+    // k = 0: bonus / free token from the row of the last clean token; k >= 1: MASK row k
     J.resid = false;
     J.tagpos = k == 0 ? ((ISD_TAG_FINAL << 16) | (uint32_t)(nv + 1)) : ((ISD_TAG_PROPOSE << 16) | (uint32_t)k);
   }
   J.prow = cur + (size_t)r * row_bytes;
 
-  // the first stages of this CTA's piece of the row are on their way while thread 0 works out the seed
   int lo, hi;
   chunk_range(P.V, P.sample_splits, split, lo, hi);
   RowStream<DT, 1, kSampleRingBytes> in;
   in.start(sm_ring, J.prow, lo, hi);
-
-  // ---- seed: the true noisy score of the row's argmax (for the residual: if it has residual mass)
-  if (threadIdx.x == 0) {
-    float seed = -INFINITY;
-    const int i0 = sm_dec.i0;
-    if (i0 >= 0 && i0 < P.V) {
-      const uint4 rnd = philox4x32_10((uint32_t)i0 >> 2, J.step, (uint32_t)b, J.tagpos, P.seed_lo, P.seed_hi);
-      seed = job_score(P, J, load_logit(J.prow, P.logits_dtype, (size_t)i0), i0, philox_word(rnd, i0 & 3));
-    }
-    sm_best = seed > -INFINITY ? enc_ordered(seed) : 0u;
-  }
-  __syncthreads();
   const float best0 = dec_ordered(sm_best);  // NaN when there is no seed
 
   Top2 top;
@@ -794,7 +830,7 @@ __device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
     sm_last = (arrived == P.sample_splits - 1);
   }
   __syncthreads();
-  if (!sm_last) return;
+  if (!sm_last) return false;
   __threadfence();
 
   // ---- last CTA of the (slot, k): merge, fp64 tie-break, write the token
@@ -843,31 +879,34 @@ __device__ __forceinline__ void verify_sample_body(const VerifyParams& P) {
       atomicOr(P.global_status, ISD_ST_EMPTY_RESIDUAL);
     }
   }
-  if (threadIdx.x != 0) return;
-  if (k == 0) {
-    const int a = rej > 0 ? rej - 1 : nv;
-    P.out.repl_tok[b] = y;
-    P.out.out_tok[(size_t)b * P.N + a] = y;
-  } else {
-    P.out.new_prop_tok[(size_t)b * NP + k - 1] = y;
-    P.out.new_q_stats[((size_t)b * NP + k - 1) * 2 + 1] =
-        y >= 0 ? load_logit(J.prow, P.logits_dtype, (size_t)y) * P.inv_t : NAN;
+  if (threadIdx.x == 0) {
+    if (k == 0) {
+      const int a = rej > 0 ? rej - 1 : nv;
+      P.out.repl_tok[b] = y;
+      P.out.out_tok[(size_t)b * P.N + a] = y;
+    } else {
+      P.out.new_prop_tok[(size_t)b * NP + k - 1] = y;
+      P.out.new_q_stats[((size_t)b * NP + k - 1) * 2 + 1] =
+          y >= 0 ? load_logit(J.prow, P.logits_dtype, (size_t)y) * P.inv_t : NAN;
+    }
   }
+  return true;
 }
 
 template <int DT>
 __global__ void __launch_bounds__(kThreads, kSampleMinBlocks) verify_sample_kernel(const VerifyParams P) {
   pdl_wait();
   pdl_launch_dependents();
-  verify_sample_body<DT>(P);
-  if (!P.fuse_commit) return;
-  // ---- isd_step: the CTA that finishes last (a ticket over the whole grid; nobody waits) has every slot's
-  // decision and tokens in front of it and commits the batch, which saves the launch of a kernel for it
+  const bool reports = verify_sample_body<DT>(P);
+  if (!P.fuse_commit || !reports) return;
+  // ---- isd_step: every (slot, k) is reported once to a ticket over the grid, after its token is written; the
+  // CTA that reports last (nobody waits) has every slot's decision and tokens in front of it and commits the
+  // batch, which saves the launch of a kernel for it
   __shared__ int sm_commit[36];
   if (threadIdx.x == 0) {
-    __threadfence();  // thread 0 wrote everything this CTA contributes (tokens, status bits)
+    __threadfence();  // what this CTA wrote (tokens, status bits) comes before its report
     const int arrived = atomicAdd(P.step_ticket, 1);
-    sm_commit[35] = (arrived == (int)(gridDim.x * gridDim.y * gridDim.z) - 1);
+    sm_commit[35] = (arrived == (int)(gridDim.y * gridDim.z) - 1);
   }
   __syncthreads();
   if (!sm_commit[35]) return;
