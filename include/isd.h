@@ -339,7 +339,7 @@ int isd_set_profile_events(isd_ctx* ctx, void* attn_start, void* attn_stop, void
  * isd_verify without any allocation (the paper has no counterpart; this serves hosts of the
  * library).  Same computation, arguments and outputs as isd_verify, but it needs no isd_ctx: the
  * scratch of the two verification kernels lives in a fixed array inside the library's device image
- * (about 0.8 MB on every GPU that loads the library, held until the process exits).
+ * (about 0.65 MB on every GPU that loads the library, held until the process exits).
  *
  * Who needs it: callers that cannot call cudaMalloc when they verify -- an engine that has given
  * all free device memory to its own KV-cache allocator, a latency-critical thread on which

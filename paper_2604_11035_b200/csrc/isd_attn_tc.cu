@@ -140,12 +140,6 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
 }
 
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
-}
 
 // K-major / MN-major shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -201,15 +195,6 @@ __device__ __forceinline__ float ex2f(float x) {
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
-}
-// bf16 pair of two non-negative finite floats, rounded half up, with integer ALU operations only: the
-// conversion instruction shares the transcendental unit with ex2, which is the busiest pipe of the
-// softmax warps.
-__device__ __forceinline__ uint32_t pack_bf16_alu(float a, float b) {
-  const uint32_t ra = __float_as_uint(a) + 0x8000u, rb = __float_as_uint(b) + 0x8000u;
-  uint32_t d;
-  asm("prmt.b32 %0, %1, %2, 0x7632;" : "=r"(d) : "r"(ra), "r"(rb));
-  return d;
 }
 
 // bf16 pair (a in the low half, b in the high half) with the conversion instruction: one instruction instead of

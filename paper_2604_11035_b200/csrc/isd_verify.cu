@@ -5,19 +5,20 @@
 // Two launches, neither of which waits on anything:
 //   1. verify_rows_kernel   one CTA per (slot, block row, split): a single streaming pass over the
 //      logits row that yields the online-softmax pair (max, sum) -> LSE and the argmax of the row.
-//      Every row has the same role here, so the kernel is a lean HBM stream.  The last CTA of a slot
-//      to finish (atomic ticket, nobody waits) merges the partials, runs the sequential accept test
-//      and writes every output that needs no random sample: accept flags, alpha, accept length, the
-//      accepted tokens, argmax proposals and the proposal-law statistics.
-//   2. verify_sample_kernel one CTA per (slot, sampled row, split).  Each slot draws exactly one
-//      token for its emission: the replacement from normalize(max(0, p - q)) when a proposal was
-//      rejected, else the bonus / free token from the row of the last clean token; with sampled
-//      proposals the N - 1 MASK rows are drawn here too.  The pass re-reads the row (mostly from L2:
-//      the rows kernel reads the rows that are sampled last).
+//      Every row has the same role here, so the kernel is a lean HBM stream; every warp ends with one
+//      store of its partial and nothing else (no merge, no fence, no ticket).
+//   2. verify_sample_kernel one CTA per (slot, sampled row, split).  At its head one warp merges the
+//      partials of the slot's rows, runs the accept tests of all proposals at once (Algorithm 1's
+//      sequence ends at the first that fails) and, in the CTA with split 0, writes every output that
+//      needs no random sample: accept flags, alpha, accept length, the accepted tokens, argmax
+//      proposals and the proposal-law statistics.  Then each slot draws exactly one token for its
+//      emission: the replacement from normalize(max(0, p - q)) when a proposal was rejected, else the
+//      bonus / free token from the row of the last clean token; with sampled proposals the N - 1 MASK
+//      rows are drawn here too.  The pass reads the row again.
 //
 // Gumbel noise is a pure function of (seed, step, slot, tag, position, vocab index), so any
 // reduction order gives the same sample, and it is evaluated only for elements that can still win.
-// The sampling pass starts from the true noisy score of the row's argmax (known from pass 1), which
+// The sampling pass starts from the true noisy score of the row's argmax (its logit is the row's maximum), which
 // is a lower bound of the winner's score from the first element on.  (1) No variate on the 24-bit
 // lattice exceeds 25 ln 2 = 17.33, so a group of four logits whose maximum is more than 17.34 below
 // the running best needs no random numbers at all; the groups that survive are compacted into a
@@ -996,7 +997,7 @@ unsigned char* g_static_ptr[kMaxDevices] = {};
 
 }  // namespace
 
-// File-scope device array (about 0.8 MB per GPU).  In host code this name is only a handle for
+// File-scope device array (about 0.65 MB per GPU).  In host code this name is only a handle for
 // cudaGetSymbolAddress; it is never passed to a kernel directly.
 static __device__ __align__(256) unsigned char g_isd_verify_static_scratch[kStaticBytes];
 
