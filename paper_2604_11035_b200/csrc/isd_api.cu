@@ -8,6 +8,9 @@
 int isd_attn_tc_create(isd_ctx* ctx);
 void isd_attn_tc_destroy(isd_ctx* ctx);
 
+// pieces per sampled row of the verification's second pass (isd_verify.cu)
+int isd_pick_sample_splits(const isd_config& c, int num_sms);
+
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -79,10 +82,8 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   rs = rs > max_by_len ? max_by_len : rs;
   ctx->row_splits = rs;
   // every slot samples one row (bonus token or residual replacement; N rows with sampled proposals)
-  // in the second pass; those passes are light, so they are cut as finely as the row length allows
-  // (four pieces per row: every further piece re-learns the running best score; eight cost 45 % more)
-  int ps = 4;
-  ps = ps > max_by_len ? max_by_len : ps;
+  // in the second pass
+  const int ps = isd_pick_sample_splits(c, ctx->num_sms);
   ctx->sample_splits = ps;
 
   int rc = ISD_OK;
