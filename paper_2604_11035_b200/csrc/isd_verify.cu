@@ -156,16 +156,40 @@ __device__ __forceinline__ void chunk_range(int V, int splits, int split, int& l
   hi = min(V, lo + per);
 }
 
-// Block-wide merge helpers (8 worker warps) -------------------------------------------------------
+// Top-2 merges ----------------------------------------------------------------------------------------
+// The two best of the union of the lanes' candidate pairs, in every lane: the winner is the best first
+// candidate (highest score, lowest index among equals), the runner-up the best of the other lanes' first
+// candidates and the winner lane's second.  On order-preserving integer codes of the scores each place is one
+// max- and one min-reduction of the warp, where five shuffle rounds of compare-and-swap on pairs cost some
+// three hundred dependent instructions at the end of every CTA.  (Indices are distinct across lanes: they are
+// different elements of a row.)
+__device__ __forceinline__ void warp_top2(Top2& t) {
+  const unsigned full = 0xffffffffu;
+  const unsigned k1 = t.i1 >= 0 ? enc_ordered(t.s1) : 0u;
+  const unsigned K1 = __reduce_max_sync(full, k1);
+  const int I1 = __reduce_min_sync(full, (t.i1 >= 0 && k1 == K1) ? t.i1 : 0x7FFFFFFF);
+  const bool won = t.i1 >= 0 && t.i1 == I1;
+  const float cs = won ? t.s2 : t.s1;
+  const int ci = won ? t.i2 : t.i1;
+  const unsigned k2 = ci >= 0 ? enc_ordered(cs) : 0u;
+  const unsigned K2 = __reduce_max_sync(full, k2);
+  const int I2 = __reduce_min_sync(full, (ci >= 0 && k2 == K2) ? ci : 0x7FFFFFFF);
+  t.s1 = K1 ? dec_ordered(K1) : -INFINITY; t.i1 = K1 ? I1 : -1;
+  t.s2 = K2 ? dec_ordered(K2) : -INFINITY; t.i2 = K2 ? I2 : -1;
+}
+
+// Over the 8 worker warps of a CTA; the result is valid in warp 0.  One barrier: the arrays are not touched
+// again before the next CTA-wide barrier of the caller.
 __device__ __forceinline__ void block_merge_top2(Top2& t, float* sm_s1, int* sm_i1, float* sm_s2, int* sm_i2) {
-  warp_merge_top2(t);
+  warp_top2(t);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (lane == 0) { sm_s1[warp] = t.s1; sm_i1[warp] = t.i1; sm_s2[warp] = t.s2; sm_i2[warp] = t.i2; }
   worker_sync();
-  if (threadIdx.x == 0) {
-    for (int w = 1; w < kThreads / 32; ++w) t.merge(sm_s1[w], sm_i1[w], sm_s2[w], sm_i2[w]);
+  if (warp == 0) {
+    t.init();
+    if (lane < kThreads / 32) { t.s1 = sm_s1[lane]; t.i1 = sm_i1[lane]; t.s2 = sm_s2[lane]; t.i2 = sm_i2[lane]; }
+    warp_top2(t);
   }
-  worker_sync();
 }
 
 // fp64 score of vocabulary index i of a Gumbel row: logit * invT + g
@@ -389,12 +413,29 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) S += __shfl_xor_sync(0xffffffffu, S, off);
   const int widx = __reduce_min_sync(0xffffffffu, (raw_idx >= 0 && raw_max == wmax) ? raw_idx : 0x7FFFFFFF);
-  if (lane == 0) {
-    if (!ok) row_timeout(P, b);
-    RowPartial rp;
-    rp.m = wmax * P.inv_t; rp.s = S; rp.raw_max = wmax; rp.idx = widx == 0x7FFFFFFF ? -1 : widx;
-    P.row_part[(((size_t)b * P.Q + r) * P.row_splits + split) * kWarps + warp] = rp;
+  if (lane == 0 && !ok) row_timeout(P, b);
+  const float4 mine = make_float4(wmax * P.inv_t, S, wmax, __int_as_float(widx == 0x7FFFFFFF ? -1 : widx));
+  float4* parts = reinterpret_cast<float4*>(P.row_part);
+  if (P.row_splits == 1) {  // large batches: one partial per warp, see above
+    if (lane == 0) parts[((size_t)b * P.Q + r) * kWarps + warp] = mine;
+    return;
   }
+  // Small batches cut a row into several CTAs and are bound by latency, not by copies in flight: one partial per
+  // CTA keeps the merge at the head of the sampling kernel short.
+  __shared__ float4 sm_part[kWarps];
+  if (lane == 0) sm_part[warp] = mine;
+  worker_sync();
+  if (warp != 0) return;
+  float4 v = lane < kWarps ? sm_part[lane] : make_float4(-INFINITY, 0.f, -INFINITY, __int_as_float(-1));
+#pragma unroll
+  for (int off = kWarps / 2; off > 0; off >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, v.x, off), os = __shfl_xor_sync(0xffffffffu, v.y, off);
+    const float orw = __shfl_xor_sync(0xffffffffu, v.z, off);
+    const int oi = __float_as_int(__shfl_xor_sync(0xffffffffu, v.w, off)), mi = __float_as_int(v.w);
+    lse_merge(v.x, v.y, om, os);
+    if (oi >= 0 && (mi < 0 || orw > v.z || (orw == v.z && oi < mi))) { v.z = orw; v.w = __int_as_float(oi); }
+  }
+  if (lane == 0) parts[((size_t)b * P.Q + r) * P.row_splits + split] = v;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -454,7 +495,7 @@ struct SampleHead {
   unsigned best;  // ordered code of the seed score (0: none)
 };
 
-constexpr int kHeadChunk = 8;  // partials of a row merged per pass (one pass when the row pass ran one CTA per row)
+constexpr int kHeadChunk = 8;  // partials of a row merged per pass (one pass unless the row pass cut a row into more than eight CTAs)
 
 // Called by all 32 lanes of warp 0.  d_*: 32 entries of shared memory each.
 template <int DT>
@@ -471,12 +512,13 @@ __device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k,
   // ---- first trip: nothing here depends on anything else that is read
   const int act = P.active[b];
   const int nv = P.n_ver[b];
-  const int n_part = P.row_splits * (kThreads / 32);
+  const int n_part = P.row_splits == 1 ? kThreads / 32 : P.row_splits;  // per warp of the row's CTA, or per CTA
   const bool has_row = lane < P.Q;  // lane = block row (rows beyond the slot's block hold stale partials, unused)
   const float4* rp = reinterpret_cast<const float4*>(P.row_part) + ((size_t)b * P.Q + (has_row ? lane : 0)) * n_part;
+  const float4 neutral = make_float4(-INFINITY, 0.f, -INFINITY, __int_as_float(-1));
   float4 part[kHeadChunk];
 #pragma unroll
-  for (int i = 0; i < kHeadChunk; ++i) part[i] = __ldcg(rp + i);  // n_part is a multiple of kHeadChunk
+  for (int i = 0; i < kHeadChunk; ++i) part[i] = i < n_part ? __ldcg(rp + i) : neutral;
   const bool is_pos = k == 0 && lane >= 1 && lane <= NP;  // lane = proposal position j (valid when j <= nv)
   int x = 0;
   float logq = 0.f, lse_q = 0.f;
@@ -530,7 +572,7 @@ __device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k,
       c += kHeadChunk;
       if (c >= n_part) break;
 #pragma unroll
-      for (int i = 0; i < kHeadChunk; ++i) part[i] = __ldcg(rp + c + i);
+      for (int i = 0; i < kHeadChunk; ++i) part[i] = c + i < n_part ? __ldcg(rp + c + i) : neutral;
     }
     const bool valid = lane < q_len;
     // NaN anywhere poisons s; +inf logits give m = +inf
@@ -835,27 +877,30 @@ __device__ __forceinline__ bool verify_sample_body(const VerifyParams& P) {
   __threadfence();
 
   // ---- last CTA of the (slot, k): merge, fp64 tie-break, write the token
-  if (threadIdx.x == 0) {
-    *ticket = 0;  // ready for the next call
+  if (threadIdx.x < 32) {
     Top2 t;
     t.init();
-    for (int i = 0; i < P.sample_splits; ++i) {
-      const volatile SamplePartial* sp = parts + i;
-      t.merge(sp->best1, sp->idx1, sp->best2, sp->idx2);
+    if ((int)threadIdx.x < P.sample_splits) {  // at most 16 pieces: one per lane
+      const volatile SamplePartial* sp = parts + threadIdx.x;
+      t.s1 = sp->best1; t.i1 = sp->idx1; t.s2 = sp->best2; t.i2 = sp->idx2;
     }
-    int y = t.i1;
-    if (t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
-      double s1, s2;
-      if (J.resid) {
-        s1 = resid_score_f64(P, J.prow, J.qrow, t.i1, J.x, J.lse_p, J.lse_q, J.step, (uint32_t)b, J.tagpos);
-        s2 = resid_score_f64(P, J.prow, J.qrow, t.i2, J.x, J.lse_p, J.lse_q, J.step, (uint32_t)b, J.tagpos);
-      } else {
-        s1 = noisy_score_f64(P, J.prow, t.i1, J.step, (uint32_t)b, J.tagpos);
-        s2 = noisy_score_f64(P, J.prow, t.i2, J.step, (uint32_t)b, J.tagpos);
+    warp_top2(t);
+    if (threadIdx.x == 0) {
+      *ticket = 0;  // ready for the next call
+      int y = t.i1;
+      if (t.i1 >= 0 && t.i2 >= 0 && (t.s1 - t.s2) < ISD_TIE_EPS) {
+        double s1, s2;
+        if (J.resid) {
+          s1 = resid_score_f64(P, J.prow, J.qrow, t.i1, J.x, J.lse_p, J.lse_q, J.step, (uint32_t)b, J.tagpos);
+          s2 = resid_score_f64(P, J.prow, J.qrow, t.i2, J.x, J.lse_p, J.lse_q, J.step, (uint32_t)b, J.tagpos);
+        } else {
+          s1 = noisy_score_f64(P, J.prow, t.i1, J.step, (uint32_t)b, J.tagpos);
+          s2 = noisy_score_f64(P, J.prow, t.i2, J.step, (uint32_t)b, J.tagpos);
+        }
+        if (s2 > s1 || (s2 == s1 && t.i2 < t.i1)) y = t.i2;
       }
-      if (s2 > s1 || (s2 == s1 && t.i2 < t.i1)) y = t.i2;
+      sm_tok = y;
     }
-    sm_tok = y;
   }
   __syncthreads();
   int y = sm_tok;
