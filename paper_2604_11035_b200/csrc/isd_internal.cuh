@@ -304,22 +304,7 @@ struct Top2 {
       s2 = s; i2 = i;
     }
   }
-  __device__ __forceinline__ void merge(float os1, int oi1, float os2, int oi2) {
-    push(os1, oi1);
-    push(os2, oi2);
-  }
 };
-
-__device__ __forceinline__ void warp_merge_top2(Top2& t) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    const float os1 = __shfl_xor_sync(0xffffffffu, t.s1, off);
-    const int oi1 = __shfl_xor_sync(0xffffffffu, t.i1, off);
-    const float os2 = __shfl_xor_sync(0xffffffffu, t.s2, off);
-    const int oi2 = __shfl_xor_sync(0xffffffffu, t.i2, off);
-    t.merge(os1, oi1, os2, oi2);
-  }
-}
 
 // (m, s) pairs of an online softmax: combine two partial sums of exp(l - m).
 __device__ __forceinline__ void lse_merge(float& m, float& s, float om, float os) {
