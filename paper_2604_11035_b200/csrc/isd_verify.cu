@@ -965,11 +965,12 @@ __global__ void __launch_bounds__(kThreads, kSampleMinBlocks) verify_sample_kern
 
 // Pieces a sampled row is cut into.  Large batches: four (every further piece starts again from the seed alone
 // and re-learns the running best; eight cost 45 % more work on flat rows).  Small batches are latency-bound and
-// leave most SMs idle, so their rows are cut finer, up to sixteen pieces (batch 1: 50 -> 42 us of verification).
+// leave most SMs idle, so their rows are cut finer, up to sixteen pieces, as long as all CTAs are resident at once
+// (four per SM; batch 1: 50 -> 42 us of verification).
 int isd_pick_sample_splits(const isd_config& c, int num_sms) {
   const int rows = c.batch * (c.propose_mode == 0 ? c.stride : 1);
   const int max_by_len = (c.vocab + 8191) / 8192;  // keep at least 8k elements per CTA
-  int ps = (4 * num_sms + rows - 1) / rows;
+  int ps = 4 * num_sms / rows;  // rounded down: a few CTAs more than the SMs hold at once would double the pass
   ps = ps < 4 ? 4 : (ps > 16 ? 16 : ps);
   return ps > max_by_len ? max_by_len : ps;
 }
