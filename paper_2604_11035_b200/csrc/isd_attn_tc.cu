@@ -218,6 +218,15 @@ struct Segment {
   int part_slot; // scratch slot when the segment does not cover the whole pair, else -1
 };
 
+// Units of the split axis per CTA.  Small batches do not fill the machine: below kMinShare units a share would
+// be mostly fixed cost (Q staging, pipeline fill, a partial result of 64 KB that the combine kernel reads back), so
+// fewer CTAs take longer shares and the rest leave at once.
+constexpr int kMinShare = 8;  // 12 and 16 measured slower at batch 1, equal at batch 8
+__device__ __forceinline__ long long share_units(long long total, int num_ctas) {
+  const long long per = (total + num_ctas - 1) / num_ctas;
+  return per < kMinShare ? kMinShare : per;
+}
+
 struct WorkIter {
   const int* prefix;
   const int* slot_info;  // ctx_len | q_len << 24 per slot in shared memory, or nullptr (read the state arrays)
@@ -228,7 +237,7 @@ struct WorkIter {
     slot_info = slot_info_;
     B = P.B; Hkv = P.Hkv;
     const long long total = (long long)prefix[B] * Hkv;
-    const long long per = (total + P.num_ctas - 1) / P.num_ctas;
+    const long long per = share_units(total, P.num_ctas);
     t_begin = t = (long long)cta * per;
     t_end = t + per < total ? t + per : total;
     // first slot whose range ends after t
@@ -886,7 +895,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const TcP
   pdl_launch_dependents();
   const long long total = (long long)P.tile_prefix[P.B] * P.Hkv;
   if (total == 0) return;
-  const long long per = (total + P.num_ctas - 1) / P.num_ctas;
+  const long long per = share_units(total, P.num_ctas);
   const long long t_last = ((long long)(c0 + 1) * per < total ? (long long)(c0 + 1) * per : total) - 1;
   if (t_last < (long long)c0 * per) return;  // empty share
   // slot of the share's last tile = number of slots whose tiles all lie at or before t_last
