@@ -328,6 +328,14 @@ int isd_test_preset_lora_counter(isd_ctx* ctx, int32_t row_block, uint32_t value
 int isd_test_lora_work_item(int32_t m, int32_t n, int32_t rank, int32_t num_sms, int32_t unit_index, int32_t item,
                             int32_t* out);
 
+/*
+ * Test hook, host only (the paper has no counterpart; needs no GPU): the launch shape isd_verify picks for a
+ * configuration on a GPU of num_sms SMs.  out[0] = CTAs a row of the first pass is cut into, out[1] = pieces a
+ * sampled row of the second pass is cut into, out[2] / out[3] = CTAs of the two launches.  Only batch, stride, vocab
+ * and propose_mode of cfg are read.  Errors: ISD_ERR_INVALID_ARG.
+ */
+int isd_test_verify_grid(const isd_config* cfg, int32_t num_sms, int32_t* out);
+
 /* Optional instrumentation (the paper has no counterpart): cudaEvent_t handles, passed as void*,
  * that later calls record on their stream immediately before / after the attention main kernel
  * (attn_*) and the kernels of isd_verify together (verify_*).  NULL switches a pair off.

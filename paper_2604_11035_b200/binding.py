@@ -21,7 +21,7 @@ ST_KERNEL_TIMEOUT = 0x80000000
 EXPORTS = ["isd_create", "isd_destroy", "isd_attn", "isd_verify", "isd_commit", "isd_step",
            "isd_release", "isd_read_status", "isd_set_profile_events", "isd_launch_count", "isd_strerror",
            "isd_verify_static", "isd_step_layers", "isd_set_step_counter", "isd_lora_linear", "isd_set_wait_limit",
-           "isd_test_preset_lora_counter", "isd_test_lora_work_item"]
+           "isd_test_preset_lora_counter", "isd_test_lora_work_item", "isd_test_verify_grid"]
 
 
 class IsdConfig(C.Structure):
@@ -95,6 +95,8 @@ def load():
         lib.isd_test_preset_lora_counter.restype = C.c_int
         lib.isd_test_lora_work_item.argtypes = [C.c_int32] * 6 + [C.POINTER(C.c_int32)]
         lib.isd_test_lora_work_item.restype = C.c_int
+        lib.isd_test_verify_grid.argtypes = [C.POINTER(IsdConfig), C.c_int32, C.POINTER(C.c_int32)]
+        lib.isd_test_verify_grid.restype = C.c_int
         lib.isd_launch_count.argtypes = [vp]
         lib.isd_launch_count.restype = C.c_int64
         lib.isd_strerror.argtypes = [C.c_int]
@@ -117,6 +119,17 @@ def lora_work_item(m: int, n: int, rank: int, num_sms: int, unit_index: int, ite
         raise IsdError(f"isd_test_lora_work_item failed: {load().isd_strerror(rc).decode()} ({rc})")
     keys = ("form", "units", "n_items", "pre", "m0", "n0", "cols", "tile_rows", "tile_cols")
     return dict(zip(keys, [int(x) for x in out]))
+
+
+def verify_grid(batch: int, stride: int, vocab: int, propose_mode: int, num_sms: int) -> dict:
+    """Host-only view of the launch shape isd_verify picks (see isd_test_verify_grid in include/isd.h)."""
+    cfg = IsdConfig()
+    cfg.batch, cfg.stride, cfg.vocab, cfg.propose_mode = batch, stride, vocab, propose_mode
+    out = (C.c_int32 * 4)()
+    rc = load().isd_test_verify_grid(C.byref(cfg), num_sms, out)
+    if rc != 0:
+        raise IsdError(f"isd_test_verify_grid failed: {load().isd_strerror(rc).decode()} ({rc})")
+    return dict(zip(("row_splits", "sample_splits", "row_ctas", "sample_ctas"), [int(x) for x in out]))
 
 
 def _check(rc: int, what: str):

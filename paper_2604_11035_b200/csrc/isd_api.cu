@@ -8,7 +8,8 @@
 int isd_attn_tc_create(isd_ctx* ctx);
 void isd_attn_tc_destroy(isd_ctx* ctx);
 
-// pieces per sampled row of the verification's second pass (isd_verify.cu)
+// CTAs per row of the verification's first pass and pieces per sampled row of its second (isd_verify.cu)
+int isd_pick_row_splits(const isd_config& c, int num_sms);
 int isd_pick_sample_splits(const isd_config& c, int num_sms);
 
 namespace {
@@ -72,14 +73,8 @@ int isd_create(const isd_config* cfg, isd_ctx** out) {
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
   ctx->num_sms = sms > 0 ? sms : ISD_NUM_SMS_DEFAULT;
 
-  // Enough CTAs to fill the machine at small batch; one CTA per row once rows are plentiful.
   const int rows = c.batch * Q;
-  const int target = ctx->num_sms * 4;
-  int rs = (target + rows - 1) / rows;
-  const int max_by_len = (c.vocab + 8191) / 8192;  // keep at least 8k elements per CTA
-  rs = rs < 1 ? 1 : rs;
-  rs = rs > 16 ? 16 : rs;
-  rs = rs > max_by_len ? max_by_len : rs;
+  const int rs = isd_pick_row_splits(c, ctx->num_sms);
   ctx->row_splits = rs;
   // every slot samples one row (bonus token or residual replacement; N rows with sampled proposals)
   // in the second pass

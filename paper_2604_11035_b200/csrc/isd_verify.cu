@@ -963,6 +963,16 @@ __global__ void __launch_bounds__(kThreads, kSampleMinBlocks) verify_sample_kern
 
 }  // namespace
 
+// CTAs a row of the row pass is cut into: enough CTAs to fill the machine (five per SM run at once) at small
+// batch, one CTA per row once rows are plentiful; a piece keeps at least 8k elements.
+int isd_pick_row_splits(const isd_config& c, int num_sms) {
+  const int rows = c.batch * (2 * c.stride - 1);
+  const int max_by_len = (c.vocab + 8191) / 8192;
+  int rs = (4 * num_sms + rows - 1) / rows;
+  rs = rs < 1 ? 1 : (rs > 16 ? 16 : rs);
+  return rs > max_by_len ? max_by_len : rs;
+}
+
 // Pieces a sampled row is cut into.  Large batches: four (every further piece starts again from the seed alone
 // and re-learns the running best; eight cost 45 % more work on flat rows).  Small batches are latency-bound and
 // leave most SMs idle, so their rows are cut finer, up to sixteen pieces, as long as all CTAs are resident at once
@@ -1098,11 +1108,8 @@ extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* s
   int sms = 0;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   tmp.num_sms = sms > 0 ? sms : ISD_NUM_SMS_DEFAULT;
-  const int rows = c.batch * tmp.Q, target = tmp.num_sms * 4;
-  const int max_by_len = (c.vocab + 8191) / 8192;
-  int rs = (target + rows - 1) / rows;
-  rs = rs < 1 ? 1 : (rs > kStaticMaxSplits ? kStaticMaxSplits : rs);
-  rs = rs > max_by_len ? max_by_len : rs;
+  const int rows = c.batch * tmp.Q;
+  int rs = isd_pick_row_splits(c, tmp.num_sms);  // <= kStaticMaxSplits
   if (rows * rs > kStaticMaxRowPieces) rs = kStaticMaxRowPieces / rows;  // >= 1: rows <= 64 * ISD_MAX_Q
   tmp.row_splits = rs;
   tmp.sample_splits = isd_pick_sample_splits(c, tmp.num_sms);  // same cut as isd_create uses (<= kStaticMaxSplits)
@@ -1116,4 +1123,15 @@ extern "C" int isd_verify_static(const isd_config* cfg, const isd_batch_state* s
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(base, 0, kZeroedBytes, stream) != cudaSuccess) return ISD_ERR_CUDA;
   return isd_launch_verify(&tmp, st, logits_cur, q_prev_logits, (uint32_t)step, out, stream);
+}
+
+extern "C" int isd_test_verify_grid(const isd_config* cfg, int32_t num_sms, int32_t* out) {
+  if (!cfg || !out || num_sms < 1 || cfg->batch < 1 || cfg->stride < 1 || cfg->vocab < 8) return ISD_ERR_INVALID_ARG;
+  const isd_config& c = *cfg;
+  const int rs = isd_pick_row_splits(c, num_sms), ps = isd_pick_sample_splits(c, num_sms);
+  out[0] = rs;
+  out[1] = ps;
+  out[2] = rs * c.batch * (2 * c.stride - 1);
+  out[3] = ps * c.batch * (c.propose_mode == 0 ? c.stride : 1);
+  return ISD_OK;
 }
