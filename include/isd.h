@@ -137,8 +137,11 @@ typedef struct isd_verify_out {
   int32_t* repl_tok;     /* [B] resampled (on rejection) or bonus token               */
   int32_t* out_tok;      /* [B, N] finalised tokens (accepted proposals, then
                             repl_tok), -1 padded                                      */
-  int32_t* new_prop_tok; /* [B, N-1] proposals made by this step's MASK rows          */
-  float* new_q_stats;    /* [B, N-1, 2] their {LSE, logit}                            */
+  int32_t* new_prop_tok; /* [B, N-1] proposals made by this step's MASK rows; -1 where
+                            a proposal of the slot was rejected: the MASK rows were
+                            conditioned on tokens that are discarded, and the next
+                            step is a pure stride step (Sec. 3.2, adaptive stride)   */
+  float* new_q_stats;    /* [B, N-1, 2] their {LSE, logit}; NaN where none was made   */
 } isd_verify_out;
 
 /* Everything one step consumes and produces besides the state. */

@@ -390,10 +390,14 @@ static void verify_slot(const verify_args* A, int b, double* lp, double* lq) {
   for (int j = 1; j <= a; ++j) A->out_tok[(size_t)b * N + (j - 1)] = A->block_tok[(size_t)b * Q + j];
   A->out_tok[(size_t)b * N + a] = y;
 
-  /* Stride: each MASK row proposes the token after its position. */
+  /* Stride: each MASK row proposes the token after its position.  After a rejection "all subsequent tokens are
+   * discarded; the next step becomes a pure stride with no tokens to introspect" (Sec. 3.2, adaptive stride): the
+   * MASK rows were conditioned on the discarded tokens, so no proposals are made from them and the outputs keep
+   * their defaults (-1 / NaN).  The rows are still checked for non-finite logits. */
   for (int m = 1; m <= NP; ++m) {
     if (load_row(A->logits_cur, A->logits_dtype, cur_base + (size_t)(nv + m) * V, V, A->invT, lp))
       status |= ORC_ST_NONFINITE_LOGIT;
+    if (a != nv) continue;
     orc_filter_row(lp, V, A->top_k, A->top_p);
     double margin;
     int xh;
@@ -592,6 +596,7 @@ int orc_commit(int B, int N, int page_size, int max_pages, int mask_token, int32
     block_tok[(size_t)b * Q + 0] = repl_tok[b];
     for (int m = 1; m <= NP; ++m) {
       block_tok[(size_t)b * Q + m] = all_accepted ? new_prop_tok[(size_t)b * NP + (m - 1)] : mask_token;
+      if (!all_accepted) continue; /* no proposals were made: the statistics of the old ones stay (unused) */
       q_stats[((size_t)b * NP + (m - 1)) * 2 + 0] = new_q_stats[((size_t)b * NP + (m - 1)) * 2 + 0];
       q_stats[((size_t)b * NP + (m - 1)) * 2 + 1] = new_q_stats[((size_t)b * NP + (m - 1)) * 2 + 1];
     }

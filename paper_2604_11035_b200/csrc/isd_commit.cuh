@@ -129,6 +129,7 @@ __device__ __forceinline__ void commit_block(const CommitParams& P, int* sm_warp
         bt[0] = __ldcg(P.repl_tok + b);
         for (int m = 1; m <= NP; ++m) {
           bt[m] = all_accepted ? __ldcg(P.new_prop_tok + (size_t)b * NP + m - 1) : P.mask_token;
+          if (!all_accepted) continue;  // no proposals were made after a rejection: nothing to keep statistics of
           P.q_stats[((size_t)b * NP + m - 1) * 2 + 0] = __ldcg(P.new_q_stats + ((size_t)b * NP + m - 1) * 2 + 0);
           P.q_stats[((size_t)b * NP + m - 1) * 2 + 1] = __ldcg(P.new_q_stats + ((size_t)b * NP + m - 1) * 2 + 1);
         }

@@ -485,8 +485,9 @@ __device__ __forceinline__ float job_score(const VerifyParams& P, const SampleJo
 // reads is fetched in one go, so that the head costs two trips to memory (three for a residual against softmax q).
 // ------------------------------------------------------------------------------------------------
 struct SampleHead {
-  int rej;        // -2: slot inactive or invalid; -1: frozen, nothing is drawn for the emission; 0: nothing rejected;
-                  // j: first rejected proposal
+  int rej;        // -2: nothing for this CTA to draw (slot inactive or invalid; MASK row of a slot that makes no
+                  // proposals); -1: frozen, nothing is drawn for the emission; 0: nothing rejected; j: first
+                  // rejected proposal
   int nv;
   int r;          // row of this step's logits that the CTA draws from
   int x;          // residual: the rejected token
@@ -519,7 +520,7 @@ __device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k,
   float4 part[kHeadChunk];
 #pragma unroll
   for (int i = 0; i < kHeadChunk; ++i) part[i] = i < n_part ? __ldcg(rp + i) : neutral;
-  const bool is_pos = k == 0 && lane >= 1 && lane <= NP;  // lane = proposal position j (valid when j <= nv)
+  const bool is_pos = lane >= 1 && lane <= NP;  // lane = proposal position j (valid when j <= nv)
   int x = 0;
   float logq = 0.f, lse_q = 0.f;
   if (is_pos) {
@@ -530,13 +531,9 @@ __device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k,
       logq = qs[1] - lse_q;
     }
   }
-  uint32_t timeout = 0;
-  int q_row0 = 0;
-  if (k == 0) {
-    // a warp of the row pass gave up on a wait: a partial is incomplete, nothing of the slot may be committed
-    timeout = *reinterpret_cast<volatile uint32_t*>(&P.slot_status[b]) & ISD_ST_KERNEL_TIMEOUT;
-    if (P.q_mode == 0) q_row0 = P.q_row0[b];
-  }
+  // a warp of the row pass gave up on a wait: a partial is incomplete, nothing of the slot may be committed
+  const uint32_t timeout = *reinterpret_cast<volatile uint32_t*>(&P.slot_status[b]) & ISD_ST_KERNEL_TIMEOUT;
+  const int q_row0 = (k == 0 && P.q_mode == 0) ? P.q_row0[b] : 0;
 
   if (!act || nv < 0 || nv > NP) {  // an invalid n_ver was flagged by the row pass
     if (lane == 0) H->rej = -2;
@@ -585,20 +582,7 @@ __device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k,
 
   int rej = 0, a = nv;
   bool frozen = false;
-  if (k == 0) {
-    // proposal-law statistics (lanes 1..N-1 = MASK row m); argmax proposals are final here, sampled ones
-    // and their logit are written by the CTAs that draw them
-    if (write && lane >= 1 && lane <= NP) {
-      const int rr = nv + lane;
-      P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 0] = d_lse[rr];
-      if (P.propose_mode == 1) {
-        const int xh = d_tok[rr];
-        P.out.new_prop_tok[(size_t)b * NP + lane - 1] = xh;
-        // the raw logit at the first argmax is the row's maximum
-        P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 1] = xh >= 0 ? d_raw[rr] * P.inv_t : NAN;
-      }
-    }
-
+  {
     // The accept tests of all positions at once (a test depends on nothing an earlier one decides); the first
     // position that rejects, or whose token id is out of range, ends the sequence.
     float al = NAN;
@@ -638,6 +622,19 @@ __device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k,
       if (lane >= 1 && lane <= NP) {
         P.out.accept[(size_t)b * NP + lane - 1] = evald ? (lane == rej ? 0 : 1) : -1;
         P.out.alpha[(size_t)b * NP + lane - 1] = evald ? al : NAN;
+        // Proposals of the MASK rows (lanes 1..N-1 = MASK row m) and their law's statistics.  After a rejection
+        // the rows were conditioned on discarded tokens and the next step is a pure stride step (Sec. 3.2): no
+        // proposals are made.  Argmax proposals are final here; sampled ones and their logit are written by the
+        // CTAs that draw them.
+        const bool proposes = !frozen && rej == 0;
+        const int rr = nv + lane;
+        P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 0] = proposes ? d_lse[rr] : NAN;
+        if (P.propose_mode == 1 || !proposes) {
+          const int xh = proposes ? d_tok[rr] : -1;
+          P.out.new_prop_tok[(size_t)b * NP + lane - 1] = xh;
+          // the raw logit at the first argmax is the row's maximum
+          P.out.new_q_stats[((size_t)b * NP + lane - 1) * 2 + 1] = xh >= 0 ? d_raw[rr] * P.inv_t : NAN;
+        }
       }
       // the emission: accepted proposals now; the drawn token and the copy of it in repl_tok come from the CTA
       // of the sampling pass that finishes the draw, unless nothing is drawn
@@ -661,6 +658,10 @@ __device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k,
   // row's maximum (for the residual: if it has residual mass)
   H->nv = nv;
   H->rej = frozen ? -1 : rej;
+  if (k > 0 && (frozen || rej != 0)) {  // a MASK row of a slot that makes no proposals
+    H->rej = -2;
+    return;
+  }
   const int r = (k == 0 && rej > 0) ? rej - 1 : nv + k;
   H->r = r;
   H->q_row = q_row0 + rej - 1;
@@ -820,7 +821,7 @@ __device__ __forceinline__ bool verify_sample_body(const VerifyParams& P) {
   }
   __syncthreads();
   const int rej = sm_head.rej;
-  if (rej == -2) return split == 0;             // inactive or invalid slot
+  if (rej == -2) return split == 0;             // inactive or invalid slot, or no proposals to draw
   if (k == 0 && rej < 0) return split == 0;     // frozen slot: no emission
   const int nv = sm_head.nv;
 

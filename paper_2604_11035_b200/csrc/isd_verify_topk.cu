@@ -647,7 +647,9 @@ __device__ __forceinline__ double gumbel_at(const TopkParams& P, uint32_t step, 
 // L2: in the row kernel other CTAs of the same launch have written them.
 //
 // Proposals of the MASK rows: Gumbel-max over the support (warp m - 1 draws row nv + m), or its head.
-__device__ void draw_proposals(const TopkParams& P, const int* s_n, const double* s_lse, int b, int nv, uint32_t step) {
+// After a rejection (or on a frozen slot) the MASK rows were conditioned on discarded tokens: no proposals are made
+// (Sec. 3.2: the next step is a pure stride step) and the outputs are set to -1 / NaN (used = false).
+__device__ void draw_proposals(const TopkParams& P, const int* s_n, const double* s_lse, int b, int nv, uint32_t step, bool used) {
   const int NP = P.N - 1, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const double inv_t = (double)P.inv_t;
   const float* LV = P.list_val + (size_t)b * P.Q * kMaxTopK;
@@ -660,6 +662,14 @@ __device__ void draw_proposals(const TopkParams& P, const int* s_n, const double
     double best = -INFINITY;
     int tok = -1;
     float ltok = NAN;
+    if (!used) {
+      if (lane == 0) {
+        P.out.new_prop_tok[(size_t)b * NP + m - 1] = -1;
+        P.out.new_q_stats[((size_t)b * NP + m - 1) * 2 + 0] = NAN;
+        P.out.new_q_stats[((size_t)b * NP + m - 1) * 2 + 1] = NAN;
+      }
+      continue;
+    }
     if (P.propose_mode == 1) {
       if (n > 0) tok = ldcg_i(ix);
     } else {
@@ -800,7 +810,7 @@ __device__ __forceinline__ void topk_rows_body(const TopkParams& P, TopkShared& 
   // ---- and the slot's draws, unless the proposal-law row of a rejection has to be streamed (decide kernel)
   const uint32_t step = P.step_dev ? *P.step_dev : P.step;
   const int a = S.a, rej = S.rej;
-  draw_proposals(P, S.n, S.lse, b, nv, step);
+  draw_proposals(P, S.n, S.lse, b, nv, step, a >= 0 && rej == 0);
   if (a < 0) return;  // frozen: no emission
   if (rej == 0) {
     draw_bonus(P, S.n, b, nv, a, step);

@@ -22,7 +22,7 @@ import torch
 import oracle
 import paper_2604_11035_b200 as isd_pkg
 from paper_2604_11035_b200 import workloads as wl
-from helpers import STATE_KEYS, bits16, logits_np, oracle_step, state_to_np
+from helpers import STATE_KEYS, abs_diff_nan_aware, bits16, logits_np, oracle_step, state_to_np
 
 TOL = 2e-2
 EXEMPT = 1e-4
@@ -176,7 +176,7 @@ def run_chain_parity(w: wl.Workload, steps: int, device="cuda:0", attn_slots=Non
                         f"(final margin {vr.final_margin[b]:.3e})")
                     resync = True
             if NP:
-                dq = np.abs(g["new_q_stats"][b] - vr.new_q_stats[b]).max()
+                dq = abs_diff_nan_aware(g["new_q_stats"][b], vr.new_q_stats[b]).max()  # NaN: no proposals made
                 rep["qstats_max_abs_err"] = max(rep["qstats_max_abs_err"], float(dq))
                 if not (dq < TOL):
                     bad(f"step {t} slot {b}: q_stats err {dq:.3e}")

@@ -228,7 +228,14 @@ def test_commit_allocator_against_dictionary_model():
             assert s["n_ver"][b] == (N - 1 if a[b] == before["n_ver"][b] else 0)
             assert s["q_row0"][b] == before["n_ver"][b] + 1
             assert s["block_tok"][b, 0] == repl[b]
-            assert np.array_equal(s["q_stats"][b], nq[b])
+            # the proposal-law statistics follow the proposals: kept when the proposals are (nothing rejected),
+            # otherwise no proposals were made and the old ones stay
+            if a[b] == before["n_ver"][b]:
+                assert np.array_equal(s["q_stats"][b], nq[b])
+                assert np.array_equal(s["block_tok"][b, 1:N], newp[b])
+            else:
+                assert np.array_equal(s["q_stats"][b], before["q_stats"][b])
+                assert np.all(s["block_tok"][b, 1:N] == V - 1)
         if not np.any(s["slot_status"] & oracle.ST_POOL_EXHAUSTED):
             assert list(s["free_stack"][:int(s["free_top"][0])]) == model_free
             check_conservation(s, Q)

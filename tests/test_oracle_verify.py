@@ -369,9 +369,23 @@ def test_proposal_law_statistics_are_lse_and_logit_of_the_mask_rows(propose_mode
         s = tiny_state(B, N, V, n_ver=n_ver)
         s["block_tok"][:, 1:n_ver + 1] = rng.integers(0, V, (B, n_ver))
         prev = rng.normal(0, 2.0, (B, Q, V)).astype(np.float32)
+        # even slots: the proposal law of every proposal is the law that judges it (p / q = 1: all accepted);
+        # odd slots: unrelated laws and random proposals (rejected, except by luck)
+        for j in range(1, n_ver + 1):
+            prev[0::2, int(s["q_row0"][0]) + j - 1] = lg[0::2, j - 1]
+            s["block_tok"][0::2, j] = lg[0::2, j - 1].argmax(-1)   # inside the support of any filter
+        q_stats_before = s["q_stats"].copy()
         _, _, v, _ = oracle_step(w, s, None, None, None, lg, prev, 4, do_attn=False, inv_temperature=inv_t,
                                  top_k=top_k, top_p=top_p)
+        proposes = v.accept_len == n_ver
+        assert np.all(proposes[0::2]) and (n_ver == 0 or not np.all(proposes[1::2]))
         for b in range(B):
+            if not proposes[b]:
+                # Sec. 3.2 (adaptive stride): after a rejection the later tokens are discarded and the next step is
+                # a pure stride step, so no proposals are made from MASK rows conditioned on them
+                assert np.all(v.new_prop_tok[b] == -1) and np.all(np.isnan(v.new_q_stats[b]))
+                assert s["n_ver"][b] == 0 and np.array_equal(s["q_stats"][b], q_stats_before[b])
+                continue
             for m in range(1, N):
                 row = lg[b, n_ver + m].astype(np.float64) * float(np.float32(inv_t))
                 if top_k:
@@ -388,8 +402,9 @@ def test_proposal_law_statistics_are_lse_and_logit_of_the_mask_rows(propose_mode
                     assert xh == int(np.argmax(row))
                 assert abs(v.new_q_stats[b, m - 1, 0] - scipy.special.logsumexp(row)) < 1e-12
                 assert v.new_q_stats[b, m - 1, 1] == row[xh]
-        # and the next step's accept test consumes exactly these two numbers through commit
-        assert np.array_equal(s["q_stats"], v.new_q_stats)
+            # and the next step's accept test consumes exactly these two numbers through commit
+            assert np.array_equal(s["q_stats"][b], v.new_q_stats[b])
+            assert np.array_equal(s["block_tok"][b, 1:N], v.new_prop_tok[b])
 
 
 # --------------------------------------------------------------------------- data faults
