@@ -59,6 +59,7 @@ struct VerifyParams {
   int* samp_ticket;
   // isd_step: the CTA of the sampling pass that finishes last commits the batch (fuse_commit != 0)
   int fuse_commit;
+  int rows_early;  // isd_step: the row pass starts before the kernel ahead of it has completed (see verify_rows_kernel)
   int* step_ticket;
   CommitParams commit;
 };
@@ -354,21 +355,10 @@ __device__ __forceinline__ void row_timeout(const VerifyParams& P, int b) {
 // Pass 1: row statistics
 // ------------------------------------------------------------------------------------------------
 template <int DT>
-__global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const VerifyParams P) {
+__device__ __forceinline__ void verify_rows_body(const VerifyParams& P, RowRing& sm_ring) {
   // Launch order = (split, slot, k): the rows that the sampling pass reads again come last, so that
   // they are the most recent lines in L2 when it starts.
   const int split = blockIdx.x, b = blockIdx.y, k = blockIdx.z;
-  __shared__ RowRing sm_ring;
-  if (threadIdx.x == kThreads) {  // needs nothing from memory: runs while the kernel before this one drains
-    for (int i = 0; i < kRowStages; ++i) {
-      ring_mbar_init(ring_smem_u32(&sm_ring.full[i]), 1);
-      ring_mbar_init(ring_smem_u32(&sm_ring.empty[i]), kThreads / 32);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();  // the only CTA-wide barrier of the kernel, still ahead of the wait
-  pdl_wait();
-  pdl_launch_dependents();
   const int act = P.active[b];
   const int nv = P.n_ver[b];  // both loads in flight together
   if (!act) return;
@@ -436,6 +426,30 @@ __global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const Ver
     if (oi >= 0 && (mi < 0 || orw > v.z || (orw == v.z && oi < mi))) { v.z = orw; v.w = __int_as_float(oi); }
   }
   if (lane == 0) parts[((size_t)b * P.Q + r) * P.row_splits + split] = v;
+}
+
+// Inside isd_step the kernel before this one is the attention's combine kernel, of which the row pass needs
+// nothing: what it reads - the step's logits and the slots' state - was complete and visible before the step's
+// first kernel returned from its own wait.  There the pass starts streaming at once (rows_early), beside the
+// last CTAs of the combine kernel, and waits for it only before it ends, which keeps the order of completion
+// along the chain: the sampling kernel, whose last CTA rewrites the state the attention read, still cannot start
+// before the attention is done.  On its own (isd_verify) the pass may follow the very kernel that wrote the
+// logits, so it waits first.
+template <int DT>
+__global__ void __launch_bounds__(kThreads + 32, 5) verify_rows_kernel(const VerifyParams P) {
+  __shared__ RowRing sm_ring;
+  if (threadIdx.x == kThreads) {  // needs nothing from memory: runs while the kernel before this one drains
+    for (int i = 0; i < kRowStages; ++i) {
+      ring_mbar_init(ring_smem_u32(&sm_ring.full[i]), 1);
+      ring_mbar_init(ring_smem_u32(&sm_ring.empty[i]), kThreads / 32);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();  // the only CTA-wide barrier of the kernel, still ahead of the wait
+  if (!P.rows_early) pdl_wait();
+  pdl_launch_dependents();
+  verify_rows_body<DT>(P, sm_ring);
+  if (P.rows_early) pdl_wait();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1004,6 +1018,7 @@ int isd_launch_verify(isd_ctx* ctx, const isd_batch_state* st, const void* logit
   P.logits_cur = logits_cur; P.q_prev = q_prev_logits; P.out = *out;
   P.row_part = ctx->row_part; P.samp_part = ctx->samp_part; P.samp_ticket = ctx->samp_ticket;
   P.fuse_commit = commit_st != nullptr && ctx->step_ticket != nullptr;
+  P.rows_early = commit_st != nullptr;  // called from isd_step / isd_step_layers, behind the step's attention
   P.step_ticket = ctx->step_ticket;
   P.commit = make_commit_params(ctx, P.fuse_commit ? commit_st : st, out);
 
