@@ -524,16 +524,11 @@ __device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k,
   const char* cur = reinterpret_cast<const char*>(P.logits_cur) + (size_t)b * P.Q * row_bytes;
   const bool write = (k == 0 && split == 0);
 
-  // ---- first trip: nothing here depends on anything else that is read
+  // ---- before the wait: the slots' state and the step's logits were complete before the kernel ahead of this one
+  // could start (see verify_rows_kernel), so the proposals and their logits in the rows that judge them are
+  // fetched while that kernel drains
   const int act = P.active[b];
   const int nv = P.n_ver[b];
-  const int n_part = P.row_splits == 1 ? kThreads / 32 : P.row_splits;  // per warp of the row's CTA, or per CTA
-  const bool has_row = lane < P.Q;  // lane = block row (rows beyond the slot's block hold stale partials, unused)
-  const float4* rp = reinterpret_cast<const float4*>(P.row_part) + ((size_t)b * P.Q + (has_row ? lane : 0)) * n_part;
-  const float4 neutral = make_float4(-INFINITY, 0.f, -INFINITY, __int_as_float(-1));
-  float4 part[kHeadChunk];
-#pragma unroll
-  for (int i = 0; i < kHeadChunk; ++i) part[i] = i < n_part ? __ldcg(rp + i) : neutral;
   const bool is_pos = lane >= 1 && lane <= NP;  // lane = proposal position j (valid when j <= nv)
   int x = 0;
   float logq = 0.f, lse_q = 0.f;
@@ -545,20 +540,30 @@ __device__ __forceinline__ void sample_head(const VerifyParams& P, int b, int k,
       logq = qs[1] - lse_q;
     }
   }
+  const int q_row0 = (k == 0 && P.q_mode == 0) ? P.q_row0[b] : 0;
+  const bool slot_ok = act && nv >= 0 && nv <= NP;  // an invalid n_ver was flagged by the row pass
+  const bool pos = slot_ok && is_pos && lane <= nv;
+  const bool badtok = pos && (x < 0 || x >= P.V);
+  float lx = 0.f;  // the raw logit of the proposal in the row that judges it
+  if (pos && !badtok) lx = load_logit(cur + (size_t)(lane - 1) * row_bytes, P.logits_dtype, (size_t)x);
+
+  pdl_wait();
+  // ---- after it: what the row pass wrote, in one trip
+  const int n_part = P.row_splits == 1 ? kThreads / 32 : P.row_splits;  // per warp of the row's CTA, or per CTA
+  const bool has_row = lane < P.Q;  // lane = block row (rows beyond the slot's block hold stale partials, unused)
+  const float4* rp = reinterpret_cast<const float4*>(P.row_part) + ((size_t)b * P.Q + (has_row ? lane : 0)) * n_part;
+  const float4 neutral = make_float4(-INFINITY, 0.f, -INFINITY, __int_as_float(-1));
+  float4 part[kHeadChunk];
+#pragma unroll
+  for (int i = 0; i < kHeadChunk; ++i) part[i] = i < n_part ? __ldcg(rp + i) : neutral;
   // a warp of the row pass gave up on a wait: a partial is incomplete, nothing of the slot may be committed
   const uint32_t timeout = *reinterpret_cast<volatile uint32_t*>(&P.slot_status[b]) & ISD_ST_KERNEL_TIMEOUT;
-  const int q_row0 = (k == 0 && P.q_mode == 0) ? P.q_row0[b] : 0;
 
-  if (!act || nv < 0 || nv > NP) {  // an invalid n_ver was flagged by the row pass
+  if (!slot_ok) {
     if (lane == 0) H->rej = -2;
     return;
   }
   const int q_len = nv + P.N;
-  const bool pos = is_pos && lane <= nv;
-  const bool badtok = pos && (x < 0 || x >= P.V);
-  // ---- second trip: the raw logit of the proposal in the row that judges it
-  float lx = 0.f;
-  if (pos && !badtok) lx = load_logit(cur + (size_t)(lane - 1) * row_bytes, P.logits_dtype, (size_t)x);
 
   {  // lane = block row: merge its partials (max and sum of the online softmax, first argmax)
     float m = -INFINITY, s = 0.f, best = -INFINITY;
@@ -830,8 +835,10 @@ __device__ __forceinline__ bool verify_sample_body(const VerifyParams& P) {
 
   // ---- what the row pass found, the slot's decision, this CTA's job and its seed (the other warps wait)
   if (threadIdx.x < 32) {
-    sample_head<DT>(P, b, k, split, d_lse, d_raw, d_tok, d_bad, &sm_head);
+    sample_head<DT>(P, b, k, split, d_lse, d_raw, d_tok, d_bad, &sm_head);  // executes the wait
     if (threadIdx.x == 0) sm_best = sm_head.rej >= 0 ? sm_head.best : 0u;
+  } else {
+    pdl_wait();
   }
   __syncthreads();
   const int rej = sm_head.rej;
@@ -956,9 +963,8 @@ __device__ __forceinline__ bool verify_sample_body(const VerifyParams& P) {
 
 template <int DT>
 __global__ void __launch_bounds__(kThreads, kSampleMinBlocks) verify_sample_kernel(const VerifyParams P) {
-  pdl_wait();
   pdl_launch_dependents();
-  const bool reports = verify_sample_body<DT>(P);
+  const bool reports = verify_sample_body<DT>(P);  // executes griddepcontrol.wait after its first loads
   if (!P.fuse_commit || !reports) return;
   // ---- isd_step: every (slot, k) is reported once to a ticket over the grid, after its token is written; the
   // CTA that reports last (nobody waits) has every slot's decision and tokens in front of it and commits the
