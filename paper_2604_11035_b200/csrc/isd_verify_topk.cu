@@ -64,6 +64,7 @@ struct TopkParams {
   int* row_ticket;            // [B] rows of the slot that are done (zero between launches)
   // isd_step: the CTA of the row kernel that finishes last commits the batch (fuse_commit != 0)
   int fuse_commit;
+  int rows_early;  // isd_step: the row kernel starts before the kernel ahead of it has completed (see topk_rows_kernel)
   int* step_ticket;
   CommitParams commit;
 };
@@ -839,9 +840,14 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads + 32, 5) topk_rows_kernel(const TopkParams P) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
-  pdl_wait();
+  // Inside isd_step the kernel ahead of this one is the attention's combine kernel, of which the selection and
+  // the draws need nothing (the step's logits and the slots' state were complete before the step's first kernel
+  // returned from its own wait): the pass starts at once and waits before it ends - before the commit rewrites the
+  // state the attention read - which keeps the order of completion along the chain.
+  if (!P.rows_early) pdl_wait();
   pdl_launch_dependents();
   topk_rows_body<DT>(P, sh);
+  if (P.rows_early) pdl_wait();
   if (!P.fuse_commit) return;
   // ---- isd_step, when this kernel is the whole verification: the CTA that finishes last (a ticket over the grid;
   // nobody waits) commits the batch
@@ -1011,6 +1017,7 @@ int isd_launch_verify_topk(isd_ctx* ctx, const isd_batch_state* st, const void* 
   const bool stream_q = c.q_mode == 0 && q_prev_logits != nullptr && !P.prev_valid;
   // the row kernel commits by itself when it is the whole verification (no decide kernel after it)
   P.fuse_commit = (commit_st != nullptr && !stream_q && ctx->step_ticket != nullptr) ? 1 : 0;
+  P.rows_early = commit_st != nullptr;  // called from isd_step / isd_step_layers, behind the step's attention
   P.step_ticket = ctx->step_ticket;
   P.commit = make_commit_params(ctx, P.fuse_commit ? commit_st : st, out);
   if (committed) *committed = P.fuse_commit != 0;
