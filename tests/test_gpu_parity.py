@@ -356,3 +356,16 @@ def test_invalid_arguments_return_error_codes():
     with pytest.raises(isd_pkg.IsdError, match="invalid"):
         isd_pkg.Isd(batch=0, stride=2, n_q_heads=8, n_kv_heads=2, vocab=64, max_pages_per_slot=4, num_pages=8,
                     logits_dtype="f32")
+
+
+@pytest.mark.parametrize("seed", [300, 301, 302])
+@pytest.mark.parametrize("propose_mode,q_mode,N,B", [(1, 1, 8, 1), (0, 0, 4, 2), (1, 0, 16, 1), (0, 0, 2, 3), (1, 1, 4, 20)])
+def test_small_batches_at_the_full_vocabulary(seed, propose_mode, q_mode, N, B):
+    # Small batches take other launch shapes than the benchmark's batch: a row of the row pass is cut into up to
+    # sixteen CTAs (one partial per CTA, merged in chunks at the head of the sampling kernel) and a sampled row into
+    # up to sixteen pieces; steps that reject make no proposals.  Several seeds, five chained steps each.
+    w = Workload("small_full_vocab", batch=B, stride=N, n_q_heads=8, n_kv_heads=2, vocab=151936, ctx_min=3, ctx_max=300,
+                 logits_dtype="bf16", logit_sigma=3.0, peaked_frac=0.7, steps=5, propose_mode=propose_mode,
+                 q_mode=q_mode, seed=seed)
+    rep = run_chain_parity(w, steps=5, device=DEV)
+    assert_clean(rep)
